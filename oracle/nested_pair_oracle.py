@@ -1,0 +1,275 @@
+"""CPU oracle for the forward pass of a Pairformer-style block on a packed multi-ragged pair state.
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, per-sample NumPy restatement of what the
+method computes.  It shares no code with the CUDA library and the library never calls it; only
+the tests, the smoke check and the benchmark's CPU-baseline leg may import it.
+
+Form: one Python loop over samples; inside a sample, ordinary dense ``matmul``/``einsum`` on the
+sample's own ``[N, N, C]`` view of the packed buffer (Eq. 2, packing: ``V[o_s:o_{s+1}]`` is the
+sample's row-major reshape).  No padded ``B x N_max^2`` tensor is ever built here.  Working
+precision is the ``dtype`` argument (float64 by default).
+
+What each function follows:
+  offsets_build        Sec. 3.1 (sample offsets ``o``), Fig. 2 (two-level row splits), Eq. 3
+                       (coordinate map), App. A (invariants ``o_0 = 0``, ``o_{i+1}-o_i = p_i``, ``o_B = T``).
+  pair_broadcast       Eq. 1 line 1 and Sec. 3.2 "Creating axes through broadcasting"; the
+                       explicit-packed form ``u[rows] + v[cols]`` of the program figure; feature-wise
+                       LayerNorm on the static tail (Sec. 3.3).  No activation at construction (App. A.1).
+  tri_mul_out          Sec. 4.3 names the triangle multiplicative update of the Pairformer block;
+                       its internals are the standard gated outgoing form (a reading; see below).
+  row_attn_pairbias    Sec. 3.3 "Attention through packed blocks" (segments from cumulative lengths;
+                       output adopts the query structure) and Sec. 4.3 (triangle attention with a
+                       pair bias); internals are a reading (see below).
+  segment_reduce       Eq. 4 (pair reduction) and the mean of Eq. 1 line 3; App. A batch-axis
+                       convention (``[1,2],[3,4]`` sums to ``[3,7]``).
+  token_update         Eq. 1 line 3: ``X~ = X + g(mean_b P~[a,b,:])`` with ``g`` a bias-free projection.
+
+Pins (tests/test_oracle_pins.py): the paper's printed (2,3) example, the ``[3,7]`` reduction,
+structural invariants, closed forms, brute-force triple loops, an independent padded-and-masked
+dense implementation (oracle/bruteforce_padded.py), and batch-composition invariance.
+
+Parity unpinned: the *choice* of sub-layer internals (which gated form the triangle update takes,
+that the row-wise attention is starting-node attention with a bias shared by all rows of a sample,
+how blocks stack, the LayerNorm parameter draw).  The paper prints no value that depends on them;
+they are pinned only by the agreement between this file and the brute-force padded computation.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+LN_EPS = 1e-5
+
+
+# --------------------------------------------------------------------------------------------
+# structure
+# --------------------------------------------------------------------------------------------
+def offsets_build(lengths):
+    """Offsets, level-2 row splits, position decode and gather maps for square pairs.
+
+    tok_off[s]  = sum_{s'<s} N_s'            (token offsets, eta of Eq. 4)
+    pair_off[s] = sum_{s'<s} N_s'^2          (sample offsets o in packed-cell space)
+    row_splits[tok_off[s] + i] = pair_off[s] + i N_s, row_splits[T1] = T2   (1 + sum N entries)
+    For packed position p = pair_off[s] + i N_s + j (Eq. 3): pos_sample[p] = s, pos_i[p] = i,
+    pos_j[p] = j, rows[p] = tok_off[s] + i, cols[p] = tok_off[s] + j.
+    Written as the literal nested loops over (s, i, j).
+    """
+    lengths = [int(n) for n in lengths]
+    if any(n < 0 for n in lengths):
+        raise ValueError("negative length")
+    tok_off, pair_off = [0], [0]
+    for n in lengths:
+        tok_off.append(tok_off[-1] + n)
+        pair_off.append(pair_off[-1] + n * n)
+    row_splits, pos_s, pos_i, pos_j, rows, cols = [], [], [], [], [], []
+    for s, n in enumerate(lengths):
+        for i in range(n):
+            row_splits.append(pair_off[s] + i * n)
+            for j in range(n):
+                pos_s.append(s)
+                pos_i.append(i)
+                pos_j.append(j)
+                rows.append(tok_off[s] + i)
+                cols.append(tok_off[s] + j)
+    row_splits.append(pair_off[-1])
+    return dict(
+        tok_off=np.asarray(tok_off, dtype=np.int64),
+        pair_off=np.asarray(pair_off, dtype=np.int64),
+        row_splits=np.asarray(row_splits, dtype=np.int64),
+        pos_sample=np.asarray(pos_s, dtype=np.int32),
+        pos_i=np.asarray(pos_i, dtype=np.int32),
+        pos_j=np.asarray(pos_j, dtype=np.int32),
+        rows=np.asarray(rows, dtype=np.int64),
+        cols=np.asarray(cols, dtype=np.int64),
+    )
+
+
+def offsets_only(lengths):
+    """tok_off, pair_off and row_splits without the per-position maps (for large batches)."""
+    lengths = [int(n) for n in lengths]
+    tok_off, pair_off = [0], [0]
+    for n in lengths:
+        tok_off.append(tok_off[-1] + n)
+        pair_off.append(pair_off[-1] + n * n)
+    row_splits = []
+    for s, n in enumerate(lengths):
+        for i in range(n):
+            row_splits.append(pair_off[s] + i * n)
+    row_splits.append(pair_off[-1])
+    return (np.asarray(tok_off, dtype=np.int64), np.asarray(pair_off, dtype=np.int64),
+            np.asarray(row_splits, dtype=np.int64))
+
+
+def decode_position(lengths, p):
+    """(s, i, j) of one packed position p: the unique sample with pair_off[s] <= p < pair_off[s+1]
+    (empty samples are never selected), then i = r div N_s, j = r mod N_s."""
+    o = 0
+    for s, n in enumerate(int(v) for v in lengths):
+        if o <= p < o + n * n:
+            r = p - o
+            return s, r // n, r % n
+        o += n * n
+    raise IndexError("position outside the packed range")
+
+
+# --------------------------------------------------------------------------------------------
+# feature-wise pieces
+# --------------------------------------------------------------------------------------------
+def layer_norm(v, gamma, beta, eps=LN_EPS):
+    """LayerNorm over the last (static feature) axis, biased variance, then affine."""
+    mu = v.mean(axis=-1, keepdims=True)
+    var = ((v - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (v - mu) / np.sqrt(var + eps) * gamma + beta
+
+
+def sigmoid(v):
+    return 1.0 / (1.0 + np.exp(-v))
+
+
+def _as(dtype, *arrs):
+    return [np.asarray(a, dtype=dtype) for a in arrs]
+
+
+# --------------------------------------------------------------------------------------------
+# the five calls
+# --------------------------------------------------------------------------------------------
+def pair_broadcast(x, lengths, W_a, W_b, ln_gamma, ln_beta, eps=LN_EPS, dtype=np.float64):
+    """z[p,:] = LN_{c_z}(W_a x_i + W_b x_j) for p = (s,i,j).  Returns packed [T2, c_z]."""
+    x, W_a, W_b, ln_gamma, ln_beta = _as(dtype, x, W_a, W_b, ln_gamma, ln_beta)
+    out, t0 = [], 0
+    for n in (int(v) for v in lengths):
+        xs = x[t0:t0 + n]
+        u = xs @ W_a.T                       # [n, c_z]  left projection
+        v = xs @ W_b.T                       # [n, c_z]  right projection
+        P = u[:, None, :] + v[None, :, :]    # (N,1,C)+(1,N,C) -> (N,N,C)
+        out.append(layer_norm(P, ln_gamma, ln_beta, eps).reshape(n * n, W_a.shape[0]))
+        t0 += n
+    c_z = W_a.shape[0]
+    return np.concatenate(out, axis=0) if out else np.zeros((0, c_z), dtype=dtype)
+
+
+def tri_mul_out(z, lengths, W, eps=LN_EPS, dtype=np.float64, return_parts=False):
+    """Outgoing triangle multiplicative update with residual, per sample:
+        zh = LN_in(z);  a = sig(zh W_ag^T) * (zh W_ap^T);  b = sig(zh W_bg^T) * (zh W_bp^T)
+        g = sig(zh W_g^T);  t[i,j,c] = sum_k a[i,k,c] b[j,k,c];  z <- z + g * (LN_out(t) W_o^T)
+    """
+    z = np.asarray(z, dtype=dtype)
+    Wd = {k: np.asarray(v, dtype=dtype) for k, v in W.items()}
+    out, parts, o = [], [], 0
+    for n in (int(v) for v in lengths):
+        zs = z[o:o + n * n].reshape(n, n, z.shape[1])
+        zh = layer_norm(zs, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)
+        a = sigmoid(zh @ Wd["W_ag"].T) * (zh @ Wd["W_ap"].T)
+        b = sigmoid(zh @ Wd["W_bg"].T) * (zh @ Wd["W_bp"].T)
+        g = sigmoid(zh @ Wd["W_g"].T)
+        # per channel c the contraction is the matrix product A_c B_c^T; move c to the front so a
+        # BLAS-backed batched matmul can serve as the step (still the plain per-sample definition)
+        t = np.matmul(a.transpose(2, 0, 1), b.transpose(2, 1, 0)).transpose(1, 2, 0)
+        upd = g * (layer_norm(t, Wd["ln_out_gamma"], Wd["ln_out_beta"], eps) @ Wd["W_o"].T)
+        out.append((zs + upd).reshape(n * n, z.shape[1]))
+        if return_parts:
+            parts.append(dict(a=a, b=b, g=g, t=t))
+        o += n * n
+    res = np.concatenate(out, axis=0) if out else z.copy()
+    return (res, parts) if return_parts else res
+
+
+def row_attn_pairbias(zx, lengths, W, H, d, eps=LN_EPS, order="pair", dtype=np.float64, return_parts=False):
+    """Row-wise pair-biased softmax attention with residual.
+
+    order="pair": zx is the packed pair state [T2, c].  For each sample, each pair row i and head h,
+    the N positions j of the row attend over the positions k of the same row:
+        zh = LN(z); q,k,v = zh W_{q,k,v}^T viewed [N,N,H,d]; bias = zh W_b^T [N,N,H]; g = sig(zh W_g^T)
+        S[i,h,j,k] = <q[i,j,h,:], k[i,k,h,:]>/sqrt(d) + bias[j,k,h];  A = softmax_k S
+        o[i,j,h,:] = sum_k A[i,h,j,k] v[i,k,h,:];  z <- z + (g * o) W_o^T
+    The bias is shared by all rows i of the sample.
+    order="token": zx is the packed token buffer [T1, c]; one attention row per sample
+    (textbook variable-length self-attention over segments).
+    ln_gamma/ln_beta absent -> no LN; W_b absent -> zero bias; W_g absent -> no gate.
+    """
+    zx = np.asarray(zx, dtype=dtype)
+    Wd = {k: (None if v is None else np.asarray(v, dtype=dtype)) for k, v in W.items()}
+    has_ln = Wd.get("ln_gamma") is not None
+    W_b, W_g = Wd.get("W_b"), Wd.get("W_g")
+    scale = 1.0 / np.sqrt(float(d))
+    out, parts, o = [], [], 0
+    for n in (int(v) for v in lengths):
+        if n == 0:
+            continue                              # an empty sample has no rows
+        rows = n * n if order == "pair" else n
+        R = n if order == "pair" else 1          # number of attention rows in this sample
+        zs = zx[o:o + rows].reshape(R, n, zx.shape[1])
+        zh = layer_norm(zs, Wd["ln_gamma"], Wd["ln_beta"], eps) if has_ln else zs
+        q = (zh @ Wd["W_q"].T).reshape(R, n, H, d)
+        k = (zh @ Wd["W_k"].T).reshape(R, n, H, d)
+        v = (zh @ Wd["W_v"].T).reshape(R, n, H, d)
+        S = np.einsum("ijhe,ikhe->ihjk", q, k) * scale
+        if W_b is not None:
+            bias = zh @ W_b.T                    # [n, n, H] (pair order only: R == n)
+            S = S + bias.transpose(2, 0, 1)[None, :, :, :]
+        S = S - S.max(axis=-1, keepdims=True)
+        A = np.exp(S)
+        A = A / A.sum(axis=-1, keepdims=True)
+        ov = np.einsum("ihjk,ikhe->ijhe", A, v).reshape(R, n, H * d)
+        if W_g is not None:
+            ov = sigmoid(zh @ W_g.T) * ov
+        out.append((zs + ov @ Wd["W_o"].T).reshape(rows, zx.shape[1]))
+        if return_parts:
+            parts.append(dict(q=q, k=k, v=v, A=A, o=ov))
+        o += rows
+    res = np.concatenate(out, axis=0) if out else zx.copy()
+    return (res, parts) if return_parts else res
+
+
+def segment_reduce(v, splits, op="mean", dtype=np.float64):
+    """out[g,:] = sum (or mean) of rows splits[g] .. splits[g+1]-1 of v.  An empty segment gives
+    zeros (there is nothing to average; the pair path never produces one because an empty
+    sample has no rows)."""
+    v = np.asarray(v, dtype=dtype)
+    splits = [int(t) for t in splits]
+    G = len(splits) - 1
+    out = np.zeros((G,) + v.shape[1:], dtype=dtype)
+    for g in range(G):
+        lo, hi = splits[g], splits[g + 1]
+        if hi > lo:
+            acc = v[lo:hi].sum(axis=0)
+            out[g] = acc / (hi - lo) if op == "mean" else acc
+    return out
+
+
+def token_update(x, m, W_r, dtype=np.float64):
+    """x' = x + m W_r^T  (the projection g of Eq. 1 line 3, bias-free)."""
+    x, m, W_r = _as(dtype, x, m, W_r)
+    return x + m @ W_r.T
+
+
+# --------------------------------------------------------------------------------------------
+# compositions
+# --------------------------------------------------------------------------------------------
+def block_forward(x, lengths, w, H, d, eps=LN_EPS, dtype=np.float64):
+    """One Pairformer-style block: broadcast+LN, outgoing triangle update, row-wise pair-biased
+    attention, segmented mean over j and token update.  Returns (x', z)."""
+    _, _, row_splits = offsets_only(lengths)
+    z = pair_broadcast(x, lengths, eps=eps, dtype=dtype, **w["broadcast"])
+    z = tri_mul_out(z, lengths, w["trimul"], eps=eps, dtype=dtype)
+    z = row_attn_pairbias(z, lengths, w["attn"], H, d, eps=eps, order="pair", dtype=dtype)
+    m = segment_reduce(z, row_splits, "mean", dtype=dtype)
+    x2 = token_update(x, m, w["reduce"]["W_r"], dtype=dtype)
+    return x2, z
+
+
+def stack_forward(x, lengths, blocks, H, d, eps=LN_EPS, dtype=np.float64):
+    """Stacked blocks: block b+1 rebuilds the pair state from the tokens block b returned."""
+    z = None
+    x = np.asarray(x, dtype=dtype)
+    for w in blocks:
+        x, z = block_forward(x, lengths, w, H, d, eps=eps, dtype=dtype)
+    return x, z
+
+
+def token_forward(x, lengths, w, H, d, dtype=np.float64):
+    """Single-ragged special case: zero-bias attention over each sample's tokens, residual,
+    then a segmented mean over the token axis.  Returns (x', pooled [B, c])."""
+    x2 = row_attn_pairbias(x, lengths, w, H, d, order="token", dtype=dtype)
+    tok_off, _, _ = offsets_only(lengths)
+    pooled = segment_reduce(x2, tok_off, "mean", dtype=dtype)
+    return x2, pooled

@@ -1,0 +1,349 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, library routines, brute force,
+an independent padded-and-masked implementation, and batch-composition invariance.  No GPU."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import nested_pair_oracle as orc
+from oracle import bruteforce_padded as bf
+from paper_2609_30379_b200 import workloads as wl
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, v = line.split(":")
+            out[k.strip()] = [float(t) for t in v.split()]
+    return out
+
+
+def tiny_inputs(lengths, seed=7, c_s=6, c_z=8, c_h=4, H=2, d=4):
+    cfg = wl.Config("tiny", "f32", tuple(lengths), c_s=c_s, c_z=c_z, c_h=c_h, H=H, d=d, blocks=1, seed=seed)
+    return cfg, wl.make_inputs(cfg)
+
+
+# ------------------------------------------------------------------ offsets / decode
+def test_offsets_printed_example():
+    g = read_golden("fig2_lengths_2_3.txt")
+    r = orc.offsets_build([int(v) for v in g["lengths"]])
+    for key in ("tok_off", "pair_off", "row_splits", "rows", "cols", "pos_sample", "pos_i", "pos_j"):
+        assert r[key].tolist() == [int(v) for v in g[key]], key
+    assert len(r["rows"]) == 13 and r["tok_off"][-1] == 5
+    assert len(r["row_splits"]) == 1 + 5
+
+
+@pytest.mark.parametrize("lengths", [(5, 9, 13, 16), (0, 3, 0, 0, 4, 1), (1,), (), (0, 0), (7, 7, 7)])
+def test_offsets_invariants_and_closed_form(lengths):
+    r = orc.offsets_build(lengths)
+    n = np.asarray(lengths, dtype=np.int64)
+    assert r["pair_off"][0] == 0 and r["tok_off"][0] == 0
+    assert np.array_equal(np.diff(r["pair_off"]), n * n)
+    assert np.array_equal(np.diff(r["tok_off"]), n)
+    assert np.array_equal(r["pair_off"], np.concatenate([[0], np.cumsum(n * n)]))
+    assert np.array_equal(r["tok_off"], np.concatenate([[0], np.cumsum(n)]))
+    T1, T2 = int(n.sum()), int((n * n).sum())
+    assert len(r["row_splits"]) == T1 + 1 and r["row_splits"][-1] == T2
+    assert len(r["rows"]) == T2
+    # coordinate map (Eq. 3) composed with the decode is the identity on every packed position
+    for p in range(T2):
+        s, i, j = r["pos_sample"][p], r["pos_i"][p], r["pos_j"][p]
+        assert r["pair_off"][s] + i * n[s] + j == p
+        assert n[s] > 0 and 0 <= i < n[s] and 0 <= j < n[s]
+        assert (s, i, j) == orc.decode_position(lengths, p)
+        assert r["rows"][p] == r["tok_off"][s] + i and r["cols"][p] == r["tok_off"][s] + j
+    # every pair row's cells are exactly the level-2 segment
+    assert np.all(np.diff(r["row_splits"]) == np.repeat(n, n))
+    a, b, c = orc.offsets_only(lengths)
+    assert np.array_equal(a, r["tok_off"]) and np.array_equal(b, r["pair_off"]) and np.array_equal(c, r["row_splits"])
+
+
+def test_config_totals():
+    assert wl.CONFIGS["cfg1"].T2 == 531 and wl.CONFIGS["cfg1"].T1 == 43
+    assert wl.CONFIGS["cfg5"].T2 == 7_749_632
+    assert wl.CONFIGS["cfg2"].T2 == 368_250 and wl.CONFIGS["cfg3"].T2 == 1_023_931
+    assert wl.CONFIGS["cfg4"].T1 == 6411
+
+
+def test_same_rows_different_structure():
+    # (2,6,C) and (3,4,C) both flatten to twelve feature rows yet are different structures;
+    # for square pairs: lengths (1,7) and (5,5) both pack 50 cells with different partitions
+    a, b = orc.offsets_build((1, 7)), orc.offsets_build((5, 5))
+    assert a["pair_off"][-1] == b["pair_off"][-1] == 50
+    assert a["pair_off"].tolist() != b["pair_off"].tolist()
+    assert a["rows"].tolist() != b["rows"].tolist()
+
+
+# ------------------------------------------------------------------ layer norm / reduce
+def test_layer_norm_matches_library():
+    rng = np.random.default_rng(0)
+    v = rng.standard_normal((11, 3, 24)) * 3 + 1.5
+    g, b = rng.standard_normal(24), rng.standard_normal(24)
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(v), (24,), torch.from_numpy(g), torch.from_numpy(b), 1e-5)
+    assert np.allclose(orc.layer_norm(v, g, b, 1e-5), ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_segment_reduce_printed_example():
+    g = read_golden("appA_batch_axis_sum.txt")
+    v = np.asarray(g["values"])[:, None]
+    sp = [int(t) for t in g["splits"]]
+    assert orc.segment_reduce(v, sp, "sum")[:, 0].tolist() == g["sum"]
+    assert orc.segment_reduce(v, sp, "mean")[:, 0].tolist() == g["mean"]
+
+
+def test_segment_reduce_closed_forms():
+    rng = np.random.default_rng(1)
+    v = rng.standard_normal((40, 5))
+    sp = np.array([0, 3, 3, 10, 11, 40])
+    got = orc.segment_reduce(v, sp, "sum")
+    nz = np.diff(sp) > 0
+    ref = np.add.reduceat(v, sp[:-1][nz], axis=0)
+    assert np.allclose(got[nz], ref, rtol=1e-13, atol=1e-13)
+    assert np.all(got[~nz] == 0)
+    const = np.full((9, 3), 2.5)
+    assert np.allclose(orc.segment_reduce(const, [0, 4, 9], "mean"), 2.5)
+    # Eq. 4 with counts: pair state of lengths (2,3), mean over j divides by N_s
+    L = (2, 3)
+    r = orc.offsets_build(L)
+    P = rng.standard_normal((13, 2))
+    m = orc.segment_reduce(P, r["row_splits"], "mean")
+    for s, n in enumerate(L):
+        for a in range(n):
+            acc = sum(P[r["pair_off"][s] + a * n + b] for b in range(n))
+            assert np.allclose(m[r["tok_off"][s] + a], acc / n)
+
+
+# ------------------------------------------------------------------ broadcast
+def test_broadcast_packed_size_and_gather_form():
+    cfg, inp = tiny_inputs((3, 5, 1, 4))
+    w = inp["blocks"][0]["broadcast"]
+    z = orc.pair_broadcast(inp["x"], cfg.lengths, **w)
+    assert z.shape == (cfg.T2, cfg.c_z)
+    r = orc.offsets_build(cfg.lengths)
+    x = inp["x"].astype(np.float64)
+    u, v = x @ w["W_a"].astype(np.float64).T, x @ w["W_b"].astype(np.float64).T
+    pre = u[r["rows"]] + v[r["cols"]]          # the explicit-packed form of the program figure
+    ref = torch.nn.functional.layer_norm(torch.from_numpy(pre), (cfg.c_z,),
+                                         torch.from_numpy(w["ln_gamma"].astype(np.float64)),
+                                         torch.from_numpy(w["ln_beta"].astype(np.float64)), 1e-5).numpy()
+    assert np.allclose(z, ref, rtol=1e-11, atol=1e-11)
+
+
+def test_broadcast_special_cases():
+    cfg, inp = tiny_inputs((4, 6))
+    w = dict(inp["blocks"][0]["broadcast"])
+    w0 = dict(w, W_b=np.zeros_like(w["W_b"]))
+    z = orc.pair_broadcast(inp["x"], cfg.lengths, **w0)
+    o = 0
+    for n in cfg.lengths:
+        zs = z[o:o + n * n].reshape(n, n, -1)
+        assert np.allclose(zs, zs[:, :1, :])       # constant along j when the column term vanishes
+        o += n * n
+    w1 = dict(w, ln_gamma=np.ones(cfg.c_z), ln_beta=np.zeros(cfg.c_z))
+    z = orc.pair_broadcast(inp["x"], cfg.lengths, **w1)
+    assert np.allclose(z.mean(-1), 0, atol=1e-12)
+    r = orc.offsets_build(cfg.lengths)
+    x = inp["x"].astype(np.float64)
+    pre = (x @ w["W_a"].T.astype(np.float64))[r["rows"]] + (x @ w["W_b"].T.astype(np.float64))[r["cols"]]
+    var = pre.var(-1)
+    assert np.allclose(z.var(-1), 1 - 1e-5 / (var + 1e-5), rtol=1e-10)
+
+
+# ------------------------------------------------------------------ triangle update
+def test_trimul_contraction_bruteforce_and_symmetry():
+    cfg, inp = tiny_inputs((3, 5, 2))
+    rng = np.random.default_rng(3)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    W = inp["blocks"][0]["trimul"]
+    znew, parts = orc.tri_mul_out(z, cfg.lengths, W, return_parts=True)
+    for n, p in zip(cfg.lengths, parts):
+        a, b, t = p["a"], p["b"], p["t"]
+        ref = np.zeros_like(t)
+        for i in range(n):
+            for j in range(n):
+                for k in range(n):
+                    ref[i, j, :] += a[i, k, :] * b[j, k, :]
+        assert np.allclose(t, ref, rtol=1e-12, atol=1e-12)
+        for c in range(cfg.c_h):                               # per channel: a library matmul A_c B_c^T
+            assert np.allclose(t[:, :, c], a[:, :, c] @ b[:, :, c].T, rtol=1e-12, atol=1e-12)
+    # a == b  ->  t symmetric in (i, j)
+    Ws = dict(W, W_bp=W["W_ap"], W_bg=W["W_ag"])
+    _, parts = orc.tri_mul_out(z, cfg.lengths, Ws, return_parts=True)
+    for p in parts:
+        assert np.allclose(p["t"], p["t"].transpose(1, 0, 2), rtol=1e-12, atol=1e-12)
+    # zero output projection -> pure residual
+    W0 = dict(W, W_o=np.zeros_like(W["W_o"]))
+    assert np.array_equal(orc.tri_mul_out(z, cfg.lengths, W0), z)
+
+
+def test_trimul_full_formula_via_torch():
+    # the same update written with torch float64 primitives on one sample (library einsum,
+    # library layer_norm, library sigmoid)
+    cfg, inp = tiny_inputs((6,))
+    rng = np.random.default_rng(4)
+    z = rng.standard_normal((36, cfg.c_z))
+    W = {k: torch.from_numpy(np.asarray(v, dtype=np.float64)) for k, v in inp["blocks"][0]["trimul"].items()}
+    zt = torch.from_numpy(z).reshape(6, 6, -1)
+    F = torch.nn.functional
+    zh = F.layer_norm(zt, (cfg.c_z,), W["ln_in_gamma"], W["ln_in_beta"], 1e-5)
+    a = torch.sigmoid(F.linear(zh, W["W_ag"])) * F.linear(zh, W["W_ap"])
+    b = torch.sigmoid(F.linear(zh, W["W_bg"])) * F.linear(zh, W["W_bp"])
+    t = torch.einsum("ikc,jkc->ijc", a, b)
+    upd = torch.sigmoid(F.linear(zh, W["W_g"])) * F.linear(F.layer_norm(t, (cfg.c_h,), W["ln_out_gamma"], W["ln_out_beta"], 1e-5), W["W_o"])
+    ref = (zt + upd).reshape(36, -1).numpy()
+    got = orc.tri_mul_out(z, cfg.lengths, inp["blocks"][0]["trimul"])
+    assert np.allclose(got, ref, rtol=1e-11, atol=1e-11)
+
+
+# ------------------------------------------------------------------ attention
+def test_attention_matches_library_sdpa():
+    cfg, inp = tiny_inputs((4, 7, 1))
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    Wn = inp["blocks"][0]["attn"]
+    got, parts = orc.row_attn_pairbias(z, cfg.lengths, Wn, cfg.H, cfg.d, return_parts=True)
+    W = {k: torch.from_numpy(np.asarray(v, dtype=np.float64)) for k, v in Wn.items()}
+    F = torch.nn.functional
+    o = 0
+    for n, p in zip(cfg.lengths, parts):
+        zt = torch.from_numpy(z[o:o + n * n]).reshape(n, n, -1)
+        zh = F.layer_norm(zt, (cfg.c_z,), W["ln_gamma"], W["ln_beta"], 1e-5)
+        q = F.linear(zh, W["W_q"]).reshape(n, n, cfg.H, cfg.d).permute(0, 2, 1, 3)     # [i, h, j, e]
+        k = F.linear(zh, W["W_k"]).reshape(n, n, cfg.H, cfg.d).permute(0, 2, 1, 3)
+        v = F.linear(zh, W["W_v"]).reshape(n, n, cfg.H, cfg.d).permute(0, 2, 1, 3)
+        bias = F.linear(zh, W["W_b"]).permute(2, 0, 1)[None]                          # [1, h, j, k]
+        att = F.scaled_dot_product_attention(q, k, v, attn_mask=bias)                 # scale 1/sqrt(d)
+        ov = att.permute(0, 2, 1, 3).reshape(n, n, cfg.H * cfg.d)
+        ref = zt + F.linear(torch.sigmoid(F.linear(zh, W["W_g"])) * ov, W["W_o"])
+        assert np.allclose(got[o:o + n * n], ref.reshape(n * n, -1).numpy(), rtol=1e-10, atol=1e-10)
+        assert np.allclose(p["A"].sum(-1), 1.0, rtol=1e-12)
+        o += n * n
+
+
+def test_attention_special_cases():
+    cfg, inp = tiny_inputs((5, 3))
+    rng = np.random.default_rng(6)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    W = dict(inp["blocks"][0]["attn"])
+    # (a) zero bias and zero W_v rows except through beta: all v rows equal -> o equals that row
+    Wv = dict(W, ln_gamma=np.zeros(cfg.c_z), W_g=None)   # LN output = beta for every position
+    _, parts = orc.row_attn_pairbias(z, cfg.lengths, Wv, cfg.H, cfg.d, return_parts=True)
+    vrow = np.asarray(W["W_v"], dtype=np.float64) @ np.asarray(W["ln_beta"], dtype=np.float64)
+    for p in parts:
+        assert np.allclose(p["o"], vrow[None, None, :], rtol=1e-12, atol=1e-12)
+    # (b) softmax shift invariance: adding a constant to every bias[j,:,h] leaves the output unchanged.
+    #     A channel that is constant over positions cannot be built after LN, so test it on the
+    #     un-normalised path: no LN, z gets an extra constant feature read only by W_b.
+    zc = np.concatenate([z, np.ones((cfg.T2, 1))], axis=1)
+    Wn = {k: (None if v is None else np.concatenate([np.asarray(v, dtype=np.float64), np.zeros((v.shape[0], 1))], axis=1))
+          for k, v in W.items() if k.startswith("W_") and k != "W_o"}
+    Wn["W_o"] = np.concatenate([np.asarray(W["W_o"], dtype=np.float64), np.zeros((1, cfg.H * cfg.d))], axis=0)
+    Wn["ln_gamma"] = None
+    Wn["ln_beta"] = None
+    base = orc.row_attn_pairbias(zc, cfg.lengths, Wn, cfg.H, cfg.d)
+    Wn2 = dict(Wn)
+    Wn2["W_b"] = Wn["W_b"].copy()
+    Wn2["W_b"][:, -1] = 3.7
+    assert np.allclose(orc.row_attn_pairbias(zc, cfg.lengths, Wn2, cfg.H, cfg.d), base, rtol=1e-11, atol=1e-11)
+
+
+def test_token_attention_is_textbook_varlen():
+    cfg = wl.Config("tok", "f32", (7, 3, 12), c_s=16, c_z=16, c_h=0, H=2, d=8, blocks=1, seed=11, kind="token")
+    inp = wl.make_inputs(cfg)
+    w = inp["blocks"][0]
+    x2, pooled = orc.token_forward(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    F = torch.nn.functional
+    t0 = 0
+    for s, n in enumerate(cfg.lengths):
+        xs = torch.from_numpy(inp["x"][t0:t0 + n].astype(np.float64))
+        q, k, v = (F.linear(xs, torch.from_numpy(w[nm].astype(np.float64))).reshape(n, cfg.H, cfg.d).transpose(0, 1)
+                   for nm in ("W_q", "W_k", "W_v"))
+        att = F.scaled_dot_product_attention(q, k, v).transpose(0, 1).reshape(n, -1)
+        ref = xs + F.linear(att, torch.from_numpy(w["W_o"].astype(np.float64)))
+        assert np.allclose(x2[t0:t0 + n], ref.numpy(), rtol=1e-10, atol=1e-10)
+        assert np.allclose(pooled[s], ref.numpy().mean(0), rtol=1e-10, atol=1e-10)
+        t0 += n
+    xb, pb = bf.token_forward_padded(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    assert np.allclose(x2, xb, rtol=1e-10, atol=1e-10) and np.allclose(pooled, pb, rtol=1e-10, atol=1e-10)
+
+
+# ------------------------------------------------------------------ whole block
+@pytest.mark.parametrize("lengths", [(2, 3), (5, 1, 4, 7), (6, 6, 6), (1, 7), (5, 5)])
+def test_block_equals_padded_bruteforce(lengths):
+    cfg, inp = tiny_inputs(lengths)
+    w = inp["blocks"][0]
+    x2, z = orc.block_forward(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    xb, zb = bf.block_forward_padded(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    assert z.shape == (cfg.T2, cfg.c_z) and x2.shape == (cfg.T1, cfg.c_s)
+    assert np.allclose(z, zb, rtol=1e-9, atol=1e-9)
+    assert np.allclose(x2, xb, rtol=1e-9, atol=1e-9)
+
+
+def test_block_cfg1_equals_padded_bruteforce():
+    cfg = wl.CONFIGS["cfg1"]
+    inp = wl.make_inputs(cfg)
+    w = inp["blocks"][0]
+    x2, z = orc.block_forward(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    xb, zb = bf.block_forward_padded(inp["x"], cfg.lengths, w, cfg.H, cfg.d)
+    assert z.size == 531 * 16
+    assert np.allclose(z, zb, rtol=1e-9, atol=1e-9) and np.allclose(x2, xb, rtol=1e-9, atol=1e-9)
+
+
+def test_sample_local_invariance():
+    # each sample's output is the same alone, with batch-mates, and under permutation of the batch
+    cfg, inp = tiny_inputs((4, 2, 6, 3))
+    w = inp["blocks"][0]
+    x = inp["x"]
+    x2, z = orc.block_forward(x, cfg.lengths, w, cfg.H, cfg.d)
+    tok = np.concatenate([[0], np.cumsum(cfg.lengths)])
+    po = np.concatenate([[0], np.cumsum(np.square(cfg.lengths))])
+    for s, n in enumerate(cfg.lengths):
+        xs, zs = orc.block_forward(x[tok[s]:tok[s + 1]], (n,), w, cfg.H, cfg.d)
+        assert np.allclose(xs, x2[tok[s]:tok[s + 1]], rtol=1e-11, atol=1e-11)
+        assert np.allclose(zs, z[po[s]:po[s + 1]], rtol=1e-11, atol=1e-11)
+    perm = [2, 0, 3, 1]
+    xp = np.concatenate([x[tok[s]:tok[s + 1]] for s in perm])
+    lp = [cfg.lengths[s] for s in perm]
+    x2p, zp = orc.block_forward(xp, lp, w, cfg.H, cfg.d)
+    t = 0
+    o = 0
+    for s in perm:
+        n = cfg.lengths[s]
+        assert np.allclose(x2p[t:t + n], x2[tok[s]:tok[s + 1]], rtol=1e-11, atol=1e-11)
+        assert np.allclose(zp[o:o + n * n], z[po[s]:po[s + 1]], rtol=1e-11, atol=1e-11)
+        t += n
+        o += n * n
+
+
+def test_empty_samples_contribute_nothing():
+    cfg, inp = tiny_inputs((3, 4))
+    w = inp["blocks"][0]
+    x2, z = orc.block_forward(inp["x"], (3, 4), w, cfg.H, cfg.d)
+    x2e, ze = orc.block_forward(inp["x"], (0, 3, 0, 4, 0), w, cfg.H, cfg.d)
+    assert np.array_equal(x2, x2e) and np.array_equal(z, ze)
+    x0, z0 = orc.block_forward(np.zeros((0, cfg.c_s)), (), w, cfg.H, cfg.d)
+    assert x0.shape == (0, cfg.c_s) and z0.shape == (0, cfg.c_z)
+
+
+def test_stack_rebuilds_pair_state_from_tokens():
+    cfg = wl.Config("two", "f32", (3, 5), c_s=6, c_z=8, c_h=4, H=2, d=4, blocks=2, seed=21)
+    inp = wl.make_inputs(cfg)
+    x2, z2 = orc.stack_forward(inp["x"], cfg.lengths, inp["blocks"], cfg.H, cfg.d)
+    xa, _ = orc.block_forward(inp["x"], cfg.lengths, inp["blocks"][0], cfg.H, cfg.d)
+    xb, zb = orc.block_forward(xa, cfg.lengths, inp["blocks"][1], cfg.H, cfg.d)
+    assert np.array_equal(x2, xb) and np.array_equal(z2, zb)
+
+
+def test_bf16_rounding_helpers():
+    a = np.array([1.0, 1.00390625, 1.001953125, 3.1415927, -2.7182817, 1e-3], dtype=np.float32)
+    ref = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    r = wl.round_to_bf16(a)
+    assert np.array_equal(r, ref)
+    assert np.array_equal(wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(r)), r)
