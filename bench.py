@@ -1,0 +1,370 @@
+"""Benchmark of the packed Pairformer-style block forward (libnested_pair) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg2] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one synthetic batch: every stacked block of the
+configuration (pair broadcast + LN, triangle multiplicative update, row-wise pair-biased attention,
+segmented mean + token update).  The metric is packed pair positions per second per block:
+(#blocks * T2 * steps * n_gpus) / time.  The path does not shard (one GPU per batch, no
+collectives): with N > 1 every rank runs an independent replica ("replicas only").
+
+One JSON line is printed by rank 0.  Besides the base keys it carries
+  roofline      for the kernel with the largest share of the step (timed live with CUDA events)
+  cpu_baseline  the NumPy oracle timed on the host cores on a bounded sample of the same workload
+  e2e           the same metric through the public API with host buffers and copies in the timed region
+  kernels       per-kernel share of the step
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2609_30379_b200 import workloads as wl  # noqa: E402
+
+METRIC = "packed pair positions/sec per Pairformer-style block (fwd)"
+UNIT = "positions/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# algorithmic work per launch of every kernel (bytes the packed method must move, flops it must do)
+# ----------------------------------------------------------------------------------------------
+def kernel_work(cfg: wl.Config):
+    e = 4 if cfg.dtype == "f32" else 2
+    T1, T2, N3 = cfg.T1, cfg.T2, cfg.N3
+    c_s, c_z, c_h, H, d = cfg.c_s, cfg.c_z, cfg.c_h, cfg.H, cfg.d
+    Hd = H * d
+    w = {}
+    tok = dict(bytes=T1 * c_s * e + c_z * c_s * e + T1 * c_z * 4, flops=2 * T1 * c_s * c_z)
+    w["tok_proj_u"] = w["tok_proj_v"] = tok
+    bc = dict(bytes=T2 * c_z * e + 2 * T1 * c_z * 4, flops=8 * T2 * c_z)
+    w["broadcast_ln"] = w["generic_broadcast_ln"] = bc
+    w["generic_tri_in_a"] = w["generic_tri_in_b"] = dict(bytes=T2 * (c_z + c_h) * e, flops=2 * T2 * c_z * 2 * c_h)
+    w["generic_tri_in_g"] = dict(bytes=2 * T2 * c_z * e, flops=2 * T2 * c_z * c_z)
+    w["tri_in"] = dict(bytes=T2 * (c_z + 2 * c_h) * e, flops=2 * T2 * c_z * 4 * c_h)
+    w["generic_tri_contract"] = w["tri_contract"] = dict(bytes=3 * T2 * c_h * e, flops=2 * N3 * c_h)
+    w["generic_tri_out"] = dict(bytes=T2 * (c_h + 3 * c_z) * e, flops=2 * T2 * c_h * c_z)
+    w["tri_out"] = dict(bytes=T2 * (c_h + 2 * c_z) * e, flops=2 * T2 * (c_h + c_z) * c_z)
+    for n in ("q", "k", "v", "g"):
+        w[f"generic_attn_in_{n}"] = dict(bytes=T2 * (c_z + Hd) * e, flops=2 * T2 * c_z * Hd)
+    w["generic_attn_in_bias"] = dict(bytes=T2 * (c_z + H) * e, flops=2 * T2 * c_z * H)
+    w["attn_in"] = dict(bytes=T2 * (c_z + 4 * Hd + H) * e, flops=2 * T2 * c_z * (4 * Hd + H))
+    w["generic_attn_core"] = w["attn_core"] = dict(bytes=T2 * (4 * Hd + H) * e, flops=4 * N3 * Hd)
+    w["generic_attn_out"] = w["attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)
+    sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
+    w["segment_reduce"] = w["generic_segment_reduce"] = sr
+    w["token_update"] = dict(bytes=T1 * (c_z + 2 * c_s) * e + c_s * c_z * e, flops=2 * T1 * c_s * c_z)
+    return w
+
+
+def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
+    if name not in work or launches == 0:
+        return None
+    wk = work[name]
+    t = total_ms / launches * 1e-3
+    hbm = peaks["hbm_gbs"] * 1e9
+    tens = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
+    t_hbm, t_tensor = wk["bytes"] / hbm, wk["flops"] / tens
+    if t_hbm >= t_tensor:
+        ach = wk["bytes"] / t / 1e9
+        return dict(kernel=name, bound="hbm", achieved=round(ach, 1), peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=round(ach / peaks["hbm_gbs"], 4), traffic=None, peak_source=f"of {peak_kind}",
+                    us_per_launch=round(t * 1e6, 2), launches=launches)
+    ach = wk["flops"] / t / 1e12
+    pk = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    return dict(kernel=name, bound="tensor", achieved=round(ach, 2), peak=pk, unit="TFLOP/s",
+                frac=round(ach / pk, 4), traffic=None, peak_source=f"of {peak_kind} (sustained)",
+                us_per_launch=round(t * 1e6, 2), launches=launches)
+
+
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+            time.sleep(0.25)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, r[4:8]):
+                if val.strip().lower() == "active":
+                    reasons.add(nm)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_rate(cfg, inp, n_samples, repeats=1):
+    """Times the NumPy oracle (as it stands, float32 on the same bf16-rounded inputs) on one block over
+    the first n_samples samples of the batch.  Returns (positions/s, seconds, sample description)."""
+    from oracle import nested_pair_oracle as orc
+    lengths = list(cfg.lengths[:n_samples])
+    T1s = sum(lengths)
+    x = inp["x"][:T1s]
+    dt = np.float64 if cfg.dtype == "f32" else np.float32
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        if cfg.kind == "pair":
+            orc.block_forward(x, lengths, inp["blocks"][0], cfg.H, cfg.d, dtype=dt)
+        else:
+            orc.token_forward(x, lengths, inp["blocks"][0], cfg.H, cfg.d, dtype=dt)
+        el = time.perf_counter() - t0
+        best = el if best is None else min(best, el)
+    units = sum(n * n for n in lengths)
+    return units / best, best, f"one block over the first {n_samples} of {cfg.B} samples ({units} positions), oracle in {np.dtype(dt).name}"
+
+
+def run_reference(args):
+    """The reference arm of this tier is the CPU oracle, timed as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = wl.CONFIGS[args.config]
+    inp = wl.make_inputs(cfg)
+    warm = max(args.warmup, 0)
+    for _ in range(min(warm, 1)):
+        oracle_sample_rate(cfg, inp, 1)
+    t0 = time.perf_counter()
+    units = 0
+    desc = ""
+    for _ in range(args.steps):
+        rate, sec, desc = oracle_sample_rate(cfg, inp, 1)
+        units += rate * sec
+    el = time.perf_counter() - t0
+    value = units / el
+    cores = len(os.sched_getaffinity(0))
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=min(warm, 1), ms_per_step=el / max(args.steps, 1) * 1e3, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                config=dict(workload=f"{cfg.name}: per step {desc}", lengths=list(cfg.lengths[:1])),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=desc),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="cfg2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2609_30379_b200 import build
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        dist.barrier()
+    from paper_2609_30379_b200 import binding as nt, runner
+
+    if args.force_generic:
+        nt.nt_force_generic(True)
+    cfg = wl.CONFIGS[args.config]
+    inp = wl.make_inputs(cfg)
+    stack = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    x0 = runner.to_device(inp["x"], stack.dtype)
+    x = torch.empty_like(x0)
+    warmup = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+
+    def step():
+        x.copy_(x0)
+        return stack.forward(x)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    torch.cuda.reset_peak_memory_stats()
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = nt.nt_launch_count()
+    barrier()
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    barrier()
+    launches = nt.nt_launch_count() - launches0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    unit_count = cfg.T2 if cfg.kind == "pair" else cfg.T1
+    value = world * cfg.blocks * unit_count * steps / (ms * 1e-3)
+    peak_alloc = torch.cuda.max_memory_allocated()
+
+    # ---- per-kernel timing pass (CUDA events around every launch, on the launching stream)
+    barrier()
+    nt.nt_profile_begin()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    prof = nt.nt_profile_end()
+    tot_prof = sum(v[0] for v in prof.values()) or 1.0
+    peaks, peak_kind = load_peaks()
+    work = kernel_work(cfg)
+    kernels = {k: dict(ms_per_step=round(v[0] / steps, 4), launches_per_step=v[1] / steps, share=round(v[0] / tot_prof, 4))
+               for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])}
+    roofs = {k: roofline_entry(k, v[0], v[1], work, peaks, peak_kind) for k, v in prof.items()}
+    roofs = {k: r for k, r in roofs.items() if r}
+    for k in kernels:
+        if k in roofs:
+            kernels[k]["frac"] = roofs[k]["frac"]
+            kernels[k]["bound"] = roofs[k]["bound"]
+    dominant = max(prof.items(), key=lambda kv: kv[1][0])[0] if prof else None
+    roofline = roofs.get(dominant) if dominant else None
+
+    # ---- end to end through the public API with host buffers
+    x_pin = torch.from_numpy(np.ascontiguousarray(inp["x"])).to(stack.dtype).pin_memory()
+    out_pin = torch.empty_like(x_pin).pin_memory()
+    h2d = x_pin.numel() * x_pin.element_size() + 8 * cfg.B
+    d2h = out_pin.numel() * out_pin.element_size()
+
+    def e2e_step():
+        stack.L = nt.Layout(cfg.lengths)          # lengths to the device + offsets build
+        x.copy_(x_pin, non_blocking=True)
+        xo, _ = stack.forward(x)
+        out_pin.copy_(xo, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * cfg.blocks * unit_count * steps / e2e_s
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_s = {"cfg1": cfg.B, "cfg2": 4, "cfg3": 8, "cfg4": cfg.B, "cfg5": 1}[cfg.name]
+        rate, sec, desc = oracle_sample_rate(cfg, inp, n_s)
+        cpu = dict(value=rate, unit=UNIT, cores=len(os.sched_getaffinity(0)), kind="oracle",
+                   sample=f"{desc}; {sec:.1f} s")
+
+    nmax = cfg.N_max
+    esz = 4 if cfg.dtype == "f32" else 2
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup,
+        ms_per_step=ms / steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16 storage, f32 accumulate" if cfg.dtype == "bf16" else "f32", data="synthetic",
+        config=dict(workload=f"{cfg.name}: B={cfg.B}, lengths {min(cfg.lengths)}..{max(cfg.lengths)}, "
+                             f"c_s={cfg.c_s}, c_z={cfg.c_z}, c_h={cfg.c_h}, H={cfg.H}x{cfg.d}, {cfg.blocks} blocks",
+                    T1=cfg.T1, T2=cfg.T2, rho_pair=round(wl.pair_occupancy(cfg.lengths), 4),
+                    parallelism="replicas only" if world > 1 else "single GPU",
+                    l2="per-step working set (pair state + intermediates) exceeds the 126 MB L2; no explicit flush",
+                    kernels_path="generic" if args.force_generic else "default"),
+        tokens_per_s=world * cfg.blocks * cfg.T1 * steps / (ms * 1e-3),
+        peak_alloc_bytes=peak_alloc, padded_envelope_z_bytes=cfg.B * nmax * nmax * cfg.c_z * esz,
+        gpu_launches=launches, clocks=clocks, roofline=roofline, kernels=kernels, cpu_baseline=cpu,
+        e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                 note="host pinned tokens + lengths in, offsets rebuilt, updated tokens out; wall clock"),
+    )
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

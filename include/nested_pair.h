@@ -1,0 +1,189 @@
+/*
+ * libnested_pair -- forward pass of a Pairformer-style block on a packed multi-ragged pair state.
+ *
+ * The pair state of a batch of B samples with lengths N_s is stored as T2 = sum_s N_s^2 packed
+ * positions (never as a padded B x N_max^2 envelope).  Storage follows the paper's packed
+ * representation (Sec. 3.1, Eq. 2): ragged axes first, static feature axis last, row-major,
+ * samples concatenated; sample offsets o_0 = 0, o_{s+1} - o_s = N_s^2, o_B = T2 (App. A).
+ * The packed row of logical coordinate (s, i, j) is  p = pair_off[s] + i * N_s + j  (Eq. 3).
+ *
+ * Common conventions for every call
+ *   - All value / weight pointers are DEVICE pointers unless the name ends in _h (host).
+ *   - Buffers are contiguous, channel-last; weights are [out, in] row-major (V' = V W^T, Sec. 3.3);
+ *     there are no linear bias vectors anywhere.
+ *   - dtype NT_F32: float storage, float arithmetic.  NT_BF16: bf16 storage of values, weights and
+ *     intermediates, float accumulation, float LayerNorm / softmax statistics.
+ *   - The caller owns every buffer.  No call allocates, frees or synchronises; all work is
+ *     enqueued on `stream` (a cudaStream_t passed as an opaque pointer; NULL = default stream).
+ *   - Pointers must be 16-byte aligned.
+ *   - Host-checkable errors are returned with nothing launched.  Device-detected conditions
+ *     (offset totals that disagree with T1/T2, a bounded wait that expired) are written to
+ *     *status_d (sticky; first error wins) and the kernel exits normally.
+ *   - B = 0 or T2 = 0 is a valid no-op.  Zero-length samples are legal (coincident offsets) and
+ *     contribute nothing.
+ *   - Canonical sizes stay on the host with device mirrors (App. A): the layout carries both.
+ */
+#ifndef NESTED_PAIR_H
+#define NESTED_PAIR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  NT_OK = 0,
+  NT_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer            */
+  NT_ERR_UNSUPPORTED = 2,   /* dtype / width / order not implemented                       */
+  NT_ERR_WORKSPACE = 3,     /* workspace smaller than nt_workspace_bytes()                 */
+  NT_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed                         */
+  NT_ERR_TIMEOUT = 5,       /* device: a bounded wait expired                              */
+  NT_ERR_INCONSISTENT = 6   /* T1 / T2 disagree with the lengths                           */
+} nt_status;
+
+typedef enum { NT_F32 = 0, NT_BF16 = 1 } nt_dtype;
+
+/* logical dimension order of a packed buffer (ragged axes first, then the static feature axis) */
+typedef enum {
+  NT_ORDER_TOKEN_NC = 0,    /* [sum N, C]                                                  */
+  NT_ORDER_PAIR_IJC = 1     /* [sum N^2, C], i major, j minor                              */
+} nt_order;
+
+typedef enum { NT_REDUCE_MEAN = 0, NT_REDUCE_SUM = 1 } nt_reduce;
+
+typedef enum {
+  NT_OP_PAIR_BROADCAST = 0, NT_OP_TRI_MUL_OUT = 1, NT_OP_ROW_ATTN = 2, NT_OP_BLOCK = 3 /* max of the three */
+} nt_op;
+
+typedef void *nt_stream;    /* cudaStream_t */
+
+/* The partitions of one batch (Sec. 3.1 "Structural metadata"). */
+typedef struct {
+  int32_t B;                    /* samples                                                  */
+  int64_t T1, T2;               /* sum N_s and sum N_s^2, computed by the caller            */
+  const int64_t *lengths_h;     /* host   [B]    canonical sizes                            */
+  const int64_t *lengths_d;     /* device [B]                                               */
+  const int64_t *tok_off_d;     /* device [B+1]  exclusive prefix of N_s                    */
+  const int64_t *pair_off_d;    /* device [B+1]  exclusive prefix of N_s^2                  */
+  const int64_t *row_splits_d;  /* device [T1+1] level-2 splits: start of every pair row    */
+  int32_t *status_d;            /* device [1], nullable                                     */
+} nt_layout;
+
+typedef struct {                /* triangle multiplicative update; all device, dtype = dt   */
+  const void *ln_in_gamma, *ln_in_beta;     /* [c_z]                                        */
+  const void *W_ap, *W_ag, *W_bp, *W_bg;    /* [c_h, c_z]                                   */
+  const void *W_g;                          /* [c_z, c_z]                                   */
+  const void *ln_out_gamma, *ln_out_beta;   /* [c_h]                                        */
+  const void *W_o;                          /* [c_z, c_h]                                   */
+} nt_trimul_weights;
+
+typedef struct {                /* row-wise attention; all device, dtype = dt               */
+  const void *ln_gamma, *ln_beta;           /* [c]      both NULL -> no LayerNorm           */
+  const void *W_q, *W_k, *W_v;              /* [H*d, c]                                     */
+  const void *W_b;                          /* [H, c]   NULL -> zero bias                   */
+  const void *W_g;                          /* [H*d, c] NULL -> no gate                     */
+  const void *W_o;                          /* [c, H*d]                                     */
+} nt_attn_weights;
+
+/*
+ * nt_offsets_build -- prefix sums and position decode (Sec. 3.1 offsets o; Fig. 2 two-level row
+ * splits; Eq. 3 coordinate map; the rows/columns gather indices of the program figure).
+ *   tok_off[s]  = sum_{s'<s} N_s',  pair_off[s] = sum_{s'<s} N_s'^2            (each [B+1])
+ *   row_splits[tok_off[s]+i] = pair_off[s] + i N_s,  row_splits[T1] = T2        ([T1+1], nullable)
+ *   for p = pair_off[s] + i N_s + j: pos_sample[p]=s, pos_i[p]=i, pos_j[p]=j    (int32 [T2], nullable as a group)
+ *                                    gather_rows[p]=tok_off[s]+i, gather_cols[p]=tok_off[s]+j (int64 [T2], nullable as a group)
+ * Integer work, bit-exact.  If the scanned totals differ from T1 / T2, NT_ERR_INCONSISTENT is
+ * written to *status_d and only the two offset arrays are produced.
+ */
+nt_status nt_offsets_build(const int64_t *lengths_d, int32_t B, int64_t T1, int64_t T2,
+                           int64_t *tok_off_d, int64_t *pair_off_d, int64_t *row_splits_d,
+                           int32_t *pos_sample_d, int32_t *pos_i_d, int32_t *pos_j_d,
+                           int64_t *gather_rows_d, int64_t *gather_cols_d,
+                           int32_t *status_d, nt_stream stream);
+
+/*
+ * nt_pair_broadcast -- ragged outer broadcast that creates the N_s x N_s axes from packed token
+ * features, fused with LayerNorm (Eq. 1 line 1; Sec. 3.2 "Creating axes through broadcasting";
+ * no activation at construction, App. A.1):
+ *   u = x W_a^T, v = x W_b^T ([T1, c_z]);  z[p,:] = LN_{c_z}(u[tok_off[s]+i] + v[tok_off[s]+j]) * gamma + beta.
+ *   x [T1, c_s] in;  z [T2, c_z] out (exactly T2 * c_z elements).
+ */
+nt_status nt_pair_broadcast(const nt_layout *L, nt_dtype dt, int32_t c_s, int32_t c_z,
+                            const void *x, const void *W_a, const void *W_b,
+                            const void *ln_gamma, const void *ln_beta, float ln_eps,
+                            void *z, void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
+ * nt_tri_mul_out -- outgoing triangle multiplicative update (the Pairformer block's triangle
+ * multiplication, Sec. 4.3), a per-sample grouped contraction over channels:
+ *   zh = LN_in(z); a = sig(zh W_ag^T) * (zh W_ap^T); b = sig(zh W_bg^T) * (zh W_bp^T); g = sig(zh W_g^T)
+ *   t_s[i,j,c] = sum_k a_s[i,k,c] b_s[j,k,c];   z += g * (LN_out(t) W_o^T)      (in place)
+ *   z [T2, c_z] in/out.  No weight pointer may be NULL.
+ */
+nt_status nt_tri_mul_out(const nt_layout *L, nt_dtype dt, int32_t c_z, int32_t c_h,
+                         const nt_trimul_weights *W, float ln_eps, void *z,
+                         void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
+ * nt_row_attn_pairbias -- row-wise pair-biased softmax attention over ragged N_s (Sec. 3.3
+ * "Attention through packed blocks": segments from the offsets, output adopts the query
+ * structure; Sec. 4.3 triangle attention, starting node).
+ *   order = NT_ORDER_PAIR_IJC: zx = z [T2, c]; attention rows are the pair rows (s, i); for each
+ *     row and head h: S[j,k] = <q_ij, k_ik>/sqrt(d) + bias[j,k,h] with bias = LN(z) W_b^T shared by
+ *     all rows of the sample; P = softmax_k S; o_ij = sum_k P[j,k] v_ik; z += (g * o) W_o^T.
+ *   order = NT_ORDER_TOKEN_NC: zx = x [T1, c]; one attention row per sample (variable-length
+ *     self-attention over the token segments); W_b must be NULL.
+ *   zx in/out (in place).  H * d need not equal c.
+ */
+nt_status nt_row_attn_pairbias(const nt_layout *L, nt_order order, nt_dtype dt,
+                               int32_t c, int32_t H, int32_t d,
+                               const nt_attn_weights *W, float ln_eps, void *zx,
+                               void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
+ * nt_segment_reduce -- segmented sum or mean of contiguous row groups (Eq. 4 pair reduction; the
+ * mean over j of Eq. 1 line 3 divides by the group's count; App. A batch-axis convention).
+ *   out[g,:] = (1/len_g or 1) * sum_{r = splits[g]}^{splits[g+1]-1} v[r,:],  empty group -> 0.
+ *   splits [G+1] device, nondecreasing, splits[0] = 0, splits[G] = rows.  v [rows, C]; out [G, C].
+ *   With splits = row_splits this is the mean over j back to the token axis; with
+ *   splits = tok_off it pools a token buffer per sample.  Accumulation is in float.
+ */
+nt_status nt_segment_reduce(nt_dtype dt, nt_reduce op, int32_t C, int64_t G, int64_t rows,
+                            const int64_t *splits_d, const void *v, void *out,
+                            int32_t *status_d, nt_stream stream);
+
+/* ------------------------------- auxiliaries (not among the five) ------------------------------- */
+
+/* x[T1, c_s] += m[T1, c_z] W_r^T  -- the projection g of Eq. 1 line 3 applied to the reduced
+ * features and added to the tokens.  W_r is [c_s, c_z]. */
+nt_status nt_token_update(nt_dtype dt, int32_t c_s, int32_t c_z, int64_t T1,
+                          const void *m, const void *W_r, void *x, nt_stream stream);
+
+/* Bytes of workspace a call needs for this batch.  dims = {c_s, c_z, c_h, H, d}; entries an op
+ * does not use are ignored.  Host only.  Returns 0 for an empty batch. */
+size_t nt_workspace_bytes(nt_op op, nt_dtype dt, nt_order order, const int64_t *lengths_h, int32_t B,
+                          const int32_t *dims);
+
+const char *nt_status_string(nt_status st);
+
+/* Number of kernels the library has launched in this process since load (all calls). */
+int64_t nt_launch_count(void);
+
+/* Per-kernel timing for benchmarks.  Between nt_profile_begin() and nt_profile_end() every kernel the
+ * library launches is bracketed by a pair of CUDA events on its stream.  nt_profile_end() waits for
+ * those events and aggregates by kernel name: names are written to `names` separated by '\n', with
+ * total milliseconds and launch counts in the parallel arrays; it returns the number of entries.
+ * Host-side only; off by default; not thread-safe against concurrent library calls. */
+int32_t nt_profile_begin(void);
+int32_t nt_profile_end(char *names, size_t names_bytes, float *total_ms, int64_t *launches, int32_t max_entries);
+
+/* Testing aid: non-zero forces the shape-generic CUDA-core kernels even where a tensor-core
+ * kernel exists for the shape.  Returns the previous value.  Both settings run on the GPU. */
+int32_t nt_force_generic(int32_t on);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NESTED_PAIR_H */

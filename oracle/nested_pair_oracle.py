@@ -202,14 +202,15 @@ def row_attn_pairbias(zx, lengths, W, H, d, eps=LN_EPS, order="pair", dtype=np.f
         q = (zh @ Wd["W_q"].T).reshape(R, n, H, d)
         k = (zh @ Wd["W_k"].T).reshape(R, n, H, d)
         v = (zh @ Wd["W_v"].T).reshape(R, n, H, d)
-        S = np.einsum("ijhe,ikhe->ihjk", q, k) * scale
+        # scores per (row, head) as a batched matrix product Q K^T (BLAS-backed, still the definition)
+        S = np.matmul(q.transpose(0, 2, 1, 3), k.transpose(0, 2, 3, 1)) * scale      # [R, H, j, k]
         if W_b is not None:
             bias = zh @ W_b.T                    # [n, n, H] (pair order only: R == n)
             S = S + bias.transpose(2, 0, 1)[None, :, :, :]
         S = S - S.max(axis=-1, keepdims=True)
         A = np.exp(S)
         A = A / A.sum(axis=-1, keepdims=True)
-        ov = np.einsum("ihjk,ikhe->ijhe", A, v).reshape(R, n, H * d)
+        ov = np.matmul(A, v.transpose(0, 2, 1, 3)).transpose(0, 2, 1, 3).reshape(R, n, H * d)
         if W_g is not None:
             ov = sigmoid(zh @ W_g.T) * ov
         out.append((zs + ov @ Wd["W_o"].T).reshape(rows, zx.shape[1]))
@@ -240,6 +241,54 @@ def token_update(x, m, W_r, dtype=np.float64):
     """x' = x + m W_r^T  (the projection g of Eq. 1 line 3, bias-free)."""
     x, m, W_r = _as(dtype, x, m, W_r)
     return x + m @ W_r.T
+
+
+# --------------------------------------------------------------------------------------------
+# the same definitions evaluated at selected positions of one sample (for samples too large to
+# run whole on the CPU); pinned to the full functions above in tests/test_oracle_pins.py
+# --------------------------------------------------------------------------------------------
+def tri_mul_out_at(zs, W, positions, eps=LN_EPS, dtype=np.float64):
+    """Outgoing triangle update of one sample at the listed (i, j).  ``zs[i]`` is pair row i of the
+    sample's state, an [n, c_z] array (``zs`` may be the [n, n, c_z] array or a mapping that holds
+    only the rows needed): only rows i and j enter t[i,j,:] = sum_k a[i,k,:] b[j,k,:]."""
+    Wd = {k: np.asarray(v, dtype=dtype) for k, v in W.items()}
+    out = []
+    for (i, j) in positions:
+        ri, rj = np.asarray(zs[i], dtype=dtype), np.asarray(zs[j], dtype=dtype)
+        zi = layer_norm(ri, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)        # [n, c_z]
+        zj = layer_norm(rj, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)
+        a_i = sigmoid(zi @ Wd["W_ag"].T) * (zi @ Wd["W_ap"].T)               # a[i, k, :]
+        b_j = sigmoid(zj @ Wd["W_bg"].T) * (zj @ Wd["W_bp"].T)               # b[j, k, :]
+        t = (a_i * b_j).sum(axis=0)
+        g = sigmoid(zi[j] @ Wd["W_g"].T)
+        out.append(ri[j] + g * (layer_norm(t, Wd["ln_out_gamma"], Wd["ln_out_beta"], eps) @ Wd["W_o"].T))
+    return np.stack(out)
+
+
+def row_attn_pairbias_at(zs, W, H, d, positions, eps=LN_EPS, dtype=np.float64):
+    """Row-wise pair-biased attention of one sample at the listed (i, j) (``zs`` as in
+    tri_mul_out_at): query j of row i attends over the keys of row i with bias[j, :, h] taken
+    from pair row j."""
+    Wd = {k: (None if v is None else np.asarray(v, dtype=dtype)) for k, v in W.items()}
+    out = []
+    for (i, j) in positions:
+        ri, rj = np.asarray(zs[i], dtype=dtype), np.asarray(zs[j], dtype=dtype)
+        n = ri.shape[0]
+        zi = layer_norm(ri, Wd["ln_gamma"], Wd["ln_beta"], eps)
+        zj = layer_norm(rj, Wd["ln_gamma"], Wd["ln_beta"], eps)
+        q = (zi[j] @ Wd["W_q"].T).reshape(H, d)
+        k = (zi @ Wd["W_k"].T).reshape(n, H, d)
+        v = (zi @ Wd["W_v"].T).reshape(n, H, d)
+        bias = zj @ Wd["W_b"].T                                               # [n(k), H]
+        o = np.zeros((H, d), dtype=dtype)
+        for h in range(H):
+            sc = k[:, h, :] @ q[h] / np.sqrt(float(d)) + bias[:, h]
+            sc = sc - sc.max()
+            e = np.exp(sc)
+            o[h] = (e / e.sum()) @ v[:, h, :]
+        gate = sigmoid(zi[j] @ Wd["W_g"].T)
+        out.append(ri[j] + (gate * o.reshape(H * d)) @ Wd["W_o"].T)
+    return np.stack(out)
 
 
 # --------------------------------------------------------------------------------------------

@@ -1,0 +1,221 @@
+"""ctypes binding of libnested_pair.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (include/nested_pair.h) and does
+nothing but convert torch tensors to device pointers and check the returned status.  torch is
+used for device memory and streams; all arithmetic runs in the library's CUDA kernels.  If the
+shared library is missing the import fails: there is no CPU or eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+NT_OK = 0
+NT_F32, NT_BF16 = 0, 1
+NT_ORDER_TOKEN_NC, NT_ORDER_PAIR_IJC = 0, 1
+NT_REDUCE_MEAN, NT_REDUCE_SUM = 0, 1
+NT_OP_PAIR_BROADCAST, NT_OP_TRI_MUL_OUT, NT_OP_ROW_ATTN, NT_OP_BLOCK = 0, 1, 2, 3
+
+STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3: "NT_ERR_WORKSPACE",
+                4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
+
+EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_tri_mul_out", "nt_row_attn_pairbias",
+           "nt_segment_reduce", "nt_token_update", "nt_workspace_bytes", "nt_status_string",
+           "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
+
+
+class NtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class nt_layout(C.Structure):
+    _fields_ = [("B", C.c_int32), ("T1", C.c_int64), ("T2", C.c_int64),
+                ("lengths_h", C.c_void_p), ("lengths_d", C.c_void_p), ("tok_off_d", C.c_void_p),
+                ("pair_off_d", C.c_void_p), ("row_splits_d", C.c_void_p), ("status_d", C.c_void_p)]
+
+
+class nt_trimul_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln_in_gamma", "ln_in_beta", "W_ap", "W_ag", "W_bp", "W_bg", "W_g",
+                                          "ln_out_gamma", "ln_out_beta", "W_o")]
+
+
+class nt_attn_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln_gamma", "ln_beta", "W_q", "W_k", "W_v", "W_b", "W_g", "W_o")]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with __graft_entry__.build() "
+                          "(python -m paper_2609_30379_b200.build); there is no fallback path")
+    lib = C.CDLL(path)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    lib.nt_offsets_build.argtypes = [vp, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.nt_pair_broadcast.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp, sz, vp]
+    lib.nt_tri_mul_out.argtypes = [C.POINTER(nt_layout), i32, i32, i32, C.POINTER(nt_trimul_weights), f32, vp, vp, sz, vp]
+    lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
+                                         f32, vp, vp, sz, vp]
+    lib.nt_segment_reduce.argtypes = [i32, i32, i32, i64, i64, vp, vp, vp, vp, vp]
+    lib.nt_token_update.argtypes = [i32, i32, i32, i64, vp, vp, vp, vp]
+    lib.nt_workspace_bytes.argtypes = [i32, i32, i32, vp, i32, vp]
+    lib.nt_workspace_bytes.restype = sz
+    lib.nt_status_string.argtypes = [i32]
+    lib.nt_status_string.restype = C.c_char_p
+    lib.nt_launch_count.argtypes = []
+    lib.nt_launch_count.restype = i64
+    lib.nt_force_generic.argtypes = [i32]
+    lib.nt_force_generic.restype = i32
+    lib.nt_profile_begin.argtypes = []
+    lib.nt_profile_begin.restype = i32
+    lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
+    lib.nt_profile_end.restype = i32
+    for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_tri_mul_out", "nt_row_attn_pairbias",
+                 "nt_segment_reduce", "nt_token_update"):
+        getattr(lib, name).restype = i32
+    return lib
+
+
+lib = _load()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("device tensor expected")
+    if not t.is_contiguous():
+        raise ValueError("contiguous tensor expected")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(st: int, where: str):
+    if st != NT_OK:
+        raise NtError(st, where)
+
+
+def dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return NT_F32
+    if t == torch.bfloat16:
+        return NT_BF16
+    raise ValueError(f"unsupported dtype {t}")
+
+
+class Layout:
+    """Host lengths plus the device mirrors of one batch; owns the buffers nt_layout points at."""
+
+    def __init__(self, lengths: Sequence[int], device="cuda", stream=None, with_maps: bool = False):
+        self.lengths_h = np.ascontiguousarray(np.asarray(lengths, dtype=np.int64))
+        self.B = int(self.lengths_h.shape[0])
+        self.T1 = int(self.lengths_h.sum())
+        self.T2 = int((self.lengths_h * self.lengths_h).sum())
+        dev = torch.device(device)
+        self.lengths_d = torch.from_numpy(self.lengths_h).to(dev) if self.B else torch.zeros(0, dtype=torch.int64, device=dev)
+        self.tok_off = torch.empty(self.B + 1, dtype=torch.int64, device=dev)
+        self.pair_off = torch.empty(self.B + 1, dtype=torch.int64, device=dev)
+        self.row_splits = torch.empty(self.T1 + 1, dtype=torch.int64, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.pos_sample = self.pos_i = self.pos_j = self.gather_rows = self.gather_cols = None
+        if with_maps:
+            self.pos_sample = torch.empty(self.T2, dtype=torch.int32, device=dev)
+            self.pos_i = torch.empty(self.T2, dtype=torch.int32, device=dev)
+            self.pos_j = torch.empty(self.T2, dtype=torch.int32, device=dev)
+            self.gather_rows = torch.empty(self.T2, dtype=torch.int64, device=dev)
+            self.gather_cols = torch.empty(self.T2, dtype=torch.int64, device=dev)
+        nt_offsets_build(self.lengths_d, self.B, self.T1, self.T2, self.tok_off, self.pair_off, self.row_splits,
+                         self.pos_sample, self.pos_i, self.pos_j, self.gather_rows, self.gather_cols,
+                         self.status, stream)
+        self.c = nt_layout(self.B, self.T1, self.T2, self.lengths_h.ctypes.data if self.B else None,
+                           _ptr(self.lengths_d) if self.B else None, _ptr(self.tok_off), _ptr(self.pair_off),
+                           _ptr(self.row_splits), _ptr(self.status))
+
+    def device_status(self) -> int:
+        return int(self.status.item())
+
+
+def nt_offsets_build(lengths_d, B, T1, T2, tok_off_d, pair_off_d, row_splits_d=None, pos_sample_d=None,
+                     pos_i_d=None, pos_j_d=None, gather_rows_d=None, gather_cols_d=None, status_d=None, stream=None):
+    st = lib.nt_offsets_build(_ptr(lengths_d) if B else None, B, T1, T2, _ptr(tok_off_d), _ptr(pair_off_d),
+                              _ptr(row_splits_d), _ptr(pos_sample_d), _ptr(pos_i_d), _ptr(pos_j_d),
+                              _ptr(gather_rows_d), _ptr(gather_cols_d), _ptr(status_d), _stream(stream))
+    _check(st, "nt_offsets_build")
+
+
+def nt_workspace_bytes(op: int, dt: int, order: int, lengths_h: np.ndarray, dims: Sequence[int]) -> int:
+    lengths_h = np.ascontiguousarray(lengths_h, dtype=np.int64)
+    d = (C.c_int32 * 5)(*[int(v) for v in dims])
+    return int(lib.nt_workspace_bytes(op, dt, order, lengths_h.ctypes.data, int(lengths_h.shape[0]), C.addressof(d)))
+
+
+def nt_pair_broadcast(L: Layout, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, stream=None):
+    c_s, c_z = int(W_a.shape[1]), int(W_a.shape[0])
+    st = lib.nt_pair_broadcast(C.byref(L.c), dtype_code(x.dtype), c_s, c_z, _ptr(x), _ptr(W_a), _ptr(W_b),
+                               _ptr(ln_gamma), _ptr(ln_beta), float(ln_eps), _ptr(z), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_pair_broadcast")
+
+
+def nt_tri_mul_out(L: Layout, W: dict, ln_eps, z, workspace, stream=None):
+    c_h, c_z = int(W["W_ap"].shape[0]), int(W["W_ap"].shape[1])
+    w = nt_trimul_weights(*[_ptr(W[n]) for n, _ in nt_trimul_weights._fields_])
+    st = lib.nt_tri_mul_out(C.byref(L.c), dtype_code(z.dtype), c_z, c_h, C.byref(w), float(ln_eps), _ptr(z),
+                            _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_tri_mul_out")
+
+
+def nt_row_attn_pairbias(L: Layout, order: int, W: dict, H: int, d: int, ln_eps, zx, workspace, stream=None):
+    c = int(W["W_q"].shape[1])
+    w = nt_attn_weights(*[_ptr(W.get(n)) for n, _ in nt_attn_weights._fields_])
+    st = lib.nt_row_attn_pairbias(C.byref(L.c), order, dtype_code(zx.dtype), c, H, d, C.byref(w), float(ln_eps),
+                                  _ptr(zx), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream))
+    _check(st, "nt_row_attn_pairbias")
+
+
+def nt_segment_reduce(op: int, splits_d, v, out, status_d=None, stream=None):
+    G, Cc, rows = int(splits_d.shape[0]) - 1, int(v.shape[1]), int(v.shape[0])
+    st = lib.nt_segment_reduce(dtype_code(v.dtype), op, Cc, G, rows, _ptr(splits_d), _ptr(v) if rows else None,
+                               _ptr(out), _ptr(status_d), _stream(stream))
+    _check(st, "nt_segment_reduce")
+
+
+def nt_token_update(m, W_r, x, stream=None):
+    st = lib.nt_token_update(dtype_code(x.dtype), int(W_r.shape[0]), int(W_r.shape[1]), int(x.shape[0]),
+                             _ptr(m), _ptr(W_r), _ptr(x), _stream(stream))
+    _check(st, "nt_token_update")
+
+
+def nt_launch_count() -> int:
+    return int(lib.nt_launch_count())
+
+
+def nt_force_generic(on: bool) -> bool:
+    return bool(lib.nt_force_generic(1 if on else 0))
+
+
+def nt_profile_begin():
+    lib.nt_profile_begin()
+
+
+def nt_profile_end(max_entries: int = 256) -> dict:
+    """{kernel name: (total milliseconds, launches)} since nt_profile_begin()."""
+    names = C.create_string_buffer(64 * max_entries)
+    ms = (C.c_float * max_entries)()
+    cnt = (C.c_int64 * max_entries)()
+    n = lib.nt_profile_end(C.addressof(names), len(names), C.addressof(ms), C.addressof(cnt), max_entries)
+    keys = names.value.decode().split("\n")[:n]
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(keys)}

@@ -1,0 +1,433 @@
+// C-ABI entry points of libnested_pair: argument validation, workspace carving and the launch
+// sequence of every call.  Nothing here allocates or synchronises.
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "fast.cuh"
+#include "generic.cuh"
+
+namespace ntp {
+
+std::atomic<long long> g_launches{0};
+int g_force_generic = 0;
+
+// ---- per-kernel event timing (off unless nt_profile_begin was called) ----------------------
+struct ProfRecord { const char* name; cudaEvent_t e0, e1; };
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<ProfRecord> g_prof;
+
+LaunchScope::LaunchScope(const char* name, cudaStream_t s) : st(s), slot(-1) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (!g_prof_on) return;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  ProfRecord r{name, nullptr, nullptr};
+  if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
+  cudaEventRecord(r.e0, st);
+  slot = (int)g_prof.size();
+  g_prof.push_back(r);
+}
+
+LaunchScope::~LaunchScope() {
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  cudaEventRecord(g_prof[slot].e1, st);
+}
+
+void fill_meta(BatchMeta& m, const int64_t* len, int s0, int s1, long long tok0, long long pair0, long long cm0) {
+  m.B = s1 - s0;
+  m.tok_off[0] = tok0;
+  m.pair_off[0] = pair0;
+  m.cm_off[0] = cm0;
+  for (int s = s0; s < s1; ++s) {
+    const int l = s - s0;
+    const long long n = len[s];
+    m.N[l] = (int)n;
+    m.tok_off[l + 1] = m.tok_off[l] + n;
+    m.pair_off[l + 1] = m.pair_off[l] + n * n;
+    m.cm_off[l + 1] = m.cm_off[l] + n * round_up8((int)n);
+  }
+  for (int l = m.B; l < MAXB; ++l) {
+    m.N[l] = 0;
+    m.tok_off[l + 1] = m.tok_off[m.B];
+    m.pair_off[l + 1] = m.pair_off[m.B];
+    m.cm_off[l + 1] = m.cm_off[m.B];
+  }
+}
+
+bool GroupIter::next(BatchMeta& m) {
+  if (s0 >= B) return false;
+  const int s1 = s0 + MAXB < B ? s0 + MAXB : B;
+  fill_meta(m, len, s0, s1, tok, pair, cm);
+  tok = m.tok_off[m.B];
+  pair = m.pair_off[m.B];
+  cm = m.cm_off[m.B];
+  s0 = s1;
+  return true;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+struct Totals { long long T1 = 0, T2 = 0, cm = 0; int nmax = 0; };
+
+static nt_status totals_of(const int64_t* len, int B, Totals& t) {
+  for (int s = 0; s < B; ++s) {
+    const long long n = len[s];
+    if (n < 0) return NT_ERR_INVALID_ARG;
+    if (n > 0x3FFFFFFF) return NT_ERR_UNSUPPORTED;
+    t.T1 += n;
+    t.T2 += n * n;
+    t.cm += n * round_up8((int)n);
+    if (n > t.nmax) t.nmax = (int)n;
+  }
+  return NT_OK;
+}
+
+static nt_status check_layout(const nt_layout* L, Totals& t) {
+  if (!L || L->B < 0) return NT_ERR_INVALID_ARG;
+  if (L->B > 0 && !L->lengths_h) return NT_ERR_INVALID_ARG;
+  nt_status st = totals_of(L->lengths_h, L->B, t);
+  if (st != NT_OK) return st;
+  if (t.T1 != L->T1 || t.T2 != L->T2) return NT_ERR_INCONSISTENT;
+  return NT_OK;
+}
+
+static size_t esize(nt_dtype dt) { return dt == NT_F32 ? 4 : 2; }
+
+struct Carver {   // hands out 256-byte aligned slices of the caller's workspace
+  char* base;
+  size_t off = 0;
+  explicit Carver(void* p) : base((char*)p) {}
+  void* take(size_t bytes) {
+    void* r = base ? base + off : nullptr;
+    off += align_up(bytes, 256);
+    return r;
+  }
+};
+
+struct TriWs { void *a, *b, *t, *g; size_t bytes; };
+static TriWs carve_trimul(void* ws, nt_dtype dt, const Totals& t, int c_z, int c_h) {
+  Carver c(ws);
+  TriWs w;
+  const size_t e = esize(dt);
+  w.a = c.take((size_t)c_h * t.cm * e);
+  w.b = c.take((size_t)c_h * t.cm * e);
+  w.t = c.take((size_t)c_h * t.cm * e);
+  w.g = c.take((size_t)t.T2 * c_z * e);
+  w.bytes = c.off;
+  return w;
+}
+
+struct AttnWs { void *q, *k, *v, *o, *g, *bias; size_t bytes; };
+static AttnWs carve_attn(void* ws, nt_dtype dt, const Totals& t, nt_order order, int H, int d) {
+  Carver c(ws);
+  AttnWs w;
+  const size_t e = esize(dt);
+  const size_t rows = order == NT_ORDER_PAIR_IJC ? t.T2 : t.T1;
+  const size_t Hd = (size_t)H * d;
+  w.q = c.take(rows * Hd * e);
+  w.k = c.take(rows * Hd * e);
+  w.v = c.take(rows * Hd * e);
+  w.o = c.take(rows * Hd * e);
+  w.g = c.take(rows * Hd * e);
+  w.bias = c.take(order == NT_ORDER_PAIR_IJC ? (size_t)H * t.cm * e : 0);
+  w.bytes = c.off;
+  return w;
+}
+
+static size_t broadcast_ws_bytes(const Totals& t, int c_z) {
+  return 2 * align_up((size_t)t.T1 * c_z * sizeof(float), 256);
+}
+
+// ------------------------------------------------------------------------------------------
+template <typename T>
+static nt_status pair_broadcast_impl(const nt_layout* L, const Totals& tot, int c_s, int c_z, const void* x,
+                                     const void* W_a, const void* W_b, const void* g, const void* b, float eps,
+                                     void* z, void* ws, cudaStream_t st, bool fast) {
+  Carver c(ws);
+  float* u = (float*)c.take((size_t)tot.T1 * c_z * sizeof(float));
+  float* v = (float*)c.take((size_t)tot.T1 * c_z * sizeof(float));
+  BatchMeta dummy;
+  fill_meta(dummy, nullptr, 0, 0, 0, 0, 0);
+  ProjArgs pa{};
+  pa.A = x; pa.a_mode = A_ROWMAJOR; pa.row0 = 0; pa.rows = tot.T1; pa.K = c_s;
+  pa.W1 = W_a; pa.Nout = c_z; pa.act = ACT_NONE; pa.out = u; pa.out_mode = O_STORE; pa.out_f32 = 1;
+  nt_status r = launch_proj<T>(pa, dummy, st, "tok_proj_u");
+  if (r != NT_OK) return r;
+  pa.W1 = W_b; pa.out = v;
+  r = launch_proj<T>(pa, dummy, st, "tok_proj_v");
+  if (r != NT_OK) return r;
+  GroupIter it(L->lengths_h, L->B);
+  BatchMeta m;
+  while (it.next(m)) {
+    if (fast) r = fast_broadcast_ln(u, v, g, b, eps, c_z, z, m, st);
+    else r = launch_broadcast_ln<T>(u, v, (const T*)g, (const T*)b, eps, c_z, (T*)z, m, st);
+    if (r != NT_OK) return r;
+  }
+  return NT_OK;
+}
+
+template <typename T>
+static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z, int c_h, const nt_trimul_weights* W,
+                                 float eps, void* z, void* ws, nt_dtype dt, cudaStream_t st) {
+  TriWs w = carve_trimul(ws, dt, tot, c_z, c_h);
+  GroupIter it(L->lengths_h, L->B);
+  BatchMeta m;
+  while (it.next(m)) {
+    const long long row0 = m.pair_off[0], rows = m.pair_off[m.B] - row0;
+    if (rows == 0) continue;
+    ProjArgs pa{};
+    pa.A = z; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c_z;
+    pa.ln_g = W->ln_in_gamma; pa.ln_b = W->ln_in_beta; pa.eps = eps;
+    pa.W1 = W->W_ag; pa.W2 = W->W_ap; pa.Nout = c_h; pa.out = w.a; pa.out_mode = O_CHANNEL_MAJOR;
+    nt_status r = launch_proj<T>(pa, m, st, "generic_tri_in_a");
+    if (r != NT_OK) return r;
+    pa.W1 = W->W_bg; pa.W2 = W->W_bp; pa.out = w.b;
+    r = launch_proj<T>(pa, m, st, "generic_tri_in_b");
+    if (r != NT_OK) return r;
+    pa.W1 = W->W_g; pa.W2 = nullptr; pa.act = ACT_SIGMOID; pa.Nout = c_z; pa.out = w.g; pa.out_mode = O_STORE;
+    r = launch_proj<T>(pa, m, st, "generic_tri_in_g");
+    if (r != NT_OK) return r;
+    r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st);
+    if (r != NT_OK) return r;
+    ProjArgs po{};
+    po.A = w.t; po.a_mode = A_CHANNEL_MAJOR; po.row0 = row0; po.rows = rows; po.K = c_h;
+    po.ln_g = W->ln_out_gamma; po.ln_b = W->ln_out_beta; po.eps = eps;
+    po.W1 = W->W_o; po.Nout = c_z; po.act = ACT_NONE; po.out = z; po.out_mode = O_ACCUM; po.gateO = w.g;
+    r = launch_proj<T>(po, m, st, "generic_tri_out");
+    if (r != NT_OK) return r;
+  }
+  return NT_OK;
+}
+
+template <typename T>
+static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order order, int c, int H, int d,
+                              const nt_attn_weights* W, float eps, void* zx, void* ws, nt_dtype dt,
+                              cudaStream_t st) {
+  AttnWs w = carve_attn(ws, dt, tot, order, H, d);
+  const int Hd = H * d;
+  const bool pair = order == NT_ORDER_PAIR_IJC;
+  GroupIter it(L->lengths_h, L->B);
+  BatchMeta m;
+  while (it.next(m)) {
+    const long long row0 = pair ? m.pair_off[0] : m.tok_off[0];
+    const long long rows = (pair ? m.pair_off[m.B] : m.tok_off[m.B]) - row0;
+    if (rows == 0) continue;
+    ProjArgs pa{};
+    pa.A = zx; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c;
+    pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = eps;
+    pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
+    nt_status r;
+    pa.W1 = W->W_q; pa.out = w.q;
+    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_q")) != NT_OK) return r;
+    pa.W1 = W->W_k; pa.out = w.k;
+    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_k")) != NT_OK) return r;
+    pa.W1 = W->W_v; pa.out = w.v;
+    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_v")) != NT_OK) return r;
+    if (W->W_g) {
+      pa.W1 = W->W_g; pa.out = w.g; pa.act = ACT_SIGMOID;
+      if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_g")) != NT_OK) return r;
+      pa.act = ACT_NONE;
+    }
+    if (W->W_b) {
+      pa.W1 = W->W_b; pa.Nout = H; pa.out = w.bias; pa.out_mode = O_CHANNEL_MAJOR;
+      if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
+    }
+    r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
+                            (T*)w.o, H, d, pair ? 1 : 0, m, st);
+    if (r != NT_OK) return r;
+    ProjArgs po{};
+    po.A = w.o; po.a_mode = A_ROWMAJOR; po.row0 = row0; po.rows = rows; po.K = Hd;
+    po.gateA = W->W_g ? w.g : nullptr;
+    po.W1 = W->W_o; po.Nout = c; po.act = ACT_NONE; po.out = zx; po.out_mode = O_ACCUM;
+    if ((r = launch_proj<T>(po, m, st, "generic_attn_out")) != NT_OK) return r;
+  }
+  return NT_OK;
+}
+
+}  // namespace ntp
+
+using namespace ntp;
+
+extern "C" {
+
+nt_status nt_pair_broadcast(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_t c_z, const void* x,
+                            const void* W_a, const void* W_b, const void* ln_gamma, const void* ln_beta,
+                            float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c_s <= 0 || c_z <= 0) return NT_ERR_INVALID_ARG;
+  if (tot.T2 == 0) return NT_OK;
+  if (!x || !W_a || !W_b || !ln_gamma || !ln_beta || !z || !workspace) return NT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(z) || !aligned16(workspace) || !aligned16(W_a) || !aligned16(W_b))
+    return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < broadcast_ws_bytes(tot, c_z)) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32)
+    return pair_broadcast_impl<float>(L, tot, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, st, false);
+  const bool fast = !g_force_generic && fast_broadcast_supported(c_z);
+  return pair_broadcast_impl<__nv_bfloat16>(L, tot, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, st,
+                                            fast);
+}
+
+nt_status nt_tri_mul_out(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,
+                         float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c_z <= 0 || c_h <= 0 || !W) return NT_ERR_INVALID_ARG;
+  if (!W->ln_in_gamma || !W->ln_in_beta || !W->W_ap || !W->W_ag || !W->W_bp || !W->W_bg || !W->W_g ||
+      !W->ln_out_gamma || !W->ln_out_beta || !W->W_o)
+    return NT_ERR_INVALID_ARG;
+  if (tot.T2 == 0) return NT_OK;
+  if (!z || !workspace || !aligned16(z) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < carve_trimul(nullptr, dt, tot, c_z, c_h).bytes) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32) return tri_mul_generic<float>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st);
+  return tri_mul_generic<__nv_bfloat16>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st);
+}
+
+nt_status nt_row_attn_pairbias(const nt_layout* L, nt_order order, nt_dtype dt, int32_t c, int32_t H, int32_t d,
+                               const nt_attn_weights* W, float ln_eps, void* zx, void* workspace,
+                               size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (order != NT_ORDER_PAIR_IJC && order != NT_ORDER_TOKEN_NC) return NT_ERR_UNSUPPORTED;
+  if (c <= 0 || H <= 0 || d <= 0 || !W) return NT_ERR_INVALID_ARG;
+  if (!W->W_q || !W->W_k || !W->W_v || !W->W_o) return NT_ERR_INVALID_ARG;
+  if ((W->ln_gamma == nullptr) != (W->ln_beta == nullptr)) return NT_ERR_INVALID_ARG;
+  if (order == NT_ORDER_TOKEN_NC && W->W_b) return NT_ERR_INVALID_ARG;
+  if (d > 128) return NT_ERR_UNSUPPORTED;
+  const long long rows = order == NT_ORDER_PAIR_IJC ? tot.T2 : tot.T1;
+  if (rows == 0) return NT_OK;
+  if (!zx || !workspace || !aligned16(zx) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < carve_attn(nullptr, dt, tot, order, H, d).bytes) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32) return attn_generic<float>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st);
+  return attn_generic<__nv_bfloat16>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st);
+}
+
+nt_status nt_segment_reduce(nt_dtype dt, nt_reduce op, int32_t C, int64_t G, int64_t rows, const int64_t* splits_d,
+                            const void* v, void* out, int32_t* status_d, nt_stream stream) {
+  (void)status_d;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (op != NT_REDUCE_MEAN && op != NT_REDUCE_SUM) return NT_ERR_UNSUPPORTED;
+  if (C <= 0 || G < 0 || rows < 0) return NT_ERR_INVALID_ARG;
+  if (G == 0) return NT_OK;
+  if (!splits_d || !out || (rows > 0 && !v)) return NT_ERR_INVALID_ARG;
+  if (!aligned16(v) || !aligned16(out)) return NT_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int mean = op == NT_REDUCE_MEAN;
+  if (dt == NT_F32) return launch_segment_reduce<float>((const float*)v, (float*)out, splits_d, G, C, mean, st);
+  if (!g_force_generic && fast_segment_reduce_supported(C))
+    return fast_segment_reduce(v, out, splits_d, G, C, mean, st);
+  return launch_segment_reduce<__nv_bfloat16>((const __nv_bfloat16*)v, (__nv_bfloat16*)out, splits_d, G, C, mean, st);
+}
+
+nt_status nt_token_update(nt_dtype dt, int32_t c_s, int32_t c_z, int64_t T1, const void* mvals, const void* W_r,
+                          void* x, nt_stream stream) {
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c_s <= 0 || c_z <= 0 || T1 < 0) return NT_ERR_INVALID_ARG;
+  if (T1 == 0) return NT_OK;
+  if (!mvals || !W_r || !x) return NT_ERR_INVALID_ARG;
+  BatchMeta dummy;
+  fill_meta(dummy, nullptr, 0, 0, 0, 0, 0);
+  ProjArgs pa{};
+  pa.A = mvals; pa.a_mode = A_ROWMAJOR; pa.row0 = 0; pa.rows = T1; pa.K = c_z;
+  pa.W1 = W_r; pa.Nout = c_s; pa.act = ACT_NONE; pa.out = x; pa.out_mode = O_ACCUM;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32) return launch_proj<float>(pa, dummy, st, "token_update");
+  return launch_proj<__nv_bfloat16>(pa, dummy, st, "token_update");
+}
+
+size_t nt_workspace_bytes(nt_op op, nt_dtype dt, nt_order order, const int64_t* lengths_h, int32_t B,
+                          const int32_t* dims) {
+  if (B <= 0 || !lengths_h || !dims) return 0;
+  Totals tot;
+  if (totals_of(lengths_h, B, tot) != NT_OK) return 0;
+  const int c_z = dims[1], c_h = dims[2], H = dims[3], d = dims[4];
+  size_t bb = broadcast_ws_bytes(tot, c_z);
+  size_t tb = carve_trimul(nullptr, dt, tot, c_z, c_h).bytes;
+  size_t ab = carve_attn(nullptr, dt, tot, order, H, d).bytes;
+  switch (op) {
+    case NT_OP_PAIR_BROADCAST: return bb;
+    case NT_OP_TRI_MUL_OUT: return tb;
+    case NT_OP_ROW_ATTN: return ab;
+    case NT_OP_BLOCK: { size_t mx = bb > tb ? bb : tb; return mx > ab ? mx : ab; }
+  }
+  return 0;
+}
+
+const char* nt_status_string(nt_status st) {
+  switch (st) {
+    case NT_OK: return "ok";
+    case NT_ERR_INVALID_ARG: return "invalid argument";
+    case NT_ERR_UNSUPPORTED: return "unsupported dtype, width or order";
+    case NT_ERR_WORKSPACE: return "workspace too small";
+    case NT_ERR_CUDA: return "CUDA call failed";
+    case NT_ERR_TIMEOUT: return "device wait timed out";
+    case NT_ERR_INCONSISTENT: return "totals disagree with lengths";
+  }
+  return "unknown status";
+}
+
+int64_t nt_launch_count(void) { return g_launches.load(); }
+
+int32_t nt_profile_begin(void) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  for (auto& r : g_prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  g_prof.clear();
+  g_prof_on = true;
+  return 0;
+}
+
+int32_t nt_profile_end(char* names, size_t names_bytes, float* total_ms, int64_t* launches, int32_t max_entries) {
+  std::lock_guard<std::mutex> lk(g_prof_mu);
+  g_prof_on = false;
+  std::vector<std::string> nm;
+  std::vector<float> ms;
+  std::vector<long long> cnt;
+  for (auto& r : g_prof) {
+    float t = 0.f;
+    cudaEventSynchronize(r.e1);
+    cudaEventElapsedTime(&t, r.e0, r.e1);
+    size_t k = 0;
+    for (; k < nm.size(); ++k) if (nm[k] == r.name) break;
+    if (k == nm.size()) { nm.push_back(r.name); ms.push_back(0.f); cnt.push_back(0); }
+    ms[k] += t;
+    cnt[k] += 1;
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  g_prof.clear();
+  std::string joined;
+  int32_t n = 0;
+  for (size_t k = 0; k < nm.size() && n < max_entries; ++k) {
+    if (joined.size() + nm[k].size() + 2 > names_bytes) break;
+    joined += nm[k];
+    joined += '\n';
+    if (total_ms) total_ms[n] = ms[k];
+    if (launches) launches[n] = cnt[k];
+    ++n;
+  }
+  if (names && names_bytes) {
+    std::memcpy(names, joined.c_str(), joined.size() + 1);
+  }
+  return n;
+}
+
+int32_t nt_force_generic(int32_t on) {
+  int32_t prev = g_force_generic;
+  g_force_generic = on;
+  return prev;
+}
+
+}  // extern "C"

@@ -1,0 +1,82 @@
+// Shared declarations of libnested_pair's CUDA sources: batch metadata passed by value to
+// kernels, dtype helpers, launch bookkeeping.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/nested_pair.h"
+
+namespace ntp {
+
+constexpr int MAXB = 64;  // samples per launch group; larger batches are processed in groups
+
+// Per-group batch metadata, computed on the host from the canonical lengths (App. A: canonical
+// sizes stay on the host) and passed by value, so kernels decode positions without a global read.
+// Offsets are absolute (they index the caller's full packed buffers).
+struct BatchMeta {
+  int B;
+  int N[MAXB];
+  long long tok_off[MAXB + 1];
+  long long pair_off[MAXB + 1];
+  // prefix of N_s * ld_s with ld_s = round_up(N_s, 8): size of one channel plane of the
+  // channel-major intermediates; element (s, c, i, k) of a C-channel buffer lives at
+  // C * cm_off[s] + c * N_s * ld_s + i * ld_s + k.
+  long long cm_off[MAXB + 1];
+};
+
+__host__ __device__ inline int round_up8(int n) { return (n + 7) & ~7; }
+
+// largest s with off[s] <= p (p < off[B]); empty samples are skipped because their successor
+// shares the offset.
+__device__ inline int find_sample(const long long* off, int B, long long p) {
+  int lo = 0, hi = B;  // invariant: off[lo] <= p < off[hi]
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (off[mid] <= p) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+template <typename T> struct Cvt;
+template <> struct Cvt<float> {
+  __device__ static inline float ld(const float* p) { return *p; }
+  __device__ static inline void st(float* p, float v) { *p = v; }
+};
+template <> struct Cvt<__nv_bfloat16> {
+  __device__ static inline float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+  __device__ static inline void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+extern std::atomic<long long> g_launches;
+extern int g_force_generic;
+
+// Counts a kernel launch and, while per-kernel profiling is on (nt_profile_begin), brackets it with
+// CUDA events on the launching stream.  Construct before the launch, destroy after it.
+struct LaunchScope {
+  LaunchScope(const char* name, cudaStream_t st);
+  ~LaunchScope();
+  cudaStream_t st;
+  int slot;
+};
+
+inline nt_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? NT_OK : NT_ERR_CUDA; }
+
+// Builds the metadata of samples [s0, s1) (s1 - s0 <= MAXB) given absolute prefix arrays.
+void fill_meta(BatchMeta& m, const int64_t* lengths_h, int s0, int s1, long long tok0, long long pair0,
+               long long cm0);
+
+struct GroupIter {  // walks a batch in groups of MAXB samples
+  const int64_t* len;
+  int B, s0 = 0;
+  long long tok = 0, pair = 0, cm = 0;
+  GroupIter(const int64_t* l, int b) : len(l), B(b) {}
+  bool next(BatchMeta& m);
+};
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace ntp

@@ -1,0 +1,16 @@
+// bf16 kernels tuned for sm_100a.  Memory-bound steps stay on CUDA cores with 16-byte vector
+// access; dense contractions use tcgen05 tensor-core tiles with TMEM accumulators.
+#pragma once
+#include "common.cuh"
+
+namespace ntp {
+
+bool fast_broadcast_supported(int c_z);
+nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
+                            void* z, const BatchMeta& m, cudaStream_t st);
+
+bool fast_segment_reduce_supported(int C);
+nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,
+                              cudaStream_t st);
+
+}  // namespace ntp

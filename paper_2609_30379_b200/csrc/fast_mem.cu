@@ -1,0 +1,186 @@
+// Memory-bound bf16 kernels on CUDA cores: the gather + LayerNorm pair broadcast (pure streaming
+// write of the packed pair state) and the segmented mean/sum (pure streaming read).
+#include "fast.cuh"
+
+namespace ntp {
+
+// ------------------------------------------------------------------------------------------
+// z[p,:] = LN(u[tok_off[s]+i] + v[tok_off[s]+j]) * gamma + beta, bf16 out, 16-byte stores.
+// A work item is a run of up to BJ consecutive j of one pair row (s, i); LP = c_z / 8 lanes share a
+// position, so a warp normalises 32 / LP positions per step with shuffle reductions inside the
+// lane group.  The row term u is held in registers for the whole run.
+// ------------------------------------------------------------------------------------------
+constexpr int BJ = 64;
+
+template <int LP>
+__global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __restrict__ u,
+                                                                const float* __restrict__ v,
+                                                                const __nv_bfloat16* __restrict__ gamma,
+                                                                const __nv_bfloat16* __restrict__ beta, float eps,
+                                                                __nv_bfloat16* __restrict__ z, BatchMeta m,
+                                                                long long n_items) {
+  constexpr int C = LP * 8;
+  constexpr int PPW = 32 / LP;   // positions per warp step
+  __shared__ long long item_off[MAXB + 1];
+  if (threadIdx.x == 0) {
+    long long acc = 0;
+    for (int s = 0; s < m.B; ++s) {
+      item_off[s] = acc;
+      acc += (long long)m.N[s] * ((m.N[s] + BJ - 1) / BJ);
+    }
+    item_off[m.B] = acc;
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, sub = lane / LP, cl = lane % LP;
+  float g[8], b[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    g[e] = __bfloat162float(gamma[cl * 8 + e]);
+    b[e] = __bfloat162float(beta[cl * 8 + e]);
+  }
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long it = wid; it < n_items; it += nw) {
+    const int s = find_sample(item_off, m.B, it);
+    const int N = m.N[s];
+    const int cps = (N + BJ - 1) / BJ;
+    const long long r = it - item_off[s];
+    const int i = (int)(r / cps), j0 = (int)(r - (long long)i * cps) * BJ;
+    const int j1 = min(N, j0 + BJ);
+    const float4* up = reinterpret_cast<const float4*>(u + (m.tok_off[s] + i) * C + cl * 8);
+    const float4 u0 = up[0], u1 = up[1];
+    const float ur[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+    __nv_bfloat16* zrow = z + (m.pair_off[s] + (long long)i * N) * C;
+    for (int jb = j0; jb < j1; jb += PPW) {
+      const int j = jb + sub;
+      const bool ok = j < j1;
+      const int jj = ok ? j : j1 - 1;
+      const float4* vp = reinterpret_cast<const float4*>(v + (m.tok_off[s] + jj) * C + cl * 8);
+      const float4 v0 = vp[0], v1 = vp[1];
+      float x[8] = {ur[0] + v0.x, ur[1] + v0.y, ur[2] + v0.z, ur[3] + v0.w,
+                    ur[4] + v1.x, ur[5] + v1.y, ur[6] + v1.z, ur[7] + v1.w};
+      float sum = ((x[0] + x[1]) + (x[2] + x[3])) + ((x[4] + x[5]) + (x[6] + x[7]));
+#pragma unroll
+      for (int o = LP / 2; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float mean = sum * (1.0f / C);
+      float q = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        x[e] -= mean;
+        q = fmaf(x[e], x[e], q);
+      }
+#pragma unroll
+      for (int o = LP / 2; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+      const float rs = rsqrtf(q * (1.0f / C) + eps);
+      uint4 pk;
+      __nv_bfloat162 h;
+      h = __floats2bfloat162_rn(fmaf(x[0] * rs, g[0], b[0]), fmaf(x[1] * rs, g[1], b[1]));
+      pk.x = *reinterpret_cast<unsigned*>(&h);
+      h = __floats2bfloat162_rn(fmaf(x[2] * rs, g[2], b[2]), fmaf(x[3] * rs, g[3], b[3]));
+      pk.y = *reinterpret_cast<unsigned*>(&h);
+      h = __floats2bfloat162_rn(fmaf(x[4] * rs, g[4], b[4]), fmaf(x[5] * rs, g[5], b[5]));
+      pk.z = *reinterpret_cast<unsigned*>(&h);
+      h = __floats2bfloat162_rn(fmaf(x[6] * rs, g[6], b[6]), fmaf(x[7] * rs, g[7], b[7]));
+      pk.w = *reinterpret_cast<unsigned*>(&h);
+      if (ok) *reinterpret_cast<uint4*>(zrow + (long long)j * C + cl * 8) = pk;
+    }
+  }
+}
+
+bool fast_broadcast_supported(int c_z) { return c_z == 64 || c_z == 128 || c_z == 256; }
+
+nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
+                            void* z, const BatchMeta& m, cudaStream_t st) {
+  long long items = 0;
+  for (int s = 0; s < m.B; ++s) items += (long long)m.N[s] * ((m.N[s] + BJ - 1) / BJ);
+  if (items == 0) return NT_OK;
+  long long blocks = (items + 7) / 8;
+  const long long cap = 148 * 8;
+  if (blocks > cap) blocks = cap;
+  const __nv_bfloat16* g = (const __nv_bfloat16*)gamma;
+  const __nv_bfloat16* b = (const __nv_bfloat16*)beta;
+  __nv_bfloat16* zz = (__nv_bfloat16*)z;
+  {
+    LaunchScope ls("broadcast_ln", st);
+    if (c_z == 64) broadcast_ln_fast_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+    else if (c_z == 128) broadcast_ln_fast_kernel<16><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+    else broadcast_ln_fast_kernel<32><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+  }
+  return cuda_ok();
+}
+
+// ------------------------------------------------------------------------------------------
+// segmented mean / sum over contiguous row groups, bf16 in, float accumulate, bf16 out.
+// One block per group; VL = C / 8 lanes cover a row with 16-byte loads, 256 / VL rows in flight.
+// ------------------------------------------------------------------------------------------
+constexpr int SR_THREADS = 256;
+constexpr int SR_UNROLL = 4;
+
+__global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const __nv_bfloat16* __restrict__ v,
+                                                                        __nv_bfloat16* __restrict__ out,
+                                                                        const int64_t* __restrict__ splits, int C,
+                                                                        int mean) {
+  extern __shared__ float part[];   // [RS][C]
+  const int VL = C >> 3;
+  const int RS = SR_THREADS / VL;
+  const int t = threadIdx.x;
+  const int slot = t / VL, vl = t - slot * VL;
+  const long long g = blockIdx.x;
+  const long long lo = splits[g], hi = splits[g + 1];
+  float acc[8] = {};
+  if (slot < RS) {
+    const uint4* base = reinterpret_cast<const uint4*>(v) + vl;
+    long long r = lo + slot;
+    for (; r + (long long)(SR_UNROLL - 1) * RS < hi; r += (long long)SR_UNROLL * RS) {
+      uint4 d[SR_UNROLL];
+#pragma unroll
+      for (int uu = 0; uu < SR_UNROLL; ++uu) d[uu] = __ldg(base + (r + (long long)uu * RS) * VL);
+#pragma unroll
+      for (int uu = 0; uu < SR_UNROLL; ++uu) {
+        const unsigned w[4] = {d[uu].x, d[uu].y, d[uu].z, d[uu].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          acc[2 * e] += __uint_as_float(w[e] << 16);
+          acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+        }
+      }
+    }
+    for (; r < hi; r += RS) {
+      const uint4 d = __ldg(base + r * VL);
+      const unsigned w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        acc[2 * e] += __uint_as_float(w[e] << 16);
+        acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) part[slot * C + vl * 8 + e] = acc[e];
+  }
+  __syncthreads();
+  const long long n = hi - lo;
+  const float sc = (mean && n > 0) ? 1.0f / (float)n : 1.0f;
+  for (int c = t; c < C; c += SR_THREADS) {
+    float tot = 0.f;
+    for (int sl = 0; sl < RS; ++sl) tot += part[sl * C + c];
+    out[g * C + c] = __float2bfloat16_rn(tot * sc);
+  }
+}
+
+bool fast_segment_reduce_supported(int C) { return C % 8 == 0 && C >= 8 && C <= 2048; }
+
+nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,
+                              cudaStream_t st) {
+  if (G <= 0) return NT_OK;
+  if (G > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  const int VL = C / 8, RS = SR_THREADS / VL;
+  const size_t smem = (size_t)RS * C * sizeof(float);
+  {
+    LaunchScope ls("segment_reduce", st);
+    segment_reduce_fast_kernel<<<(unsigned)G, SR_THREADS, smem, st>>>((const __nv_bfloat16*)v, (__nv_bfloat16*)out,
+                                                                     splits, C, mean);
+  }
+  return cuda_ok();
+}
+
+}  // namespace ntp

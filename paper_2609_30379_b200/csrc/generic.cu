@@ -1,0 +1,455 @@
+// Shape-generic CUDA-core kernels: tiled projection with LayerNorm / gate prologues and
+// row-major or channel-major epilogues, the per-(sample, channel) triangle contraction, the
+// gather + LayerNorm broadcast, an online-softmax attention core and the segmented reduction.
+#include "generic.cuh"
+
+namespace ntp {
+
+// ------------------------------------------------------------------------------------------
+// projection
+// ------------------------------------------------------------------------------------------
+constexpr int PBM = 64, PBN = 64, PBK = 16, PTHREADS = 256;
+
+__device__ inline float sigmoidf_acc(float x) { return 1.0f / (1.0f + expf(-x)); }
+
+template <typename T>
+__global__ void __launch_bounds__(PTHREADS) proj_kernel(ProjArgs a, BatchMeta m) {
+  __shared__ __align__(16) float As[PBK][PBM + 4];
+  __shared__ __align__(16) float W1s[PBK][PBN + 4];
+  __shared__ __align__(16) float W2s[PBK][PBN + 4];
+  __shared__ float mu[PBM], rstd[PBM];
+  __shared__ long long cmbase[PBM], inpl[PBM], plane[PBM];
+
+  const int t = threadIdx.x;
+  const long long r0 = a.row0 + (long long)blockIdx.x * PBM;
+  const long long rend = a.row0 + a.rows;
+  const int n0 = blockIdx.y * PBN;
+  const T* A = (const T*)a.A;
+  const T* gA = (const T*)a.gateA;
+  const int K = a.K;
+  const bool need_cm = a.a_mode == A_CHANNEL_MAJOR || a.out_mode == O_CHANNEL_MAJOR;
+
+  if (t < PBM) {
+    long long p = r0 + t;
+    if (need_cm && p < rend) {
+      int s = find_sample(m.pair_off, m.B, p);
+      int N = m.N[s], ld = round_up8(N);
+      long long r = p - m.pair_off[s];
+      long long i = r / N, j = r - i * N;
+      cmbase[t] = m.cm_off[s];
+      plane[t] = (long long)N * ld;
+      inpl[t] = i * ld + j;
+    }
+  }
+  __syncthreads();
+
+  auto loadA = [&](int rl, int k) -> float {
+    long long p = r0 + rl;
+    if (p >= rend || k >= K) return 0.f;
+    float v;
+    if (a.a_mode == A_ROWMAJOR) {
+      v = Cvt<T>::ld(A + p * K + k);
+      if (gA) v *= Cvt<T>::ld(gA + p * K + k);
+    } else {
+      v = Cvt<T>::ld(A + (long long)K * cmbase[rl] + (long long)k * plane[rl] + inpl[rl]);
+    }
+    return v;
+  };
+
+  const bool has_ln = a.ln_g != nullptr;
+  if (has_ln) {   // two-pass row statistics
+    const int w = t >> 5, lane = t & 31;
+    for (int rl = w; rl < PBM; rl += PTHREADS / 32) {
+      float s = 0.f;
+      for (int k = lane; k < K; k += 32) s += loadA(rl, k);
+#pragma unroll
+      for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const float mean = s / (float)K;
+      float q = 0.f;
+      for (int k = lane; k < K; k += 32) {
+        float dlt = loadA(rl, k) - mean;
+        q += dlt * dlt;
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+      if (lane == 0) {
+        mu[rl] = mean;
+        rstd[rl] = rsqrtf(q / (float)K + a.eps);
+      }
+    }
+    __syncthreads();
+  }
+
+  const T* W1 = (const T*)a.W1;
+  const T* W2 = (const T*)a.W2;
+  const T* lng = (const T*)a.ln_g;
+  const T* lnb = (const T*)a.ln_b;
+  const int ty = t >> 4, tx = t & 15;
+  float acc1[4][4] = {}, acc2[4][4] = {};
+
+  for (int k0 = 0; k0 < K; k0 += PBK) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int rl, kk;
+      if (a.a_mode == A_ROWMAJOR) { rl = t >> 2; kk = (t & 3) * 4 + u; }
+      else { rl = t & 63; kk = (t >> 6) + 4 * u; }
+      const int k = k0 + kk;
+      float v = loadA(rl, k);
+      if (has_ln && k < K) v = (v - mu[rl]) * rstd[rl] * Cvt<T>::ld(lng + k) + Cvt<T>::ld(lnb + k);
+      As[kk][rl] = v;
+      const int nl = t >> 2, kw = (t & 3) * 4 + u, n = n0 + nl, k2 = k0 + kw;
+      const bool ok = n < a.Nout && k2 < K;
+      W1s[kw][nl] = ok ? Cvt<T>::ld(W1 + (long long)n * K + k2) : 0.f;
+      if (W2) W2s[kw][nl] = ok ? Cvt<T>::ld(W2 + (long long)n * K + k2) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < PBK; ++kk) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 wv = *reinterpret_cast<const float4*>(&W1s[kk][tx * 4]);
+      const float ar[4] = {av.x, av.y, av.z, av.w};
+      const float wr[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc1[i][j] = fmaf(ar[i], wr[j], acc1[i][j]);
+      if (W2) {
+        const float4 w2 = *reinterpret_cast<const float4*>(&W2s[kk][tx * 4]);
+        const float w2r[4] = {w2.x, w2.y, w2.z, w2.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc2[i][j] = fmaf(ar[i], w2r[j], acc2[i][j]);
+      }
+    }
+    __syncthreads();
+  }
+
+  const T* gO = (const T*)a.gateO;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int rl = ty * 4 + i;
+    const long long p = r0 + rl;
+    if (p >= rend) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tx * 4 + j;
+      if (n >= a.Nout) continue;
+      float v = acc1[i][j];
+      if (W2) v = sigmoidf_acc(v) * acc2[i][j];
+      else if (a.act == ACT_SIGMOID) v = sigmoidf_acc(v);
+      if (gO) v *= Cvt<T>::ld(gO + p * a.Nout + n);
+      if (a.out_mode == O_CHANNEL_MAJOR) {
+        Cvt<T>::st((T*)a.out + (long long)a.Nout * cmbase[rl] + (long long)n * plane[rl] + inpl[rl], v);
+      } else if (a.out_f32) {
+        float* o = (float*)a.out + p * a.Nout + n;
+        *o = (a.out_mode == O_ACCUM) ? *o + v : v;
+      } else {
+        T* o = (T*)a.out + p * a.Nout + n;
+        if (a.out_mode == O_ACCUM) v += Cvt<T>::ld(o);
+        Cvt<T>::st(o, v);
+      }
+    }
+  }
+}
+
+template <typename T>
+nt_status launch_proj(const ProjArgs& a, const BatchMeta& m, cudaStream_t st, const char* name) {
+  if (a.rows <= 0 || a.Nout <= 0) return NT_OK;
+  long long bx = (a.rows + PBM - 1) / PBM;
+  if (bx > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)bx, (unsigned)((a.Nout + PBN - 1) / PBN));
+  {
+    LaunchScope ls(name, st);
+    proj_kernel<T><<<grid, PTHREADS, 0, st>>>(a, m);
+  }
+  return cuda_ok();
+}
+template nt_status launch_proj<float>(const ProjArgs&, const BatchMeta&, cudaStream_t, const char*);
+template nt_status launch_proj<__nv_bfloat16>(const ProjArgs&, const BatchMeta&, cudaStream_t, const char*);
+
+// ------------------------------------------------------------------------------------------
+// triangle contraction  t[c][i][j] = sum_k a[c][i][k] b[c][j][k]
+// ------------------------------------------------------------------------------------------
+constexpr int CT = 64, CK = 16;
+
+template <typename T>
+__global__ void __launch_bounds__(256) contract_kernel(const T* __restrict__ a, const T* __restrict__ b,
+                                                      T* __restrict__ tout, int C, BatchMeta m) {
+  __shared__ __align__(16) float As[CK][CT + 4];
+  __shared__ __align__(16) float Bs[CK][CT + 4];
+  long long w = blockIdx.x;
+  int s = 0, nt = 0;
+  for (; s < m.B; ++s) {   // tile -> sample
+    nt = (m.N[s] + CT - 1) / CT;
+    long long cnt = (long long)C * nt * nt;
+    if (w < cnt) break;
+    w -= cnt;
+  }
+  if (s >= m.B) return;
+  const int N = m.N[s], ld = round_up8(N);
+  const int c = (int)(w / (nt * nt));
+  const int rem = (int)(w - (long long)c * nt * nt);
+  const int i0 = (rem / nt) * CT, j0 = (rem % nt) * CT;
+  const long long base = (long long)C * m.cm_off[s] + (long long)c * N * ld;
+  const T* Ap = a + base;
+  const T* Bp = b + base;
+  const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < N; k0 += CK) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int rl = t >> 2, kk = (t & 3) * 4 + u, k = k0 + kk;
+      const int i = i0 + rl, j = j0 + rl;
+      As[kk][rl] = (i < N && k < N) ? Cvt<T>::ld(Ap + (long long)i * ld + k) : 0.f;
+      Bs[kk][rl] = (j < N && k < N) ? Cvt<T>::ld(Bp + (long long)j * ld + k) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < CK; ++kk) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float ar[4] = {av.x, av.y, av.z, av.w};
+      const float br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  T* Tp = tout + base;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int ii = i0 + ty * 4 + i, jj = j0 + tx * 4 + j;
+      if (ii < N && jj < N) Cvt<T>::st(Tp + (long long)ii * ld + jj, acc[i][j]);
+    }
+}
+
+template <typename T>
+nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& m, cudaStream_t st) {
+  long long tiles = 0;
+  for (int s = 0; s < m.B; ++s) {
+    long long nt = (m.N[s] + CT - 1) / CT;
+    tiles += (long long)C * nt * nt;
+  }
+  if (tiles == 0) return NT_OK;
+  if (tiles > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("generic_tri_contract", st);
+    contract_kernel<T><<<(unsigned)tiles, 256, 0, st>>>(a, b, t, C, m);
+  }
+  return cuda_ok();
+}
+template nt_status launch_contract<float>(const float*, const float*, float*, int, const BatchMeta&, cudaStream_t);
+template nt_status launch_contract<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, __nv_bfloat16*, int,
+                                                  const BatchMeta&, cudaStream_t);
+
+// ------------------------------------------------------------------------------------------
+// broadcast + LayerNorm (generic widths): one warp per packed position
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) broadcast_ln_kernel(const float* __restrict__ u, const float* __restrict__ v,
+                                                          const T* __restrict__ gamma, const T* __restrict__ beta,
+                                                          float eps, int c_z, T* __restrict__ z, BatchMeta m) {
+  const int lane = threadIdx.x & 31;
+  const long long p = m.pair_off[0] + (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (p >= m.pair_off[m.B]) return;
+  const int s = find_sample(m.pair_off, m.B, p);
+  const int N = m.N[s];
+  const long long r = p - m.pair_off[s];
+  const long long i = r / N, j = r - i * N;
+  const float* ur = u + (m.tok_off[s] + i) * c_z;
+  const float* vr = v + (m.tok_off[s] + j) * c_z;
+  float sum = 0.f;
+  for (int c = lane; c < c_z; c += 32) sum += ur[c] + vr[c];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum / (float)c_z;
+  float q = 0.f;
+  for (int c = lane; c < c_z; c += 32) {
+    float dlt = ur[c] + vr[c] - mean;
+    q += dlt * dlt;
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+  const float rs = rsqrtf(q / (float)c_z + eps);
+  T* zr = z + p * c_z;
+  for (int c = lane; c < c_z; c += 32)
+    Cvt<T>::st(zr + c, (ur[c] + vr[c] - mean) * rs * Cvt<T>::ld(gamma + c) + Cvt<T>::ld(beta + c));
+}
+
+template <typename T>
+nt_status launch_broadcast_ln(const float* u, const float* v, const T* gamma, const T* beta, float eps, int c_z,
+                              T* z, const BatchMeta& m, cudaStream_t st) {
+  long long npos = m.pair_off[m.B] - m.pair_off[0];
+  if (npos <= 0) return NT_OK;
+  long long blocks = (npos + 7) / 8;
+  if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("generic_broadcast_ln", st);
+    broadcast_ln_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(u, v, gamma, beta, eps, c_z, z, m);
+  }
+  return cuda_ok();
+}
+template nt_status launch_broadcast_ln<float>(const float*, const float*, const float*, const float*, float, int,
+                                              float*, const BatchMeta&, cudaStream_t);
+template nt_status launch_broadcast_ln<__nv_bfloat16>(const float*, const float*, const __nv_bfloat16*,
+                                                      const __nv_bfloat16*, float, int, __nv_bfloat16*,
+                                                      const BatchMeta&, cudaStream_t);
+
+// ------------------------------------------------------------------------------------------
+// attention core: one warp per (attention row, head, query); lanes over keys; online softmax
+// ------------------------------------------------------------------------------------------
+constexpr int AQB = 8;      // queries (warps) per block
+constexpr int AD_MAX = 128; // head dim limit of the generic core
+
+template <typename T>
+__global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                            const T* __restrict__ v, const T* __restrict__ bias,
+                                                            T* __restrict__ o, int H, int d, int pair_order,
+                                                            BatchMeta m) {
+  __shared__ float qs[AQB][AD_MAX];
+  long long w = blockIdx.x;
+  int s = 0, N = 0, nqb = 0;
+  for (; s < m.B; ++s) {
+    N = m.N[s];
+    nqb = (N + AQB - 1) / AQB;
+    long long cnt = (long long)(pair_order ? N : (N > 0 ? 1 : 0)) * H * nqb;
+    if (w < cnt) break;
+    w -= cnt;
+  }
+  if (s >= m.B) return;
+  const int jb = (int)(w % nqb);
+  const int h = (int)((w / nqb) % H);
+  const long long i = w / ((long long)nqb * H);
+  const long long base = pair_order ? m.pair_off[s] + i * N : m.tok_off[s];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j = jb * AQB + warp;
+  const int Hd = H * d;
+  const bool active = j < N;
+  if (active)
+    for (int e = lane; e < d; e += 32) qs[warp][e] = Cvt<T>::ld(q + (base + j) * Hd + h * d + e);
+  __syncwarp();
+  if (!active) return;
+  const int ld = round_up8(N);
+  const T* brow = bias ? bias + (long long)H * m.cm_off[s] + (long long)h * N * ld + (long long)j * ld : nullptr;
+  const float scale = rsqrtf((float)d);
+  float mrun = -INFINITY, lrun = 0.f;
+  float oacc[AD_MAX / 32] = {};
+  const int ne = (d + 31) / 32;
+  for (int c0 = 0; c0 < N; c0 += 32) {
+    const int kk = c0 + lane;
+    float sc = -INFINITY;
+    if (kk < N) {
+      const T* kr = k + (base + kk) * Hd + h * d;
+      float dot = 0.f;
+      for (int e = 0; e < d; ++e) dot = fmaf(qs[warp][e], Cvt<T>::ld(kr + e), dot);
+      sc = dot * scale;
+      if (brow) sc += Cvt<T>::ld(brow + kk);
+    }
+    float cmax = sc;
+#pragma unroll
+    for (int of = 16; of; of >>= 1) cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, of));
+    const float mnew = fmaxf(mrun, cmax);
+    const float corr = expf(mrun - mnew);   // first chunk: exp(-inf) = 0
+    const float pr = (kk < N) ? expf(sc - mnew) : 0.f;
+    float psum = pr;
+#pragma unroll
+    for (int of = 16; of; of >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, of);
+    lrun = lrun * corr + psum;
+    mrun = mnew;
+    for (int u = 0; u < ne; ++u) oacc[u] *= corr;
+    const int lim = min(32, N - c0);
+    for (int k2 = 0; k2 < lim; ++k2) {
+      const float pk = __shfl_sync(0xffffffffu, pr, k2);
+      const T* vr = v + (base + c0 + k2) * Hd + h * d;
+      for (int u = 0; u < ne; ++u) {
+        const int e = u * 32 + lane;
+        if (e < d) oacc[u] = fmaf(pk, Cvt<T>::ld(vr + e), oacc[u]);
+      }
+    }
+  }
+  const float inv = 1.0f / lrun;
+  for (int u = 0; u < ne; ++u) {
+    const int e = u * 32 + lane;
+    if (e < d) Cvt<T>::st(o + (base + j) * Hd + h * d + e, oacc[u] * inv);
+  }
+}
+
+template <typename T>
+nt_status launch_attn_core(const T* q, const T* k, const T* v, const T* bias, T* o, int H, int d, int pair_order,
+                           const BatchMeta& m, cudaStream_t st) {
+  if (d > AD_MAX) return NT_ERR_UNSUPPORTED;
+  long long blocks = 0;
+  for (int s = 0; s < m.B; ++s) {
+    long long N = m.N[s], nqb = (N + AQB - 1) / AQB;
+    blocks += (pair_order ? N : (N > 0 ? 1 : 0)) * H * nqb;
+  }
+  if (blocks == 0) return NT_OK;
+  if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("generic_attn_core", st);
+    attn_core_kernel<T><<<(unsigned)blocks, AQB * 32, 0, st>>>(q, k, v, bias, o, H, d, pair_order, m);
+  }
+  return cuda_ok();
+}
+template nt_status launch_attn_core<float>(const float*, const float*, const float*, const float*, float*, int, int,
+                                           int, const BatchMeta&, cudaStream_t);
+template nt_status launch_attn_core<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
+                                                   const __nv_bfloat16*, __nv_bfloat16*, int, int, int,
+                                                   const BatchMeta&, cudaStream_t);
+
+// ------------------------------------------------------------------------------------------
+// segmented reduction (generic widths): one block per group
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) segment_reduce_kernel(const T* __restrict__ v, T* __restrict__ out,
+                                                            const int64_t* __restrict__ splits, int C, int mean) {
+  __shared__ float part[256];
+  const long long g = blockIdx.x;
+  const long long lo = splits[g], hi = splits[g + 1];
+  const long long n = hi - lo;
+  const float sc = (mean && n > 0) ? 1.0f / (float)n : 1.0f;
+  const int t = threadIdx.x;
+  if (C >= 256) {
+    for (int c = t; c < C; c += 256) {
+      float acc = 0.f;
+      for (long long r = lo; r < hi; ++r) acc += Cvt<T>::ld(v + r * C + c);
+      Cvt<T>::st(out + g * C + c, acc * sc);
+    }
+    return;
+  }
+  const int RS = 256 / C;
+  const int ch = t % C, slot = t / C;
+  float acc = 0.f;
+  if (slot < RS)
+    for (long long r = lo + slot; r < hi; r += RS) acc += Cvt<T>::ld(v + r * C + ch);
+  part[t] = acc;
+  __syncthreads();
+  if (t < C) {
+    float tot = 0.f;
+    for (int sl = 0; sl < RS; ++sl) tot += part[sl * C + t];
+    Cvt<T>::st(out + g * C + t, tot * sc);
+  }
+}
+
+template <typename T>
+nt_status launch_segment_reduce(const T* v, T* out, const int64_t* splits, long long G, int C, int mean,
+                                cudaStream_t st) {
+  if (G <= 0) return NT_OK;
+  if (G > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("generic_segment_reduce", st);
+    segment_reduce_kernel<T><<<(unsigned)G, 256, 0, st>>>(v, out, splits, C, mean);
+  }
+  return cuda_ok();
+}
+template nt_status launch_segment_reduce<float>(const float*, float*, const int64_t*, long long, int, int,
+                                                cudaStream_t);
+template nt_status launch_segment_reduce<__nv_bfloat16>(const __nv_bfloat16*, __nv_bfloat16*, const int64_t*,
+                                                        long long, int, int, cudaStream_t);
+
+}  // namespace ntp

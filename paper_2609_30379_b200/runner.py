@@ -1,0 +1,84 @@
+"""Sequencing of the library calls for one block / a stack of blocks (the call a user makes).
+
+Only orchestration lives here: buffers come from torch, every arithmetic step is a call into
+libnested_pair through ``binding``.  One block (all asynchronous on one stream):
+    nt_pair_broadcast -> nt_tri_mul_out -> nt_row_attn_pairbias -> nt_segment_reduce -> nt_token_update
+Stacked blocks rebuild the pair state from the tokens the previous block returned and reuse the
+same ``z`` and workspace buffers, so peak memory is one block's.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as nt
+from .workloads import Config
+
+LN_EPS = 1e-5
+
+
+def torch_dtype(cfg_dtype: str) -> torch.dtype:
+    return torch.float32 if cfg_dtype == "f32" else torch.bfloat16
+
+
+def to_device(arr: Optional[np.ndarray], dtype: torch.dtype, device="cuda") -> Optional[torch.Tensor]:
+    if arr is None:
+        return None
+    return torch.from_numpy(np.ascontiguousarray(arr)).to(device=device, dtype=dtype).contiguous()
+
+
+def upload_weights(blocks: List[dict], dtype: torch.dtype, device="cuda") -> List[dict]:
+    out = []
+    for w in blocks:
+        if all(isinstance(v, dict) for v in w.values()):
+            out.append({k: {kk: to_device(vv, dtype, device) for kk, vv in v.items()} for k, v in w.items()})
+        else:
+            out.append({k: to_device(v, dtype, device) for k, v in w.items()})
+    return out
+
+
+class PairStack:
+    """Device state for running a configuration's stacked blocks on one batch layout."""
+
+    def __init__(self, cfg: Config, lengths, weights_host: List[dict], device="cuda"):
+        self.cfg = cfg
+        self.dtype = torch_dtype(cfg.dtype)
+        self.device = torch.device(device)
+        self.L = nt.Layout(lengths, device=device)
+        self.W = upload_weights(weights_host, self.dtype, device)
+        dt = nt.dtype_code(self.dtype)
+        dims = (cfg.c_s, cfg.c_z, cfg.c_h, cfg.H, cfg.d)
+        if cfg.kind == "pair":
+            nbytes = nt.nt_workspace_bytes(nt.NT_OP_BLOCK, dt, nt.NT_ORDER_PAIR_IJC, self.L.lengths_h, dims)
+            self.z = torch.empty((self.L.T2, cfg.c_z), dtype=self.dtype, device=self.device)
+            self.m = torch.empty((self.L.T1, cfg.c_z), dtype=self.dtype, device=self.device)
+        else:
+            nbytes = nt.nt_workspace_bytes(nt.NT_OP_ROW_ATTN, dt, nt.NT_ORDER_TOKEN_NC, self.L.lengths_h, dims)
+            self.z = None
+            self.pooled = torch.empty((self.L.B, cfg.c_z), dtype=self.dtype, device=self.device)
+        self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+
+    # one block, in place on x; z is rebuilt from x
+    def block(self, x: torch.Tensor, w: dict, stream=None):
+        cfg, L = self.cfg, self.L
+        b = w["broadcast"]
+        nt.nt_pair_broadcast(L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], LN_EPS, self.z, self.workspace, stream)
+        nt.nt_tri_mul_out(L, w["trimul"], LN_EPS, self.z, self.workspace, stream)
+        nt.nt_row_attn_pairbias(L, nt.NT_ORDER_PAIR_IJC, w["attn"], cfg.H, cfg.d, LN_EPS, self.z, self.workspace, stream)
+        nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, self.z, self.m, L.status, stream)
+        nt.nt_token_update(self.m, w["reduce"]["W_r"], x, stream)
+
+    def forward(self, x: torch.Tensor, stream=None):
+        """Runs every block in place on ``x`` [T1, c_s]; returns (x, z) for pair configs or
+        (x, pooled) for the token-only configuration."""
+        if self.cfg.kind == "pair":
+            for w in self.W:
+                self.block(x, w, stream)
+            return x, self.z
+        for w in self.W:
+            nt.nt_row_attn_pairbias(self.L, nt.NT_ORDER_TOKEN_NC, w, self.cfg.H, self.cfg.d, LN_EPS, x,
+                                    self.workspace, stream)
+        nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, self.L.tok_off, x, self.pooled, self.L.status, stream)
+        return x, self.pooled

@@ -1,0 +1,109 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and its host-side
+argument validation returns the documented codes before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_30379_b200 import build
+    build.build_library()
+    from paper_2609_30379_b200 import binding
+    return binding
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "nested_pair.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(nt_[a-z_]+)\s*\(", text)))
+
+
+def test_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert {"nt_offsets_build", "nt_pair_broadcast", "nt_tri_mul_out", "nt_row_attn_pairbias",
+            "nt_segment_reduce"} <= set(names)
+    for n in names:
+        assert hasattr(lib.lib, n), n
+    assert set(lib.EXPORTS) == set(names)
+
+
+def test_status_strings(lib):
+    for code in range(7):
+        assert lib.lib.nt_status_string(code)
+
+
+def _layout(lib, lengths, T1=None, T2=None):
+    lengths = np.asarray(lengths, dtype=np.int64)
+    L = lib.nt_layout()
+    L.B = len(lengths)
+    L.T1 = int(lengths.sum()) if T1 is None else T1
+    L.T2 = int((lengths * lengths).sum()) if T2 is None else T2
+    L.lengths_h = lengths.ctypes.data if len(lengths) else None
+    return L, lengths
+
+
+FAKE = 0x10000   # aligned non-null value; validation fails before anything dereferences it
+
+
+def test_host_validation_codes(lib):
+    L, keep = _layout(lib, [3, 4], T2=26)            # true T2 is 25
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 6   # NT_ERR_INCONSISTENT
+    L, keep = _layout(lib, [3, -1], T1=2, T2=10)
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 1   # negative length
+    L, keep = _layout(lib, [3, 4])
+    st = lib.lib.nt_pair_broadcast(C.byref(L), 7, 8, 8, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 2   # unknown dtype
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, None, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 1   # null x
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE + 2, FAKE, 1 << 20, None)
+    assert st == 1   # misaligned z
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 16, None)
+    assert st == 3   # workspace too small
+    w = lib.nt_trimul_weights()
+    st = lib.lib.nt_tri_mul_out(C.byref(L), lib.NT_BF16, 8, 8, C.byref(w), 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 1   # null weights
+    aw = lib.nt_attn_weights(*([FAKE] * 8))
+    st = lib.lib.nt_row_attn_pairbias(C.byref(L), lib.NT_ORDER_TOKEN_NC, lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 1   # bias weights with token order
+    st = lib.lib.nt_row_attn_pairbias(C.byref(L), 5, lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None)
+    assert st == 2   # unknown order
+    st = lib.lib.nt_row_attn_pairbias(C.byref(L), lib.NT_ORDER_PAIR_IJC, lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 8, None)
+    assert st == 3
+    st = lib.lib.nt_segment_reduce(lib.NT_BF16, 9, 8, 4, 10, FAKE, FAKE, FAKE, None, None)
+    assert st == 2
+    st = lib.lib.nt_segment_reduce(lib.NT_BF16, 0, 8, 4, 10, None, FAKE, FAKE, None, None)
+    assert st == 1
+    st = lib.lib.nt_offsets_build(FAKE, -1, 0, 0, FAKE, FAKE, None, None, None, None, None, None, None, None)
+    assert st == 1
+    st = lib.lib.nt_offsets_build(FAKE, 2, 5, 13, FAKE, FAKE, None, FAKE, None, None, None, None, None, None)
+    assert st == 1   # decode outputs must be given as a group
+
+
+def test_empty_batch_is_a_noop(lib):
+    L, keep = _layout(lib, [])
+    st = lib.lib.nt_pair_broadcast(C.byref(L), lib.NT_BF16, 8, 8, None, None, None, None, None, 1e-5, None, None, 0, None)
+    assert st == 0
+    L, keep = _layout(lib, [0, 0])
+    w = lib.nt_trimul_weights(*([FAKE] * 10))
+    st = lib.lib.nt_tri_mul_out(C.byref(L), lib.NT_BF16, 8, 8, C.byref(w), 1e-5, None, None, 0, None)
+    assert st == 0
+
+
+def test_workspace_bytes_scale_with_packed_size_not_envelope(lib):
+    dims = (384, 128, 128, 4, 32)
+    a = lib.nt_workspace_bytes(lib.NT_OP_BLOCK, lib.NT_BF16, lib.NT_ORDER_PAIR_IJC, np.array([64, 64, 64, 64]), dims)
+    b = lib.nt_workspace_bytes(lib.NT_OP_BLOCK, lib.NT_BF16, lib.NT_ORDER_PAIR_IJC, np.array([128, 8, 8, 8]), dims)
+    # same packed size up to 1.2%, very different N_max: workspace follows sum N^2, not B * N_max^2
+    assert abs(a - b) / a < 0.05
+    assert lib.nt_workspace_bytes(lib.NT_OP_BLOCK, lib.NT_BF16, lib.NT_ORDER_PAIR_IJC, np.array([], dtype=np.int64), dims) == 0
+    T2 = 4 * 64 * 64
+    assert a >= T2 * 128 * 2 * 5     # q, k, v, o, g
+    assert a < T2 * 128 * 2 * 8

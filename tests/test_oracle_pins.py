@@ -347,3 +347,16 @@ def test_bf16_rounding_helpers():
     r = wl.round_to_bf16(a)
     assert np.array_equal(r, ref)
     assert np.array_equal(wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(r)), r)
+
+
+def test_sampled_evaluators_equal_full_functions():
+    cfg, inp = tiny_inputs((7,))
+    rng = np.random.default_rng(9)
+    z = rng.standard_normal((49, cfg.c_z))
+    pos = [(0, 0), (3, 5), (6, 2), (6, 6), (1, 0)]
+    full = orc.tri_mul_out(z, cfg.lengths, inp["blocks"][0]["trimul"]).reshape(7, 7, -1)
+    got = orc.tri_mul_out_at(z.reshape(7, 7, -1), inp["blocks"][0]["trimul"], pos)
+    assert np.allclose(got, np.stack([full[i, j] for i, j in pos]), rtol=1e-12, atol=1e-12)
+    full = orc.row_attn_pairbias(z, cfg.lengths, inp["blocks"][0]["attn"], cfg.H, cfg.d).reshape(7, 7, -1)
+    got = orc.row_attn_pairbias_at(z.reshape(7, 7, -1), inp["blocks"][0]["attn"], cfg.H, cfg.d, pos)
+    assert np.allclose(got, np.stack([full[i, j] for i, j in pos]), rtol=1e-12, atol=1e-12)

@@ -1,0 +1,346 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs.
+
+Each call is gated separately ("teacher forcing"): the oracle step is applied to exactly the
+inputs the GPU call consumed (the GPU's own previous output, up-cast), so bf16 rounding of one
+call does not leak into the verdict on the next.  Whole samples are checked where the oracle
+finishes in seconds (every step is sample-local, so a sample's slice is compared with the oracle
+run on that sample alone); larger samples are checked at sampled positions.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nested_pair_oracle as orc
+from paper_2609_30379_b200 import workloads as wl
+from tests.parity_utils import check
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nt():
+    from paper_2609_30379_b200 import build
+    build.build_library()
+    from paper_2609_30379_b200 import binding
+    return binding
+
+
+def host(t):
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def offsets_np(lengths):
+    n = np.asarray(lengths, dtype=np.int64)
+    return np.concatenate([[0], np.cumsum(n)]), np.concatenate([[0], np.cumsum(n * n)])
+
+
+class RowFetcher:
+    """zs[i] -> pair row i of sample s from a device buffer, as float64 [n, c]."""
+
+    def __init__(self, z_d, pair_off, n):
+        self.z, self.o, self.n, self.cache = z_d, int(pair_off), int(n), {}
+
+    def __getitem__(self, i):
+        if i not in self.cache:
+            a = self.o + i * self.n
+            self.cache[i] = host(self.z[a:a + self.n])
+        return self.cache[i]
+
+
+def run_block_teacher_forced(nt, cfg, inp, full_samples, sampled=None, force_generic=False, rng_seed=0):
+    """Runs one block call by call on the GPU and checks each call against the oracle."""
+    from paper_2609_30379_b200 import runner
+    lengths = [int(v) for v in inp["lengths"]]
+    tok, po = offsets_np(lengths)
+    prev = nt.nt_force_generic(force_generic)
+    try:
+        st = runner.PairStack(cfg, lengths, inp["blocks"][:1])
+        w_d, w_h = st.W[0], inp["blocks"][0]
+        x_d = runner.to_device(inp["x"], st.dtype)
+        L = st.L
+        worst = {}
+        sampled = sampled or {}
+        rng = np.random.default_rng(rng_seed)
+
+        # ---- nt_pair_broadcast
+        b = w_d["broadcast"]
+        nt.nt_pair_broadcast(L, x_d, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, st.z, st.workspace)
+        z0 = st.z.clone()
+        assert st.z.numel() == cfg.c_z * sum(n * n for n in lengths)
+        for s in full_samples:
+            n = lengths[s]
+            ref = orc.pair_broadcast(inp["x"][tok[s]:tok[s + 1]], (n,), **w_h["broadcast"])
+            worst["broadcast"] = max(worst.get("broadcast", 0), check(cfg.dtype, host(z0[po[s]:po[s + 1]]), ref,
+                                                                      f"broadcast s={s}", already_normalised=True))
+        for s, npos in sampled.items():
+            n = lengths[s]
+            xs = inp["x"][tok[s]:tok[s + 1]].astype(np.float64)
+            u = xs @ w_h["broadcast"]["W_a"].astype(np.float64).T
+            v = xs @ w_h["broadcast"]["W_b"].astype(np.float64).T
+            ii, jj = rng.integers(0, n, npos), rng.integers(0, n, npos)
+            ref = orc.layer_norm(u[ii] + v[jj], w_h["broadcast"]["ln_gamma"].astype(np.float64),
+                                 w_h["broadcast"]["ln_beta"].astype(np.float64))
+            got = host(z0[torch.as_tensor(po[s] + ii * n + jj, device=z0.device)])
+            check(cfg.dtype, got, ref, f"broadcast sampled s={s}", already_normalised=True)
+
+        # ---- nt_tri_mul_out
+        nt.nt_tri_mul_out(L, w_d["trimul"], 1e-5, st.z, st.workspace)
+        z1 = st.z.clone()
+        for s in full_samples:
+            n = lengths[s]
+            ref = orc.tri_mul_out(host(z0[po[s]:po[s + 1]]), (n,), w_h["trimul"])
+            worst["trimul"] = max(worst.get("trimul", 0), check(cfg.dtype, host(z1[po[s]:po[s + 1]]), ref, f"tri_mul s={s}"))
+        for s, npos in sampled.items():
+            n = lengths[s]
+            pos = [(int(a), int(b_)) for a, b_ in zip(rng.integers(0, n, npos), rng.integers(0, n, npos))]
+            pos += [(0, 0), (n - 1, n - 1), (0, n - 1)]
+            ref = orc.tri_mul_out_at(RowFetcher(z0, po[s], n), w_h["trimul"], pos)
+            got = host(z1[torch.as_tensor([po[s] + i * n + j for i, j in pos], device=z1.device)])
+            check(cfg.dtype, got, ref, f"tri_mul sampled s={s}")
+
+        # ---- nt_row_attn_pairbias
+        nt.nt_row_attn_pairbias(L, nt.NT_ORDER_PAIR_IJC, w_d["attn"], cfg.H, cfg.d, 1e-5, st.z, st.workspace)
+        z2 = st.z.clone()
+        for s in full_samples:
+            n = lengths[s]
+            ref = orc.row_attn_pairbias(host(z1[po[s]:po[s + 1]]), (n,), w_h["attn"], cfg.H, cfg.d)
+            worst["attn"] = max(worst.get("attn", 0), check(cfg.dtype, host(z2[po[s]:po[s + 1]]), ref, f"attn s={s}"))
+        for s, npos in sampled.items():
+            n = lengths[s]
+            pos = [(int(a), int(b_)) for a, b_ in zip(rng.integers(0, n, npos), rng.integers(0, n, npos))]
+            pos += [(0, 0), (n - 1, n - 1), (n - 1, 0)]
+            ref = orc.row_attn_pairbias_at(RowFetcher(z1, po[s], n), w_h["attn"], cfg.H, cfg.d, pos)
+            got = host(z2[torch.as_tensor([po[s] + i * n + j for i, j in pos], device=z2.device)])
+            check(cfg.dtype, got, ref, f"attn sampled s={s}")
+
+        # ---- nt_segment_reduce (mean over j back to the token axis) + token update
+        nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, st.z, st.m, L.status)
+        m_gpu = st.m.clone()
+        rows_checked = []
+        for s in list(full_samples) + list(sampled.keys()):
+            n = lengths[s]
+            if n == 0:
+                continue
+            sel = np.arange(n) if s in full_samples else np.unique(rng.integers(0, n, 8))
+            for i in sel:
+                a = po[s] + i * n
+                ref = orc.segment_reduce(host(z2[a:a + n]), [0, n], "mean")
+                check(cfg.dtype, host(m_gpu[tok[s] + i:tok[s] + i + 1]), ref, f"segment mean s={s} i={i}")
+                rows_checked.append(tok[s] + i)
+        x_before = x_d.clone()
+        nt.nt_token_update(st.m, w_d["reduce"]["W_r"], x_d)
+        ref = orc.token_update(host(x_before), host(m_gpu), w_h["reduce"]["W_r"])
+        check(cfg.dtype, host(x_d), ref, "token update")
+        assert L.device_status() == 0
+        torch.cuda.synchronize()
+        return worst
+    finally:
+        nt.nt_force_generic(prev)
+
+
+# ------------------------------------------------------------------------------------------------
+# offsets / decode: bit-exact
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("lengths", [(2, 3), (5, 9, 13, 16), (0, 3, 0, 0, 4, 1), (1,), (0, 0), (7, 7, 7),
+                                     tuple(wl.CONFIGS["cfg3"].lengths), tuple(range(1, 90))])
+def test_offsets_bit_exact(nt, lengths):
+    L = nt.Layout(lengths, with_maps=True)
+    ref = orc.offsets_build(lengths)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    assert np.array_equal(L.tok_off.cpu().numpy(), ref["tok_off"])
+    assert np.array_equal(L.pair_off.cpu().numpy(), ref["pair_off"])
+    assert np.array_equal(L.row_splits.cpu().numpy(), ref["row_splits"])
+    for got, key in ((L.pos_sample, "pos_sample"), (L.pos_i, "pos_i"), (L.pos_j, "pos_j"),
+                     (L.gather_rows, "rows"), (L.gather_cols, "cols")):
+        g = got.cpu().numpy()
+        assert g.dtype == ref[key].dtype and np.array_equal(g, ref[key]), key
+
+
+def test_offsets_empty_batch(nt):
+    L = nt.Layout((), with_maps=True)
+    assert L.tok_off.cpu().tolist() == [0] and L.pair_off.cpu().tolist() == [0]
+    assert L.row_splits.cpu().tolist() == [0] and L.device_status() == 0
+
+
+def test_offsets_large_sampled(nt):
+    cfg = wl.CONFIGS["cfg5"]
+    L = nt.Layout(cfg.lengths, with_maps=True)
+    tok, po, rs = orc.offsets_only(cfg.lengths)
+    assert L.T2 == 7_749_632
+    assert np.array_equal(L.tok_off.cpu().numpy(), tok) and np.array_equal(L.pair_off.cpu().numpy(), po)
+    assert np.array_equal(L.row_splits.cpu().numpy(), rs)
+    rng = np.random.default_rng(0)
+    ps = np.concatenate([rng.integers(0, L.T2, 4000), po[:-1], po[1:] - 1])
+    gs, gi, gj = (t.cpu().numpy() for t in (L.pos_sample, L.pos_i, L.pos_j))
+    gr, gc = L.gather_rows.cpu().numpy(), L.gather_cols.cpu().numpy()
+    for p in ps:
+        s, i, j = orc.decode_position(cfg.lengths, int(p))
+        assert (gs[p], gi[p], gj[p]) == (s, i, j)
+        assert gr[p] == tok[s] + i and gc[p] == tok[s] + j
+    # properties that hold at any size: the coordinate map inverts the decode everywhere
+    n = np.asarray(cfg.lengths, dtype=np.int64)
+    assert np.array_equal(po[gs] + gi.astype(np.int64) * n[gs] + gj, np.arange(L.T2))
+    assert np.all(gi < n[gs]) and np.all(gj < n[gs]) and np.all(gi >= 0) and np.all(gj >= 0)
+
+
+def test_offsets_device_detects_inconsistent_totals(nt):
+    lengths = torch.tensor([3, 4], dtype=torch.int64, device="cuda")
+    tok = torch.zeros(3, dtype=torch.int64, device="cuda")
+    po = torch.zeros(3, dtype=torch.int64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    nt.nt_offsets_build(lengths, 2, 7, 26, tok, po, status_d=status)      # true T2 is 25
+    assert int(status.item()) == 6
+    assert po.cpu().tolist() == [0, 9, 25]
+
+
+# ------------------------------------------------------------------------------------------------
+# per-call parity
+# ------------------------------------------------------------------------------------------------
+def test_cfg1_fp32_every_call(nt):
+    cfg = wl.CONFIGS["cfg1"]
+    inp = wl.make_inputs(cfg)
+    worst = run_block_teacher_forced(nt, cfg, inp, full_samples=range(cfg.B))
+    print("cfg1 worst error / bound:", worst)
+
+
+EDGE_LENGTHS = (1, 7, 17, 0, 33, 64, 65, 129, 2, 0)
+
+
+@pytest.mark.parametrize("dtype,generic", [("f32", False), ("bf16", False), ("bf16", True)])
+def test_edge_lengths_every_call(nt, dtype, generic):
+    cfg = wl.Config("edge", dtype, EDGE_LENGTHS, c_s=64, c_z=64, c_h=64, H=4, d=16, blocks=1, seed=77)
+    inp = wl.make_inputs(cfg)
+    run_block_teacher_forced(nt, cfg, inp, full_samples=range(cfg.B), force_generic=generic)
+
+
+def test_cfg2_bf16_every_call(nt):
+    cfg = wl.CONFIGS["cfg2"]
+    inp = wl.make_inputs(cfg)
+    worst = run_block_teacher_forced(nt, cfg, inp, full_samples=(0, 5), sampled={1: 24, 2: 24, 3: 24, 4: 24, 6: 24, 7: 24})
+    print("cfg2 worst abs error after LN:", worst)
+
+
+def test_cfg2_bf16_generic_kernels(nt):
+    cfg = wl.CONFIGS["cfg2"]
+    inp = wl.make_inputs(cfg)
+    run_block_teacher_forced(nt, cfg, inp, full_samples=(2,), sampled={7: 16}, force_generic=True)
+
+
+def test_cfg3_bf16_sampled(nt):
+    cfg = wl.CONFIGS["cfg3"]
+    inp = wl.make_inputs(cfg)
+    small = [s for s, n in enumerate(cfg.lengths) if n <= 130]
+    big = {s: 12 for s, n in enumerate(cfg.lengths) if n > 130}
+    run_block_teacher_forced(nt, cfg, inp, full_samples=small, sampled=big)
+
+
+def test_cfg5_bf16_sampled(nt):
+    cfg = wl.CONFIGS["cfg5"]
+    inp = wl.make_inputs(cfg)
+    run_block_teacher_forced(nt, cfg, inp, full_samples=(), sampled={0: 24, 1: 12, 2: 8, 3: 8})
+
+
+def test_cfg4_token_special_case(nt):
+    from paper_2609_30379_b200 import runner
+    cfg = wl.CONFIGS["cfg4"]
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    x_d = runner.to_device(inp["x"], st.dtype)
+    x_in = host(x_d)
+    x_out, pooled = st.forward(x_d)
+    ref_x = orc.row_attn_pairbias(x_in, cfg.lengths, inp["blocks"][0], cfg.H, cfg.d, order="token")
+    check("bf16", host(x_out), ref_x, "token attention")
+    tok, _, _ = orc.offsets_only(cfg.lengths)
+    ref_p = orc.segment_reduce(host(x_out), tok, "mean")
+    check("bf16", host(pooled), ref_p, "token pooled mean")
+    assert pooled.shape == (cfg.B, cfg.c_z)
+
+
+# ------------------------------------------------------------------------------------------------
+# whole stack, structure, determinism
+# ------------------------------------------------------------------------------------------------
+def test_cfg1_whole_block_end_to_end(nt):
+    from paper_2609_30379_b200 import runner
+    cfg = wl.CONFIGS["cfg1"]
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    x_d = runner.to_device(inp["x"], st.dtype)
+    x_out, z = st.forward(x_d)
+    rx, rz = orc.stack_forward(inp["x"], cfg.lengths, inp["blocks"], cfg.H, cfg.d)
+    check("f32", host(z), rz, "cfg1 z end to end")
+    check("f32", host(x_out), rx, "cfg1 x end to end")
+    assert z.shape == (531, 16)
+
+
+def test_two_block_stack_drift_bf16(nt):
+    from paper_2609_30379_b200 import runner
+    cfg = wl.Config("stack", "bf16", (40, 72, 9, 130), c_s=128, c_z=128, c_h=128, H=4, d=32, blocks=2, seed=5)
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    x_d = runner.to_device(inp["x"], st.dtype)
+    x_out, z = st.forward(x_d)
+    rx, rz = orc.stack_forward(inp["x"], cfg.lengths, inp["blocks"], cfg.H, cfg.d)
+    from tests.parity_utils import ln0
+    drift_z = float(np.abs(ln0(host(z)) - ln0(rz)).max())
+    drift_x = float(np.abs(ln0(host(x_out)) - ln0(rx)).max())
+    print(f"end-to-end drift over 2 blocks (no teacher forcing): z {drift_z:.4f}, x {drift_x:.4f}")
+    assert drift_z < 0.25 and drift_x < 0.25    # a loose guard; per-call parity is the gate
+
+
+def test_deterministic_and_sample_local(nt):
+    from paper_2609_30379_b200 import runner
+    cfg = wl.Config("det", "bf16", (33, 70, 12), c_s=64, c_z=128, c_h=128, H=4, d=32, blocks=1, seed=9)
+    inp = wl.make_inputs(cfg)
+    outs = []
+    for _ in range(2):
+        st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+        x_d = runner.to_device(inp["x"], st.dtype)
+        x_out, z = st.forward(x_d)
+        outs.append((x_out.clone(), z.clone()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    # a sample run alone gives the same result as inside the batch (sample-local semantics)
+    tok, po = offsets_np(cfg.lengths)
+    s = 1
+    st = runner.PairStack(cfg, (cfg.lengths[s],), inp["blocks"])
+    x_d = runner.to_device(inp["x"][tok[s]:tok[s + 1]], st.dtype)
+    x_alone, z_alone = st.forward(x_d)
+    check("bf16", host(z_alone), host(outs[0][1][po[s]:po[s + 1]]), "sample alone vs in batch (z)")
+    check("bf16", host(x_alone), host(outs[0][0][tok[s]:tok[s + 1]]), "sample alone vs in batch (x)")
+
+
+def test_outputs_stay_inside_packed_size(nt):
+    """Canary words after z: nothing may be written beyond sum N^2 * c_z elements."""
+    from paper_2609_30379_b200 import runner
+    cfg = wl.Config("canary", "bf16", (19, 37, 5), c_s=64, c_z=64, c_h=64, H=4, d=16, blocks=1, seed=3)
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    pad = 4096
+    big = torch.full((cfg.T2 * cfg.c_z + pad,), 1.5, dtype=st.dtype, device="cuda")
+    st.z = big[:cfg.T2 * cfg.c_z].view(cfg.T2, cfg.c_z)
+    x_d = runner.to_device(inp["x"], st.dtype)
+    st.forward(x_d)
+    torch.cuda.synchronize()
+    assert torch.all(big[cfg.T2 * cfg.c_z:] == 1.5)
+    assert torch.isfinite(st.z.float()).all()
+
+
+def test_segment_reduce_sum_and_empty_groups(nt):
+    rng = np.random.default_rng(2)
+    v = wl.round_to_bf16(rng.standard_normal((300, 64)).astype(np.float32))
+    splits = np.array([0, 0, 10, 10, 137, 300], dtype=np.int64)
+    for dt in (torch.float32, torch.bfloat16):
+        v_d = torch.from_numpy(v).to("cuda", dt)
+        sp = torch.from_numpy(splits).cuda()
+        for op, name in ((nt.NT_REDUCE_SUM, "sum"), (nt.NT_REDUCE_MEAN, "mean")):
+            out = torch.empty((5, 64), dtype=dt, device="cuda")
+            nt.nt_segment_reduce(op, sp, v_d, out)
+            ref = orc.segment_reduce(v, splits, name)
+            check("f32" if dt == torch.float32 else "bf16", host(out), ref, f"segment {name}")
+            assert torch.all(out[0] == 0) and torch.all(out[2] == 0)
+
+
+def test_launch_counter_counts_kernels(nt):
+    before = nt.nt_launch_count()
+    nt.Layout((3, 4))
+    assert nt.nt_launch_count() - before == 2     # scan + row splits
