@@ -236,8 +236,11 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       pa.W1 = W->W_b; pa.Nout = H; pa.out = w.bias; pa.out_mode = O_CHANNEL_MAJOR;
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
     }
-    r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
-                            (T*)w.o, H, d, pair ? 1 : 0, m, st);
+    if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d))
+      r = fast_attn_core(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, pair ? 1 : 0, m, st);
+    else
+      r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
+                              (T*)w.o, H, d, pair ? 1 : 0, m, st);
     if (r != NT_OK) return r;
     ProjArgs po{};
     po.A = w.o; po.a_mode = A_ROWMAJOR; po.row0 = row0; po.rows = rows; po.K = Hd;

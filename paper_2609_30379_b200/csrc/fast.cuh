@@ -13,4 +13,10 @@ bool fast_segment_reduce_supported(int C);
 nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,
                               cudaStream_t st);
 
+// attention core on tensor cores (bf16, d in {16, 32, 64}); q, k, v, o row-major [rows, H*d], bias
+// head-major channel-major (nullable)
+bool fast_attn_core_supported(int H, int d);
+nt_status fast_attn_core(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
+                         int pair_order, const BatchMeta& m, cudaStream_t st);
+
 }  // namespace ntp
