@@ -19,4 +19,10 @@ bool fast_attn_core_supported(int H, int d);
 nt_status fast_attn_core(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
                          int pair_order, const BatchMeta& m, cudaStream_t st);
 
+// triangle contraction on tcgen05: a, b, t are three equally spaced channel-major buffers
+// (b = a + stride, t = a + 2 * stride)
+bool fast_contract_supported(int C);
+nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
+                        cudaStream_t st);
+
 }  // namespace ntp

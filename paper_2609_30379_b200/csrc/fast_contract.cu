@@ -1,0 +1,237 @@
+// Triangle contraction t[c][i][j] = sum_k a[c][i][k] b[c][j][k] per (sample, channel) on the
+// tcgen05 tensor cores (bf16 operands, float accumulators in TMEM).
+//
+// Operands are the channel-major intermediates: for one (sample, channel) a and b are N x N
+// matrices with k contiguous (K-major for both MMA operands).  A persistent CTA per SM walks jobs
+// (sample, channel, 128-row block of i, up-to-256-column block of j) taken from the host lengths:
+//   warp 0   TMA producer: 64-wide k slabs of the a rows and b rows into a 3-stage ring
+//   warp 1   MMA issuer: 128 x Nt x 16 tcgen05.mma steps, accumulating into one of two TMEM buffers
+//   warps 2-5 epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store into t
+// One 4-D tensor map per sample {k, i, channel, which of a/b/t} serves loads and stores; rows and
+// columns past N are zero-filled on load and clipped on store, so no padded tile is ever moved.
+#include <cstring>
+
+#include "fast.cuh"
+#include "tc_common.cuh"
+
+namespace ntp {
+
+constexpr int CT_STAGES = 3;
+constexpr int CT_A_BYTES = 128 * 128;            // 128 rows x 64 bf16
+constexpr int CT_B_BYTES = 256 * 128;
+constexpr int CT_STAGE_BYTES = CT_A_BYTES + CT_B_BYTES;
+constexpr int CT_STAGING_BYTES = 4 * CT_A_BYTES; // 128 x 256 bf16 in four swizzled 64-column panels
+constexpr int CT_SMEM = CT_STAGES * CT_STAGE_BYTES + CT_STAGING_BYTES + 1024;
+constexpr int CT_THREADS = 192;
+constexpr int TMA_MAXB = 16;
+
+struct ContractParams {
+  CUtensorMap maps[TMA_MAXB];
+  long long job_off[TMA_MAXB + 1];
+  int N[TMA_MAXB];
+  int B, C;
+  int* status;
+};
+
+__device__ inline void contract_decode(const ContractParams& p, long long job, int& s, int& c, int& i0, int& j0,
+                                       int& Nt) {
+  s = 0;
+  while (s + 1 < p.B && job >= p.job_off[s + 1]) ++s;
+  const int N = p.N[s];
+  const int nib = (N + 127) / 128, njb = (N + 255) / 256;
+  long long r = job - p.job_off[s];
+  c = (int)(r / (nib * njb));
+  const int rem = (int)(r - (long long)c * nib * njb);
+  i0 = (rem / njb) * 128;
+  j0 = (rem % njb) * 256;
+  const int left = N - j0;
+  Nt = left >= 256 ? 256 : ((left + 15) & ~15);
+}
+
+__global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __grid_constant__ ContractParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[2 * CT_STAGES + 4];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_flag;
+  unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+  unsigned char* staging = smem + CT_STAGES * CT_STAGE_BYTES;
+  unsigned long long* full = bars;
+  unsigned long long* empty = bars + CT_STAGES;
+  unsigned long long* tfull = bars + 2 * CT_STAGES;
+  unsigned long long* tempty = bars + 2 * CT_STAGES + 2;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < CT_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 4); }
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_s, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_s;
+  AbortCtx ab{p.status, &abort_flag};
+  const long long njobs = p.job_off[p.B];
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long job = blockIdx.x; job < njobs; job += gridDim.x) {
+      int s, c, i0, j0, Nt;
+      contract_decode(p, job, s, c, i0, j0, Nt);
+      const int nkc = (p.N[s] + 63) / 64;
+      const CUtensorMap* map = &p.maps[s];
+      for (int kc = 0; kc < nkc; ++kc) {
+        mbar_wait(&empty[stage], phase ^ 1, ab);
+        unsigned char* As = smem + stage * CT_STAGE_BYTES;
+        unsigned char* Bs = As + CT_A_BYTES;
+        mbar_expect_tx(&full[stage], CT_A_BYTES + (Nt > 128 ? CT_B_BYTES : CT_B_BYTES / 2));
+        tma_load_4d(As, map, &full[stage], kc * 64, i0, c, 0);
+        tma_load_4d(Bs, map, &full[stage], kc * 64, j0, c, 1);
+        if (Nt > 128) tma_load_4d(Bs + CT_B_BYTES / 2, map, &full[stage], kc * 64, j0 + 128, c, 1);
+        if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0};
+    long long n = 0;
+    for (long long job = blockIdx.x; job < njobs; job += gridDim.x, ++n) {
+      int s, c, i0, j0, Nt;
+      contract_decode(p, job, s, c, i0, j0, Nt);
+      const int N = p.N[s];
+      const int nkc = (N + 63) / 64;
+      const int buf = (int)(n & 1);
+      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
+      tph[buf] ^= 1;
+      tc_fence_after();
+      const unsigned idesc = idesc_bf16(128, Nt, 0, 0);
+      const unsigned d_tmem = tmem_base + buf * 256;
+      for (int kc = 0; kc < nkc; ++kc) {
+        mbar_wait(&full[stage], phase, ab);
+        tc_fence_after();
+        const unsigned a_addr = smem_u32(smem + stage * CT_STAGE_BYTES);
+        const unsigned b_addr = a_addr + CT_A_BYTES;
+        const int ksteps = min(4, (N - kc * 64 + 15) / 16);
+        for (int k4 = 0; k4 < ksteps; ++k4)
+          umma_bf16(d_tmem, desc_kmajor_sw128(a_addr + k4 * 32), desc_kmajor_sw128(b_addr + k4 * 32), idesc,
+                    (kc | k4) != 0);
+        tc_commit(&empty[stage]);
+        if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
+      }
+      tc_commit(&tfull[buf]);
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int ep_tid = threadIdx.x - 64;
+    unsigned tph[2] = {0, 0};
+    long long n = 0;
+    for (long long job = blockIdx.x; job < njobs; job += gridDim.x, ++n) {
+      int s, c, i0, j0, Nt;
+      contract_decode(p, job, s, c, i0, j0, Nt);
+      const int buf = (int)(n & 1);
+      mbar_wait(&tfull[buf], tph[buf], ab);
+      tph[buf] ^= 1;
+      tc_fence_after();
+      if (n > 0) {                          // staging tile still being read by the previous store?
+        if (ep_tid == 0) tma_store_wait_read0();
+        named_bar_sync(1, 128);
+      }
+      const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
+      const int ncg = (Nt + 63) / 64;
+      for (int cg = 0; cg < ncg; ++cg) {
+        unsigned r0[32], r1[32];
+        tmem_ld32(taddr + cg * 64, r0);
+        tmem_ld32(taddr + cg * 64 + 32, r1);
+        tmem_ld_wait();
+        unsigned char* panel = staging + cg * CT_A_BYTES;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4 v;
+          v.x = pack2(r0[ch * 8 + 0], r0[ch * 8 + 1]);
+          v.y = pack2(r0[ch * 8 + 2], r0[ch * 8 + 3]);
+          v.z = pack2(r0[ch * 8 + 4], r0[ch * 8 + 5]);
+          v.w = pack2(r0[ch * 8 + 6], r0[ch * 8 + 7]);
+          *reinterpret_cast<uint4*>(panel + sw128_off(row, ch)) = v;
+        }
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4 v;
+          v.x = pack2(r1[ch * 8 + 0], r1[ch * 8 + 1]);
+          v.y = pack2(r1[ch * 8 + 2], r1[ch * 8 + 3]);
+          v.z = pack2(r1[ch * 8 + 4], r1[ch * 8 + 5]);
+          v.w = pack2(r1[ch * 8 + 6], r1[ch * 8 + 7]);
+          *reinterpret_cast<uint4*>(panel + sw128_off(row, 4 + ch)) = v;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+      fence_proxy_async_smem();
+      named_bar_sync(1, 128);
+      if (ep_tid == 0) {
+        for (int cg = 0; cg < ncg; ++cg)
+          tma_store_4d(&p.maps[s], staging + cg * CT_A_BYTES, j0 + cg * 64, i0, c, 2);
+        tma_store_commit();
+      }
+    }
+    if (ep_tid == 0) tma_store_wait_all0();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+bool fast_contract_supported(int C) { return C >= 1; }
+
+nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
+                        cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tri_contract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CT_SMEM) != cudaSuccess)
+      return NT_ERR_CUDA;
+    attr_set = true;
+  }
+  for (int g0 = 0; g0 < m.B; g0 += TMA_MAXB) {
+    ContractParams p;
+    p.B = m.B - g0 < TMA_MAXB ? m.B - g0 : TMA_MAXB;
+    p.C = C;
+    p.status = status;
+    p.job_off[0] = 0;
+    for (int l = 0; l < TMA_MAXB; ++l) {
+      const int N = l < p.B ? m.N[g0 + l] : 0;
+      p.N[l] = N;
+      const long long nib = (N + 127) / 128, njb = (N + 255) / 256;
+      p.job_off[l + 1] = p.job_off[l] + (long long)C * nib * njb;
+      if (l < p.B && N > 0) {
+        const int ld = round_up8(N);
+        const unsigned long long dims[4] = {(unsigned long long)N, (unsigned long long)N, (unsigned long long)C, 3};
+        const unsigned long long strides[3] = {(unsigned long long)ld * 2, (unsigned long long)N * ld * 2,
+                                               (unsigned long long)buf_stride_bytes};
+        const unsigned box[4] = {64, 128, 1, 1};
+        const char* base = (const char*)a + (size_t)C * m.cm_off[g0 + l] * 2;
+        if (!make_tmap_bf16(&p.maps[l], base, 4, dims, strides, box)) return NT_ERR_CUDA;
+      } else {
+        memset(&p.maps[l], 0, sizeof(CUtensorMap));
+      }
+    }
+    const long long njobs = p.job_off[p.B];
+    if (njobs == 0) continue;
+    const unsigned grid = (unsigned)(njobs < 148 ? njobs : 148);
+    {
+      LaunchScope ls("tri_contract", st);
+      tri_contract_kernel<<<grid, CT_THREADS, CT_SMEM, st>>>(p);
+    }
+    if (cudaGetLastError() != cudaSuccess) return NT_ERR_CUDA;
+  }
+  return NT_OK;
+}
+
+}  // namespace ntp

@@ -1,0 +1,180 @@
+// sm_100a building blocks for the tensor-core kernels: mbarrier with bounded waits, TMA tiled
+// loads / stores, tcgen05 MMA with shared-memory operand descriptors, TMEM allocation and loads.
+// Every wait has an iteration limit; on expiry the kernel records NT_ERR_TIMEOUT in the status
+// word, raises a CTA-wide abort flag (later waits give up after a short spin) and still runs to
+// its normal end, so TMEM is released and the context stays usable.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace ntp {
+
+// ---------------------------------------------------------------------------------- host: TMA maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_tiled();
+
+// bf16 tensor map with 128-byte swizzle; dims / strides fastest first (strides in bytes for dims 1..rank-1)
+bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+                    const unsigned long long* strides_bytes, const unsigned* box);
+
+#ifdef __CUDACC__
+// ---------------------------------------------------------------------------------- device helpers
+constexpr unsigned WAIT_LIMIT = 1u << 22;        // polls before a wait gives up (~ tens of ms)
+constexpr unsigned WAIT_LIMIT_ABORTED = 1u << 10;
+
+struct AbortCtx {
+  int* status;            // global status word (nullable)
+  volatile int* flag;     // CTA-shared abort flag
+};
+
+__device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(void* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ inline void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::); }
+__device__ inline void mbar_expect_tx(void* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ inline void mbar_arrive(void* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline bool mbar_try(void* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait; returns false (after flagging) if the limit was reached
+__device__ inline bool mbar_wait(void* bar, unsigned parity, const AbortCtx& ab) {
+  const unsigned limit = *ab.flag ? WAIT_LIMIT_ABORTED : WAIT_LIMIT;
+  for (unsigned it = 0; it < limit; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *ab.flag) break;
+  }
+  if (!*ab.flag) {
+    *ab.flag = 1;
+    if (ab.status) atomicCAS(ab.status, 0, (int)NT_ERR_TIMEOUT);
+  }
+  return false;
+}
+
+__device__ inline void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ inline void tma_load_4d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ inline void tma_store_2d(const CUtensorMap* map, const void* src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];\n"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ inline void tma_store_4d(const CUtensorMap* map, const void* src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];\n"
+               ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ inline void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+__device__ inline void tma_store_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;\n" ::: "memory"); }
+__device__ inline void tma_store_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;\n" ::: "memory"); }
+__device__ inline void tma_prefetch_map(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];\n" ::"l"(map) : "memory");
+}
+
+// ---- TMEM
+__device__ inline void tmem_alloc(unsigned* dst_smem, unsigned ncols) {   // whole warp
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(dst_smem)), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ inline void tmem_dealloc(unsigned taddr, unsigned ncols) {     // whole warp
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ inline void tc_commit(void* bar) {   // arrives on the mbarrier when all prior MMAs of this thread finish
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+
+// 32 lanes x 32 consecutive columns of 32-bit: thread t gets row (lane base + t), columns c..c+31
+__device__ inline void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+
+// ---- MMA descriptors (bf16 operands, float accumulate)
+// K-major operand tile in the 128-byte-swizzled layout TMA writes for a {64 elements, rows} box:
+// row r at r * 128 bytes, 16-byte chunks XOR-swizzled by (r & 7); groups of 8 rows are 1024 bytes
+// apart (stride byte offset).  The tile base must be 1024-byte aligned; advancing K by 16 elements
+// adds 32 bytes to the start address.
+__device__ inline unsigned long long desc_kmajor_sw128(unsigned saddr) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((saddr & 0x3FFFFu) >> 4);            // start address, bits [0,14)
+  d |= (unsigned long long)1 << 16;                              // leading byte offset (unused with swizzle)
+  d |= (unsigned long long)(1024 >> 4) << 32;                    // stride byte offset, bits [32,46)
+  d |= (unsigned long long)1 << 46;                              // descriptor version (Blackwell)
+  d |= (unsigned long long)2 << 61;                              // SWIZZLE_128B
+  return d;
+}
+// MN-major operand: 64 MN-elements (128 bytes) contiguous per K row, 8 K rows form a 1024-byte
+// swizzle atom; the next 64 MN-elements live `lbo` bytes further, the next 8 K rows `sbo` bytes further.
+__device__ inline unsigned long long desc_mnmajor_sw128(unsigned saddr, unsigned lbo, unsigned sbo) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((saddr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (unsigned long long)((sbo >> 4) & 0x3FFF) << 32;
+  d |= (unsigned long long)1 << 46;
+  d |= (unsigned long long)2 << 61;
+  return d;
+}
+// instruction descriptor: D = f32, A = B = bf16, M x N tile, operand majors (0 = K-major, 1 = MN-major)
+__device__ inline unsigned idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)a_mn_major << 15) | ((unsigned)b_mn_major << 16) |
+         ((unsigned)(N >> 3) << 17) | ((unsigned)(M >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem]; issued by one thread
+__device__ inline void umma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
+                                 unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ inline void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;\n" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// two floats (given as bit patterns) -> packed bf16x2, first in the low half
+__device__ inline unsigned pack2(unsigned lo, unsigned hi) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(lo), __uint_as_float(hi));
+  return *reinterpret_cast<unsigned*>(&h);
+}
+
+// byte offset of 16-byte chunk `chunk` of row `row` inside a 128-byte-swizzled tile
+__device__ inline unsigned sw128_off(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+#endif  // __CUDACC__
+
+}  // namespace ntp
