@@ -37,6 +37,12 @@ LaunchScope::~LaunchScope() {
   cudaEventRecord(g_prof[slot].e1, st);
 }
 
+nt_status cuda_fail(const char* where) {
+  const cudaError_t e = cudaGetLastError();   // also clears a non-sticky error
+  fprintf(stderr, "libnested_pair: CUDA failure at %s: %s\n", where, cudaGetErrorString(e));
+  return NT_ERR_CUDA;
+}
+
 void fill_meta(BatchMeta& m, const int64_t* len, int s0, int s1, long long tok0, long long pair0, long long cm0) {
   m.B = s1 - s0;
   m.tok_off[0] = tok0;
@@ -108,7 +114,7 @@ struct Carver {   // hands out 256-byte aligned slices of the caller's workspace
   }
 };
 
-struct TriWs { void *a, *b, *t, *g; size_t bytes; };
+struct TriWs { void *a, *b, *t, *g, *prep; size_t bytes; };
 static TriWs carve_trimul(void* ws, nt_dtype dt, const Totals& t, int c_z, int c_h) {
   Carver c(ws);
   TriWs w;
@@ -117,6 +123,7 @@ static TriWs carve_trimul(void* ws, nt_dtype dt, const Totals& t, int c_z, int c
   w.b = c.take((size_t)c_h * t.cm * e);
   w.t = c.take((size_t)c_h * t.cm * e);
   w.g = c.take((size_t)t.T2 * c_z * e);
+  w.prep = c.take(1 << 20);   // folded weights of the tensor-core projections
   w.bytes = c.off;
   return w;
 }
@@ -182,12 +189,19 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
     ProjArgs pa{};
     pa.A = z; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c_z;
     pa.ln_g = W->ln_in_gamma; pa.ln_b = W->ln_in_beta; pa.eps = eps;
-    pa.W1 = W->W_ag; pa.W2 = W->W_ap; pa.Nout = c_h; pa.out = w.a; pa.out_mode = O_CHANNEL_MAJOR;
-    nt_status r = launch_proj<T>(pa, m, st, "generic_tri_in_a");
-    if (r != NT_OK) return r;
-    pa.W1 = W->W_bg; pa.W2 = W->W_bp; pa.out = w.b;
-    r = launch_proj<T>(pa, m, st, "generic_tri_in_b");
-    if (r != NT_OK) return r;
+    nt_status r;
+    const bool tc = dt == NT_BF16 && !g_force_generic;
+    if (tc && fast_tri_in_supported(c_z, c_h)) {
+      r = fast_tri_in(z, W, eps, c_z, c_h, w.a, w.b, w.prep, m, L->status_d, st);
+      if (r != NT_OK) return r;
+    } else {
+      pa.W1 = W->W_ag; pa.W2 = W->W_ap; pa.Nout = c_h; pa.out = w.a; pa.out_mode = O_CHANNEL_MAJOR;
+      r = launch_proj<T>(pa, m, st, "generic_tri_in_a");
+      if (r != NT_OK) return r;
+      pa.W1 = W->W_bg; pa.W2 = W->W_bp; pa.out = w.b;
+      r = launch_proj<T>(pa, m, st, "generic_tri_in_b");
+      if (r != NT_OK) return r;
+    }
     pa.W1 = W->W_g; pa.W2 = nullptr; pa.act = ACT_SIGMOID; pa.Nout = c_z; pa.out = w.g; pa.out_mode = O_STORE;
     r = launch_proj<T>(pa, m, st, "generic_tri_in_g");
     if (r != NT_OK) return r;

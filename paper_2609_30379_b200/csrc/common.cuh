@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include <atomic>
 
@@ -63,7 +64,12 @@ struct LaunchScope {
   int slot;
 };
 
-inline nt_status cuda_ok() { return cudaGetLastError() == cudaSuccess ? NT_OK : NT_ERR_CUDA; }
+// Reports the pending CUDA error (and where it was seen) on stderr and maps it to NT_ERR_CUDA.
+nt_status cuda_fail(const char* where);
+
+inline nt_status cuda_ok(const char* where = "kernel launch") {
+  return cudaPeekAtLastError() == cudaSuccess ? NT_OK : cuda_fail(where);
+}
 
 // Builds the metadata of samples [s0, s1) (s1 - s0 <= MAXB) given absolute prefix arrays.
 void fill_meta(BatchMeta& m, const int64_t* lengths_h, int s0, int s1, long long tok0, long long pair0,

@@ -25,4 +25,13 @@ bool fast_contract_supported(int C);
 nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
                         cudaStream_t st);
 
+// triangle input projection on tcgen05 (LayerNorm folded into the weights); `prep` is scratch of
+// fast_tri_in_prep_bytes() for the folded weights
+bool fast_tri_in_supported(int c_z, int c_h);
+size_t fast_tri_in_prep_bytes(int c_z, int c_h);
+nt_status fast_tri_in(const void* z, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* a, void* b,
+                      void* prep, const BatchMeta& m, int* status, cudaStream_t st);
+nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
+                            const void* beta, void* out, void* c01, cudaStream_t st);
+
 }  // namespace ntp

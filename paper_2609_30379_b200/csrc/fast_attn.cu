@@ -349,7 +349,7 @@ static nt_status launch_attn_mma(const __nv_bfloat16* q, const __nv_bfloat16* k,
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_core_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) !=
         cudaSuccess)
-      return NT_ERR_CUDA;
+      return cuda_fail("shared memory attribute");
     attr_set = true;
   }
   {

@@ -196,7 +196,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(tri_contract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CT_SMEM) != cudaSuccess)
-      return NT_ERR_CUDA;
+      return cuda_fail("shared memory attribute");
     attr_set = true;
   }
   for (int g0 = 0; g0 < m.B; g0 += TMA_MAXB) {
@@ -217,7 +217,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
                                                (unsigned long long)buf_stride_bytes};
         const unsigned box[4] = {64, 128, 1, 1};
         const char* base = (const char*)a + (size_t)C * m.cm_off[g0 + l] * 2;
-        if (!make_tmap_bf16(&p.maps[l], base, 4, dims, strides, box)) return NT_ERR_CUDA;
+        if (!make_tmap_bf16(&p.maps[l], base, 4, dims, strides, box)) { fprintf(stderr, "libnested_pair: tensor map encode failed (%s:%d)\n", __FILE__, __LINE__); return NT_ERR_CUDA; }
       } else {
         memset(&p.maps[l], 0, sizeof(CUtensorMap));
       }
@@ -229,7 +229,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
       LaunchScope ls("tri_contract", st);
       tri_contract_kernel<<<grid, CT_THREADS, CT_SMEM, st>>>(p);
     }
-    if (cudaGetLastError() != cudaSuccess) return NT_ERR_CUDA;
+    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("tensor-core kernel launch");
   }
   return NT_OK;
 }
