@@ -202,14 +202,22 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
       r = launch_proj<T>(pa, m, st, "generic_tri_in_b");
       if (r != NT_OK) return r;
     }
-    pa.W1 = W->W_g; pa.W2 = nullptr; pa.act = ACT_SIGMOID; pa.Nout = c_z; pa.out = w.g; pa.out_mode = O_STORE;
-    r = launch_proj<T>(pa, m, st, "generic_tri_in_g");
-    if (r != NT_OK) return r;
-    if (dt == NT_BF16 && !g_force_generic && fast_contract_supported(c_h))
+    const bool tc_out = tc && fast_tri_out_supported(c_z, c_h);   // recomputes the output gate from z
+    if (!tc_out) {
+      pa.W1 = W->W_g; pa.W2 = nullptr; pa.act = ACT_SIGMOID; pa.Nout = c_z; pa.out = w.g; pa.out_mode = O_STORE;
+      r = launch_proj<T>(pa, m, st, "generic_tri_in_g");
+      if (r != NT_OK) return r;
+    }
+    if (tc && fast_contract_supported(c_h))
       r = fast_contract(w.a, (size_t)((char*)w.b - (char*)w.a), c_h, m, L->status_d, st);
     else
       r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st);
     if (r != NT_OK) return r;
+    if (tc_out) {
+      r = fast_tri_out(z, w.t, W, eps, c_z, c_h, (char*)w.prep + (512 << 10), m, L->status_d, st);
+      if (r != NT_OK) return r;
+      continue;
+    }
     ProjArgs po{};
     po.A = w.t; po.a_mode = A_CHANNEL_MAJOR; po.row0 = row0; po.rows = rows; po.K = c_h;
     po.ln_g = W->ln_out_gamma; po.ln_b = W->ln_out_beta; po.eps = eps;

@@ -34,4 +34,10 @@ nt_status fast_tri_in(const void* z, const nt_trimul_weights* W, float eps, int 
 nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
                             const void* beta, void* out, void* c01, cudaStream_t st);
 
+// triangle output stage on tcgen05, in place on z: z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T)
+bool fast_tri_out_supported(int c_z, int c_h);
+size_t fast_tri_out_prep_bytes(int c_z, int c_h);
+nt_status fast_tri_out(void* z, const void* t, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* prep,
+                       const BatchMeta& m, int* status, cudaStream_t st);
+
 }  // namespace ntp

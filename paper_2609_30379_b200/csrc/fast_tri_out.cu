@@ -1,0 +1,352 @@
+// Triangle-update output stage on tcgen05 (bf16, float accumulate), in place on the pair state:
+//   z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T)
+// t is the contraction result in channel-major layout (t[c][i][j], j contiguous), so a run of 64
+// positions of one pair row is, per channel, 128 contiguous bytes: exactly the MN-major operand
+// form of the MMA (positions are M, channels are K).  The output gate is recomputed here from z
+// instead of being stored by the input projection, which saves one write and one read of a
+// [T2, c_z] buffer.  Both LayerNorms are folded into the weights (see fast_tri_in.cu); the row
+// statistics come from the shared-memory tiles.
+//
+// A tile is two 64-position chunks (s, i, j0).  Per tile the producer brings the t chunk
+// [c_h][64] and the z chunk [64][c_z]; the MMA warp issues t^T W_o'^T and z W_g'^T into one TMEM
+// buffer; eight epilogue warps combine them with the residual, write the new z into the z tile in
+// shared memory and TMA-store it (clipped at the row end, so nothing outside sum N^2 is touched).
+#include <cstring>
+
+#include "fast.cuh"
+#include "tc_common.cuh"
+
+namespace ntp {
+
+constexpr int TO_THREADS = 64 + 256;
+constexpr int TO_MAXB = 12;
+
+struct TriOutParams {
+  CUtensorMap zmap[TO_MAXB];     // {c_z, N (j), N (i), 1}, box {64, 64, 1, 1}
+  CUtensorMap tmap[TO_MAXB];     // {N (j), N (i), c_h, 1}, box {64, 1, c_h, 1}
+  CUtensorMap womap;             // {c_h, c_z}, box {64, c_z}
+  CUtensorMap wgmap;             // {c_z, c_z}, box {64, c_z}
+  long long chunk_off[TO_MAXB + 1];
+  int N[TO_MAXB];
+  int B, c_z, c_h;
+  float eps;
+  const float2* c01o;            // [c_z]
+  const float2* c01g;            // [c_z]
+  int* status;
+};
+
+__device__ inline bool to_decode(const TriOutParams& p, long long q, int& s, int& i, int& j0) {
+  if (q >= p.chunk_off[p.B]) return false;
+  s = 0;
+  while (s + 1 < p.B && q >= p.chunk_off[s + 1]) ++s;
+  const int cpr = (p.N[s] + 63) / 64;
+  const long long r = q - p.chunk_off[s];
+  i = (int)(r / cpr);
+  j0 = (int)(r - (long long)i * cpr) * 64;
+  return true;
+}
+
+__device__ inline float sigmoid_fast2(float x) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(0.5f * x));
+  return fmaf(0.5f, t, 0.5f);
+}
+
+__global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_constant__ TriOutParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_flag;
+  unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+  const int c_z = p.c_z, c_h = p.c_h;
+  const int zslab = c_z / 64, hslab = c_h / 64;
+  const int wo_slab = c_z * 128, wg_slab = c_z * 128;        // one 64-wide K slab of [c_z rows]
+  const int wo_bytes = hslab * wo_slab, wg_bytes = zslab * wg_slab;
+  const int t_chunk = c_h * 128;                             // [c_h][64 positions]
+  const int z_slab = 128 * 128;                              // [128 positions][64 channels]
+  const int stage_bytes = 2 * t_chunk + zslab * z_slab;
+  unsigned char* sWo = smem;
+  unsigned char* sWg = sWo + wo_bytes;
+  unsigned char* sSt = sWg + wg_bytes;                       // 2 stages: t chunks then z slabs
+  float2* sCo = reinterpret_cast<float2*>(sSt + 2 * stage_bytes);
+  float2* sCg = sCo + c_z;
+  unsigned long long* afull = bars;
+  unsigned long long* aempty = bars + 2;
+  unsigned long long* tfull = bars + 4;
+  unsigned long long* tempty = bars + 6;
+  unsigned long long* wfull = bars + 8;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&afull[s], 1);
+      mbar_init(&aempty[s], 2);            // MMA commit + the storing epilogue thread
+      mbar_init(&tfull[s], 1);
+      mbar_init(&tempty[s], 8);
+    }
+    mbar_init(wfull, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_s, 512);
+  for (int n = threadIdx.x; n < c_z; n += TO_THREADS) {
+    sCo[n] = p.c01o[n];
+    sCg[n] = p.c01g[n];
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_s;
+  AbortCtx ab{p.status, &abort_flag};
+  const long long nchunks = p.chunk_off[p.B];
+  const long long ntiles = (nchunks + 1) / 2;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer
+    mbar_expect_tx(wfull, wo_bytes + wg_bytes);
+    for (int sl = 0; sl < hslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
+    for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&aempty[stage], phase ^ 1, ab);
+      const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
+      mbar_expect_tx(&afull[stage], nvalid * (t_chunk + zslab * 64 * 128));
+      unsigned char* st = sSt + stage * stage_bytes;
+      for (int q = 0; q < nvalid; ++q) {
+        int s, i, j0;
+        to_decode(p, 2 * t + q, s, i, j0);
+        tma_load_4d(st + q * t_chunk, &p.tmap[s], &afull[stage], j0, i, 0, 0);
+        for (int sl = 0; sl < zslab; ++sl)
+          tma_load_4d(st + 2 * t_chunk + sl * z_slab + q * 64 * 128, &p.zmap[s], &afull[stage], sl * 64, j0, i, 0);
+      }
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    mbar_wait(wfull, 0, ab);
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0};
+    long long n = 0;
+    const unsigned idesc_t = idesc_bf16(128, c_z, 1, 0);     // A = t, MN-major
+    const unsigned idesc_z = idesc_bf16(128, c_z, 0, 0);
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
+      const int buf = (int)(n & 1);
+      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
+      tph[buf] ^= 1;
+      mbar_wait(&afull[stage], phase, ab);
+      tc_fence_after();
+      const unsigned st = smem_u32(sSt + stage * stage_bytes);
+      const unsigned d1 = tmem_base + buf * 256, d2 = d1 + c_z;
+      for (int ks = 0; ks < c_h / 16; ++ks) {                // K = channels of t, 16 per step
+        const unsigned long long ad = desc_mnmajor_sw128(st + ks * 2048, t_chunk, 1024);
+        const unsigned long long bd = desc_kmajor_sw128(smem_u32(sWo) + (ks >> 2) * wo_slab + (ks & 3) * 32);
+        umma_bf16(d1, ad, bd, idesc_t, ks != 0);
+      }
+      for (int ks = 0; ks < c_z / 16; ++ks) {
+        const unsigned long long ad = desc_kmajor_sw128(st + 2 * t_chunk + (ks >> 2) * z_slab + (ks & 3) * 32);
+        const unsigned long long bd = desc_kmajor_sw128(smem_u32(sWg) + (ks >> 2) * wg_slab + (ks & 3) * 32);
+        umma_bf16(d2, ad, bd, idesc_z, ks != 0);
+      }
+      tc_commit(&tfull[buf]);
+      tc_commit(&aempty[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue (8 warps)
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int row = quarter * 32 + lane;           // position inside the tile
+    const int q = quarter >> 1;                    // chunk of this row
+    const int pos = (quarter & 1) * 32 + lane;     // position inside the chunk
+    const int ep_tid = threadIdx.x - 64;
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0};
+    long long n = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
+      const int buf = (int)(n & 1);
+      mbar_wait(&afull[stage], phase, ab);
+      unsigned char* st = sSt + stage * stage_bytes;
+      // statistics of t over channels (column of the MN-major tile) and of z over channels (row)
+      float ts = 0.f, tq = 0.f;
+      const unsigned char* tcol = st + q * t_chunk + (pos & 7) * 2;
+      for (int c = 0; c < c_h; ++c) {
+        const unsigned short hv = *reinterpret_cast<const unsigned short*>(tcol + c * 128 + (((pos >> 3) ^ (c & 7)) << 4));
+        const float v = __uint_as_float((unsigned)hv << 16);
+        ts += v;
+        tq = fmaf(v, v, tq);
+      }
+      float zs = 0.f, zq = 0.f;
+      unsigned char* zrow = st + 2 * t_chunk;
+      for (int sl = 0; sl < zslab; ++sl) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = *reinterpret_cast<const uint4*>(zrow + sl * z_slab + sw128_off(row, ch));
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            zs += lo + hi;
+            zq = fmaf(lo, lo, zq);
+            zq = fmaf(hi, hi, zq);
+          }
+        }
+      }
+      const float tmean = ts / (float)c_h;
+      const float trstd = rsqrtf(fmaxf(tq / (float)c_h - tmean * tmean, 0.f) + p.eps);
+      const float zmean = zs / (float)c_z;
+      const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
+      named_bar_sync(2, 256);                      // every row's statistics are taken before z is overwritten
+      mbar_wait(&tfull[buf], tph[buf], ab);
+      tph[buf] ^= 1;
+      tc_fence_after();
+      const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
+      for (int c0 = half * (c_z / 2); c0 < (half + 1) * (c_z / 2); c0 += 32) {
+        unsigned r1[32], r2[32];
+        tmem_ld32(taddr + c0, r1);
+        tmem_ld32(taddr + c_z + c0, r2);
+        tmem_ld_wait();
+        unsigned char* zp = zrow + (c0 >> 6) * z_slab;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int chunk16 = ((c0 & 63) >> 3) + ch;
+          uint4* ptr = reinterpret_cast<uint4*>(zp + sw128_off(row, chunk16));
+          uint4 v = *ptr;
+          unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int n0 = ch * 8 + e * 2;
+            float out[2];
+#pragma unroll
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const float2 ko = sCo[c0 + n0 + h2], kg = sCg[c0 + n0 + h2];
+              const float o = fmaf(trstd, __uint_as_float(r1[n0 + h2]) - tmean * ko.y, ko.x);
+              const float g = sigmoid_fast2(fmaf(zrstd, __uint_as_float(r2[n0 + h2]) - zmean * kg.y, kg.x));
+              const float zold = h2 == 0 ? __uint_as_float(w[e] << 16) : __uint_as_float(w[e] & 0xffff0000u);
+              out[h2] = fmaf(g, o, zold);
+            }
+            __nv_bfloat162 hh = __floats2bfloat162_rn(out[0], out[1]);
+            w[e] = *reinterpret_cast<unsigned*>(&hh);
+          }
+          *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+      fence_proxy_async_smem();
+      named_bar_sync(1, 256);
+      if (ep_tid == 0) {
+        const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
+        for (int qq = 0; qq < nvalid; ++qq) {
+          int s, i, j0;
+          to_decode(p, 2 * t + qq, s, i, j0);
+          for (int sl = 0; sl < zslab; ++sl)
+            tma_store_4d(&p.zmap[s], zrow + sl * z_slab + qq * 64 * 128, sl * 64, j0, i, 0);
+        }
+        tma_store_commit();
+        tma_store_wait_read0();
+        mbar_arrive(&aempty[stage]);
+      }
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+    if (ep_tid == 0) tma_store_wait_all0();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+bool fast_tri_out_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) && (c_h == 64 || c_h == 128); }
+
+size_t fast_tri_out_prep_bytes(int c_z, int c_h) {
+  return align_up((size_t)c_z * c_h * 2, 256) + align_up((size_t)c_z * c_z * 2, 256) +
+         2 * align_up((size_t)c_z * sizeof(float2), 256);
+}
+
+nt_status fast_tri_out(void* z, const void* t, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* prep,
+                       const BatchMeta& m, int* status, cudaStream_t st) {
+  char* pp = (char*)prep;
+  __nv_bfloat16* wo = (__nv_bfloat16*)pp;
+  pp += align_up((size_t)c_z * c_h * 2, 256);
+  __nv_bfloat16* wg = (__nv_bfloat16*)pp;
+  pp += align_up((size_t)c_z * c_z * 2, 256);
+  float2* c01o = (float2*)pp;
+  pp += align_up((size_t)c_z * sizeof(float2), 256);
+  float2* c01g = (float2*)pp;
+  {
+    const void* srcs[1] = {W->W_o};
+    const int rows[1] = {c_z};
+    nt_status r = fast_ln_fold_prep(srcs, rows, 1, c_h, W->ln_out_gamma, W->ln_out_beta, wo, c01o, st);
+    if (r != NT_OK) return r;
+    const void* srcs2[1] = {W->W_g};
+    r = fast_ln_fold_prep(srcs2, rows, 1, c_z, W->ln_in_gamma, W->ln_in_beta, wg, c01g, st);
+    if (r != NT_OK) return r;
+  }
+  const int zslab = c_z / 64, hslab = c_h / 64;
+  const size_t smem = (size_t)hslab * c_z * 128 + (size_t)zslab * c_z * 128 +
+                      2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 2 * c_z * 8 + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tri_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      return cuda_fail("tri_out smem attribute");
+    attr_set = true;
+  }
+  for (int g0 = 0; g0 < m.B; g0 += TO_MAXB) {
+    TriOutParams p;
+    memset(&p, 0, sizeof(p));
+    p.B = m.B - g0 < TO_MAXB ? m.B - g0 : TO_MAXB;
+    p.c_z = c_z;
+    p.c_h = c_h;
+    p.eps = eps;
+    p.c01o = c01o;
+    p.c01g = c01g;
+    p.status = status;
+    {
+      const unsigned long long dims[2] = {(unsigned long long)c_h, (unsigned long long)c_z};
+      const unsigned long long strides[1] = {(unsigned long long)c_h * 2};
+      const unsigned box[2] = {64, (unsigned)c_z};
+      if (!make_tmap_bf16(&p.womap, wo, 2, dims, strides, box)) return cuda_fail("tri_out W_o map");
+      const unsigned long long dims2[2] = {(unsigned long long)c_z, (unsigned long long)c_z};
+      const unsigned long long strides2[1] = {(unsigned long long)c_z * 2};
+      if (!make_tmap_bf16(&p.wgmap, wg, 2, dims2, strides2, box)) return cuda_fail("tri_out W_g map");
+    }
+    p.chunk_off[0] = 0;
+    for (int l = 0; l < TO_MAXB; ++l) {
+      const int N = l < p.B ? m.N[g0 + l] : 0;
+      p.N[l] = N;
+      p.chunk_off[l + 1] = p.chunk_off[l] + (long long)N * ((N + 63) / 64);
+      if (N > 0) {
+        const int ld = round_up8(N);
+        {
+          const unsigned long long dims[4] = {(unsigned long long)c_z, (unsigned long long)N, (unsigned long long)N, 1};
+          const unsigned long long strides[3] = {(unsigned long long)c_z * 2, (unsigned long long)N * c_z * 2,
+                                                 (unsigned long long)N * N * c_z * 2};
+          const unsigned box[4] = {64, 64, 1, 1};
+          const char* base = (const char*)z + (size_t)m.pair_off[g0 + l] * c_z * 2;
+          if (!make_tmap_bf16(&p.zmap[l], base, 4, dims, strides, box)) return cuda_fail("tri_out z map");
+        }
+        {
+          const unsigned long long dims[4] = {(unsigned long long)N, (unsigned long long)N, (unsigned long long)c_h, 1};
+          const unsigned long long strides[3] = {(unsigned long long)ld * 2, (unsigned long long)N * ld * 2,
+                                                 (unsigned long long)c_h * N * ld * 2};
+          const unsigned box[4] = {64, 1, (unsigned)c_h, 1};
+          const char* base = (const char*)t + (size_t)c_h * m.cm_off[g0 + l] * 2;
+          if (!make_tmap_bf16(&p.tmap[l], base, 4, dims, strides, box)) return cuda_fail("tri_out t map");
+        }
+      }
+    }
+    const long long ntiles = (p.chunk_off[p.B] + 1) / 2;
+    if (ntiles == 0) continue;
+    const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);
+    {
+      LaunchScope ls("tri_out", st);
+      tri_out_kernel<<<grid, TO_THREADS, smem, st>>>(p);
+    }
+    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("tri_out launch");
+  }
+  return NT_OK;
+}
+
+}  // namespace ntp
