@@ -128,7 +128,7 @@ static TriWs carve_trimul(void* ws, nt_dtype dt, const Totals& t, int c_z, int c
   return w;
 }
 
-struct AttnWs { void *q, *k, *v, *o, *g, *bias; size_t bytes; };
+struct AttnWs { void *q, *k, *v, *o, *g, *bias, *prep; size_t bytes; };
 static AttnWs carve_attn(void* ws, nt_dtype dt, const Totals& t, nt_order order, int H, int d) {
   Carver c(ws);
   AttnWs w;
@@ -141,6 +141,7 @@ static AttnWs carve_attn(void* ws, nt_dtype dt, const Totals& t, nt_order order,
   w.o = c.take(rows * Hd * e);
   w.g = c.take(rows * Hd * e);
   w.bias = c.take(order == NT_ORDER_PAIR_IJC ? (size_t)H * t.cm * e : 0);
+  w.prep = c.take(1 << 20);   // folded weights of the tensor-core projections
   w.bytes = c.off;
   return w;
 }
@@ -246,18 +247,26 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
     pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = eps;
     pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
     nt_status r;
-    pa.W1 = W->W_q; pa.out = w.q;
-    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_q")) != NT_OK) return r;
-    pa.W1 = W->W_k; pa.out = w.k;
-    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_k")) != NT_OK) return r;
-    pa.W1 = W->W_v; pa.out = w.v;
-    if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_v")) != NT_OK) return r;
-    if (W->W_g) {
-      pa.W1 = W->W_g; pa.out = w.g; pa.act = ACT_SIGMOID;
+    const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma;
+    const bool tc_in = tc && fast_attn_in_supported(c, H, d);
+    const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
+    if (tc_in) {
+      r = fast_attn_in(zx, W, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.prep, m, L->status_d, st);
+      if (r != NT_OK) return r;
+    } else {
+      pa.W1 = W->W_q; pa.out = w.q;
+      if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_q")) != NT_OK) return r;
+      pa.W1 = W->W_k; pa.out = w.k;
+      if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_k")) != NT_OK) return r;
+      pa.W1 = W->W_v; pa.out = w.v;
+      if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_v")) != NT_OK) return r;
+    }
+    if (W->W_g && !tc_out) {
+      pa.W1 = W->W_g; pa.out = w.g; pa.act = ACT_SIGMOID; pa.Nout = Hd; pa.out_mode = O_STORE;
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_g")) != NT_OK) return r;
       pa.act = ACT_NONE;
     }
-    if (W->W_b) {
+    if (W->W_b && !tc_in) {
       pa.W1 = W->W_b; pa.Nout = H; pa.out = w.bias; pa.out_mode = O_CHANNEL_MAJOR;
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
     }
@@ -267,6 +276,11 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
                               (T*)w.o, H, d, pair ? 1 : 0, m, st);
     if (r != NT_OK) return r;
+    if (tc_out) {
+      r = fast_attn_out(zx, w.o, W, eps, c, H, d, (char*)w.prep + (512 << 10), m, L->status_d, st);
+      if (r != NT_OK) return r;
+      continue;
+    }
     ProjArgs po{};
     po.A = w.o; po.a_mode = A_ROWMAJOR; po.row0 = row0; po.rows = rows; po.K = Hd;
     po.gateA = W->W_g ? w.g : nullptr;

@@ -34,6 +34,16 @@ nt_status fast_tri_in(const void* z, const nt_trimul_weights* W, float eps, int 
 nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
                             const void* beta, void* out, void* c01, cudaStream_t st);
 
+// attention input projection on tcgen05: q, k, v row-major, bias head-major (nullable)
+bool fast_attn_in_supported(int c, int H, int d);
+nt_status fast_attn_in(const void* z, const nt_attn_weights* W, float eps, int c, int H, int d, void* q, void* k,
+                       void* v, void* bias, void* prep, const BatchMeta& m, int* status, cudaStream_t st);
+
+// attention output stage on tcgen05, in place on z: z += (sigmoid(LN(z) W_g^T) * o) W_o^T
+bool fast_attn_out_supported(int c, int H, int d);
+nt_status fast_attn_out(void* z, const void* o, const nt_attn_weights* W, float eps, int c, int H, int d, void* prep,
+                        const BatchMeta& m, int* status, cudaStream_t st);
+
 // triangle output stage on tcgen05, in place on z: z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T)
 bool fast_tri_out_supported(int c_z, int c_h);
 size_t fast_tri_out_prep_bytes(int c_z, int c_h);

@@ -1,0 +1,332 @@
+// Attention input projection on tcgen05 (bf16, float accumulate):
+//   zh = LN(z);  q, k, v = zh W_{q,k,v}^T  (row-major [T2, H d]);  bias = zh W_b^T  (head-major, channel-major)
+// LayerNorm is folded into the weights (see fast_tri_in.cu).  The gate sigmoid(zh W_g^T) is not
+// produced here: the output projection recomputes it from z, which saves a [T2, H d] write and read.
+//
+// Tiles are 128 consecutive packed positions (the outputs are row-major, so no row alignment is
+// needed); the (3 H d + 16) x c_z weights stay resident in shared memory.  Accumulator units per
+// tile: [q | k], [v], [bias padded to 16 columns].  Eight epilogue warps apply the LayerNorm
+// correction, stage each output as swizzled 64-channel panels and TMA-store them; the bias values
+// are scattered per head as 2-byte stores that coalesce across the warp (consecutive k of a row).
+#include <cstring>
+
+#include "fast.cuh"
+#include "tc_common.cuh"
+
+namespace ntp {
+
+constexpr int AI_THREADS = 64 + 256;
+constexpr int AI_MAXB = 16;
+
+struct AttnInParams {
+  CUtensorMap zmap;              // {c, rows}, box {64, 128}
+  CUtensorMap wmap;              // {c, 3 Hd + 16}, box {64, 128} (q, k, v rows)
+  CUtensorMap wbmap;             // same tensor, box {64, 16} (bias rows)
+  CUtensorMap omap[3];           // q, k, v: {Hd, rows}, box {64, 128}
+  long long pair_off[AI_MAXB + 1];   // relative to the first position of the group
+  long long cm_off[AI_MAXB];
+  int N[AI_MAXB];
+  int B, c, H, Hd;
+  long long rows;                // positions in the group
+  float eps;
+  const float2* c01;             // [3 Hd + 16]
+  __nv_bfloat16* bias;           // nullable
+  int* status;
+};
+
+__global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_constant__ AttnInParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_flag;
+  unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+  const int c = p.c, Hd = p.Hd;
+  const int nslab = c / 64;
+  const int wrows = 3 * Hd + 16;
+  const int w_slab = wrows * 128;
+  const int a_slab = 128 * 128;
+  const int a_stage = nslab * a_slab;
+  const int npanel = Hd / 64 > 0 ? Hd / 64 : 1;
+  unsigned char* sW = smem;
+  unsigned char* sA = sW + nslab * w_slab;               // 2 stages
+  unsigned char* sOut = sA + 2 * a_stage;                // npanel panels of [128][64]
+  float2* sC = reinterpret_cast<float2*>(sOut + npanel * a_slab);
+  unsigned long long* afull = bars;
+  unsigned long long* aempty = bars + 2;
+  unsigned long long* tfull = bars + 4;
+  unsigned long long* tempty = bars + 6;
+  unsigned long long* wfull = bars + 8;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&afull[s], 1);
+      mbar_init(&aempty[s], 1 + 8);
+      mbar_init(&tfull[s], 1);
+      mbar_init(&tempty[s], 8);
+    }
+    mbar_init(wfull, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_s, 512);
+  for (int n = threadIdx.x; n < wrows; n += AI_THREADS) sC[n] = p.c01[n];
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_s;
+  AbortCtx ab{p.status, &abort_flag};
+  const long long ntiles = (p.rows + 127) / 128;
+  const int nunits = p.bias ? 3 : 2;
+  // unit u: weight row offset and accumulator width
+  const int u_row[3] = {0, 2 * Hd, 3 * Hd};
+  const int u_n[3] = {2 * Hd, Hd, 16};
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer
+    mbar_expect_tx(wfull, nslab * w_slab);
+    for (int sl = 0; sl < nslab; ++sl) {
+      for (int rb = 0; rb < 3 * Hd / 128; ++rb)
+        tma_load_2d(sW + sl * w_slab + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
+      if ((3 * Hd) % 128) {   // H d = 64: rows 128..191 via a second 128-row box would overrun; use 16-row boxes
+        for (int r16 = (3 * Hd / 128) * 128; r16 < 3 * Hd; r16 += 16)
+          tma_load_2d(sW + sl * w_slab + r16 * 128, &p.wbmap, wfull, sl * 64, r16);
+      }
+      tma_load_2d(sW + sl * w_slab + 3 * Hd * 128, &p.wbmap, wfull, sl * 64, 3 * Hd);
+    }
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&aempty[stage], phase ^ 1, ab);
+      mbar_expect_tx(&afull[stage], a_stage);
+      for (int sl = 0; sl < nslab; ++sl)
+        tma_load_2d(sA + stage * a_stage + sl * a_slab, &p.zmap, &afull[stage], sl * 64, (int)(t * 128));
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    mbar_wait(wfull, 0, ab);
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0};
+    long long unit = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      tc_fence_after();
+      const unsigned a_addr = smem_u32(sA + stage * a_stage);
+      for (int u = 0; u < nunits; ++u, ++unit) {
+        const int buf = (int)(unit & 1);
+        mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
+        tph[buf] ^= 1;
+        tc_fence_after();
+        const unsigned idesc = idesc_bf16(128, u_n[u], 0, 0);
+        const unsigned d_tmem = tmem_base + buf * 256;
+        for (int sl = 0; sl < nslab; ++sl) {
+          const unsigned w_addr = smem_u32(sW + sl * w_slab + u_row[u] * 128);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            umma_bf16(d_tmem, desc_kmajor_sw128(a_addr + sl * a_slab + k4 * 32), desc_kmajor_sw128(w_addr + k4 * 32),
+                      idesc, (sl | k4) != 0);
+        }
+        tc_commit(&tfull[buf]);
+      }
+      tc_commit(&aempty[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue (8 warps)
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int row = quarter * 32 + lane;
+    const int ep_tid = threadIdx.x - 64;
+    const int cpw = Hd / 2;                         // channels of one output handled by this warp
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0};
+    long long unit = 0;
+    bool store_pending = false;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      float sum = 0.f, sq = 0.f;
+      const unsigned char* arow = sA + stage * a_stage;
+      for (int sl = 0; sl < nslab; ++sl) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = *reinterpret_cast<const uint4*>(arow + sl * a_slab + sw128_off(row, ch));
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            sum += lo + hi;
+            sq = fmaf(lo, lo, sq);
+            sq = fmaf(hi, hi, sq);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&aempty[stage]);
+      const float mean = sum / (float)c;
+      const float rstd = rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps);
+      for (int u = 0; u < nunits; ++u, ++unit) {
+        const int buf = (int)(unit & 1);
+        mbar_wait(&tfull[buf], tph[buf], ab);
+        tph[buf] ^= 1;
+        tc_fence_after();
+        const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
+        if (u < 2) {
+          const int nout = u == 0 ? 2 : 1;
+          for (int oi = 0; oi < nout; ++oi) {
+            const int o = u == 0 ? oi : 2;          // 0 = q, 1 = k, 2 = v
+            if (store_pending) {                    // previous output still being read from the panels?
+              if (ep_tid == 0) tma_store_wait_read0();
+              named_bar_sync(1, 256);
+            }
+            const float2* cc = sC + o * Hd;
+            for (int c0 = half * cpw; c0 < (half + 1) * cpw; c0 += 32) {
+              unsigned r[32];
+              tmem_ld32(taddr + oi * Hd + c0, r);
+              tmem_ld_wait();
+              unsigned char* panel = sOut + (c0 >> 6) * a_slab;
+#pragma unroll
+              for (int ch = 0; ch < 4; ++ch) {
+                unsigned w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const int n0 = ch * 8 + e * 2;
+                  const float2 k0 = cc[c0 + n0], k1 = cc[c0 + n0 + 1];
+                  const float x0 = fmaf(rstd, __uint_as_float(r[n0]) - mean * k0.y, k0.x);
+                  const float x1 = fmaf(rstd, __uint_as_float(r[n0 + 1]) - mean * k1.y, k1.x);
+                  __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                  w[e] = *reinterpret_cast<unsigned*>(&hh);
+                }
+                *reinterpret_cast<uint4*>(panel + sw128_off(row, ((c0 & 63) >> 3) + ch)) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+            fence_proxy_async_smem();
+            named_bar_sync(1, 256);
+            if (ep_tid == 0) {
+              for (int pn = 0; pn < npanel; ++pn)
+                tma_store_2d(&p.omap[o], sOut + pn * a_slab, pn * 64, (int)(t * 128));
+              tma_store_commit();
+            }
+            store_pending = true;
+          }
+        } else if (half == 0) {
+          // bias: H values per position, written head-major / channel-major
+          unsigned r[32];
+          tmem_ld32(taddr, r);
+          tmem_ld_wait();
+          const long long P = t * 128 + row;
+          if (P < p.rows) {
+            int s = 0;
+            while (s + 1 < p.B && P >= p.pair_off[s + 1]) ++s;
+            const int N = p.N[s], ld = round_up8(N);
+            const long long rr = P - p.pair_off[s];
+            const long long i = rr / N, j = rr - i * N;
+            __nv_bfloat16* bp = p.bias + (long long)p.H * p.cm_off[s] + i * ld + j;
+            const float2* cc = sC + 3 * Hd;
+            for (int h = 0; h < p.H; ++h) {
+              const float x = fmaf(rstd, __uint_as_float(r[h]) - mean * cc[h].y, cc[h].x);
+              bp[(long long)h * N * ld] = __float2bfloat16_rn(x);
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[buf]);
+      }
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+    if (ep_tid == 0) tma_store_wait_all0();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+bool fast_attn_in_supported(int c, int H, int d) {
+  const int Hd = H * d;
+  return (c == 64 || c == 128) && (Hd == 64 || Hd == 128) && H <= 16;
+}
+
+size_t fast_attn_in_prep_bytes(int c, int H, int d) {
+  const int wrows = 3 * H * d + 16;
+  return align_up((size_t)wrows * c * 2, 256) + align_up((size_t)wrows * sizeof(float2), 256) + 256;
+}
+
+nt_status fast_attn_in(const void* z, const nt_attn_weights* W, float eps, int c, int H, int d, void* q, void* k,
+                       void* v, void* bias, void* prep, const BatchMeta& m, int* status, cudaStream_t st) {
+  const int Hd = H * d;
+  const int wrows = 3 * Hd + 16;
+  __nv_bfloat16* wprime = (__nv_bfloat16*)prep;
+  float2* c01 = (float2*)((char*)prep + align_up((size_t)wrows * c * 2, 256));
+  __nv_bfloat16* zero_rows = (__nv_bfloat16*)((char*)c01 + align_up((size_t)wrows * sizeof(float2), 256));
+  (void)zero_rows;
+  // rows: W_q, W_k, W_v, W_b (H rows), then 16 - H rows that must be zero: clear the tail first
+  if (cudaMemsetAsync((char*)wprime + (size_t)3 * Hd * c * 2, 0, (size_t)16 * c * 2, st) != cudaSuccess)
+    return cuda_fail("attn_in memset");
+  if (cudaMemsetAsync(c01 + 3 * Hd, 0, 16 * sizeof(float2), st) != cudaSuccess) return cuda_fail("attn_in memset");
+  const void* srcs[4] = {W->W_q, W->W_k, W->W_v, W->W_b};
+  const int rows[4] = {Hd, Hd, Hd, H};
+  nt_status r = fast_ln_fold_prep(srcs, rows, W->W_b ? 4 : 3, c, W->ln_gamma, W->ln_beta, wprime, c01, st);
+  if (r != NT_OK) return r;
+  const int nslab = c / 64;
+  const int npanel = Hd / 64;
+  const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)nslab * 128 * 128 + (size_t)npanel * 128 * 128 +
+                      (size_t)wrows * 8 + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      return cuda_fail("attn_in smem attribute");
+    attr_set = true;
+  }
+  for (int g0 = 0; g0 < m.B; g0 += AI_MAXB) {
+    AttnInParams p;
+    memset(&p, 0, sizeof(p));
+    p.B = m.B - g0 < AI_MAXB ? m.B - g0 : AI_MAXB;
+    p.c = c;
+    p.H = H;
+    p.Hd = Hd;
+    p.eps = eps;
+    p.c01 = c01;
+    p.bias = (__nv_bfloat16*)bias;
+    p.status = status;
+    const long long P0 = m.pair_off[g0];
+    p.pair_off[0] = 0;
+    for (int l = 0; l < AI_MAXB; ++l) {
+      const int N = l < p.B ? m.N[g0 + l] : 0;
+      p.N[l] = N;
+      p.cm_off[l] = l < p.B ? m.cm_off[g0 + l] : 0;
+      p.pair_off[l + 1] = p.pair_off[l] + (long long)N * N;
+    }
+    p.rows = p.pair_off[p.B];
+    if (p.rows == 0) continue;
+    if (p.rows > 0x7FFFFF00ll) return NT_ERR_UNSUPPORTED;
+    {
+      const unsigned long long dims[2] = {(unsigned long long)c, (unsigned long long)p.rows};
+      const unsigned long long strides[1] = {(unsigned long long)c * 2};
+      const unsigned box[2] = {64, 128};
+      if (!make_tmap_bf16(&p.zmap, (const char*)z + (size_t)P0 * c * 2, 2, dims, strides, box))
+        return cuda_fail("attn_in z map");
+      const unsigned long long wdims[2] = {(unsigned long long)c, (unsigned long long)wrows};
+      if (!make_tmap_bf16(&p.wmap, wprime, 2, wdims, strides, box)) return cuda_fail("attn_in w map");
+      const unsigned bbox[2] = {64, 16};
+      if (!make_tmap_bf16(&p.wbmap, wprime, 2, wdims, strides, bbox)) return cuda_fail("attn_in wb map");
+      const unsigned long long odims[2] = {(unsigned long long)Hd, (unsigned long long)p.rows};
+      const unsigned long long ostr[1] = {(unsigned long long)Hd * 2};
+      void* outs[3] = {q, k, v};
+      for (int o = 0; o < 3; ++o)
+        if (!make_tmap_bf16(&p.omap[o], (char*)outs[o] + (size_t)P0 * Hd * 2, 2, odims, ostr, box))
+          return cuda_fail("attn_in out map");
+    }
+    const long long ntiles = (p.rows + 127) / 128;
+    const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);
+    {
+      LaunchScope ls("attn_in", st);
+      attn_in_kernel<<<grid, AI_THREADS, smem, st>>>(p);
+    }
+    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("attn_in launch");
+  }
+  return NT_OK;
+}
+
+}  // namespace ntp

@@ -1,0 +1,300 @@
+// Attention output stage on tcgen05 (bf16, float accumulate), in place on the pair state:
+//   z += (sigmoid(LN(z) W_g^T) * o) W_o^T
+// The gate is recomputed from z here (LayerNorm folded into W_g, see fast_tri_in.cu) instead of
+// being written by the input projection.  Per 128-position tile: TMA brings the z tile and the o
+// tile; the MMA warp computes the gate pre-activation into TMEM; the epilogue warps turn it into
+// sigmoid(.) * o, written back over the o tile in shared memory; the MMA warp multiplies that by
+// W_o; the epilogue adds the residual into the z tile and TMA-stores it.
+#include <cstring>
+
+#include "fast.cuh"
+#include "tc_common.cuh"
+
+namespace ntp {
+
+constexpr int AO_THREADS = 64 + 256;
+
+struct AttnOutParams {
+  CUtensorMap zmap;              // {c, rows}, box {64, 128}: load and store
+  CUtensorMap omap;              // {Hd, rows}, box {64, 128}
+  CUtensorMap wgmap;             // {c, Hd}, box {64, Hd}
+  CUtensorMap womap;             // {Hd, c}, box {64, c}
+  int c, Hd;
+  long long rows;
+  float eps;
+  const float2* c01g;            // [Hd]
+  int* status;
+};
+
+__device__ inline float sigmoid_fast3(float x) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(0.5f * x));
+  return fmaf(0.5f, t, 0.5f);
+}
+
+__global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_constant__ AttnOutParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[13];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_flag;
+  unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+  const int c = p.c, Hd = p.Hd;
+  const int zslab = c / 64, oslab = Hd / 64;
+  const int slab = 128 * 128;
+  const int wg_slab = Hd * 128, wo_slab = c * 128;
+  const int stage_bytes = (zslab + oslab) * slab;
+  unsigned char* sWg = smem;                          // zslab slabs of [Hd rows][64]
+  unsigned char* sWo = sWg + zslab * wg_slab;         // oslab slabs of [c rows][64]
+  unsigned char* sSt = sWo + oslab * wo_slab;         // 2 stages: z slabs then o slabs
+  float2* sC = reinterpret_cast<float2*>(sSt + 2 * stage_bytes);
+  unsigned long long* afull = bars;        // [2]
+  unsigned long long* aempty = bars + 2;   // [2]
+  unsigned long long* gfull = bars + 4;    // [2]
+  unsigned long long* ogated = bars + 6;   // [2]
+  unsigned long long* ofull = bars + 8;    // [2]
+  unsigned long long* tempty = bars + 10;  // [2]
+  unsigned long long* wfull = bars + 12;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&afull[s], 1);
+      mbar_init(&aempty[s], 2);
+      mbar_init(&gfull[s], 1);
+      mbar_init(&ogated[s], 8);
+      mbar_init(&ofull[s], 1);
+      mbar_init(&tempty[s], 8);
+    }
+    mbar_init(wfull, 1);
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_s, 512);
+  for (int n = threadIdx.x; n < Hd; n += AO_THREADS) sC[n] = p.c01g[n];
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_s;
+  AbortCtx ab{p.status, &abort_flag};
+  const long long ntiles = (p.rows + 127) / 128;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------------------------------------------ producer
+    mbar_expect_tx(wfull, zslab * wg_slab + oslab * wo_slab);
+    for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
+    for (int sl = 0; sl < oslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&aempty[stage], phase ^ 1, ab);
+      mbar_expect_tx(&afull[stage], stage_bytes);
+      unsigned char* st = sSt + stage * stage_bytes;
+      for (int sl = 0; sl < zslab; ++sl) tma_load_2d(st + sl * slab, &p.zmap, &afull[stage], sl * 64, (int)(t * 128));
+      for (int sl = 0; sl < oslab; ++sl)
+        tma_load_2d(st + (zslab + sl) * slab, &p.omap, &afull[stage], sl * 64, (int)(t * 128));
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    mbar_wait(wfull, 0, ab);
+    int stage = 0;
+    unsigned phase = 0, tph[2] = {0, 0}, gph[2] = {0, 0};
+    long long n = 0;
+    const unsigned idesc_g = idesc_bf16(128, Hd, 0, 0);
+    const unsigned idesc_o = idesc_bf16(128, c, 0, 0);
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
+      const int buf = (int)(n & 1);
+      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
+      tph[buf] ^= 1;
+      mbar_wait(&afull[stage], phase, ab);
+      tc_fence_after();
+      const unsigned st = smem_u32(sSt + stage * stage_bytes);
+      const unsigned dg = tmem_base + buf * 256, dout = dg + Hd;
+      for (int ks = 0; ks < c / 16; ++ks)
+        umma_bf16(dg, desc_kmajor_sw128(st + (ks >> 2) * slab + (ks & 3) * 32),
+                  desc_kmajor_sw128(smem_u32(sWg) + (ks >> 2) * wg_slab + (ks & 3) * 32), idesc_g, ks != 0);
+      tc_commit(&gfull[buf]);
+      mbar_wait(&ogated[buf], gph[buf], ab);     // gated o tile written back by the epilogue warps
+      gph[buf] ^= 1;
+      tc_fence_after();
+      for (int ks = 0; ks < Hd / 16; ++ks)
+        umma_bf16(dout, desc_kmajor_sw128(st + (zslab + (ks >> 2)) * slab + (ks & 3) * 32),
+                  desc_kmajor_sw128(smem_u32(sWo) + (ks >> 2) * wo_slab + (ks & 3) * 32), idesc_o, ks != 0);
+      tc_commit(&ofull[buf]);
+      tc_commit(&aempty[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue (8 warps)
+    const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int row = quarter * 32 + lane;
+    const int ep_tid = threadIdx.x - 64;
+    int stage = 0;
+    unsigned phase = 0, gph[2] = {0, 0}, oph[2] = {0, 0};
+    long long n = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
+      const int buf = (int)(n & 1);
+      mbar_wait(&afull[stage], phase, ab);
+      unsigned char* st = sSt + stage * stage_bytes;
+      float sum = 0.f, sq = 0.f;
+      for (int sl = 0; sl < zslab; ++sl) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = *reinterpret_cast<const uint4*>(st + sl * slab + sw128_off(row, ch));
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            sum += lo + hi;
+            sq = fmaf(lo, lo, sq);
+            sq = fmaf(hi, hi, sq);
+          }
+        }
+      }
+      const float mean = sum / (float)c;
+      const float rstd = rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps);
+      // ---- phase 1: o <- sigmoid(gate) * o, in place in shared memory
+      mbar_wait(&gfull[buf], gph[buf], ab);
+      gph[buf] ^= 1;
+      tc_fence_after();
+      const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
+      for (int c0 = half * (Hd / 2); c0 < (half + 1) * (Hd / 2); c0 += 32) {
+        unsigned r[32];
+        tmem_ld32(taddr + c0, r);
+        tmem_ld_wait();
+        unsigned char* op = st + (zslab + (c0 >> 6)) * slab;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4* ptr = reinterpret_cast<uint4*>(op + sw128_off(row, ((c0 & 63) >> 3) + ch));
+          const uint4 v = *ptr;
+          unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int n0 = ch * 8 + e * 2;
+            const float2 k0 = sC[c0 + n0], k1 = sC[c0 + n0 + 1];
+            const float g0 = sigmoid_fast3(fmaf(rstd, __uint_as_float(r[n0]) - mean * k0.y, k0.x));
+            const float g1 = sigmoid_fast3(fmaf(rstd, __uint_as_float(r[n0 + 1]) - mean * k1.y, k1.x));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(g0 * __uint_as_float(w[e] << 16),
+                                                      g1 * __uint_as_float(w[e] & 0xffff0000u));
+            w[e] = *reinterpret_cast<unsigned*>(&hh);
+          }
+          *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      tc_fence_before();
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ogated[buf]);
+      // ---- phase 2: z += (gated o) W_o^T, in place in the z tile, then store
+      mbar_wait(&ofull[buf], oph[buf], ab);
+      oph[buf] ^= 1;
+      tc_fence_after();
+      for (int c0 = half * (c / 2); c0 < (half + 1) * (c / 2); c0 += 32) {
+        unsigned r[32];
+        tmem_ld32(taddr + Hd + c0, r);
+        tmem_ld_wait();
+        unsigned char* zp = st + (c0 >> 6) * slab;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint4* ptr = reinterpret_cast<uint4*>(zp + sw128_off(row, ((c0 & 63) >> 3) + ch));
+          const uint4 v = *ptr;
+          unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int n0 = ch * 8 + e * 2;
+            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(w[e] << 16) + __uint_as_float(r[n0]),
+                                                      __uint_as_float(w[e] & 0xffff0000u) + __uint_as_float(r[n0 + 1]));
+            w[e] = *reinterpret_cast<unsigned*>(&hh);
+          }
+          *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+      fence_proxy_async_smem();
+      named_bar_sync(1, 256);
+      if (ep_tid == 0) {
+        for (int sl = 0; sl < zslab; ++sl) tma_store_2d(&p.zmap, st + sl * slab, sl * 64, (int)(t * 128));
+        tma_store_commit();
+        tma_store_wait_read0();
+        mbar_arrive(&aempty[stage]);
+      }
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+    if (ep_tid == 0) tma_store_wait_all0();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+bool fast_attn_out_supported(int c, int H, int d) {
+  const int Hd = H * d;
+  return (c == 64 || c == 128) && (Hd == 64 || Hd == 128);
+}
+
+size_t fast_attn_out_prep_bytes(int c, int H, int d) {
+  return align_up((size_t)H * d * c * 2, 256) + align_up((size_t)H * d * sizeof(float2), 256);
+}
+
+nt_status fast_attn_out(void* z, const void* o, const nt_attn_weights* W, float eps, int c, int H, int d, void* prep,
+                        const BatchMeta& m, int* status, cudaStream_t st) {
+  const int Hd = H * d;
+  __nv_bfloat16* wg = (__nv_bfloat16*)prep;
+  float2* c01g = (float2*)((char*)prep + align_up((size_t)Hd * c * 2, 256));
+  {
+    const void* srcs[1] = {W->W_g};
+    const int rows[1] = {Hd};
+    nt_status r = fast_ln_fold_prep(srcs, rows, 1, c, W->ln_gamma, W->ln_beta, wg, c01g, st);
+    if (r != NT_OK) return r;
+  }
+  const int zslab = c / 64, oslab = Hd / 64;
+  const size_t smem = (size_t)zslab * Hd * 128 + (size_t)oslab * c * 128 + 2 * (size_t)(zslab + oslab) * 128 * 128 +
+                      (size_t)Hd * 8 + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+      return cuda_fail("attn_out smem attribute");
+    attr_set = true;
+  }
+  AttnOutParams p;
+  memset(&p, 0, sizeof(p));
+  const long long P0 = m.pair_off[0];
+  p.rows = m.pair_off[m.B] - P0;
+  if (p.rows == 0) return NT_OK;
+  if (p.rows > 0x7FFFFF00ll) return NT_ERR_UNSUPPORTED;
+  p.c = c;
+  p.Hd = Hd;
+  p.eps = eps;
+  p.c01g = c01g;
+  p.status = status;
+  {
+    const unsigned box[2] = {64, 128};
+    const unsigned long long zdims[2] = {(unsigned long long)c, (unsigned long long)p.rows};
+    const unsigned long long zstr[1] = {(unsigned long long)c * 2};
+    if (!make_tmap_bf16(&p.zmap, (char*)z + (size_t)P0 * c * 2, 2, zdims, zstr, box)) return cuda_fail("attn_out z map");
+    const unsigned long long odims[2] = {(unsigned long long)Hd, (unsigned long long)p.rows};
+    const unsigned long long ostr[1] = {(unsigned long long)Hd * 2};
+    if (!make_tmap_bf16(&p.omap, (const char*)o + (size_t)P0 * Hd * 2, 2, odims, ostr, box))
+      return cuda_fail("attn_out o map");
+    const unsigned long long gdims[2] = {(unsigned long long)c, (unsigned long long)Hd};
+    const unsigned gbox[2] = {64, (unsigned)Hd};
+    if (!make_tmap_bf16(&p.wgmap, wg, 2, gdims, zstr, gbox)) return cuda_fail("attn_out W_g map");
+    const unsigned long long wdims[2] = {(unsigned long long)Hd, (unsigned long long)c};
+    const unsigned wbox[2] = {64, (unsigned)c};
+    if (!make_tmap_bf16(&p.womap, W->W_o, 2, wdims, ostr, wbox)) return cuda_fail("attn_out W_o map");
+  }
+  const long long ntiles = (p.rows + 127) / 128;
+  const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);
+  {
+    LaunchScope ls("attn_out", st);
+    attn_out_kernel<<<grid, AO_THREADS, smem, st>>>(p);
+  }
+  if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("attn_out launch");
+  return NT_OK;
+}
+
+}  // namespace ntp
