@@ -191,8 +191,10 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
     pa.A = z; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c_z;
     pa.ln_g = W->ln_in_gamma; pa.ln_b = W->ln_in_beta; pa.eps = eps;
     nt_status r;
-    const bool tc = dt == NT_BF16 && !g_force_generic;
-    if (tc && fast_tri_in_supported(c_z, c_h)) {
+    // The tensor-core stages exchange a, b (fp16) and t (fp16, scaled by 1 / N): all three or none.
+    const bool tc = dt == NT_BF16 && !g_force_generic && fast_tri_in_supported(c_z, c_h) &&
+                    fast_contract_supported(c_h) && fast_tri_out_supported(c_z, c_h);
+    if (tc) {
       r = fast_tri_in(z, W, eps, c_z, c_h, w.a, w.b, w.prep, m, L->status_d, st);
       if (r != NT_OK) return r;
     } else {

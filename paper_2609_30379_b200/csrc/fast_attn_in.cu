@@ -15,7 +15,7 @@
 
 namespace ntp {
 
-constexpr int AI_THREADS = 64 + 256;
+constexpr int AI_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps, 8 epilogue warps
 constexpr int AI_MAXB = 16;
 
 struct AttnInParams {
@@ -36,7 +36,8 @@ struct AttnInParams {
 
 __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_constant__ AttnInParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ __align__(8) unsigned long long bars[11];
+  __shared__ float2 sStats[2][128];        // per stage: (mean, rstd) of every tile row
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
   unsigned long long* tfull = bars + 4;
   unsigned long long* tempty = bars + 6;
   unsigned long long* wfull = bars + 8;
+  unsigned long long* aconv = bars + 9;    // [2]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -65,6 +67,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
       mbar_init(&aempty[s], 1 + 8);
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
+      mbar_init(&aconv[s], 4);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -110,7 +113,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&afull[stage], phase, ab);
+      mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned a_addr = smem_u32(sA + stage * a_stage);
       for (int u = 0; u < nunits; ++u, ++unit) {
@@ -118,7 +121,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
         mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
         tph[buf] ^= 1;
         tc_fence_after();
-        const unsigned idesc = idesc_bf16(128, u_n[u], 0, 0);
+        const unsigned idesc = idesc_f16(128, u_n[u], 0, 0, FMT_F16, FMT_F16);   // z tile converted to fp16, folded weights fp16
         const unsigned d_tmem = tmem_base + buf * 256;
         for (int sl = 0; sl < nslab; ++sl) {
           const unsigned w_addr = smem_u32(sW + sl * w_slab + u_row[u] * 128);
@@ -132,39 +135,39 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
       tc_commit(&aempty[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 6) {
+    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
+    const int row = (warp - 2) * 32 + lane;
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      float sum, sq;
+      convert_row_bf16_to_f16(sA + stage * a_stage, nslab, a_slab, row, sum, sq);
+      const float mean = sum / (float)c;
+      sStats[stage][row] = make_float2(mean, rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps));
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&aconv[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 6) {
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int half = (warp - 6) >> 2;
     const int row = quarter * 32 + lane;
-    const int ep_tid = threadIdx.x - 64;
+    const int ep_tid = threadIdx.x - 192;
     const int cpw = Hd / 2;                         // channels of one output handled by this warp
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
     bool store_pending = false;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&afull[stage], phase, ab);
-      float sum = 0.f, sq = 0.f;
-      const unsigned char* arow = sA + stage * a_stage;
-      for (int sl = 0; sl < nslab; ++sl) {
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = *reinterpret_cast<const uint4*>(arow + sl * a_slab + sw128_off(row, ch));
-          const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            sum += lo + hi;
-            sq = fmaf(lo, lo, sq);
-            sq = fmaf(hi, hi, sq);
-          }
-        }
-      }
+      mbar_wait(&aconv[stage], phase, ab);          // statistics of this tile are published
+      const float2 stt = sStats[stage][row];
       __syncwarp();
       if (lane == 0) mbar_arrive(&aempty[stage]);
-      const float mean = sum / (float)c;
-      const float rstd = rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps);
+      const float mean = stt.x, rstd = stt.y;
       for (int u = 0; u < nunits; ++u, ++unit) {
         const int buf = (int)(unit & 1);
         mbar_wait(&tfull[buf], tph[buf], ab);

@@ -12,7 +12,7 @@
 
 namespace ntp {
 
-constexpr int AO_THREADS = 64 + 256;
+constexpr int AO_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps, 8 epilogue warps
 
 struct AttnOutParams {
   CUtensorMap zmap;              // {c, rows}, box {64, 128}: load and store
@@ -34,7 +34,8 @@ __device__ inline float sigmoid_fast3(float x) {
 
 __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_constant__ AttnOutParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[13];
+  __shared__ __align__(8) unsigned long long bars[15];
+  __shared__ float2 sStats[2][128];        // per stage: (mean, rstd) of every z row
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
   unsigned long long* ofull = bars + 8;    // [2]
   unsigned long long* tempty = bars + 10;  // [2]
   unsigned long long* wfull = bars + 12;
+  unsigned long long* aconv = bars + 13;   // [2]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -65,6 +67,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       mbar_init(&ogated[s], 8);
       mbar_init(&ofull[s], 1);
       mbar_init(&tempty[s], 8);
+      mbar_init(&aconv[s], 4);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -100,13 +103,13 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0}, gph[2] = {0, 0};
     long long n = 0;
-    const unsigned idesc_g = idesc_bf16(128, Hd, 0, 0);
-    const unsigned idesc_o = idesc_bf16(128, c, 0, 0);
+    const unsigned idesc_g = idesc_f16(128, Hd, 0, 0, FMT_F16, FMT_F16);    // z tile converted to fp16, folded W_g fp16
+    const unsigned idesc_o = idesc_f16(128, c, 0, 0, FMT_BF16, FMT_BF16);   // gated o bf16, W_o as given (bf16)
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const int buf = (int)(n & 1);
       mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
       tph[buf] ^= 1;
-      mbar_wait(&afull[stage], phase, ab);
+      mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned st = smem_u32(sSt + stage * stage_bytes);
       const unsigned dg = tmem_base + buf * 256, dout = dg + Hd;
@@ -124,40 +127,39 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       tc_commit(&aempty[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 6) {
+    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
+    const int row = (warp - 2) * 32 + lane;
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      float sum, sq;
+      convert_row_bf16_to_f16(sSt + stage * stage_bytes, zslab, slab, row, sum, sq);
+      const float mean = sum / (float)c;
+      sStats[stage][row] = make_float2(mean, rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps));
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&aconv[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 6) {
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int half = (warp - 6) >> 2;
     const int row = quarter * 32 + lane;
-    const int ep_tid = threadIdx.x - 64;
+    const int ep_tid = threadIdx.x - 192;
     int stage = 0;
-    unsigned phase = 0, gph[2] = {0, 0}, oph[2] = {0, 0};
+    unsigned gph[2] = {0, 0}, oph[2] = {0, 0};
     long long n = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const int buf = (int)(n & 1);
-      mbar_wait(&afull[stage], phase, ab);
       unsigned char* st = sSt + stage * stage_bytes;
-      float sum = 0.f, sq = 0.f;
-      for (int sl = 0; sl < zslab; ++sl) {
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = *reinterpret_cast<const uint4*>(st + sl * slab + sw128_off(row, ch));
-          const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            sum += lo + hi;
-            sq = fmaf(lo, lo, sq);
-            sq = fmaf(hi, hi, sq);
-          }
-        }
-      }
-      const float mean = sum / (float)c;
-      const float rstd = rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps);
       // ---- phase 1: o <- sigmoid(gate) * o, in place in shared memory
-      mbar_wait(&gfull[buf], gph[buf], ab);
+      mbar_wait(&gfull[buf], gph[buf], ab);         // gate MMA done, hence the statistics are published too
       gph[buf] ^= 1;
       tc_fence_after();
+      const float mean = sStats[stage][row].x, rstd = sStats[stage][row].y;
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       for (int c0 = half * (Hd / 2); c0 < (half + 1) * (Hd / 2); c0 += 32) {
         unsigned r[32];
@@ -203,8 +205,8 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(w[e] << 16) + __uint_as_float(r[n0]),
-                                                      __uint_as_float(w[e] & 0xffff0000u) + __uint_as_float(r[n0 + 1]));
+            const float2 zo = unpack_h2(w[e]);        // the z tile holds fp16 after conversion
+            __nv_bfloat162 hh = __floats2bfloat162_rn(zo.x + __uint_as_float(r[n0]), zo.y + __uint_as_float(r[n0 + 1]));
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);
@@ -221,7 +223,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
         tma_store_wait_read0();
         mbar_arrive(&aempty[stage]);
       }
-      if (++stage == 2) { stage = 0; phase ^= 1; }
+      if (++stage == 2) stage = 0;
     }
     if (ep_tid == 0) tma_store_wait_all0();
   }

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
       tph[buf] ^= 1;
       tc_fence_after();
-      const unsigned idesc = idesc_bf16(128, Nt, 0, 0);
+      const unsigned idesc = idesc_f16(128, Nt, 0, 0, FMT_F16, FMT_F16);   // a, b are fp16
       const unsigned d_tmem = tmem_base + buf * 256;
       for (int kc = 0; kc < nkc; ++kc) {
         mbar_wait(&full[stage], phase, ab);
@@ -145,6 +145,7 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       }
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       const int ncg = (Nt + 63) / 64;
+      const float tscale = 1.0f / (float)p.N[s];   // t is stored as t / N in fp16; the following LayerNorm is scale-free
       for (int cg = 0; cg < ncg; ++cg) {
         unsigned r0[32], r1[32];
         tmem_ld32(taddr + cg * 64, r0);
@@ -154,19 +155,19 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint4 v;
-          v.x = pack2(r0[ch * 8 + 0], r0[ch * 8 + 1]);
-          v.y = pack2(r0[ch * 8 + 2], r0[ch * 8 + 3]);
-          v.z = pack2(r0[ch * 8 + 4], r0[ch * 8 + 5]);
-          v.w = pack2(r0[ch * 8 + 6], r0[ch * 8 + 7]);
+          v.x = pack2h(r0[ch * 8 + 0], r0[ch * 8 + 1], tscale);
+          v.y = pack2h(r0[ch * 8 + 2], r0[ch * 8 + 3], tscale);
+          v.z = pack2h(r0[ch * 8 + 4], r0[ch * 8 + 5], tscale);
+          v.w = pack2h(r0[ch * 8 + 6], r0[ch * 8 + 7], tscale);
           *reinterpret_cast<uint4*>(panel + sw128_off(row, ch)) = v;
         }
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint4 v;
-          v.x = pack2(r1[ch * 8 + 0], r1[ch * 8 + 1]);
-          v.y = pack2(r1[ch * 8 + 2], r1[ch * 8 + 3]);
-          v.z = pack2(r1[ch * 8 + 4], r1[ch * 8 + 5]);
-          v.w = pack2(r1[ch * 8 + 6], r1[ch * 8 + 7]);
+          v.x = pack2h(r1[ch * 8 + 0], r1[ch * 8 + 1], tscale);
+          v.y = pack2h(r1[ch * 8 + 2], r1[ch * 8 + 3], tscale);
+          v.z = pack2h(r1[ch * 8 + 4], r1[ch * 8 + 5], tscale);
+          v.w = pack2h(r1[ch * 8 + 6], r1[ch * 8 + 7], tscale);
           *reinterpret_cast<uint4*>(panel + sw128_off(row, 4 + ch)) = v;
         }
       }

@@ -20,7 +20,7 @@
 namespace ntp {
 
 constexpr int TI_CH = 32;                  // positions per chunk
-constexpr int TI_THREADS = 64 + 256;       // producer warp, MMA warp, 8 epilogue warps
+constexpr int TI_THREADS = 64 + 128 + 256; // producer warp, MMA warp, 4 converter warps, 8 epilogue warps
 constexpr int TI_MAXB = 16;
 
 struct TriInParams {
@@ -56,7 +56,8 @@ __device__ inline float sigmoid_fast(float x) {
 
 __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_constant__ TriInParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ __align__(8) unsigned long long bars[11];
+  __shared__ float2 sStats[2][128];        // per stage: (mean, rstd) of every tile row
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   unsigned long long* tfull = bars + 4;    // [2]
   unsigned long long* tempty = bars + 6;   // [2]
   unsigned long long* wfull = bars + 8;
+  unsigned long long* aconv = bars + 9;    // [2] tile converted to fp16, statistics published
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -84,6 +86,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       mbar_init(&aempty[s], 1 + 8);        // MMA commit + one arrival per epilogue warp
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
+      mbar_init(&aconv[s], 4);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -127,9 +130,9 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
-    const unsigned idesc = idesc_bf16(128, Nu, 0, 0);
+    const unsigned idesc = idesc_f16(128, Nu, 0, 0, FMT_F16, FMT_F16);   // z tile converted to fp16, folded weights fp16
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&afull[stage], phase, ab);
+      mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned a_addr = smem_u32(sA + stage * a_stage_bytes);
       for (int u = 0; u < 2; ++u, ++unit) {
@@ -150,12 +153,29 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       tc_commit(&aempty[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 6) {
+    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
+    const int row = (warp - 2) * 32 + lane;
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      float sum, sq;
+      convert_row_bf16_to_f16(sA + stage * a_stage_bytes, nslab, a_slab_bytes, row, sum, sq);
+      const float mean = sum / (float)c_z;
+      const float var = fmaxf(sq / (float)c_z - mean * mean, 0.f);
+      sStats[stage][row] = make_float2(mean, rsqrtf(var + p.eps));
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&aconv[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 6) {
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;                  // TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;              // which half of the channels this warp handles
+    const int half = (warp - 6) >> 2;              // which half of the channels this warp handles
     const int row = quarter * 32 + lane;           // accumulator row = position inside the tile
-    unsigned char* stg = sStage + (warp - 2) * 2048;
+    unsigned char* stg = sStage + (warp - 6) * 2048;
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
@@ -163,29 +183,11 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       // chunk of this warp: quarter-th chunk of the tile
       int s = 0, i = 0, jc = 0;
       const bool valid = ti_decode(p, 4 * t + quarter, s, i, jc);
-      mbar_wait(&afull[stage], phase, ab);
-      // row statistics from the raw z tile
-      float sum = 0.f, sq = 0.f;
-      const unsigned char* arow = sA + stage * a_stage_bytes;
-      for (int sl = 0; sl < nslab; ++sl) {
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = *reinterpret_cast<const uint4*>(arow + sl * a_slab_bytes + sw128_off(row, ch));
-          const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            sum += lo + hi;
-            sq = fmaf(lo, lo, sq);
-            sq = fmaf(hi, hi, sq);
-          }
-        }
-      }
+      mbar_wait(&aconv[stage], phase, ab);         // statistics of this tile are published
+      const float2 stt = sStats[stage][row];
       __syncwarp();
       if (lane == 0) mbar_arrive(&aempty[stage]);
-      const float mean = sum / (float)c_z;
-      const float var = fmaxf(sq / (float)c_z - mean * mean, 0.f);
-      const float rstd = rsqrtf(var + p.eps);
+      const float mean = stt.x, rstd = stt.y;
       const int N = valid ? p.N[s] : 1;
       const int ld = round_up8(N);
       const long long plane = (long long)N * ld;
@@ -207,8 +209,8 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
             const float2 kg = cg[c0 + e], kv = cg[c_h + c0 + e];
             const float xg = fmaf(rstd, __uint_as_float(rg[e]) - mean * kg.y, kg.x);
             const float xv = fmaf(rstd, __uint_as_float(rv[e]) - mean * kv.y, kv.x);
-            const float val = sigmoid_fast(xg) * xv;
-            reinterpret_cast<__nv_bfloat16*>(stg)[e * 32 + lane] = __float2bfloat16_rn(val);
+            const float val = fminf(fmaxf(sigmoid_fast(xg) * xv, -65504.f), 65504.f);
+            reinterpret_cast<__half*>(stg)[e * 32 + lane] = __float2half_rn(val);
           }
           __syncwarp();
           if (valid) {
@@ -246,7 +248,7 @@ struct PrepArgs {
   int nsrc, K;
   const __nv_bfloat16* gamma;
   const __nv_bfloat16* beta;
-  __nv_bfloat16* out;
+  __half* out;     // folded weights are kept in fp16: 11 significant bits instead of 8, same MMA rate
   float2* c01;
 };
 
@@ -262,11 +264,11 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
   float c0 = 0.f, c1 = 0.f;
   for (int k = lane; k < a.K; k += 32) {
     const float wv = __bfloat162float(w[k]);
-    __nv_bfloat16 o = w[k];
+    __half o = __float2half_rn(wv);
     if (a.gamma) {
-      o = __float2bfloat16_rn(wv * __bfloat162float(a.gamma[k]));
+      o = __float2half_rn(wv * __bfloat162float(a.gamma[k]));
       c0 = fmaf(wv, __bfloat162float(a.beta[k]), c0);
-      c1 += __bfloat162float(o);
+      c1 += __half2float(o);
     }
     a.out[(long long)n * a.K + k] = o;
   }
@@ -291,7 +293,7 @@ nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, 
   a.K = K;
   a.gamma = (const __nv_bfloat16*)gamma;
   a.beta = (const __nv_bfloat16*)beta;
-  a.out = (__nv_bfloat16*)out;
+  a.out = (__half*)out;
   a.c01 = (float2*)c01;
   {
     LaunchScope ls("weight_prep", st);

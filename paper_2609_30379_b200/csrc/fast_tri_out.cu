@@ -18,7 +18,7 @@
 
 namespace ntp {
 
-constexpr int TO_THREADS = 64 + 256;
+constexpr int TO_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps, 8 epilogue warps
 constexpr int TO_MAXB = 12;
 
 struct TriOutParams {
@@ -54,7 +54,8 @@ __device__ inline float sigmoid_fast2(float x) {
 
 __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_constant__ TriOutParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[9];
+  __shared__ __align__(8) unsigned long long bars[11];
+  __shared__ float4 sStats[2][128];      // per stage and tile row: (t mean, t rstd, z mean, z rstd)
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -75,6 +76,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   unsigned long long* tfull = bars + 4;
   unsigned long long* tempty = bars + 6;
   unsigned long long* wfull = bars + 8;
+  unsigned long long* aconv = bars + 9;  // [2]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -84,6 +86,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       mbar_init(&aempty[s], 2);            // MMA commit + the storing epilogue thread
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
+      mbar_init(&aconv[s], 4);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -128,13 +131,13 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long n = 0;
-    const unsigned idesc_t = idesc_bf16(128, c_z, 1, 0);     // A = t, MN-major
-    const unsigned idesc_z = idesc_bf16(128, c_z, 0, 0);
+    const unsigned idesc_t = idesc_f16(128, c_z, 1, 0, FMT_F16, FMT_F16);   // A = t (fp16, MN-major), W_o' fp16
+    const unsigned idesc_z = idesc_f16(128, c_z, 0, 0, FMT_F16, FMT_F16);   // A = z tile converted to fp16, W_g' fp16
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const int buf = (int)(n & 1);
       mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
       tph[buf] ^= 1;
-      mbar_wait(&afull[stage], phase, ab);
+      mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned st = smem_u32(sSt + stage * stage_bytes);
       const unsigned d1 = tmem_base + buf * 256, d2 = d1 + c_z;
@@ -152,54 +155,60 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       tc_commit(&aempty[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2) {
+  } else if (warp >= 2 && warp < 6) {
+    // ------------------------------------------------------------------ converters (4 warps, one position per thread)
+    const int row = (warp - 2) * 32 + lane;
+    const int q = row >> 6, pos = row & 63;
+    int stage = 0;
+    unsigned phase = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      mbar_wait(&afull[stage], phase, ab);
+      unsigned char* st = sSt + stage * stage_bytes;
+      // statistics of t over channels: a column of the MN-major fp16 tile
+      float ts = 0.f, tq = 0.f;
+      const unsigned char* tcol = st + q * t_chunk + (pos & 7) * 2;
+      for (int c = 0; c < c_h; ++c) {
+        const float v = __half2float(*reinterpret_cast<const __half*>(tcol + c * 128 + (((pos >> 3) ^ (c & 7)) << 4)));
+        ts += v;
+        tq = fmaf(v, v, tq);
+      }
+      // t arrives scaled by 1 / N_s (see the contraction); LayerNorm is scale-free once eps is scaled alike
+      float eps_t = p.eps;
+      {
+        int s_, i_, j_;
+        if (to_decode(p, 2 * t + q, s_, i_, j_)) eps_t = p.eps / ((float)p.N[s_] * (float)p.N[s_]);
+      }
+      const float tmean = ts / (float)c_h;
+      const float trstd = rsqrtf(fmaxf(tq / (float)c_h - tmean * tmean, 0.f) + eps_t);
+      // z row: convert to fp16 in place and take its statistics
+      float zs, zq;
+      convert_row_bf16_to_f16(st + 2 * t_chunk, zslab, z_slab, row, zs, zq);
+      const float zmean = zs / (float)c_z;
+      const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
+      sStats[stage][row] = make_float4(tmean, trstd, zmean, zrstd);
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&aconv[stage]);
+      if (++stage == 2) { stage = 0; phase ^= 1; }
+    }
+  } else if (warp >= 6) {
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int half = (warp - 6) >> 2;
     const int row = quarter * 32 + lane;           // position inside the tile
-    const int q = quarter >> 1;                    // chunk of this row
-    const int pos = (quarter & 1) * 32 + lane;     // position inside the chunk
-    const int ep_tid = threadIdx.x - 64;
+    const int ep_tid = threadIdx.x - 192;
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long n = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const int buf = (int)(n & 1);
-      mbar_wait(&afull[stage], phase, ab);
       unsigned char* st = sSt + stage * stage_bytes;
-      // statistics of t over channels (column of the MN-major tile) and of z over channels (row)
-      float ts = 0.f, tq = 0.f;
-      const unsigned char* tcol = st + q * t_chunk + (pos & 7) * 2;
-      for (int c = 0; c < c_h; ++c) {
-        const unsigned short hv = *reinterpret_cast<const unsigned short*>(tcol + c * 128 + (((pos >> 3) ^ (c & 7)) << 4));
-        const float v = __uint_as_float((unsigned)hv << 16);
-        ts += v;
-        tq = fmaf(v, v, tq);
-      }
-      float zs = 0.f, zq = 0.f;
       unsigned char* zrow = st + 2 * t_chunk;
-      for (int sl = 0; sl < zslab; ++sl) {
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = *reinterpret_cast<const uint4*>(zrow + sl * z_slab + sw128_off(row, ch));
-          const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            zs += lo + hi;
-            zq = fmaf(lo, lo, zq);
-            zq = fmaf(hi, hi, zq);
-          }
-        }
-      }
-      const float tmean = ts / (float)c_h;
-      const float trstd = rsqrtf(fmaxf(tq / (float)c_h - tmean * tmean, 0.f) + p.eps);
-      const float zmean = zs / (float)c_z;
-      const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
-      named_bar_sync(2, 256);                      // every row's statistics are taken before z is overwritten
-      mbar_wait(&tfull[buf], tph[buf], ab);
+      mbar_wait(&tfull[buf], tph[buf], ab);         // MMAs done, hence the statistics are published too
       tph[buf] ^= 1;
       tc_fence_after();
+      const float4 stt = sStats[stage][row];
+      const float tmean = stt.x, trstd = stt.y, zmean = stt.z, zrstd = stt.w;
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       for (int c0 = half * (c_z / 2); c0 < (half + 1) * (c_z / 2); c0 += 32) {
         unsigned r1[32], r2[32];
@@ -222,7 +231,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
               const float2 ko = sCo[c0 + n0 + h2], kg = sCg[c0 + n0 + h2];
               const float o = fmaf(trstd, __uint_as_float(r1[n0 + h2]) - tmean * ko.y, ko.x);
               const float g = sigmoid_fast2(fmaf(zrstd, __uint_as_float(r2[n0 + h2]) - zmean * kg.y, kg.x));
-              const float zold = h2 == 0 ? __uint_as_float(w[e] << 16) : __uint_as_float(w[e] & 0xffff0000u);
+              const float2 zo = unpack_h2(w[e]);       // the z tile holds fp16 after conversion
+              const float zold = h2 == 0 ? zo.x : zo.y;
               out[h2] = fmaf(g, o, zold);
             }
             __nv_bfloat162 hh = __floats2bfloat162_rn(out[0], out[1]);

@@ -148,10 +148,12 @@ __device__ inline unsigned long long desc_mnmajor_sw128(unsigned saddr, unsigned
   d |= (unsigned long long)2 << 61;
   return d;
 }
-// instruction descriptor: D = f32, A = B = bf16, M x N tile, operand majors (0 = K-major, 1 = MN-major)
-__device__ inline unsigned idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)a_mn_major << 15) | ((unsigned)b_mn_major << 16) |
-         ((unsigned)(N >> 3) << 17) | ((unsigned)(M >> 4) << 24);
+// instruction descriptor of kind::f16: D = f32, M x N tile, operand majors (0 = K-major, 1 = MN-major)
+// and per-operand 16-bit formats (FMT_F16 or FMT_BF16; the two operands may differ)
+constexpr int FMT_F16 = 0, FMT_BF16 = 1;
+__device__ inline unsigned idesc_f16(int M, int N, int a_mn_major, int b_mn_major, int a_fmt, int b_fmt) {
+  return (1u << 4) | ((unsigned)a_fmt << 7) | ((unsigned)b_fmt << 10) | ((unsigned)a_mn_major << 15) |
+         ((unsigned)b_mn_major << 16) | ((unsigned)(N >> 3) << 17) | ((unsigned)(M >> 4) << 24);
 }
 // D[tmem] (+)= A[smem] * B[smem]; issued by one thread
 __device__ inline void umma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
@@ -173,8 +175,49 @@ __device__ inline unsigned pack2(unsigned lo, unsigned hi) {
   return *reinterpret_cast<unsigned*>(&h);
 }
 
+// two floats (bit patterns) scaled and packed as fp16x2 (saturating), first in the low half
+__device__ inline unsigned pack2h(unsigned lo, unsigned hi, float scale) {
+  const float a = fminf(fmaxf(__uint_as_float(lo) * scale, -65504.f), 65504.f);
+  const float b = fminf(fmaxf(__uint_as_float(hi) * scale, -65504.f), 65504.f);
+  __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<unsigned*>(&h);
+}
+
 // byte offset of 16-byte chunk `chunk` of row `row` inside a 128-byte-swizzled tile
 __device__ inline unsigned sw128_off(int row, int chunk) { return row * 128 + ((chunk ^ (row & 7)) << 4); }
+
+// Both MMA operands must have the same 16-bit format.  The folded weights are fp16 (three more
+// significant bits than bf16), so the bf16 activation tile is rewritten as fp16 in place before the
+// MMA; a bf16 value is exactly representable in fp16 while its magnitude is in [2^-14, 65504], and
+// loses only bits below 2^-24 otherwise.  One thread converts one row of a K-major 128-byte-swizzled
+// tile made of `nslab` 64-column slabs and returns the row's sum and sum of squares.
+__device__ inline void convert_row_bf16_to_f16(unsigned char* tile, int nslab, int slab_bytes, int row, float& sum,
+                                               float& sq) {
+  sum = 0.f;
+  sq = 0.f;
+  for (int sl = 0; sl < nslab; ++sl) {
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+      uint4* ptr = reinterpret_cast<uint4*>(tile + sl * slab_bytes + sw128_off(row, ch));
+      const uint4 v = *ptr;
+      unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+        sum += lo + hi;
+        sq = fmaf(lo, lo, sq);
+        sq = fmaf(hi, hi, sq);
+        __half2 h = __floats2half2_rn(lo, hi);
+        w[e] = *reinterpret_cast<unsigned*>(&h);
+      }
+      *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+__device__ inline float2 unpack_h2(unsigned w) {
+  return __half22float2(*reinterpret_cast<const __half2*>(&w));
+}
 #endif  // __CUDACC__
 
 }  // namespace ntp
