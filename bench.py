@@ -58,6 +58,7 @@ def kernel_work(cfg: wl.Config):
     w = {}
     tok = dict(bytes=T1 * c_s * e + c_z * c_s * e + T1 * c_z * 4, flops=2 * T1 * c_s * c_z)
     w["tok_proj_u"] = w["tok_proj_v"] = tok
+    w["tok_proj"] = dict(bytes=T1 * c_s * e + 2 * c_z * c_s * e + 2 * T1 * c_z * 4, flops=4 * T1 * c_s * c_z)
     bc = dict(bytes=T2 * c_z * e + 2 * T1 * c_z * 4, flops=8 * T2 * c_z)
     w["broadcast_ln"] = w["generic_broadcast_ln"] = bc
     w["generic_tri_in_a"] = w["generic_tri_in_b"] = dict(bytes=T2 * (c_z + c_h) * e, flops=2 * T2 * c_z * 2 * c_h)
@@ -213,6 +214,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the per-kernel timing pass, the end-to-end pass and the CPU baseline (for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -283,6 +286,14 @@ def main():
     unit_count = cfg.T2 if cfg.kind == "pair" else cfg.T1
     value = world * cfg.blocks * unit_count * steps / (ms * 1e-3)
     peak_alloc = torch.cuda.max_memory_allocated()
+
+    if args.no_extras:
+        if rank == 0:
+            print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=steps, warmup=warmup,
+                                  ms_per_step=ms / steps, gpu_launches=launches, note="--no-extras run")))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- per-kernel timing pass (CUDA events around every launch, on the launching stream)
     barrier()

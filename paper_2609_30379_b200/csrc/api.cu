@@ -163,11 +163,17 @@ static nt_status pair_broadcast_impl(const nt_layout* L, const Totals& tot, int 
   ProjArgs pa{};
   pa.A = x; pa.a_mode = A_ROWMAJOR; pa.row0 = 0; pa.rows = tot.T1; pa.K = c_s;
   pa.W1 = W_a; pa.Nout = c_z; pa.act = ACT_NONE; pa.out = u; pa.out_mode = O_STORE; pa.out_f32 = 1;
-  nt_status r = launch_proj<T>(pa, dummy, st, "tok_proj_u");
-  if (r != NT_OK) return r;
-  pa.W1 = W_b; pa.out = v;
-  r = launch_proj<T>(pa, dummy, st, "tok_proj_v");
-  if (r != NT_OK) return r;
+  nt_status r;
+  if (fast && fast_token_gemm_supported(c_s, c_z, c_z)) {
+    r = fast_token_gemm(x, tot.T1, c_s, W_a, c_z, u, W_b, c_z, v, 1, 0, "tok_proj", st);
+    if (r != NT_OK) return r;
+  } else {
+    r = launch_proj<T>(pa, dummy, st, "tok_proj_u");
+    if (r != NT_OK) return r;
+    pa.W1 = W_b; pa.out = v;
+    r = launch_proj<T>(pa, dummy, st, "tok_proj_v");
+    if (r != NT_OK) return r;
+  }
   GroupIter it(L->lengths_h, L->B);
   BatchMeta m;
   while (it.next(m)) {
@@ -182,6 +188,14 @@ template <typename T>
 static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z, int c_h, const nt_trimul_weights* W,
                                  float eps, void* z, void* ws, nt_dtype dt, cudaStream_t st) {
   TriWs w = carve_trimul(ws, dt, tot, c_z, c_h);
+  // The tensor-core stages exchange a, b (fp16) and t (fp16, scaled by 1 / N): all three or none.
+  const bool tc = dt == NT_BF16 && !g_force_generic && fast_tri_in_supported(c_z, c_h) &&
+                  fast_contract_supported(c_h) && fast_tri_out_supported(c_z, c_h);
+  TriPrep tprep{};
+  if (tc) {
+    nt_status r0 = fast_tri_prep(W, c_z, c_h, w.prep, tprep, st);
+    if (r0 != NT_OK) return r0;
+  }
   GroupIter it(L->lengths_h, L->B);
   BatchMeta m;
   while (it.next(m)) {
@@ -191,11 +205,8 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
     pa.A = z; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c_z;
     pa.ln_g = W->ln_in_gamma; pa.ln_b = W->ln_in_beta; pa.eps = eps;
     nt_status r;
-    // The tensor-core stages exchange a, b (fp16) and t (fp16, scaled by 1 / N): all three or none.
-    const bool tc = dt == NT_BF16 && !g_force_generic && fast_tri_in_supported(c_z, c_h) &&
-                    fast_contract_supported(c_h) && fast_tri_out_supported(c_z, c_h);
     if (tc) {
-      r = fast_tri_in(z, W, eps, c_z, c_h, w.a, w.b, w.prep, m, L->status_d, st);
+      r = fast_tri_in(z, tprep, eps, c_z, c_h, w.a, w.b, m, L->status_d, st);
       if (r != NT_OK) return r;
     } else {
       pa.W1 = W->W_ag; pa.W2 = W->W_ap; pa.Nout = c_h; pa.out = w.a; pa.out_mode = O_CHANNEL_MAJOR;
@@ -217,7 +228,7 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
       r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st);
     if (r != NT_OK) return r;
     if (tc_out) {
-      r = fast_tri_out(z, w.t, W, eps, c_z, c_h, (char*)w.prep + (512 << 10), m, L->status_d, st);
+      r = fast_tri_out(z, w.t, tprep, eps, c_z, c_h, m, L->status_d, st);
       if (r != NT_OK) return r;
       continue;
     }
@@ -238,6 +249,14 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
   AttnWs w = carve_attn(ws, dt, tot, order, H, d);
   const int Hd = H * d;
   const bool pair = order == NT_ORDER_PAIR_IJC;
+  const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma;
+  const bool tc_in = tc && fast_attn_in_supported(c, H, d);
+  const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
+  AttnPrep aprep{};
+  if (tc_in || tc_out) {
+    nt_status r0 = fast_attn_prep(W, c, H, d, w.prep, aprep, st);
+    if (r0 != NT_OK) return r0;
+  }
   GroupIter it(L->lengths_h, L->B);
   BatchMeta m;
   while (it.next(m)) {
@@ -249,11 +268,8 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
     pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = eps;
     pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
     nt_status r;
-    const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma;
-    const bool tc_in = tc && fast_attn_in_supported(c, H, d);
-    const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
     if (tc_in) {
-      r = fast_attn_in(zx, W, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.prep, m, L->status_d, st);
+      r = fast_attn_in(zx, aprep, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, m, L->status_d, st);
       if (r != NT_OK) return r;
     } else {
       pa.W1 = W->W_q; pa.out = w.q;
@@ -279,7 +295,7 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
                               (T*)w.o, H, d, pair ? 1 : 0, m, st);
     if (r != NT_OK) return r;
     if (tc_out) {
-      r = fast_attn_out(zx, w.o, W, eps, c, H, d, (char*)w.prep + (512 << 10), m, L->status_d, st);
+      r = fast_attn_out(zx, w.o, W->W_o, aprep, eps, c, H, d, m, L->status_d, st);
       if (r != NT_OK) return r;
       continue;
     }
@@ -389,6 +405,8 @@ nt_status nt_token_update(nt_dtype dt, int32_t c_s, int32_t c_z, int64_t T1, con
   pa.W1 = W_r; pa.Nout = c_s; pa.act = ACT_NONE; pa.out = x; pa.out_mode = O_ACCUM;
   cudaStream_t st = (cudaStream_t)stream;
   if (dt == NT_F32) return launch_proj<float>(pa, dummy, st, "token_update");
+  if (!g_force_generic && fast_token_gemm_supported(c_z, c_s, 0))
+    return fast_token_gemm(mvals, T1, c_z, W_r, c_s, x, nullptr, 0, nullptr, 0, 1, "token_update", st);
   return launch_proj<__nv_bfloat16>(pa, dummy, st, "token_update");
 }
 

@@ -13,6 +13,11 @@ bool fast_segment_reduce_supported(int C);
 nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,
                               cudaStream_t st);
 
+// token-side projections: out[r][n] (+)= sum_k A[r][k] W[n][k] for up to two (W, out) pairs sharing A
+bool fast_token_gemm_supported(int K, int N0, int N1);
+nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, int N0, void* out0, const void* W1,
+                          int N1, void* out1, int out_f32, int accumulate, const char* name, cudaStream_t st);
+
 // attention core on tensor cores (bf16, d in {16, 32, 64}); q, k, v, o row-major [rows, H*d], bias
 // head-major channel-major (nullable)
 bool fast_attn_core_supported(int H, int d);
@@ -25,29 +30,30 @@ bool fast_contract_supported(int C);
 nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
                         cudaStream_t st);
 
-// triangle input projection on tcgen05 (LayerNorm folded into the weights); `prep` is scratch of
-// fast_tri_in_prep_bytes() for the folded weights
+// ---- tensor-core projections (tcgen05, LayerNorm folded into fp16 weights prepared once per call)
+struct TriPrep { void *w1, *c01_1, *wg, *c01g, *wo, *c01o; };
+struct AttnPrep { void *w, *c01, *wg, *c01g; };
+nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep, TriPrep& out, cudaStream_t st);
+nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* prep, AttnPrep& out, cudaStream_t st);
+
+// a = sig(LN(z) W_ag^T) * (LN(z) W_ap^T), b likewise: fp16, channel-major
 bool fast_tri_in_supported(int c_z, int c_h);
-size_t fast_tri_in_prep_bytes(int c_z, int c_h);
-nt_status fast_tri_in(const void* z, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* a, void* b,
-                      void* prep, const BatchMeta& m, int* status, cudaStream_t st);
-nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
-                            const void* beta, void* out, void* c01, cudaStream_t st);
+nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int c_h, void* a, void* b,
+                      const BatchMeta& m, int* status, cudaStream_t st);
 
-// attention input projection on tcgen05: q, k, v row-major, bias head-major (nullable)
-bool fast_attn_in_supported(int c, int H, int d);
-nt_status fast_attn_in(const void* z, const nt_attn_weights* W, float eps, int c, int H, int d, void* q, void* k,
-                       void* v, void* bias, void* prep, const BatchMeta& m, int* status, cudaStream_t st);
-
-// attention output stage on tcgen05, in place on z: z += (sigmoid(LN(z) W_g^T) * o) W_o^T
-bool fast_attn_out_supported(int c, int H, int d);
-nt_status fast_attn_out(void* z, const void* o, const nt_attn_weights* W, float eps, int c, int H, int d, void* prep,
-                        const BatchMeta& m, int* status, cudaStream_t st);
-
-// triangle output stage on tcgen05, in place on z: z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T)
+// in place on z: z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T); t fp16 channel-major scaled by 1 / N
 bool fast_tri_out_supported(int c_z, int c_h);
-size_t fast_tri_out_prep_bytes(int c_z, int c_h);
-nt_status fast_tri_out(void* z, const void* t, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* prep,
-                       const BatchMeta& m, int* status, cudaStream_t st);
+nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int c_z, int c_h, const BatchMeta& m,
+                       int* status, cudaStream_t st);
+
+// q, k, v row-major bf16, bias head-major bf16 (nullable)
+bool fast_attn_in_supported(int c, int H, int d);
+nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int H, int d, void* q, void* k, void* v,
+                       void* bias, const BatchMeta& m, int* status, cudaStream_t st);
+
+// in place on z: z += (sigmoid(LN(z) W_g^T) * o) W_o^T
+bool fast_attn_out_supported(int c, int H, int d);
+nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
+                        const BatchMeta& m, int* status, cudaStream_t st);
 
 }  // namespace ntp

@@ -251,27 +251,12 @@ bool fast_attn_in_supported(int c, int H, int d) {
   return (c == 64 || c == 128) && (Hd == 64 || Hd == 128) && H <= 16;
 }
 
-size_t fast_attn_in_prep_bytes(int c, int H, int d) {
-  const int wrows = 3 * H * d + 16;
-  return align_up((size_t)wrows * c * 2, 256) + align_up((size_t)wrows * sizeof(float2), 256) + 256;
-}
-
-nt_status fast_attn_in(const void* z, const nt_attn_weights* W, float eps, int c, int H, int d, void* q, void* k,
-                       void* v, void* bias, void* prep, const BatchMeta& m, int* status, cudaStream_t st) {
+nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int H, int d, void* q, void* k, void* v,
+                       void* bias, const BatchMeta& m, int* status, cudaStream_t st) {
   const int Hd = H * d;
   const int wrows = 3 * Hd + 16;
-  __nv_bfloat16* wprime = (__nv_bfloat16*)prep;
-  float2* c01 = (float2*)((char*)prep + align_up((size_t)wrows * c * 2, 256));
-  __nv_bfloat16* zero_rows = (__nv_bfloat16*)((char*)c01 + align_up((size_t)wrows * sizeof(float2), 256));
-  (void)zero_rows;
-  // rows: W_q, W_k, W_v, W_b (H rows), then 16 - H rows that must be zero: clear the tail first
-  if (cudaMemsetAsync((char*)wprime + (size_t)3 * Hd * c * 2, 0, (size_t)16 * c * 2, st) != cudaSuccess)
-    return cuda_fail("attn_in memset");
-  if (cudaMemsetAsync(c01 + 3 * Hd, 0, 16 * sizeof(float2), st) != cudaSuccess) return cuda_fail("attn_in memset");
-  const void* srcs[4] = {W->W_q, W->W_k, W->W_v, W->W_b};
-  const int rows[4] = {Hd, Hd, Hd, H};
-  nt_status r = fast_ln_fold_prep(srcs, rows, W->W_b ? 4 : 3, c, W->ln_gamma, W->ln_beta, wprime, c01, st);
-  if (r != NT_OK) return r;
+  const void* wprime = ap.w;
+  const float2* c01 = (const float2*)ap.c01;
   const int nslab = c / 64;
   const int npanel = Hd / 64;
   const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)nslab * 128 * 128 + (size_t)npanel * 128 * 128 +

@@ -238,21 +238,11 @@ bool fast_attn_out_supported(int c, int H, int d) {
   return (c == 64 || c == 128) && (Hd == 64 || Hd == 128);
 }
 
-size_t fast_attn_out_prep_bytes(int c, int H, int d) {
-  return align_up((size_t)H * d * c * 2, 256) + align_up((size_t)H * d * sizeof(float2), 256);
-}
-
-nt_status fast_attn_out(void* z, const void* o, const nt_attn_weights* W, float eps, int c, int H, int d, void* prep,
+nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
                         const BatchMeta& m, int* status, cudaStream_t st) {
   const int Hd = H * d;
-  __nv_bfloat16* wg = (__nv_bfloat16*)prep;
-  float2* c01g = (float2*)((char*)prep + align_up((size_t)Hd * c * 2, 256));
-  {
-    const void* srcs[1] = {W->W_g};
-    const int rows[1] = {Hd};
-    nt_status r = fast_ln_fold_prep(srcs, rows, 1, c, W->ln_gamma, W->ln_beta, wg, c01g, st);
-    if (r != NT_OK) return r;
-  }
+  const void* wg = ap.wg;
+  const float2* c01g = (const float2*)ap.c01g;
   const int zslab = c / 64, oslab = Hd / 64;
   const size_t smem = (size_t)zslab * Hd * 128 + (size_t)oslab * c * 128 + 2 * (size_t)(zslab + oslab) * 128 * 128 +
                       (size_t)Hd * 8 + 1024;
@@ -287,7 +277,7 @@ nt_status fast_attn_out(void* z, const void* o, const nt_attn_weights* W, float 
     if (!make_tmap_bf16(&p.wgmap, wg, 2, gdims, zstr, gbox)) return cuda_fail("attn_out W_g map");
     const unsigned long long wdims[2] = {(unsigned long long)Hd, (unsigned long long)c};
     const unsigned wbox[2] = {64, (unsigned)c};
-    if (!make_tmap_bf16(&p.womap, W->W_o, 2, wdims, ostr, wbox)) return cuda_fail("attn_out W_o map");
+    if (!make_tmap_bf16(&p.womap, W_o, 2, wdims, ostr, wbox)) return cuda_fail("attn_out W_o map");
   }
   const long long ntiles = (p.rows + 127) / 128;
   const unsigned grid = (unsigned)(ntiles < 148 ? ntiles : 148);

@@ -184,3 +184,121 @@ nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, l
 }
 
 }  // namespace ntp
+
+namespace ntp {
+
+// ------------------------------------------------------------------------------------------
+// Token-side projection (a few thousand rows, so a fraction of a percent of a block's work):
+//   out[r][n] (+)= sum_k A[r][k] W[n][k]   for up to two weight / output pairs sharing A.
+// 32 x 32 output tiles so that even T1 ~ 1.7k rows give several hundred CTAs; the A and W tiles are
+// staged whole in shared memory (K <= 1024).
+// ------------------------------------------------------------------------------------------
+struct TokGemmArgs {
+  const __nv_bfloat16* A;
+  long long rows;
+  int K;
+  const __nv_bfloat16* W[2];
+  int N[2];
+  void* out[2];
+  int out_f32;       // outputs are float (store) instead of bf16
+  int accumulate;    // bf16 outputs: out += result
+};
+
+__global__ void __launch_bounds__(256) token_gemm_kernel(TokGemmArgs a) {
+  extern __shared__ __align__(16) unsigned char tg_smem[];
+  const int K = a.K, ldk = K + 8;
+  __nv_bfloat16* As = reinterpret_cast<__nv_bfloat16*>(tg_smem);
+  __nv_bfloat16* Ws = As + 32 * ldk;
+  const long long r0 = (long long)blockIdx.x * 32;
+  int n0 = blockIdx.y * 32, which = 0;
+  if (n0 >= a.N[0]) { n0 -= a.N[0]; which = 1; }
+  const __nv_bfloat16* W = a.W[which];
+  const int N = a.N[which];
+  const int t = threadIdx.x, kv = K / 8;
+  for (int idx = t; idx < 32 * kv; idx += 256) {
+    const int r = idx / kv, c = idx - r * kv;
+    uint4 va = make_uint4(0, 0, 0, 0), vw = make_uint4(0, 0, 0, 0);
+    if (r0 + r < a.rows) va = *reinterpret_cast<const uint4*>(a.A + (r0 + r) * K + c * 8);
+    if (n0 + r < N) vw = *reinterpret_cast<const uint4*>(W + (long long)(n0 + r) * K + c * 8);
+    *reinterpret_cast<uint4*>(As + r * ldk + c * 8) = va;
+    *reinterpret_cast<uint4*>(Ws + r * ldk + c * 8) = vw;
+  }
+  __syncthreads();
+  const int ty = t >> 4, tx = t & 15;
+  float acc[2][2] = {};
+  for (int k = 0; k < K; k += 8) {
+    uint4 av[2], wv[2];
+    av[0] = *reinterpret_cast<const uint4*>(As + ty * ldk + k);
+    av[1] = *reinterpret_cast<const uint4*>(As + (ty + 16) * ldk + k);
+    wv[0] = *reinterpret_cast<const uint4*>(Ws + tx * ldk + k);
+    wv[1] = *reinterpret_cast<const uint4*>(Ws + (tx + 16) * ldk + k);
+    const unsigned* ap0 = reinterpret_cast<const unsigned*>(&av[0]);
+    const unsigned* ap1 = reinterpret_cast<const unsigned*>(&av[1]);
+    const unsigned* wp0 = reinterpret_cast<const unsigned*>(&wv[0]);
+    const unsigned* wp1 = reinterpret_cast<const unsigned*>(&wv[1]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float a0l = __uint_as_float(ap0[e] << 16), a0h = __uint_as_float(ap0[e] & 0xffff0000u);
+      const float a1l = __uint_as_float(ap1[e] << 16), a1h = __uint_as_float(ap1[e] & 0xffff0000u);
+      const float w0l = __uint_as_float(wp0[e] << 16), w0h = __uint_as_float(wp0[e] & 0xffff0000u);
+      const float w1l = __uint_as_float(wp1[e] << 16), w1h = __uint_as_float(wp1[e] & 0xffff0000u);
+      acc[0][0] = fmaf(a0l, w0l, fmaf(a0h, w0h, acc[0][0]));
+      acc[0][1] = fmaf(a0l, w1l, fmaf(a0h, w1h, acc[0][1]));
+      acc[1][0] = fmaf(a1l, w0l, fmaf(a1h, w0h, acc[1][0]));
+      acc[1][1] = fmaf(a1l, w1l, fmaf(a1h, w1h, acc[1][1]));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const long long r = r0 + ty + 16 * i;
+      const int n = n0 + tx + 16 * j;
+      if (r >= a.rows || n >= N) continue;
+      if (a.out_f32) {
+        reinterpret_cast<float*>(a.out[which])[r * N + n] = acc[i][j];
+      } else {
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(a.out[which]) + r * N + n;
+        const float base = a.accumulate ? __bfloat162float(*o) : 0.f;
+        *o = __float2bfloat16_rn(base + acc[i][j]);
+      }
+    }
+}
+
+bool fast_token_gemm_supported(int K, int N0, int N1) {
+  return K % 8 == 0 && K >= 8 && K <= 1024 && N0 % 32 == 0 && N1 % 32 == 0;
+}
+
+nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, int N0, void* out0, const void* W1,
+                          int N1, void* out1, int out_f32, int accumulate, const char* name, cudaStream_t st) {
+  if (rows <= 0) return NT_OK;
+  TokGemmArgs a{};
+  a.A = (const __nv_bfloat16*)A;
+  a.rows = rows;
+  a.K = K;
+  a.W[0] = (const __nv_bfloat16*)W0;
+  a.W[1] = (const __nv_bfloat16*)W1;
+  a.N[0] = N0;
+  a.N[1] = N1;
+  a.out[0] = out0;
+  a.out[1] = out1;
+  a.out_f32 = out_f32;
+  a.accumulate = accumulate;
+  const size_t smem = (size_t)2 * 32 * (K + 8) * 2;
+  static size_t attr = 0;
+  if (smem > 48 * 1024 && smem > attr) {
+    if (cudaFuncSetAttribute(token_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 140 * 1024) != cudaSuccess)
+      return cuda_fail("token gemm smem attribute");
+    attr = 140 * 1024;
+  }
+  const long long bx = (rows + 31) / 32;
+  if (bx > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  dim3 grid((unsigned)bx, (unsigned)((N0 + N1) / 32));
+  {
+    LaunchScope ls(name, st);
+    token_gemm_kernel<<<grid, 256, smem, st>>>(a);
+  }
+  return cuda_ok(name);
+}
+
+}  // namespace ntp

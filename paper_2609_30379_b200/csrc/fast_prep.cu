@@ -1,0 +1,119 @@
+// Weight preparation for the tensor-core projections: LayerNorm folded into the weights.
+//   out[n][:] = fp16(W[n][:] * gamma),  c01[n] = (sum_k W[n][k] beta[k],  sum_k out[n][k])
+// so that (LN(z) W^T)[n] = rstd * (z . out[n] - mean * c01[n].y) + c01[n].x.
+// One launch prepares up to two jobs (different K / gamma / beta); a job concatenates up to six
+// source matrices; a NULL source stands for zero rows (padding).  gamma == NULL copies W.
+// The folded weights are fp16: 11 significant bits instead of bf16's 8, at the same MMA rate.
+#include "fast.cuh"
+
+namespace ntp {
+
+struct PrepJob {
+  const __nv_bfloat16* src[6];
+  int rows[6];
+  int nsrc, K, total;
+  const __nv_bfloat16* gamma;
+  const __nv_bfloat16* beta;
+  __half* out;
+  float2* c01;
+};
+struct PrepArgs { PrepJob job[2]; int njobs; };
+
+__global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
+  int n = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  int j = 0;
+  while (j < a.njobs && n >= a.job[j].total) { n -= a.job[j].total; ++j; }
+  if (j >= a.njobs) return;
+  const PrepJob& J = a.job[j];
+  int src = 0, r = n;
+  while (r >= J.rows[src]) { r -= J.rows[src]; ++src; }
+  const __nv_bfloat16* w = J.src[src] ? J.src[src] + (long long)r * J.K : nullptr;
+  float c0 = 0.f, c1 = 0.f;
+  for (int k = lane; k < J.K; k += 32) {
+    const float wv = w ? __bfloat162float(w[k]) : 0.f;
+    __half o = __float2half_rn(wv);
+    if (J.gamma) {
+      o = __float2half_rn(wv * __bfloat162float(J.gamma[k]));
+      c0 = fmaf(wv, __bfloat162float(J.beta[k]), c0);
+      c1 += __half2float(o);
+    }
+    J.out[(long long)n * J.K + k] = o;
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    c0 += __shfl_xor_sync(0xffffffffu, c0, o);
+    c1 += __shfl_xor_sync(0xffffffffu, c1, o);
+  }
+  if (lane == 0) J.c01[n] = make_float2(c0, c1);
+}
+
+static void add_job(PrepArgs& a, const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
+                    const void* beta, void* out, void* c01) {
+  PrepJob& J = a.job[a.njobs++];
+  J.total = 0;
+  for (int i = 0; i < nsrc; ++i) {
+    J.src[i] = (const __nv_bfloat16*)srcs[i];
+    J.rows[i] = rows[i];
+    J.total += rows[i];
+  }
+  J.nsrc = nsrc;
+  J.K = K;
+  J.gamma = (const __nv_bfloat16*)gamma;
+  J.beta = (const __nv_bfloat16*)beta;
+  J.out = (__half*)out;
+  J.c01 = (float2*)c01;
+}
+
+static nt_status run_prep(const PrepArgs& a, cudaStream_t st) {
+  int total = 0;
+  for (int j = 0; j < a.njobs; ++j) total += a.job[j].total;
+  {
+    LaunchScope ls("weight_prep", st);
+    ln_fold_prep_kernel<<<(total + 7) / 8, 256, 0, st>>>(a);
+  }
+  return cuda_ok("weight_prep launch");
+}
+
+// Triangle update: job 0 = [W_ag; W_ap; W_bg; W_bp; W_g] folded with LN_in (K = c_z),
+//                  job 1 = W_o folded with LN_out (K = c_h).
+nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep, TriPrep& out, cudaStream_t st) {
+  char* p = (char*)prep;
+  const int rows1 = 4 * c_h + c_z;
+  out.w1 = p;
+  out.wg = p + (size_t)4 * c_h * c_z * 2;
+  p += align_up((size_t)rows1 * c_z * 2, 256);
+  out.c01_1 = p;
+  out.c01g = p + (size_t)4 * c_h * sizeof(float2);
+  p += align_up((size_t)rows1 * sizeof(float2), 256);
+  out.wo = p;
+  p += align_up((size_t)c_z * c_h * 2, 256);
+  out.c01o = p;
+  PrepArgs a{};
+  const void* s0[5] = {W->W_ag, W->W_ap, W->W_bg, W->W_bp, W->W_g};
+  const int r0[5] = {c_h, c_h, c_h, c_h, c_z};
+  add_job(a, s0, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1);
+  const void* s1[1] = {W->W_o};
+  const int r1[1] = {c_z};
+  add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o);
+  return run_prep(a, st);
+}
+
+// Attention: [W_q; W_k; W_v; W_b (H rows); zero rows up to 16; W_g] folded with LN (K = c).
+nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* prep, AttnPrep& out, cudaStream_t st) {
+  const int Hd = H * d;
+  const int rows = 3 * Hd + 16 + Hd;
+  char* p = (char*)prep;
+  out.w = p;
+  out.wg = p + (size_t)(3 * Hd + 16) * c * 2;
+  p += align_up((size_t)rows * c * 2, 256);
+  out.c01 = p;
+  out.c01g = p + (size_t)(3 * Hd + 16) * sizeof(float2);
+  PrepArgs a{};
+  const void* s0[6] = {W->W_q, W->W_k, W->W_v, W->W_b, nullptr, W->W_g};
+  const int r0[6] = {Hd, Hd, Hd, W->W_b ? H : 0, W->W_b ? 16 - H : 16, W->W_g ? Hd : 0};
+  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01);
+  return run_prep(a, st);
+}
+
+}  // namespace ntp

@@ -238,84 +238,12 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
-// ------------------------------------------------------------------------------------------
-// weight preparation: out[n][:] = bf16(W[n][:] * gamma), c01[n] = (sum_k W[n][k] beta[k], sum_k out[n][k]);
-// gamma == NULL copies W and writes zeros.  One warp per output row; sources are concatenated.
-// ------------------------------------------------------------------------------------------
-struct PrepArgs {
-  const __nv_bfloat16* src[5];
-  int rows[5];
-  int nsrc, K;
-  const __nv_bfloat16* gamma;
-  const __nv_bfloat16* beta;
-  __half* out;     // folded weights are kept in fp16: 11 significant bits instead of 8, same MMA rate
-  float2* c01;
-};
-
-__global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
-  const int n = blockIdx.x * 8 + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  int total = 0;
-  for (int i = 0; i < a.nsrc; ++i) total += a.rows[i];
-  if (n >= total) return;
-  int src = 0, r = n;
-  while (r >= a.rows[src]) { r -= a.rows[src]; ++src; }
-  const __nv_bfloat16* w = a.src[src] + (long long)r * a.K;
-  float c0 = 0.f, c1 = 0.f;
-  for (int k = lane; k < a.K; k += 32) {
-    const float wv = __bfloat162float(w[k]);
-    __half o = __float2half_rn(wv);
-    if (a.gamma) {
-      o = __float2half_rn(wv * __bfloat162float(a.gamma[k]));
-      c0 = fmaf(wv, __bfloat162float(a.beta[k]), c0);
-      c1 += __half2float(o);
-    }
-    a.out[(long long)n * a.K + k] = o;
-  }
-#pragma unroll
-  for (int o = 16; o; o >>= 1) {
-    c0 += __shfl_xor_sync(0xffffffffu, c0, o);
-    c1 += __shfl_xor_sync(0xffffffffu, c1, o);
-  }
-  if (lane == 0) a.c01[n] = make_float2(c0, c1);
-}
-
-nt_status fast_ln_fold_prep(const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
-                            const void* beta, void* out, void* c01, cudaStream_t st) {
-  PrepArgs a{};
-  int total = 0;
-  for (int i = 0; i < nsrc; ++i) {
-    a.src[i] = (const __nv_bfloat16*)srcs[i];
-    a.rows[i] = rows[i];
-    total += rows[i];
-  }
-  a.nsrc = nsrc;
-  a.K = K;
-  a.gamma = (const __nv_bfloat16*)gamma;
-  a.beta = (const __nv_bfloat16*)beta;
-  a.out = (__half*)out;
-  a.c01 = (float2*)c01;
-  {
-    LaunchScope ls("weight_prep", st);
-    ln_fold_prep_kernel<<<(total + 7) / 8, 256, 0, st>>>(a);
-  }
-  return cuda_ok();
-}
-
 bool fast_tri_in_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) && (c_h == 64 || c_h == 128); }
 
-size_t fast_tri_in_prep_bytes(int c_z, int c_h) {
-  return align_up((size_t)4 * c_h * c_z * 2, 256) + align_up((size_t)4 * c_h * sizeof(float2), 256);
-}
-
-nt_status fast_tri_in(const void* z, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* a, void* b,
-                      void* prep, const BatchMeta& m, int* status, cudaStream_t st) {
-  __nv_bfloat16* wprime = (__nv_bfloat16*)prep;
-  float2* c01 = (float2*)((char*)prep + align_up((size_t)4 * c_h * c_z * 2, 256));
-  const void* srcs[4] = {W->W_ag, W->W_ap, W->W_bg, W->W_bp};
-  const int rows[4] = {c_h, c_h, c_h, c_h};
-  nt_status r = fast_ln_fold_prep(srcs, rows, 4, c_z, W->ln_in_gamma, W->ln_in_beta, wprime, c01, st);
-  if (r != NT_OK) return r;
+nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int c_h, void* a, void* b,
+                      const BatchMeta& m, int* status, cudaStream_t st) {
+  const void* wprime = tp.w1;
+  const float2* c01 = (const float2*)tp.c01_1;
   const int nslab = c_z / 64;
   const size_t smem = (size_t)nslab * 4 * c_h * 128 + 2 * (size_t)nslab * 128 * 128 + 8 * 2048 + 4 * c_h * 8 + 1024;
   static bool attr_set = false;

@@ -270,30 +270,12 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
 
 bool fast_tri_out_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) && (c_h == 64 || c_h == 128); }
 
-size_t fast_tri_out_prep_bytes(int c_z, int c_h) {
-  return align_up((size_t)c_z * c_h * 2, 256) + align_up((size_t)c_z * c_z * 2, 256) +
-         2 * align_up((size_t)c_z * sizeof(float2), 256);
-}
-
-nt_status fast_tri_out(void* z, const void* t, const nt_trimul_weights* W, float eps, int c_z, int c_h, void* prep,
-                       const BatchMeta& m, int* status, cudaStream_t st) {
-  char* pp = (char*)prep;
-  __nv_bfloat16* wo = (__nv_bfloat16*)pp;
-  pp += align_up((size_t)c_z * c_h * 2, 256);
-  __nv_bfloat16* wg = (__nv_bfloat16*)pp;
-  pp += align_up((size_t)c_z * c_z * 2, 256);
-  float2* c01o = (float2*)pp;
-  pp += align_up((size_t)c_z * sizeof(float2), 256);
-  float2* c01g = (float2*)pp;
-  {
-    const void* srcs[1] = {W->W_o};
-    const int rows[1] = {c_z};
-    nt_status r = fast_ln_fold_prep(srcs, rows, 1, c_h, W->ln_out_gamma, W->ln_out_beta, wo, c01o, st);
-    if (r != NT_OK) return r;
-    const void* srcs2[1] = {W->W_g};
-    r = fast_ln_fold_prep(srcs2, rows, 1, c_z, W->ln_in_gamma, W->ln_in_beta, wg, c01g, st);
-    if (r != NT_OK) return r;
-  }
+nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int c_z, int c_h, const BatchMeta& m,
+                       int* status, cudaStream_t st) {
+  const void* wo = tp.wo;
+  const void* wg = tp.wg;
+  const float2* c01o = (const float2*)tp.c01o;
+  const float2* c01g = (const float2*)tp.c01g;
   const int zslab = c_z / 64, hslab = c_h / 64;
   const size_t smem = (size_t)hslab * c_z * 128 + (size_t)zslab * c_z * 128 +
                       2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 2 * c_z * 8 + 1024;
