@@ -250,7 +250,7 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
   const int Hd = H * d;
   const bool pair = order == NT_ORDER_PAIR_IJC;
   const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma;
-  const bool tc_in = tc && fast_attn_in_supported(c, H, d);
+  const bool tc_in = tc && fast_attn_in_supported(c, H, d) && fast_attn_core_supported(H, d);   // bias goes out times sqrt(d)
   const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
   AttnPrep aprep{};
   if (tc_in || tc_out) {
@@ -289,7 +289,8 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
     }
     if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d))
-      r = fast_attn_core(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, pair ? 1 : 0, m, st);
+      r = fast_attn_core(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, pair ? 1 : 0, tc_in ? 1 : 0, m,
+                         L->status_d, st);
     else
       r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
                               (T*)w.o, H, d, pair ? 1 : 0, m, st);

@@ -22,7 +22,7 @@ nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, 
 // head-major channel-major (nullable)
 bool fast_attn_core_supported(int H, int d);
 nt_status fast_attn_core(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
-                         int pair_order, const BatchMeta& m, cudaStream_t st);
+                         int pair_order, int bias_prescaled, const BatchMeta& m, int* status, cudaStream_t st);
 
 // triangle contraction on tcgen05: a, b, t are three equally spaced channel-major buffers
 // (b = a + stride, t = a + 2 * stride)
@@ -34,6 +34,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
 struct TriPrep { void *w1, *c01_1, *wg, *c01g, *wo, *c01o; };
 struct AttnPrep { void *w, *c01, *wg, *c01g; };
 nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep, TriPrep& out, cudaStream_t st);
+// the bias rows are folded times sqrt(d): the attention core keeps scores in units of q.k
 nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* prep, AttnPrep& out, cudaStream_t st);
 
 // a = sig(LN(z) W_ag^T) * (LN(z) W_ap^T), b likewise: fp16, channel-major

@@ -11,6 +11,7 @@ namespace ntp {
 struct PrepJob {
   const __nv_bfloat16* src[6];
   int rows[6];
+  float scale[6];   // extra factor on the rows of a source (and on its c0, c1)
   int nsrc, K, total;
   const __nv_bfloat16* gamma;
   const __nv_bfloat16* beta;
@@ -31,7 +32,7 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
   const __nv_bfloat16* w = J.src[src] ? J.src[src] + (long long)r * J.K : nullptr;
   float c0 = 0.f, c1 = 0.f;
   for (int k = lane; k < J.K; k += 32) {
-    const float wv = w ? __bfloat162float(w[k]) : 0.f;
+    const float wv = w ? __bfloat162float(w[k]) * J.scale[src] : 0.f;
     __half o = __float2half_rn(wv);
     if (J.gamma) {
       o = __float2half_rn(wv * __bfloat162float(J.gamma[k]));
@@ -49,12 +50,13 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
 }
 
 static void add_job(PrepArgs& a, const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
-                    const void* beta, void* out, void* c01) {
+                    const void* beta, void* out, void* c01, const float* scale = nullptr) {
   PrepJob& J = a.job[a.njobs++];
   J.total = 0;
   for (int i = 0; i < nsrc; ++i) {
     J.src[i] = (const __nv_bfloat16*)srcs[i];
     J.rows[i] = rows[i];
+    J.scale[i] = scale ? scale[i] : 1.0f;
     J.total += rows[i];
   }
   J.nsrc = nsrc;
@@ -112,7 +114,8 @@ nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* pr
   PrepArgs a{};
   const void* s0[6] = {W->W_q, W->W_k, W->W_v, W->W_b, nullptr, W->W_g};
   const int r0[6] = {Hd, Hd, Hd, W->W_b ? H : 0, W->W_b ? 16 - H : 16, W->W_g ? Hd : 0};
-  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01);
+  const float sc[6] = {1.f, 1.f, 1.f, sqrtf((float)d), 1.f, 1.f};   // bias rows times sqrt(d)
+  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01, sc);
   return run_prep(a, st);
 }
 

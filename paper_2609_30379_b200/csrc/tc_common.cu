@@ -1,5 +1,5 @@
 // Host side of the TMA plumbing: resolves cuTensorMapEncodeTiled through the runtime (no link-time
-// dependency on the driver library) and encodes bf16 tiled maps with 128-byte swizzle.
+// dependency on the driver library) and encodes tiled maps for 16-bit elements.
 #include "tc_common.cuh"
 
 namespace ntp {
@@ -18,8 +18,8 @@ EncodeTiledFn get_encode_tiled() {
   return fn;
 }
 
-bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-                    const unsigned long long* strides_bytes, const unsigned* box) {
+bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
   EncodeTiledFn enc = get_encode_tiled();
   if (!enc) return false;
   cuuint64_t gdim[5];
@@ -31,10 +31,19 @@ bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned
     estr[i] = 1;
     if (i + 1 < rank) gstr[i] = strides_bytes[i];
   }
+  const CUtensorMapSwizzle sw = swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                               : swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                                     : CU_TENSOR_MAP_SWIZZLE_128B;
+  // bf16 and fp16 tiles move identically (no conversion on the way), so one 16-bit type serves both
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bdim,
-                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+                    const unsigned long long* strides_bytes, const unsigned* box) {
+  return make_tmap_16bit(map, base, rank, dims, strides_bytes, box, 128);
 }
 
 }  // namespace ntp

@@ -20,6 +20,9 @@ EncodeTiledFn get_encode_tiled();
 // bf16 tensor map with 128-byte swizzle; dims / strides fastest first (strides in bytes for dims 1..rank-1)
 bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                     const unsigned long long* strides_bytes, const unsigned* box);
+// same with a 32-, 64- or 128-byte swizzle span (the inner box extent in bytes must not exceed it)
+bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
+                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes);
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------- device helpers
