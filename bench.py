@@ -239,7 +239,7 @@ def main():
         build.build_library()
     if world > 1:
         dist.barrier()
-    from paper_2609_30379_b200 import binding as nt, runner
+    from paper_2609_30379_b200 import binding as nt, replicas, runner
 
     if args.force_generic:
         nt.nt_force_generic(True)
@@ -279,10 +279,7 @@ def main():
     launches = nt.nt_launch_count() - launches0
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(ms, device="cuda")
     unit_count = cfg.T2 if cfg.kind == "pair" else cfg.T1
     value = world * cfg.blocks * unit_count * steps / (ms * 1e-3)
     peak_alloc = torch.cuda.max_memory_allocated()
@@ -336,10 +333,7 @@ def main():
         e2e_step()
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = replicas.max_over_ranks(e2e_s, device="cuda")
     e2e_value = world * cfg.blocks * unit_count * steps / e2e_s
 
     if rank != 0:
