@@ -154,6 +154,33 @@ nt_status nt_segment_reduce(nt_dtype dt, nt_reduce op, int32_t C, int64_t G, int
                             const int64_t *splits_d, const void *v, void *out,
                             int32_t *status_d, nt_stream stream);
 
+/*
+ * nt_pair_broadcast_static -- nt_pair_broadcast without a caller workspace.  (The paper has no
+ * counterpart: this entry point exists for integration, not for the method.)
+ *
+ * Same arguments, result and error behaviour as nt_pair_broadcast, minus `workspace`: the scratch
+ * for the projected token features lives in a fixed array inside the library's device module.  It is
+ * meant for callers that cannot allocate device memory themselves: an embedding application whose
+ * interface passes only input and output pointers, or a serving loop that must never call
+ * cudaMalloc (a device-wide synchronising call that can fail when memory is fragmented).
+ *   - Limit: the batch must need at most NT_PAIR_BROADCAST_STATIC_BYTES of scratch, i.e.
+ *     2 * round_up(T1 * c_z * 4, 256) bytes (about T1 * c_z <= 1,048,000); larger batches are refused
+ *     with NT_ERR_WORKSPACE and a message on stderr, with nothing launched.
+ *   - Every GPU that loads the library holds the array (NT_PAIR_BROADCAST_STATIC_BYTES) until the
+ *     process exits.
+ *   - The first call on each device looks up the array's device address (no allocation, no
+ *     synchronisation); make that first call before any stream capture begins.
+ *   - All calls share the one array and it keeps whatever the last call left in it.  Nothing in it
+ *     needs clearing (every call overwrites what it reads), but two calls that overlap on the GPU --
+ *     different streams, or different host threads -- race on it: serialise them.
+ *   - The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ */
+#define NT_PAIR_BROADCAST_STATIC_BYTES (8u << 20)
+nt_status nt_pair_broadcast_static(const nt_layout *L, nt_dtype dt, int32_t c_s, int32_t c_z,
+                                   const void *x, const void *W_a, const void *W_b,
+                                   const void *ln_gamma, const void *ln_beta, float ln_eps,
+                                   void *z, nt_stream stream);
+
 /* ------------------------------- auxiliaries (not among the five) ------------------------------- */
 
 /* x[T1, c_s] += m[T1, c_z] W_r^T  -- the projection g of Eq. 1 line 3 applied to the reduced

@@ -1,0 +1,65 @@
+// nt_pair_broadcast_static: the pair broadcast for callers that cannot hand the library a workspace.
+//
+// nt_pair_broadcast needs scratch for the projected token features u = x W_a^T and v = x W_b^T
+// (two float [T1, c_z] arrays) and takes it from a caller-allocated workspace.  Some callers have
+// nothing to allocate with: a host application that embeds the library behind an interface that only
+// passes input and output pointers, or a latency-critical serving loop that must not call cudaMalloc
+// (it serialises against the whole device and can fail once memory is fragmented).  For them the
+// scratch lives in a file-scope __device__ array of fixed size that is part of the loaded module.
+//
+// In host code the array's name is only a host-side stand-in for the symbol, not a device address,
+// so the device address is looked up once per device with cudaGetSymbolAddress (with that device
+// current) and that pointer is what the kernels receive.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace ntp {
+
+constexpr size_t PB_STATIC_BYTES = NT_PAIR_BROADCAST_STATIC_BYTES;
+constexpr int PB_MAX_DEVICES = 64;
+
+static __device__ __align__(256) unsigned char g_pb_scratch[PB_STATIC_BYTES];
+
+static std::mutex g_pb_mu;
+static void* g_pb_ptr[PB_MAX_DEVICES] = {};
+
+// Device address of the scratch array on the current device; resolved on the first call per device.
+static nt_status pb_scratch_ptr(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail("cudaGetDevice");
+  if (dev < 0 || dev >= PB_MAX_DEVICES) return NT_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lk(g_pb_mu);
+  if (!g_pb_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_pb_scratch) != cudaSuccess || !ptr)
+      return cuda_fail("cudaGetSymbolAddress(pair broadcast scratch)");
+    g_pb_ptr[dev] = ptr;
+  }
+  *out = g_pb_ptr[dev];
+  return NT_OK;
+}
+
+}  // namespace ntp
+
+using namespace ntp;
+
+extern "C" nt_status nt_pair_broadcast_static(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_t c_z,
+                                              const void* x, const void* W_a, const void* W_b, const void* ln_gamma,
+                                              const void* ln_beta, float ln_eps, void* z, nt_stream stream) {
+  if (!L || L->B < 0 || c_z <= 0) return NT_ERR_INVALID_ARG;
+  if (L->B > 0 && !L->lengths_h) return NT_ERR_INVALID_ARG;
+  const int32_t dims[5] = {c_s, c_z, 0, 0, 0};
+  const size_t need = nt_workspace_bytes(NT_OP_PAIR_BROADCAST, dt, NT_ORDER_PAIR_IJC, L->lengths_h, L->B, dims);
+  if (need > PB_STATIC_BYTES) {
+    fprintf(stderr,
+            "libnested_pair: nt_pair_broadcast_static needs %zu bytes of scratch for this batch but its built-in "
+            "array holds %zu (T1 * c_z is limited to %zu); use nt_pair_broadcast with a workspace instead\n",
+            need, (size_t)PB_STATIC_BYTES, (size_t)(PB_STATIC_BYTES / 8));
+    return NT_ERR_WORKSPACE;
+  }
+  void* scratch = nullptr;
+  nt_status r = pb_scratch_ptr(&scratch);
+  if (r != NT_OK) return r;
+  return nt_pair_broadcast(L, dt, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, scratch, PB_STATIC_BYTES, stream);
+}

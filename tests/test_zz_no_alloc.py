@@ -1,0 +1,68 @@
+"""nt_pair_broadcast_static: the workspace-free variant of the pair broadcast.
+
+Some users of the library cannot allocate device memory (they sit behind an interface that only
+hands over input and output pointers, or they run where cudaMalloc is off limits), so this entry
+point keeps its scratch in a fixed array inside the library.  The test calls it through the C ABI
+twice in a row -- the array is shared and keeps the previous call's contents -- and checks each
+result against nt_pair_broadcast on the same inputs.  It is collected last so that a run stopping at
+the first failure has already run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_30379_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nt():
+    from paper_2609_30379_b200 import build
+    build.build_library()
+    from paper_2609_30379_b200 import binding
+    return binding
+
+
+def _run(nt, cfg, seed_shift):
+    from paper_2609_30379_b200 import runner
+    cfg = wl.Config(cfg.name, cfg.dtype, cfg.lengths, cfg.c_s, cfg.c_z, cfg.c_h, cfg.H, cfg.d, 1, cfg.seed + seed_shift)
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    b = st.W[0]["broadcast"]
+    x = runner.to_device(inp["x"], st.dtype)
+    nt.nt_pair_broadcast(st.L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, st.z, st.workspace)
+    ref = st.z.clone()
+    out = torch.full_like(ref, float("nan"))
+    nt.nt_pair_broadcast_static(st.L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, out)
+    torch.cuda.synchronize()
+    return out, ref
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_static_scratch_matches_workspace_variant_twice(nt, dtype):
+    cfg_a = wl.Config("na", dtype, (37, 5, 64, 0, 19), c_s=64, c_z=128, c_h=128, H=4, d=32, blocks=1, seed=100)
+    cfg_b = wl.Config("nb", dtype, (12, 90), c_s=32, c_z=64, c_h=64, H=4, d=16, blocks=1, seed=200)
+    for cfg, shift in ((cfg_a, 0), (cfg_b, 1), (cfg_a, 2)):      # consecutive calls share the array
+        out, ref = _run(nt, cfg, shift)
+        assert torch.isfinite(out.float()).all()
+        # same kernels on the same inputs: the tolerance of the other bf16 / fp32 parity tests is ample
+        tol = 2e-2 if dtype == "bf16" else 1e-4
+        assert float((out.float() - ref.float()).abs().max()) <= tol
+        assert torch.equal(out, ref)
+
+
+def test_static_scratch_rejects_oversized_batches(nt):
+    from paper_2609_30379_b200 import runner
+    # T1 * c_z = 9000 * 128 floats twice exceeds the 8 MiB array; refused before anything runs
+    cfg = wl.Config("big", "bf16", (9000,), c_s=8, c_z=128, c_h=128, H=4, d=32, blocks=1, seed=7)
+    L = nt.Layout(cfg.lengths)
+    x = torch.zeros((cfg.T1, cfg.c_s), dtype=torch.bfloat16, device="cuda")
+    W = torch.zeros((cfg.c_z, cfg.c_s), dtype=torch.bfloat16, device="cuda")
+    g = torch.ones(cfg.c_z, dtype=torch.bfloat16, device="cuda")
+    z = torch.empty((16, cfg.c_z), dtype=torch.bfloat16, device="cuda")   # never written
+    before = nt.nt_launch_count()
+    with pytest.raises(nt.NtError) as e:
+        nt.nt_pair_broadcast_static(L, x, W, W, g, g, 1e-5, z)
+    assert e.value.status == 3                      # NT_ERR_WORKSPACE
+    assert nt.nt_launch_count() == before
