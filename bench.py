@@ -79,6 +79,11 @@ def kernel_work(cfg: wl.Config):
     return w
 
 
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (cfg2 only);
+# other workloads report traffic = None.
+NCU_TRAFFIC_CFG2 = {"attn_core": 367.4e6, "tri_in": 230.2e6, "tri_contract": 256.3e6}
+
+
 def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
     if name not in work or launches == 0:
         return None
@@ -312,6 +317,8 @@ def main():
             kernels[k]["bound"] = roofs[k]["bound"]
     dominant = max(prof.items(), key=lambda kv: kv[1][0])[0] if prof else None
     roofline = roofs.get(dominant) if dominant else None
+    if roofline and cfg.name == "cfg2" and not args.force_generic:
+        roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
     # ---- end to end through the public API with host buffers
     x_pin = torch.from_numpy(np.ascontiguousarray(inp["x"])).to(stack.dtype).pin_memory()
