@@ -288,7 +288,7 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       pa.W1 = W->W_b; pa.Nout = H; pa.out = w.bias; pa.out_mode = O_CHANNEL_MAJOR;
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
     }
-    if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d))
+    if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d) && (!W->W_b || tc_in))
       r = fast_attn_core(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, pair ? 1 : 0, tc_in ? 1 : 0, m,
                          L->status_d, st);
     else

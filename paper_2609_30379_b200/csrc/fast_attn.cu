@@ -214,7 +214,9 @@ __device__ inline void attn_step_dispatch(bool masked, int rem, float (&sacc)[AT
     attn_step<D, 4, BIAS, true>(sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
 }
 
-template <int D>
+// BIAS: 0 = no bias, 1 = bias tile resident in shared memory (samples with want_resident), 2 = bias through L1/L2.
+// A launch handles the samples whose bias tile fits (BIAS == 1) or the ones whose tile does not (BIAS == 2).
+template <int D, int BIAS>
 __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_constant__ AttnCoreParams p) {
   constexpr int KV_TILE = AT_K * D * 2;      // bytes of one K or V block
   constexpr int Q_TILE = AT_Q * D * 2;
@@ -239,6 +241,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
     int s = 0;
     for (; s < m.B; ++s) {
       const int N = m.N[s];
+      if (BIAS != 0 && (AT_Q * at_bias_stride(N) <= AT_RES_CAP) != (BIAS == 1)) continue;   // other launch's sample
       const long long njb = (N + AT_Q - 1) / AT_Q;
       const long long nic = pair_order ? (N + p.ichunk - 1) / p.ichunk : (N > 0 ? 1 : 0);
       const long long cnt = njb * H * nic;
@@ -266,9 +269,9 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
   const int nkb = (N + AT_K - 1) / AT_K;
   const int n_active = min(AT_CONSUMERS, (N - j0 + 15) / 16);   // consumer warps that own valid queries
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const bool has_bias = p.bias != nullptr;
+  constexpr bool has_bias = BIAS != 0;
   const int bstride = at_bias_stride(N);
-  const bool resident = has_bias && p.bias_prescaled && AT_Q * bstride <= p.bias_bytes;
+  constexpr bool resident = BIAS == 1;
   const __nv_bfloat16* bias_h =
       has_bias ? p.bias + (long long)H * m.cm_off[s] + (long long)h * N * ld : nullptr;
   if (threadIdx.x == 0) {
@@ -333,7 +336,6 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
   const int jr0 = min(j0 + rloc, N - 1), jr1 = min(j0 + rloc + 8, N - 1);
   const __nv_bfloat16* bg0 = has_bias ? bias_h + (long long)jr0 * ld : nullptr;
   const __nv_bfloat16* bg1 = has_bias ? bias_h + (long long)jr1 * ld : nullptr;
-  const int bias_mode = !has_bias ? 0 : (resident ? 1 : 2);
   int st = 0, qs = 0;
   unsigned ph = 0, qph = 0;
   for (int i = i_begin; i < i_end; ++i) {
@@ -360,15 +362,8 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
       const int k0 = kb * AT_K;
       const bool masked = tail && kb == nkb - 1;
       const unsigned bias_s = bias_lane + k0 * 2;
-      if (bias_mode == 1)
-        attn_step_dispatch<D, 1>(masked, N - k0, sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
-                                 sc2, p.bias_mul, lane);
-      else if (bias_mode == 2)
-        attn_step_dispatch<D, 2>(masked, N - k0, sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
-                                 sc2, p.bias_mul, lane);
-      else
-        attn_step_dispatch<D, 0>(masked, N - k0, sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
-                                 sc2, p.bias_mul, lane);
+      attn_step_dispatch<D, BIAS>(masked, N - k0, sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
+                                  sc2, p.bias_mul, lane);
       __syncwarp();
       if (lane == 0) mbar_arrive(&kvempty[st]);
       if (++st == AT_STAGES) { st = 0; ph ^= 1; }
@@ -395,6 +390,40 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
 
 bool fast_attn_core_supported(int H, int d) { return (d == 16 || d == 32 || d == 64) && H >= 1; }
 
+template <int D, int BIAS>
+static nt_status launch_attn_mode(AttnCoreParams& p, int bias_bytes, cudaStream_t st) {
+  const BatchMeta& m = p.m;
+  auto count = [&](int ic) {
+    long long c = 0;
+    for (int s = 0; s < m.B; ++s) {
+      const long long N = m.N[s], njb = (N + AT_Q - 1) / AT_Q;
+      if (BIAS != 0 && (AT_Q * at_bias_stride((int)N) <= AT_RES_CAP) != (BIAS == 1)) continue;
+      const long long nic = p.pair_order ? (N + ic - 1) / ic : (N > 0 ? 1 : 0);
+      c += njb * p.H * nic;
+    }
+    return c;
+  };
+  int ichunk = 32;
+  while (p.pair_order && ichunk > 2 && count(ichunk) < 148 * 12) ichunk >>= 1;
+  p.ichunk = ichunk;
+  const long long blocks = count(ichunk);
+  if (blocks == 0) return NT_OK;
+  if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)2 * AT_STAGES * AT_K * D * 2 + 2 * (size_t)AT_Q * D * 2 + (BIAS == 1 ? bias_bytes + 128 : 0) + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_core_kernel<D, BIAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) !=
+        cudaSuccess)
+      return cuda_fail("attention core smem attribute");
+    attr_set = true;
+  }
+  {
+    LaunchScope ls("attn_core", st);
+    attn_core_kernel<D, BIAS><<<(unsigned)blocks, AT_THREADS, smem, st>>>(p);
+  }
+  return cuda_ok("attention core launch");
+}
+
 template <int D>
 static nt_status launch_attn(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                              const __nv_bfloat16* bias, __nv_bfloat16* o, int H, int pair_order, int bias_prescaled,
@@ -409,32 +438,20 @@ static nt_status launch_attn(const __nv_bfloat16* q, const __nv_bfloat16* k, con
   p.bias_prescaled = bias_prescaled;
   p.bias_mul = bias_prescaled ? 1.0f : sqrtf((float)D);
   p.status = status;
+  // a bias must come stored times sqrt(d) (as the tensor-core input projection writes it)
+  if (bias && !bias_prescaled) return NT_ERR_UNSUPPORTED;
   p.row0 = pair_order ? m.pair_off[0] : m.tok_off[0];
   const long long rows = (pair_order ? m.pair_off[m.B] : m.tok_off[m.B]) - p.row0;
   if (rows <= 0) return NT_OK;
   if (rows > 0x7FFFFF00ll) return NT_ERR_UNSUPPORTED;
   int bias_bytes = 0;
-  if (bias && bias_prescaled)
-    for (int s = 0; s < m.B; ++s) {
-      const int res = AT_Q * at_bias_stride(m.N[s]);
-      if (res <= AT_RES_CAP && res > bias_bytes) bias_bytes = res;
-    }
+  bool any_long = false;
+  for (int s = 0; s < m.B; ++s) {
+    const int res = AT_Q * at_bias_stride(m.N[s]);
+    if (res <= AT_RES_CAP) { if (res > bias_bytes) bias_bytes = res; }
+    else any_long = true;
+  }
   p.bias_bytes = bias_bytes;
-  auto count = [&](int ic) {
-    long long c = 0;
-    for (int s = 0; s < m.B; ++s) {
-      const long long N = m.N[s], njb = (N + AT_Q - 1) / AT_Q;
-      const long long nic = pair_order ? (N + ic - 1) / ic : (N > 0 ? 1 : 0);
-      c += njb * H * nic;
-    }
-    return c;
-  };
-  int ichunk = 32;
-  while (pair_order && ichunk > 2 && count(ichunk) < 148 * 12) ichunk >>= 1;
-  p.ichunk = ichunk;
-  const long long blocks = count(ichunk);
-  if (blocks == 0) return NT_OK;
-  if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
   const int Hd = H * D;
   {
     const unsigned long long dims[2] = {(unsigned long long)Hd, (unsigned long long)rows};
@@ -444,18 +461,11 @@ static nt_status launch_attn(const __nv_bfloat16* q, const __nv_bfloat16* k, con
     if (!make_tmap_16bit(&p.kmap, k + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn k map");
     if (!make_tmap_16bit(&p.vmap, v + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn v map");
   }
-  const size_t smem = (size_t)2 * AT_STAGES * AT_K * D * 2 + 2 * (size_t)AT_Q * D * 2 + bias_bytes + 128 + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_core_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-      return cuda_fail("attention core smem attribute");
-    attr_set = true;
-  }
-  {
-    LaunchScope ls("attn_core", st);
-    attn_core_kernel<D><<<(unsigned)blocks, AT_THREADS, smem, st>>>(p);
-  }
-  return cuda_ok("attention core launch");
+  if (!bias) return launch_attn_mode<D, 0>(p, 0, st);
+  nt_status r = launch_attn_mode<D, 1>(p, bias_bytes, st);
+  if (r != NT_OK) return r;
+  if (any_long) r = launch_attn_mode<D, 2>(p, 0, st);
+  return r;
 }
 
 nt_status fast_attn_core(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
