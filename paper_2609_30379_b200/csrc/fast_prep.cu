@@ -17,6 +17,7 @@ struct PrepJob {
   const __nv_bfloat16* beta;
   __half* out;
   float2* c01;
+  __half* aug;      // nullable: [2][total][8] fp16 augmentation columns (see below)
 };
 struct PrepArgs { PrepJob job[2]; int njobs; };
 
@@ -46,11 +47,24 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
     c0 += __shfl_xor_sync(0xffffffffu, c0, o);
     c1 += __shfl_xor_sync(0xffffffffu, c1, o);
   }
-  if (lane == 0) J.c01[n] = make_float2(c0, c1);
+  if (lane == 0) {
+    J.c01[n] = make_float2(c0, c1);
+    if (J.aug) {
+      // Extra K columns that make the MMA itself apply the LayerNorm correction: against activation columns
+      // (m_hi, m_lo, m_hi, 1, 1) with m = -mean * rstd they contribute m * c1 + c0 (hi/lo split keeps ~22 bits).
+      const __half c1h = __float2half_rn(c1), c1l = __float2half_rn(c1 - __half2float(c1h));
+      const __half c0h = __float2half_rn(c0), c0l = __float2half_rn(c0 - __half2float(c0h));
+      const __half z = __float2half_rn(0.f);
+      __half* r0 = J.aug + (long long)n * 8;
+      __half* r1 = J.aug + ((long long)J.total + n) * 8;
+      r0[0] = c1h; r0[1] = c1h; r0[2] = c1l; r0[3] = c0h; r0[4] = c0l; r0[5] = z; r0[6] = z; r0[7] = z;
+      for (int e = 0; e < 8; ++e) r1[e] = z;
+    }
+  }
 }
 
 static void add_job(PrepArgs& a, const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
-                    const void* beta, void* out, void* c01, const float* scale = nullptr) {
+                    const void* beta, void* out, void* c01, const float* scale = nullptr, void* aug = nullptr) {
   PrepJob& J = a.job[a.njobs++];
   J.total = 0;
   for (int i = 0; i < nsrc; ++i) {
@@ -65,6 +79,7 @@ static void add_job(PrepArgs& a, const void* const* srcs, const int* rows, int n
   J.beta = (const __nv_bfloat16*)beta;
   J.out = (__half*)out;
   J.c01 = (float2*)c01;
+  J.aug = (__half*)aug;
 }
 
 static nt_status run_prep(const PrepArgs& a, cudaStream_t st) {
@@ -91,10 +106,16 @@ nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep
   out.wo = p;
   p += align_up((size_t)c_z * c_h * 2, 256);
   out.c01o = p;
+  p += align_up((size_t)c_z * sizeof(float2), 256);
+  out.aug1 = p;                         // [2][rows1][8] fp16
+  out.aug1_rows = rows1;
   PrepArgs a{};
-  const void* s0[5] = {W->W_ag, W->W_ap, W->W_bg, W->W_bp, W->W_g};
+  // The input projection computes D^T = W' z^T with 128 weight rows per MMA and pairs the gate rows of an
+  // accumulator with the value rows of the next one: c_h = 128 -> [ag, ap, bg, bp]; c_h = 64 -> [ag, bg, ap, bp].
+  const void* s128[5] = {W->W_ag, W->W_ap, W->W_bg, W->W_bp, W->W_g};
+  const void* s64[5] = {W->W_ag, W->W_bg, W->W_ap, W->W_bp, W->W_g};
   const int r0[5] = {c_h, c_h, c_h, c_h, c_z};
-  add_job(a, s0, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1);
+  add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, nullptr, out.aug1);
   const void* s1[1] = {W->W_o};
   const int r1[1] = {c_z};
   add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o);

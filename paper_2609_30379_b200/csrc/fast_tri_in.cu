@@ -1,17 +1,23 @@
-// Triangle-update input projection on tcgen05 (bf16, float accumulate):
+// Triangle-update input projection on tcgen05 (fp16 operands, float accumulate):
 //   zh = LN(z);  a = sigmoid(zh W_ag^T) * (zh W_ap^T);  b = sigmoid(zh W_bg^T) * (zh W_bp^T)
-// written channel-major (a[c][i][k], k contiguous) so the contraction's operands are K-major.
+// written channel-major in fp16 (a[c][i][k], k contiguous) so the contraction's operands are K-major.
 //
-// LayerNorm is folded into the product: with W' = W * gamma (column scale, rounded to bf16),
-// c1[n] = sum_k W'[n][k] and c0[n] = sum_k W[n][k] beta[k],
-//   (LN(z) W^T)[n] = rstd * (z . W'[n] - mean * c1[n]) + c0[n],
-// so the raw z tile goes from TMA straight into the MMA and only per-row mean / rstd (computed by
-// the epilogue threads from the same shared-memory tile) are needed afterwards.
+// The product is computed transposed, D^T[channel][position] = W' z'^T: the accumulator row (TMEM
+// lane) is the output channel and the columns are positions, so a thread that reads 32 columns
+// holds 32 consecutive k of one channel -- exactly a 64-byte channel-major run, stored with four
+// 16-byte stores and no transposition.
+//
+// LayerNorm is folded completely into the MMA.  With W' = W * gamma (fp16), c1[n] = sum_k W'[n][k],
+// c0[n] = sum_k W[n][k] beta[k]:
+//   (LN(z) W^T)[n] = (rstd z) . W'[n] + (-mean rstd) c1[n] + c0[n].
+// Four converter warps rewrite the bf16 z tile as fp16 scaled by the row's rstd and append five
+// extra K columns (m_hi, m_lo, m_hi, 1, 1), m = -mean rstd, that meet (c1_hi, c1_hi, c1_lo, c0_hi,
+// c0_lo) on the weight side (hi / lo halves keep ~22 bits), so the accumulator already holds the
+// normalised projection and the epilogue is sigmoid * value, convert, store.
 //
 // A tile is 128 packed positions made of four 32-position chunks, each a run of consecutive k inside
-// one pair row (s, i) taken from the offset table, so a warp's 32 accumulator rows are 32 consecutive
-// k of one row and transpose into 64-byte channel-major runs.  The weights (4 c_h x c_z) stay
-// resident in shared memory; the pair state is read exactly once.
+// one pair row (s, i) taken from the offset table.  The weights (4 c_h x c_z) stay resident in
+// shared memory; the pair state is read exactly once.
 #include <cstring>
 
 #include "fast.cuh"
@@ -19,21 +25,21 @@
 
 namespace ntp {
 
-constexpr int TI_CH = 32;                  // positions per chunk
-constexpr int TI_THREADS = 64 + 128 + 256; // producer warp, MMA warp, 4 converter warps, 8 epilogue warps
+constexpr int TI_CH = 32;                       // positions per chunk
+constexpr int TI_THREADS = 64 + 128 + 256;      // producer warp, MMA warp, 4 converter warps, 8 epilogue warps
 constexpr int TI_MAXB = 16;
 
 struct TriInParams {
-  CUtensorMap zmap[TI_MAXB];               // {c_z, N (k), N (i)}, box {64, 32, 1}
+  CUtensorMap zmap[TI_MAXB];               // {c_z, N (k), N (i), 1}, box {64, 32, 1, 1}
   CUtensorMap wmap;                        // {c_z, 4 c_h}, box {64, 128}
+  CUtensorMap xmap;                        // augmentation columns {8, 2 * aug_rows}, box {8, 256}, no swizzle
   long long chunk_off[TI_MAXB + 1];
   long long cm_off[TI_MAXB];
   int N[TI_MAXB];
-  int B, c_z, c_h;
+  int B, c_z, c_h, aug_rows;
   float eps;
-  const float2* c01;                       // [4 c_h] (c0, c1)
-  __nv_bfloat16* a;
-  __nv_bfloat16* b;
+  __half* a;
+  __half* b;
   int* status;
 };
 
@@ -57,33 +63,35 @@ __device__ inline float sigmoid_fast(float x) {
 __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_constant__ TriInParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[11];
-  __shared__ float2 sStats[2][128];        // per stage: (mean, rstd) of every tile row
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
   const int c_z = p.c_z, c_h = p.c_h;
   const int nslab = c_z / 64;
-  const int w_slab_bytes = 4 * c_h * 128;          // one 64-channel slab of all 4 c_h weight rows
+  const int wrows = 4 * c_h;
+  const int w_slab_bytes = wrows * 128;            // one 64-channel slab of all weight rows
   const int w_bytes = nslab * w_slab_bytes;
-  const int a_slab_bytes = 128 * 128;
-  const int a_stage_bytes = nslab * a_slab_bytes;
+  const int wx_region = wrows * 16;                // one 8-column region of the weight augmentation
+  const int z_slab_bytes = 128 * 128;
+  const int z_stage_bytes = nslab * z_slab_bytes;
+  const int zx_region = 128 * 16;                  // one 8-column region of the activation augmentation
   unsigned char* sW = smem;
-  unsigned char* sA = sW + w_bytes;                // 2 stages
-  unsigned char* sStage = sA + 2 * a_stage_bytes;  // 8 warps x 2 KB transpose staging
-  float2* sC = reinterpret_cast<float2*>(sStage + 8 * 2048);
-  unsigned long long* afull = bars;        // [2]
-  unsigned long long* aempty = bars + 2;   // [2]
-  unsigned long long* tfull = bars + 4;    // [2]
-  unsigned long long* tempty = bars + 6;   // [2]
+  unsigned char* sWx = sW + w_bytes;               // [2 regions][wrows][8] fp16, no swizzle
+  unsigned char* sZ = sWx + 2 * wx_region;         // 2 stages of the z tile
+  unsigned char* sZx = sZ + 2 * z_stage_bytes;     // 2 stages x [2 regions][128][8] fp16
+  unsigned long long* afull = bars;        // [2] TMA landed
+  unsigned long long* aempty = bars + 2;   // [2] MMAs that read the stage are done
+  unsigned long long* tfull = bars + 4;    // [2] accumulator buffer ready
+  unsigned long long* tempty = bars + 6;   // [2] accumulator buffer drained
   unsigned long long* wfull = bars + 8;
-  unsigned long long* aconv = bars + 9;    // [2] tile converted to fp16, statistics published
+  unsigned long long* aconv = bars + 9;    // [2] tile normalised / converted, augmentation written
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(&afull[s], 1);
-      mbar_init(&aempty[s], 1 + 8);        // MMA commit + one arrival per epilogue warp
+      mbar_init(&aempty[s], 1);
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
       mbar_init(&aconv[s], 4);
@@ -92,7 +100,12 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
-  for (int n = threadIdx.x; n < 4 * c_h; n += TI_THREADS) sC[n] = p.c01[n];
+  // the second 8-column region of the activation augmentation is always zero
+  for (int idx = threadIdx.x; idx < 2 * zx_region / 16; idx += TI_THREADS) {
+    const int st = idx / (zx_region / 16), r = idx % (zx_region / 16);
+    *reinterpret_cast<uint4*>(sZx + st * 2 * zx_region + zx_region + r * 16) = make_uint4(0, 0, 0, 0);
+  }
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -100,14 +113,17 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   AbortCtx ab{p.status, &abort_flag};
   const long long nchunks = p.chunk_off[p.B];
   const long long ntiles = (nchunks + 3) / 4;
-  const int Nu = 2 * c_h;                          // accumulator columns per unit (gate | value)
+  const int nunits = c_h == 128 ? 2 : 1;           // accumulator units per tile: (gate rows | value rows) of 128 each
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ producer
-    mbar_expect_tx(wfull, w_bytes);
+    mbar_expect_tx(wfull, w_bytes + 2 * wx_region);
     for (int sl = 0; sl < nslab; ++sl)
-      for (int rb = 0; rb < 4 * c_h / 128; ++rb)
+      for (int rb = 0; rb < wrows / 128; ++rb)
         tma_load_2d(sW + sl * w_slab_bytes + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
+    for (int reg = 0; reg < 2; ++reg)
+      for (int rb = 0; rb < wrows / 256; ++rb)
+        tma_load_2d(sWx + reg * wx_region + rb * 256 * 16, &p.xmap, wfull, 0, reg * p.aug_rows + rb * 256);
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
@@ -119,7 +135,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         int s, i, jc;
         ti_decode(p, 4 * t + q, s, i, jc);
         for (int sl = 0; sl < nslab; ++sl)
-          tma_load_4d(sA + stage * a_stage_bytes + sl * a_slab_bytes + q * TI_CH * 128, &p.zmap[s], &afull[stage],
+          tma_load_4d(sZ + stage * z_stage_bytes + sl * z_slab_bytes + q * TI_CH * 128, &p.zmap[s], &afull[stage],
                       sl * 64, jc, i, 0);
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
@@ -130,23 +146,31 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
-    const unsigned idesc = idesc_f16(128, Nu, 0, 0, FMT_F16, FMT_F16);   // z tile converted to fp16, folded weights fp16
+    const unsigned idesc = idesc_f16(128, 128, 0, 0, FMT_F16, FMT_F16);   // M = 128 channels, N = 128 positions
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
-      const unsigned a_addr = smem_u32(sA + stage * a_stage_bytes);
-      for (int u = 0; u < 2; ++u, ++unit) {
+      const unsigned z_addr = smem_u32(sZ + stage * z_stage_bytes);
+      const unsigned zx_desc_addr = smem_u32(sZx + stage * 2 * zx_region);
+      for (int u = 0; u < nunits; ++u, ++unit) {
         const int buf = (int)(unit & 1);
         mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
         tph[buf] ^= 1;
         tc_fence_after();
-        const unsigned d_tmem = tmem_base + buf * 256;
-        for (int sl = 0; sl < nslab; ++sl) {
-          const unsigned w_addr = smem_u32(sW + sl * w_slab_bytes + u * Nu * 128);
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            umma_bf16(d_tmem, desc_kmajor_sw128(a_addr + sl * a_slab_bytes + k4 * 32),
-                      desc_kmajor_sw128(w_addr + k4 * 32), idesc, (sl | k4) != 0);
+        for (int part = 0; part < 2; ++part) {                 // 0 = gate rows, 1 = value rows
+          const int row0 = u * 256 + part * 128;
+          const unsigned d_tmem = tmem_base + buf * 256 + part * 128;
+          for (int sl = 0; sl < nslab; ++sl) {
+            const unsigned w_addr = smem_u32(sW + sl * w_slab_bytes + row0 * 128);
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4)
+              umma_bf16(d_tmem, desc_kmajor_sw128(w_addr + k4 * 32), desc_kmajor_sw128(z_addr + sl * z_slab_bytes + k4 * 32),
+                        idesc, (sl | k4) != 0);
+          }
+          // augmentation K step: c1 / c0 columns against the (-mean rstd, 1) columns
+          umma_bf16(d_tmem, desc_kmajor_nosw(smem_u32(sWx + row0 * 16), wx_region, 128),
+                    desc_kmajor_nosw(zx_desc_addr, zx_region, 128), idesc, 1);
         }
         tc_commit(&tfull[buf]);
       }
@@ -154,17 +178,54 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
+    // ------------------------------------------------------------------ converters (4 warps, one position per thread)
     const int row = (warp - 2) * 32 + lane;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
-      float sum, sq;
-      convert_row_bf16_to_f16(sA + stage * a_stage_bytes, nslab, a_slab_bytes, row, sum, sq);
+      unsigned char* tile = sZ + stage * z_stage_bytes;
+      float sum = 0.f, sq = 0.f;
+      for (int sl = 0; sl < nslab; ++sl) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint4 v = *reinterpret_cast<const uint4*>(tile + sl * z_slab_bytes + sw128_off(row, ch));
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            sum += lo + hi;
+            sq = fmaf(lo, lo, sq);
+            sq = fmaf(hi, hi, sq);
+          }
+        }
+      }
       const float mean = sum / (float)c_z;
-      const float var = fmaxf(sq / (float)c_z - mean * mean, 0.f);
-      sStats[stage][row] = make_float2(mean, rsqrtf(var + p.eps));
+      const float rstd = rsqrtf(fmaxf(sq / (float)c_z - mean * mean, 0.f) + p.eps);
+      for (int sl = 0; sl < nslab; ++sl) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          uint4* ptr = reinterpret_cast<uint4*>(tile + sl * z_slab_bytes + sw128_off(row, ch));
+          const uint4 v = *ptr;
+          unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __half2 h = __floats2half2_rn(__uint_as_float(w[e] << 16) * rstd, __uint_as_float(w[e] & 0xffff0000u) * rstd);
+            w[e] = *reinterpret_cast<unsigned*>(&h);
+          }
+          *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      {
+        const float mm = -mean * rstd;
+        const __half mh = __float2half_rn(mm), ml = __float2half_rn(mm - __half2float(mh));
+        const __half one = __float2half_rn(1.0f), zero = __float2half_rn(0.0f);
+        __half2 p0 = __halves2half2(mh, ml), p1 = __halves2half2(mh, one), p2 = __halves2half2(one, zero),
+                p3 = __halves2half2(zero, zero);
+        *reinterpret_cast<uint4*>(sZx + stage * 2 * zx_region + row * 16) =
+            make_uint4(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1),
+                       *reinterpret_cast<unsigned*>(&p2), *reinterpret_cast<unsigned*>(&p3));
+      }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&aconv[stage]);
@@ -172,64 +233,52 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     }
   } else if (warp >= 6) {
     // ------------------------------------------------------------------ epilogue (8 warps)
-    const int quarter = warp & 3;                  // TMEM lane quarter this warp may read
-    const int half = (warp - 6) >> 2;              // which half of the channels this warp handles
-    const int row = quarter * 32 + lane;           // accumulator row = position inside the tile
-    unsigned char* stg = sStage + (warp - 6) * 2048;
-    int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0};
+    const int quarter = warp & 3;                  // TMEM lane quarter = 32 output channels
+    const int half = (warp - 6) >> 2;              // which two of the tile's four chunks this warp stores
+    const int lane_ch = quarter * 32 + lane;       // accumulator row
+    unsigned tph[2] = {0, 0};
     long long unit = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      // chunk of this warp: quarter-th chunk of the tile
-      int s = 0, i = 0, jc = 0;
-      const bool valid = ti_decode(p, 4 * t + quarter, s, i, jc);
-      mbar_wait(&aconv[stage], phase, ab);         // statistics of this tile are published
-      const float2 stt = sStats[stage][row];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&aempty[stage]);
-      const float mean = stt.x, rstd = stt.y;
-      const int N = valid ? p.N[s] : 1;
-      const int ld = round_up8(N);
-      const long long plane = (long long)N * ld;
-      for (int u = 0; u < 2; ++u, ++unit) {
+      for (int u = 0; u < nunits; ++u, ++unit) {
         const int buf = (int)(unit & 1);
         mbar_wait(&tfull[buf], tph[buf], ab);
         tph[buf] ^= 1;
         tc_fence_after();
+        // c_h = 128: unit 0 -> a, unit 1 -> b, channel = accumulator row; c_h = 64: rows 0-63 -> a, 64-127 -> b
+        const int ch = c_h == 128 ? lane_ch : (lane_ch & 63);
+        __half* obase = (c_h == 128 ? (u == 0) : (lane_ch < 64)) ? p.a : p.b;
         const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
-        __nv_bfloat16* outp = (u == 0 ? p.a : p.b) + (valid ? (long long)c_h * p.cm_off[s] + (long long)i * ld + jc : 0);
-        const float2* cg = sC + u * Nu;            // gate rows first, value rows c_h later
-        for (int c0 = half * (c_h / 2); c0 < (half + 1) * (c_h / 2); c0 += 32) {
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          const int q = half * 2 + qq;
+          int s = 0, i = 0, jc = 0;
+          const bool valid = ti_decode(p, 4 * t + q, s, i, jc);
           unsigned rg[32], rv[32];
-          tmem_ld32(taddr + c0, rg);
-          tmem_ld32(taddr + c_h + c0, rv);
+          tmem_ld32(taddr + q * 32, rg);
+          tmem_ld32(taddr + 128 + q * 32, rv);
           tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float2 kg = cg[c0 + e], kv = cg[c_h + c0 + e];
-            const float xg = fmaf(rstd, __uint_as_float(rg[e]) - mean * kg.y, kg.x);
-            const float xv = fmaf(rstd, __uint_as_float(rv[e]) - mean * kv.y, kv.x);
-            const float val = fminf(fmaxf(sigmoid_fast(xg) * xv, -65504.f), 65504.f);
-            reinterpret_cast<__half*>(stg)[e * 32 + lane] = __float2half_rn(val);
-          }
-          __syncwarp();
           if (valid) {
+            const int N = p.N[s], ld = round_up8(N);
+            __half* outp = obase + (long long)c_h * p.cm_off[s] + (long long)ch * N * ld + (long long)i * ld + jc;
 #pragma unroll
-            for (int it = 0; it < 4; ++it) {
-              const int cl = it * 8 + (lane >> 2), vec = lane & 3;
-              if (jc + vec * 8 < ld) {
-                const uint4 v = *reinterpret_cast<const uint4*>(stg + cl * 64 + vec * 16);
-                *reinterpret_cast<uint4*>(outp + (long long)(c0 + cl) * plane + vec * 8) = v;
+            for (int vec = 0; vec < 4; ++vec) {
+              unsigned w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int n0 = vec * 8 + e * 2;
+                const float v0 = sigmoid_fast(__uint_as_float(rg[n0])) * __uint_as_float(rv[n0]);
+                const float v1 = sigmoid_fast(__uint_as_float(rg[n0 + 1])) * __uint_as_float(rv[n0 + 1]);
+                __half2 h = __floats2half2_rn(fminf(fmaxf(v0, -65504.f), 65504.f), fminf(fmaxf(v1, -65504.f), 65504.f));
+                w[e] = *reinterpret_cast<unsigned*>(&h);
               }
+              if (jc + vec * 8 < ld) *reinterpret_cast<uint4*>(outp + vec * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
-          __syncwarp();
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty[buf]);
       }
-      if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   }
   tc_fence_before();
@@ -242,13 +291,13 @@ bool fast_tri_in_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) 
 
 nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int c_h, void* a, void* b,
                       const BatchMeta& m, int* status, cudaStream_t st) {
-  const void* wprime = tp.w1;
-  const float2* c01 = (const float2*)tp.c01_1;
   const int nslab = c_z / 64;
-  const size_t smem = (size_t)nslab * 4 * c_h * 128 + 2 * (size_t)nslab * 128 * 128 + 8 * 2048 + 4 * c_h * 8 + 1024;
+  const int wrows = 4 * c_h;
+  const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)wrows * 16 + 2 * (size_t)nslab * 128 * 128 +
+                      2 * 2 * (size_t)128 * 16 + 1024;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(tri_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(tri_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) != cudaSuccess)
       return cuda_fail("tri_in smem attribute");
     attr_set = true;
   }
@@ -258,16 +307,20 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
     p.B = m.B - g0 < TI_MAXB ? m.B - g0 : TI_MAXB;
     p.c_z = c_z;
     p.c_h = c_h;
+    p.aug_rows = tp.aug1_rows;
     p.eps = eps;
-    p.c01 = c01;
-    p.a = (__nv_bfloat16*)a;
-    p.b = (__nv_bfloat16*)b;
+    p.a = (__half*)a;
+    p.b = (__half*)b;
     p.status = status;
     {
-      const unsigned long long dims[2] = {(unsigned long long)c_z, (unsigned long long)4 * c_h};
+      const unsigned long long dims[2] = {(unsigned long long)c_z, (unsigned long long)wrows};
       const unsigned long long strides[1] = {(unsigned long long)c_z * 2};
       const unsigned box[2] = {64, 128};
-      if (!make_tmap_bf16(&p.wmap, wprime, 2, dims, strides, box)) { fprintf(stderr, "libnested_pair: tensor map encode failed (%s:%d)\n", __FILE__, __LINE__); return NT_ERR_CUDA; }
+      if (!make_tmap_bf16(&p.wmap, tp.w1, 2, dims, strides, box)) return cuda_fail("tri_in weight map");
+      const unsigned long long xdims[2] = {8, (unsigned long long)2 * tp.aug1_rows};
+      const unsigned long long xstr[1] = {16};
+      const unsigned xbox[2] = {8, 256};
+      if (!make_tmap_16bit(&p.xmap, tp.aug1, 2, xdims, xstr, xbox, 0)) return cuda_fail("tri_in augmentation map");
     }
     p.chunk_off[0] = 0;
     for (int l = 0; l < TI_MAXB; ++l) {
@@ -281,7 +334,7 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
                                                (unsigned long long)N * N * c_z * 2};
         const unsigned box[4] = {64, TI_CH, 1, 1};
         const char* base = (const char*)z + (size_t)m.pair_off[g0 + l] * c_z * 2;
-        if (!make_tmap_bf16(&p.zmap[l], base, 4, dims, strides, box)) { fprintf(stderr, "libnested_pair: tensor map encode failed (%s:%d)\n", __FILE__, __LINE__); return NT_ERR_CUDA; }
+        if (!make_tmap_bf16(&p.zmap[l], base, 4, dims, strides, box)) return cuda_fail("tri_in z map");
       }
     }
     const long long ntiles = (p.chunk_off[p.B] + 3) / 4;
@@ -291,7 +344,7 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
       LaunchScope ls("tri_in", st);
       tri_in_kernel<<<grid, TI_THREADS, smem, st>>>(p);
     }
-    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("tensor-core kernel launch");
+    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("tri_in launch");
   }
   return NT_OK;
 }

@@ -20,7 +20,7 @@ EncodeTiledFn get_encode_tiled();
 // bf16 tensor map with 128-byte swizzle; dims / strides fastest first (strides in bytes for dims 1..rank-1)
 bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                     const unsigned long long* strides_bytes, const unsigned* box);
-// same with a 32-, 64- or 128-byte swizzle span (the inner box extent in bytes must not exceed it)
+// same with a 32-, 64- or 128-byte swizzle span (the inner box extent in bytes must not exceed it); 0 = no swizzle
 bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                      const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes);
 
@@ -149,6 +149,16 @@ __device__ inline unsigned long long desc_mnmajor_sw128(unsigned saddr, unsigned
   d |= (unsigned long long)((sbo >> 4) & 0x3FFF) << 32;
   d |= (unsigned long long)1 << 46;
   d |= (unsigned long long)2 << 61;
+  return d;
+}
+// K-major operand without swizzle ("interleaved" core matrices): a core matrix is 8 rows x 16 bytes stored
+// contiguously (128 bytes); the next 8 rows are `sbo` bytes further, the next 8 K-elements `lbo` bytes further.
+__device__ inline unsigned long long desc_kmajor_nosw(unsigned saddr, unsigned lbo, unsigned sbo) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((saddr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)((lbo >> 4) & 0x3FFF) << 16;
+  d |= (unsigned long long)((sbo >> 4) & 0x3FFF) << 32;
+  d |= (unsigned long long)1 << 46;
   return d;
 }
 // instruction descriptor of kind::f16: D = f32, M x N tile, operand majors (0 = K-major, 1 = MN-major)
