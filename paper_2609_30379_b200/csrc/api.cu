@@ -189,7 +189,8 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
                                  float eps, void* z, void* ws, nt_dtype dt, cudaStream_t st) {
   TriWs w = carve_trimul(ws, dt, tot, c_z, c_h);
   // The tensor-core stages exchange a, b (fp16) and t (fp16, scaled by 1 / N): all three or none.
-  const bool tc = dt == NT_BF16 && !g_force_generic && fast_tri_in_supported(c_z, c_h) &&
+  // (the tensor-core kernels index positions inside a sample with 32 bits: N below 2^16)
+  const bool tc = dt == NT_BF16 && !g_force_generic && tot.nmax < 60000 && fast_tri_in_supported(c_z, c_h) &&
                   fast_contract_supported(c_h) && fast_tri_out_supported(c_z, c_h);
   TriPrep tprep{};
   if (tc) {
@@ -249,7 +250,7 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
   AttnWs w = carve_attn(ws, dt, tot, order, H, d);
   const int Hd = H * d;
   const bool pair = order == NT_ORDER_PAIR_IJC;
-  const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma;
+  const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma && tot.nmax < 60000;
   const bool tc_in = tc && fast_attn_in_supported(c, H, d) && fast_attn_core_supported(H, d);   // bias goes out times sqrt(d)
   const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
   AttnPrep aprep{};

@@ -222,9 +222,9 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
             int s = 0;
             while (s + 1 < p.B && P >= p.pair_off[s + 1]) ++s;
             const int N = p.N[s], ld = round_up8(N);
-            const long long rr = P - p.pair_off[s];
-            const long long i = rr / N, j = rr - i * N;
-            __nv_bfloat16* bp = p.bias + (long long)p.H * p.cm_off[s] + i * ld + j;
+            const unsigned rr = (unsigned)(P - p.pair_off[s]);      // N^2 < 2^32 (N < 2^16 for this path)
+            const unsigned i = rr / (unsigned)N, j = rr - i * (unsigned)N;
+            __nv_bfloat16* bp = p.bias + (long long)p.H * p.cm_off[s] + (long long)i * ld + j;
             const float2* cc = sC + 3 * Hd;
             for (int h = 0; h < p.H; ++h) {
               const float x = fmaf(rstd, __uint_as_float(r[h]) - mean * cc[h].y, cc[h].x);

@@ -115,7 +115,9 @@ nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep
   const void* s128[5] = {W->W_ag, W->W_ap, W->W_bg, W->W_bp, W->W_g};
   const void* s64[5] = {W->W_ag, W->W_bg, W->W_ap, W->W_bp, W->W_g};
   const int r0[5] = {c_h, c_h, c_h, c_h, c_z};
-  add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, nullptr, out.aug1);
+  // gate and value rows are folded times 1/2 (exact): sigmoid(g) v = (tanh(g / 2) + 1) (v / 2) costs one MUFU and one FMA
+  const float sc[5] = {0.5f, 0.5f, 0.5f, 0.5f, 1.0f};
+  add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, sc, out.aug1);
   const void* s1[1] = {W->W_o};
   const int r1[1] = {c_z};
   add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o);

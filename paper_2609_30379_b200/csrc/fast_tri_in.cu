@@ -48,16 +48,17 @@ __device__ inline bool ti_decode(const TriInParams& p, long long q, int& s, int&
   s = 0;
   while (s + 1 < p.B && q >= p.chunk_off[s + 1]) ++s;
   const int cpr = (p.N[s] + TI_CH - 1) / TI_CH;
-  const long long r = q - p.chunk_off[s];
-  i = (int)(r / cpr);
-  jc = (int)(r - (long long)i * cpr) * TI_CH;
+  // a sample's chunk count N * ceil(N / chunk) is far below 2^32 (N < 2^20 is checked on the host): 32-bit division
+  const unsigned r = (unsigned)(q - p.chunk_off[s]);
+  i = (int)(r / (unsigned)cpr);
+  jc = (int)(r - (unsigned)i * (unsigned)cpr) * TI_CH;
   return true;
 }
 
-__device__ inline float sigmoid_fast(float x) {
+__device__ inline float tanh_fast(float x) {
   float t;
-  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(0.5f * x));
-  return fmaf(0.5f, t, 0.5f);
+  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(x));
+  return t;
 }
 
 __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_constant__ TriInParams p) {
@@ -236,6 +237,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     const int quarter = warp & 3;                  // TMEM lane quarter = 32 output channels
     const int half = (warp - 6) >> 2;              // which two of the tile's four chunks this warp stores
     const int lane_ch = quarter * 32 + lane;       // accumulator row
+    const __half2 hmax2 = __float2half2_rn(65504.f), hmin2 = __float2half2_rn(-65504.f);
     unsigned tph[2] = {0, 0};
     long long unit = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
@@ -266,9 +268,13 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const int n0 = vec * 8 + e * 2;
-                const float v0 = sigmoid_fast(__uint_as_float(rg[n0])) * __uint_as_float(rv[n0]);
-                const float v1 = sigmoid_fast(__uint_as_float(rg[n0 + 1])) * __uint_as_float(rv[n0 + 1]);
-                __half2 h = __floats2half2_rn(fminf(fmaxf(v0, -65504.f), 65504.f), fminf(fmaxf(v1, -65504.f), 65504.f));
+                // the gate and value weight rows were folded times 1/2, so with g' = g / 2, v' = v / 2:
+                // sigmoid(g) * v = (tanh(g') + 1) * v' = fma(v', tanh(g'), v')
+                const float h0 = __uint_as_float(rv[n0]), h1 = __uint_as_float(rv[n0 + 1]);
+                const float v0 = fmaf(h0, tanh_fast(__uint_as_float(rg[n0])), h0);
+                const float v1 = fmaf(h1, tanh_fast(__uint_as_float(rg[n0 + 1])), h1);
+                __half2 h = __floats2half2_rn(v0, v1);          // overflow gives inf, clamped below
+                h = __hmax2(__hmin2(h, hmax2), hmin2);
                 w[e] = *reinterpret_cast<unsigned*>(&h);
               }
               if (jc + vec * 8 < ld) *reinterpret_cast<uint4*>(outp + vec * 8) = make_uint4(w[0], w[1], w[2], w[3]);

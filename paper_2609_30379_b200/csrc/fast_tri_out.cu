@@ -40,9 +40,10 @@ __device__ inline bool to_decode(const TriOutParams& p, long long q, int& s, int
   s = 0;
   while (s + 1 < p.B && q >= p.chunk_off[s + 1]) ++s;
   const int cpr = (p.N[s] + 63) / 64;
-  const long long r = q - p.chunk_off[s];
-  i = (int)(r / cpr);
-  j0 = (int)(r - (long long)i * cpr) * 64;
+  // a sample's chunk count N * ceil(N / chunk) is far below 2^32 (N < 2^20 is checked on the host): 32-bit division
+  const unsigned r = (unsigned)(q - p.chunk_off[s]);
+  i = (int)(r / (unsigned)cpr);
+  j0 = (int)(r - (unsigned)i * (unsigned)cpr) * 64;
   return true;
 }
 

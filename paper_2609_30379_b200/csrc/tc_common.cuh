@@ -60,6 +60,7 @@ __device__ inline bool mbar_wait(void* bar, unsigned parity, const AbortCtx& ab)
   const unsigned limit = *ab.flag ? WAIT_LIMIT_ABORTED : WAIT_LIMIT;
   for (unsigned it = 0; it < limit; ++it) {
     if (mbar_try(bar, parity)) return true;
+    if (it >= 4) __nanosleep(40);          // waiting roles should not steal issue slots from working warps
     if ((it & 1023u) == 1023u && *ab.flag) break;
   }
   if (!*ab.flag) {
