@@ -69,6 +69,14 @@ __device__ inline unsigned pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<unsigned*>(&h);
 }
+// two exponentials at once: the arguments are rounded to bf16 (they are <= 0, so the absolute error grows
+// only where the weight is already small) and the results come back packed as the bf16 pair the PV MMA takes
+__device__ inline unsigned exp2_bf16x2(float lo, float hi) {
+  unsigned x, y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(x) : "f"(hi), "f"(lo));
+  asm("ex2.approx.ftz.bf16x2 %0, %1;\n" : "=r"(y) : "r"(x));
+  return y;
+}
 __device__ inline float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
@@ -96,7 +104,7 @@ __device__ inline void mma_bf16_zero(float (&d)[4], const unsigned (&a)[4], unsi
 // Scores stay in unscaled units S' = q.k + bias sqrt(d); the softmax scale log2(e) / sqrt(d) is
 // applied inside the exponent: p = exp2(sc2 S' - sc2 max').
 template <int D, int NT, int BIAS, bool MASKED>
-__device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8][4], float (&mrow)[2], float (&lrow)[2],
+__device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8][4], float (&mrow)[2], float (&lacc)[4],
                                  const unsigned (&qf)[D / 16][4], const unsigned (&idf)[4], unsigned ks_, unsigned vs_,
                                  unsigned bias_s, int ld, const __nv_bfloat16* bg0, const __nv_bfloat16* bg1, int k0,
                                  int N, float sc2, float bias_mul, int lane) {
@@ -132,7 +140,7 @@ __device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8
     }
   }
   // ---- bias through L1/L2 (long samples), mask, running max
-  float mx0 = -INFINITY, mx1 = -INFINITY;
+  float t0[2] = {-INFINITY, -INFINITY}, t1[2] = {-INFINITY, -INFINITY};   // two chains each, half the latency
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
     const int kc = k0 + nt * 8 + 2 * tq;
@@ -151,9 +159,10 @@ __device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8
       if (kc >= N) sacc[nt][0] = sacc[nt][2] = -INFINITY;
       if (kc + 1 >= N) sacc[nt][1] = sacc[nt][3] = -INFINITY;
     }
-    mx0 = fmaxf(mx0, fmaxf(sacc[nt][0], sacc[nt][1]));
-    mx1 = fmaxf(mx1, fmaxf(sacc[nt][2], sacc[nt][3]));
+    t0[nt & 1] = fmaxf(t0[nt & 1], fmaxf(sacc[nt][0], sacc[nt][1]));
+    t1[nt & 1] = fmaxf(t1[nt & 1], fmaxf(sacc[nt][2], sacc[nt][3]));
   }
+  float mx0 = fmaxf(t0[0], t0[1]), mx1 = fmaxf(t1[0], t1[1]);
   mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
   mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
   mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
@@ -163,31 +172,23 @@ __device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8
   mrow[0] = mn0;
   mrow[1] = mn1;
   const float ms0 = -mn0 * sc2, ms1 = -mn1 * sc2;
-  float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    sacc[nt][0] = fast_exp2(fmaf(sacc[nt][0], sc2, ms0));
-    sacc[nt][1] = fast_exp2(fmaf(sacc[nt][1], sc2, ms0));
-    sacc[nt][2] = fast_exp2(fmaf(sacc[nt][2], sc2, ms1));
-    sacc[nt][3] = fast_exp2(fmaf(sacc[nt][3], sc2, ms1));
-    ps0 += sacc[nt][0] + sacc[nt][1];
-    ps1 += sacc[nt][2] + sacc[nt][3];
-  }
-  lrow[0] = lrow[0] * cr0 + ps0;
-  lrow[1] = lrow[1] * cr1 + ps1;
 #pragma unroll
   for (int nd = 0; nd < D / 8; ++nd) {
     oacc[nd][0] *= cr0; oacc[nd][1] *= cr0;
     oacc[nd][2] *= cr1; oacc[nd][3] *= cr1;
   }
-  // ---- O += P V
+  lacc[0] *= cr0; lacc[1] *= cr0;
+  lacc[2] *= cr1; lacc[3] *= cr1;
+  // ---- O += P V, with the row sums of P accumulated by one more MMA against an all-ones B tile, so the
+  // denominator sums exactly the rounded weights the numerator uses
 #pragma unroll
   for (int kk = 0; kk < NT / 2; ++kk) {
     unsigned pf[4];
-    pf[0] = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
-    pf[1] = pack_bf16(sacc[2 * kk][2], sacc[2 * kk][3]);
-    pf[2] = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
-    pf[3] = pack_bf16(sacc[2 * kk + 1][2], sacc[2 * kk + 1][3]);
+    pf[0] = exp2_bf16x2(fmaf(sacc[2 * kk][0], sc2, ms0), fmaf(sacc[2 * kk][1], sc2, ms0));
+    pf[1] = exp2_bf16x2(fmaf(sacc[2 * kk][2], sc2, ms1), fmaf(sacc[2 * kk][3], sc2, ms1));
+    pf[2] = exp2_bf16x2(fmaf(sacc[2 * kk + 1][0], sc2, ms0), fmaf(sacc[2 * kk + 1][1], sc2, ms0));
+    pf[3] = exp2_bf16x2(fmaf(sacc[2 * kk + 1][2], sc2, ms1), fmaf(sacc[2 * kk + 1][3], sc2, ms1));
+    mma_bf16(lacc, pf, 0x3F803F80u, 0x3F803F80u);
 #pragma unroll
     for (int np = 0; np < D / 16; ++np) {
       const int mtx = lane >> 3;
@@ -202,16 +203,16 @@ __device__ inline void attn_step(float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8
 
 template <int D, int BIAS>
 __device__ inline void attn_step_dispatch(bool masked, int rem, float (&sacc)[AT_K / 8][4], float (&oacc)[D / 8][4],
-                                          float (&mrow)[2], float (&lrow)[2], const unsigned (&qf)[D / 16][4],
+                                          float (&mrow)[2], float (&lacc)[4], const unsigned (&qf)[D / 16][4],
                                           const unsigned (&idf)[4], unsigned ks_, unsigned vs_, unsigned bias_s, int ld,
                                           const __nv_bfloat16* bg0, const __nv_bfloat16* bg1, int k0, int N, float sc2,
                                           float bias_mul, int lane) {
   if (!masked)
-    attn_step<D, 8, BIAS, false>(sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
+    attn_step<D, 8, BIAS, false>(sacc, oacc, mrow, lacc, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
   else if (rem > 32)
-    attn_step<D, 8, BIAS, true>(sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
+    attn_step<D, 8, BIAS, true>(sacc, oacc, mrow, lacc, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
   else
-    attn_step<D, 4, BIAS, true>(sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
+    attn_step<D, 4, BIAS, true>(sacc, oacc, mrow, lacc, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N, sc2, bias_mul, lane);
 }
 
 // BIAS: 0 = no bias, 1 = bias tile resident in shared memory (samples with want_resident), 2 = bias through L1/L2.
@@ -325,7 +326,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
   unsigned qf[D / 16][4];
   float oacc[D / 8][4];
   float sacc[AT_K / 8][4];
-  float mrow[2], lrow[2];
+  float mrow[2], lacc[4];
   const int rloc = cw * 16 + g;                       // this thread's first query row inside the CTA tile
   // identity A fragment of the bias MMA: 1.0 where the query row equals the k index
   unsigned idf[4];
@@ -355,26 +356,21 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
 #pragma unroll
     for (int nd = 0; nd < D / 8; ++nd) oacc[nd][0] = oacc[nd][1] = oacc[nd][2] = oacc[nd][3] = 0.f;
     mrow[0] = mrow[1] = -INFINITY;
-    lrow[0] = lrow[1] = 0.f;
+    lacc[0] = lacc[1] = lacc[2] = lacc[3] = 0.f;
     for (int kb = 0; kb < nkb; ++kb) {
       mbar_wait(&kvfull[st], ph, ab);
       const unsigned ks_ = smem_u32(sK + st * KV_TILE), vs_ = smem_u32(sV + st * KV_TILE);
       const int k0 = kb * AT_K;
       const bool masked = tail && kb == nkb - 1;
       const unsigned bias_s = bias_lane + k0 * 2;
-      attn_step_dispatch<D, BIAS>(masked, N - k0, sacc, oacc, mrow, lrow, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
+      attn_step_dispatch<D, BIAS>(masked, N - k0, sacc, oacc, mrow, lacc, qf, idf, ks_, vs_, bias_s, ld, bg0, bg1, k0, N,
                                   sc2, p.bias_mul, lane);
       __syncwarp();
       if (lane == 0) mbar_arrive(&kvempty[st]);
       if (++st == AT_STAGES) { st = 0; ph ^= 1; }
     }
     // ---- normalise and store this row's 16 x d outputs
-    float l0 = lrow[0], l1 = lrow[1];
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    const float inv0 = 1.0f / l0, inv1 = 1.0f / l1;
+    const float inv0 = 1.0f / lacc[0], inv1 = 1.0f / lacc[2];   // every column of the ones tile holds the row sum
     const long long base = row_coord(i) + p.row0;
     const int r0 = j0 + rloc, r1 = r0 + 8;
 #pragma unroll

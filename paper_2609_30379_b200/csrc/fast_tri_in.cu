@@ -10,7 +10,7 @@
 // LayerNorm is folded completely into the MMA.  With W' = W * gamma (fp16), c1[n] = sum_k W'[n][k],
 // c0[n] = sum_k W[n][k] beta[k]:
 //   (LN(z) W^T)[n] = (rstd z) . W'[n] + (-mean rstd) c1[n] + c0[n].
-// Four converter warps rewrite the bf16 z tile as fp16 scaled by the row's rstd and append five
+// Eight converter warps (two threads per position) rewrite the bf16 z tile as fp16 scaled by the row's rstd and append five
 // extra K columns (m_hi, m_lo, m_hi, 1, 1), m = -mean rstd, that meet (c1_hi, c1_hi, c1_lo, c0_hi,
 // c0_lo) on the weight side (hi / lo halves keep ~22 bits), so the accumulator already holds the
 // normalised projection and the epilogue is sigmoid * value, convert, store.
@@ -26,7 +26,9 @@
 namespace ntp {
 
 constexpr int TI_CH = 32;                       // positions per chunk
-constexpr int TI_THREADS = 64 + 128 + 256;      // producer warp, MMA warp, 4 converter warps, 8 epilogue warps
+constexpr int TI_CONV_WARPS = 8;
+constexpr int TI_EPI_WARP0 = 2 + TI_CONV_WARPS; // first epilogue warp (a multiple of 4 plus 2: see the lane quarters below)
+constexpr int TI_THREADS = 64 + 32 * TI_CONV_WARPS + 256;   // producer warp, MMA warp, converter warps, 8 epilogue warps
 constexpr int TI_MAXB = 16;
 
 struct TriInParams {
@@ -66,6 +68,8 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   __shared__ __align__(8) unsigned long long bars[11];
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
+  __shared__ int4 tinfo[8][4];             // ring of decoded chunks {s, i, k0, valid} per tile, written by the producer up to
+                                           // five tiles ahead of the epilogue that reads it
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
   const int c_z = p.c_z, c_h = p.c_h;
   const int nslab = c_z / 64;
@@ -95,7 +99,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       mbar_init(&aempty[s], 1);
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
-      mbar_init(&aconv[s], 4);
+      mbar_init(&aconv[s], TI_CONV_WARPS);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -116,29 +120,38 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   const long long ntiles = (nchunks + 3) / 4;
   const int nunits = c_h == 128 ? 2 : 1;           // accumulator units per tile: (gate rows | value rows) of 128 each
 
-  if (warp == 0 && lane == 0) {
-    // ------------------------------------------------------------------ producer
-    mbar_expect_tx(wfull, w_bytes + 2 * wx_region);
-    for (int sl = 0; sl < nslab; ++sl)
-      for (int rb = 0; rb < wrows / 128; ++rb)
-        tma_load_2d(sW + sl * w_slab_bytes + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
-    for (int reg = 0; reg < 2; ++reg)
-      for (int rb = 0; rb < wrows / 256; ++rb)
-        tma_load_2d(sWx + reg * wx_region + rb * 256 * 16, &p.xmap, wfull, 0, reg * p.aug_rows + rb * 256);
-    int stage = 0;
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (lane q decodes and loads chunk q)
+    if (lane == 0) {
+      mbar_expect_tx(wfull, w_bytes + 2 * wx_region);
+      for (int sl = 0; sl < nslab; ++sl)
+        for (int rb = 0; rb < wrows / 128; ++rb)
+          tma_load_2d(sW + sl * w_slab_bytes + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
+      for (int reg = 0; reg < 2; ++reg)
+        for (int rb = 0; rb < wrows / 256; ++rb)
+          tma_load_2d(sWx + reg * wx_region + rb * 256 * 16, &p.xmap, wfull, 0, reg * p.aug_rows + rb * 256);
+    }
+    int stage = 0, tn = 0;
     unsigned phase = 0;
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&aempty[stage], phase ^ 1, ab);
-      int nvalid = 0;
-      for (int q = 0; q < 4; ++q) nvalid += (4 * t + q < nchunks) ? 1 : 0;
-      mbar_expect_tx(&afull[stage], nvalid * nslab * TI_CH * 128);
-      for (int q = 0; q < nvalid; ++q) {
-        int s, i, jc;
-        ti_decode(p, 4 * t + q, s, i, jc);
-        for (int sl = 0; sl < nslab; ++sl)
-          tma_load_4d(sZ + stage * z_stage_bytes + sl * z_slab_bytes + q * TI_CH * 128, &p.zmap[s], &afull[stage],
-                      sl * 64, jc, i, 0);
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++tn) {
+      int s = 0, i = 0, jc = 0;
+      bool valid = false;
+      if (lane < 4) {
+        valid = ti_decode(p, 4 * t + lane, s, i, jc);
+        tinfo[tn & 7][lane] = make_int4(s, i, jc, valid ? 1 : 0);
       }
+      __syncwarp();
+      if (lane == 0) {
+        const long long left = nchunks - 4 * t;
+        const int nvalid = left < 4 ? (int)left : 4;
+        mbar_wait(&aempty[stage], phase ^ 1, ab);
+        mbar_expect_tx(&afull[stage], nvalid * nslab * TI_CH * 128);
+      }
+      __syncwarp();
+      if (valid)
+        for (int sl = 0; sl < nslab; ++sl)
+          tma_load_4d(sZ + stage * z_stage_bytes + sl * z_slab_bytes + lane * TI_CH * 128, &p.zmap[s], &afull[stage],
+                      sl * 64, jc, i, 0);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp == 1 && lane == 0) {
@@ -178,46 +191,58 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       tc_commit(&aempty[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------------ converters (4 warps, one position per thread)
-    const int row = (warp - 2) * 32 + lane;
+  } else if (warp >= 2 && warp < TI_EPI_WARP0) {
+    // ------------------------------------------------------------------ converters: two threads per position, each
+    // owning four of the eight 16-byte chunks of every 64-channel slab
+    const int row = (warp - 2) * 16 + (lane >> 1), hf = lane & 1;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
       unsigned char* tile = sZ + stage * z_stage_bytes;
-      float sum = 0.f, sq = 0.f;
-      for (int sl = 0; sl < nslab; ++sl) {
+      uint4 raw[2][4];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint4 v = *reinterpret_cast<const uint4*>(tile + sl * z_slab_bytes + sw128_off(row, ch));
-          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+      for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          raw[sl][j] = sl < nslab ? *reinterpret_cast<const uint4*>(tile + sl * z_slab_bytes + sw128_off(row, hf * 4 + j))
+                                  : make_uint4(0, 0, 0, 0);
+      float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};   // four independent chains
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const unsigned w[4] = {raw[sl][j].x, raw[sl][j].y, raw[sl][j].z, raw[sl][j].w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-            sum += lo + hi;
-            sq = fmaf(lo, lo, sq);
-            sq = fmaf(hi, hi, sq);
+            s4[e] += lo + hi;
+            q4[e] = fmaf(lo, lo, q4[e]);
+            q4[e] = fmaf(hi, hi, q4[e]);
           }
         }
-      }
+      float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]), sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
       const float mean = sum / (float)c_z;
       const float rstd = rsqrtf(fmaxf(sq / (float)c_z - mean * mean, 0.f) + p.eps);
-      for (int sl = 0; sl < nslab; ++sl) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          uint4* ptr = reinterpret_cast<uint4*>(tile + sl * z_slab_bytes + sw128_off(row, ch));
-          const uint4 v = *ptr;
-          unsigned w[4] = {v.x, v.y, v.z, v.w};
+      for (int sl = 0; sl < 2; ++sl)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __half2 h = __floats2half2_rn(__uint_as_float(w[e] << 16) * rstd, __uint_as_float(w[e] & 0xffff0000u) * rstd);
-            w[e] = *reinterpret_cast<unsigned*>(&h);
+        for (int j = 0; j < 4; ++j) {
+          if (sl < nslab) {
+            unsigned w[4] = {raw[sl][j].x, raw[sl][j].y, raw[sl][j].z, raw[sl][j].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __half2 h =
+                  __floats2half2_rn(__uint_as_float(w[e] << 16) * rstd, __uint_as_float(w[e] & 0xffff0000u) * rstd);
+              w[e] = *reinterpret_cast<unsigned*>(&h);
+            }
+            *reinterpret_cast<uint4*>(tile + sl * z_slab_bytes + sw128_off(row, hf * 4 + j)) =
+                make_uint4(w[0], w[1], w[2], w[3]);
           }
-          *ptr = make_uint4(w[0], w[1], w[2], w[3]);
         }
-      }
-      {
+      if (hf == 0) {
         const float mm = -mean * rstd;
         const __half mh = __float2half_rn(mm), ml = __float2half_rn(mm - __half2float(mh));
         const __half one = __float2half_rn(1.0f), zero = __float2half_rn(0.0f);
@@ -232,15 +257,16 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
       if (lane == 0) mbar_arrive(&aconv[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= TI_EPI_WARP0) {
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;                  // TMEM lane quarter = 32 output channels
-    const int half = (warp - 6) >> 2;              // which two of the tile's four chunks this warp stores
+    const int half = (warp - TI_EPI_WARP0) >> 2;   // which two of the tile's four chunks this warp stores
     const int lane_ch = quarter * 32 + lane;       // accumulator row
     const __half2 hmax2 = __float2half2_rn(65504.f), hmin2 = __float2half2_rn(-65504.f);
     unsigned tph[2] = {0, 0};
     long long unit = 0;
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+    int tn = 0;
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++tn) {
       for (int u = 0; u < nunits; ++u, ++unit) {
         const int buf = (int)(unit & 1);
         mbar_wait(&tfull[buf], tph[buf], ab);
@@ -249,30 +275,34 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         // c_h = 128: unit 0 -> a, unit 1 -> b, channel = accumulator row; c_h = 64: rows 0-63 -> a, 64-127 -> b
         const int ch = c_h == 128 ? lane_ch : (lane_ch & 63);
         __half* obase = (c_h == 128 ? (u == 0) : (lane_ch < 64)) ? p.a : p.b;
-        const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
+        const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256 + half * 64;
+        // four steps of 16 positions; the TMEM loads of step k + 1 are in flight while step k is computed
+        unsigned rg[2][16], rv[2][16];
+        tmem_ld16(taddr, rg[0]);
+        tmem_ld16(taddr + 128, rv[0]);
 #pragma unroll
-        for (int qq = 0; qq < 2; ++qq) {
-          const int q = half * 2 + qq;
-          int s = 0, i = 0, jc = 0;
-          const bool valid = ti_decode(p, 4 * t + q, s, i, jc);
-          unsigned rg[32], rv[32];
-          tmem_ld32(taddr + q * 32, rg);
-          tmem_ld32(taddr + 128 + q * 32, rv);
-          tmem_ld_wait();
-          if (valid) {
+        for (int k = 0; k < 4; ++k) {
+          tmem_ld_wait2(rg[k & 1], rv[k & 1]);
+          if (k < 3) {
+            tmem_ld16(taddr + (k + 1) * 16, rg[(k + 1) & 1]);
+            tmem_ld16(taddr + 128 + (k + 1) * 16, rv[(k + 1) & 1]);
+          }
+          const int4 info = tinfo[tn & 7][half * 2 + (k >> 1)];
+          if (info.w) {
+            const int s = info.x, i = info.y, jc = info.z + (k & 1) * 16;
             const int N = p.N[s], ld = round_up8(N);
             __half* outp = obase + (long long)c_h * p.cm_off[s] + (long long)ch * N * ld + (long long)i * ld + jc;
 #pragma unroll
-            for (int vec = 0; vec < 4; ++vec) {
+            for (int vec = 0; vec < 2; ++vec) {
               unsigned w[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const int n0 = vec * 8 + e * 2;
                 // the gate and value weight rows were folded times 1/2, so with g' = g / 2, v' = v / 2:
                 // sigmoid(g) * v = (tanh(g') + 1) * v' = fma(v', tanh(g'), v')
-                const float h0 = __uint_as_float(rv[n0]), h1 = __uint_as_float(rv[n0 + 1]);
-                const float v0 = fmaf(h0, tanh_fast(__uint_as_float(rg[n0])), h0);
-                const float v1 = fmaf(h1, tanh_fast(__uint_as_float(rg[n0 + 1])), h1);
+                const float h0 = __uint_as_float(rv[k & 1][n0]), h1 = __uint_as_float(rv[k & 1][n0 + 1]);
+                const float v0 = fmaf(h0, tanh_fast(__uint_as_float(rg[k & 1][n0])), h0);
+                const float v1 = fmaf(h1, tanh_fast(__uint_as_float(rg[k & 1][n0 + 1])), h1);
                 __half2 h = __floats2half2_rn(v0, v1);          // overflow gives inf, clamped below
                 h = __hmax2(__hmin2(h, hmax2), hmin2);
                 w[e] = *reinterpret_cast<unsigned*>(&h);

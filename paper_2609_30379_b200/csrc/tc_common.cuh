@@ -127,6 +127,26 @@ __device__ inline void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
       : "r"(taddr) : "memory");
 }
 
+// 32 lanes x 16 consecutive columns
+__device__ inline void tmem_ld16(unsigned taddr, unsigned (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+
+// wait for the TMEM loads in flight; the two register sets are passed through the statement so that no use of
+// them can be scheduled ahead of the wait
+__device__ inline void tmem_ld_wait2(unsigned (&a)[16], unsigned (&b)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(a[8]),
+                 "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]), "+r"(b[0]),
+                 "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]), "+r"(b[8]), "+r"(b[9]),
+                 "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+               :: "memory");
+}
+
 // ---- MMA descriptors (bf16 operands, float accumulate)
 // K-major operand tile in the 128-byte-swizzled layout TMA writes for a {64 elements, rows} box:
 // row r at r * 128 bytes, 16-byte chunks XOR-swizzled by (r & 7); groups of 8 rows are 1024 bytes
