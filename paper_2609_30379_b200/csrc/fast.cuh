@@ -24,6 +24,12 @@ bool fast_attn_core_supported(int H, int d);
 nt_status fast_attn_core(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
                          int pair_order, int bias_prescaled, const BatchMeta& m, int* status, cudaStream_t st);
 
+// the same core on tcgen05 for the samples with 1 <= N <= n_max (pair order, d in {16, 32}, bias stored times sqrt(d));
+// fast_attn_tc_max_n gives the largest N whose score row and bias tiles fit (0: not supported)
+int fast_attn_tc_max_n(int d, bool has_bias);
+nt_status fast_attn_core_tc(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
+                            const BatchMeta& m, int n_max, int* status, cudaStream_t st);
+
 // triangle contraction on tcgen05: a, b, t are three equally spaced channel-major buffers
 // (b = a + stride, t = a + 2 * stride)
 bool fast_contract_supported(int C);

@@ -34,6 +34,7 @@ struct AttnCoreParams {
   int H, pair_order, ichunk, bias_bytes;
   float bias_mul;                 // factor that brings the stored bias to bias * sqrt(d) (1 if stored that way)
   int bias_prescaled;             // bias buffer already holds bias * sqrt(d): the resident tile can go through the MMA
+  int skip_max_n;                 // samples with N <= skip_max_n belong to the tcgen05 kernel
   int* status;
 };
 
@@ -242,6 +243,7 @@ __global__ void __launch_bounds__(AT_THREADS, 2) attn_core_kernel(const __grid_c
     int s = 0;
     for (; s < m.B; ++s) {
       const int N = m.N[s];
+      if (N <= p.skip_max_n) continue;
       if (BIAS != 0 && (AT_Q * at_bias_stride(N) <= AT_RES_CAP) != (BIAS == 1)) continue;   // other launch's sample
       const long long njb = (N + AT_Q - 1) / AT_Q;
       const long long nic = pair_order ? (N + p.ichunk - 1) / p.ichunk : (N > 0 ? 1 : 0);
@@ -393,6 +395,7 @@ static nt_status launch_attn_mode(AttnCoreParams& p, int bias_bytes, cudaStream_
     long long c = 0;
     for (int s = 0; s < m.B; ++s) {
       const long long N = m.N[s], njb = (N + AT_Q - 1) / AT_Q;
+      if (N <= p.skip_max_n) continue;
       if (BIAS != 0 && (AT_Q * at_bias_stride((int)N) <= AT_RES_CAP) != (BIAS == 1)) continue;
       const long long nic = p.pair_order ? (N + ic - 1) / ic : (N > 0 ? 1 : 0);
       c += njb * p.H * nic;
@@ -440,9 +443,27 @@ static nt_status launch_attn(const __nv_bfloat16* q, const __nv_bfloat16* k, con
   const long long rows = (pair_order ? m.pair_off[m.B] : m.tok_off[m.B]) - p.row0;
   if (rows <= 0) return NT_OK;
   if (rows > 0x7FFFFF00ll) return NT_ERR_UNSUPPORTED;
+  // short samples (pair order) go to the tcgen05 kernel, which holds a whole score row in TMEM
+  int skip = 0;
+  if (pair_order && (D == 16 || D == 32)) {
+    const int n_tc = fast_attn_tc_max_n(D, bias != nullptr);
+    bool any_short = false, any_other = false;
+    for (int s = 0; s < m.B; ++s) {
+      if (m.N[s] >= 1 && m.N[s] <= n_tc) any_short = true;
+      else if (m.N[s] > n_tc) any_other = true;
+    }
+    if (any_short) {
+      const nt_status r = fast_attn_core_tc(q, k, v, bias, o, H, D, m, n_tc, status, st);
+      if (r != NT_OK) return r;
+      skip = n_tc;
+      if (!any_other) return NT_OK;
+    }
+  }
+  p.skip_max_n = skip;
   int bias_bytes = 0;
   bool any_long = false;
   for (int s = 0; s < m.B; ++s) {
+    if (m.N[s] <= skip) continue;
     const int res = AT_Q * at_bias_stride(m.N[s]);
     if (res <= AT_RES_CAP) { if (res > bias_bytes) bias_bytes = res; }
     else any_long = true;

@@ -1,0 +1,473 @@
+// Row-wise pair-biased attention on tcgen05 for samples whose whole key range fits one accumulator
+// (N <= 224, pair order, head dim 16 or 32).
+//
+// Work item: one attention row (s, i), one head h, one block of 128 queries j.  The scores of the
+// item, S' = Q K^T (M = 128 queries, N = round_up(N_s, 16) keys, K = d), are one MMA group into a
+// 256-column TMEM buffer, so the softmax needs no running rescale:
+//   pass 1  two threads per query read their halves of the row from TMEM, add the pair bias
+//           (resident in shared memory for both query blocks of the (s, h) being processed, stored
+//           times sqrt(d)), take the row maximum and write the biased scores back;
+//   pass 2  p = exp2((s - max) log2(e) / sqrt(d)) as packed bf16 pairs, each 16-key granule written over
+//           half of its own score columns, from where the second MMA group takes P as its
+//           TMEM-resident A operand: O = P V (N = d) and the row sums l = P 1 (N = 16, a tile of
+//           ones), so numerator and denominator see the same rounded weights;
+//   output  O / l, 16 channels per thread, stored row-major.
+// Roles: warp 0 streams Q | K and warp 2 streams V of each item with TMA (32-row boxes, swizzle span =
+// 2 d bytes) through two rings (a Q | K stage is free again as soon as the scores are computed), one
+// thread of warp 1 issues the MMAs (the scores of item n + 1 before P V of item n), warps 3-10 and
+// 11-18 are two softmax groups that own one TMEM buffer each and take alternate items.  Each CTA walks a contiguous range of the items ordered (s, h, i, j block), so the
+// two query blocks of a row are neighbours (their K / V come from L2 the second time) and the bias
+// tiles are reloaded only when (s, h) changes.
+#include <cstring>
+
+#include "fast.cuh"
+#include "tc_common.cuh"
+
+namespace ntp {
+
+constexpr int TCA_THREADS = 96 + 512;
+constexpr int TCA_NMAX = 224;      // keys per item: 224 score columns + 32 output columns = one 256-column TMEM buffer
+constexpr int TCA_O_COL = 224;     // output accumulator (up to 32 columns)
+constexpr int TCA_L_COL = 8;       // row sums (16 columns): the gap between the weights of granules 0 and 1
+constexpr float TCA_LOG2E = 1.4426950408889634f;
+
+struct AttnTcParams {
+  CUtensorMap qmap;       // flat {H d, rows}, box {d, 128}
+  CUtensorMap kmap, vmap; // box {d, 32}
+  BatchMeta m;
+  long long item_off[MAXB + 1];   // prefix of N_s * H * ceil(N_s / 128) over the samples this kernel takes
+  const __nv_bfloat16* bias;      // head-major channel-major, stored times sqrt(d); nullable
+  __nv_bfloat16* o;
+  long long row0;                 // first packed row the maps cover
+  int H, nqk, nv, kv_rows;        // stages of the Q|K ring and of the V ring; rows reserved for K (and V) per stage
+  int bias_tile_bytes;            // bytes reserved per resident bias tile
+  int n_max;                      // samples with N > n_max are left to the other kernel
+  int* status;
+};
+
+__host__ __device__ inline int tca_bias_stride(int N) {   // bytes per resident bias row: an odd multiple of 16
+  int b = round_up8(N) * 2;
+  return (b / 16) % 2 == 0 ? b + 16 : b;
+}
+
+__device__ inline void tca_cp_async16(void* smem, const void* gmem, bool valid) {
+  const unsigned sa = (unsigned)__cvta_generic_to_shared(smem);
+  const int sz = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(sa), "l"(gmem), "r"(sz));
+}
+
+__device__ inline unsigned tca_exp2_bf16x2(float lo, float hi) {
+  unsigned x, y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(x) : "f"(hi), "f"(lo));
+  asm("ex2.approx.ftz.bf16x2 %0, %1;\n" : "=r"(y) : "r"(x));
+  return y;
+}
+
+// swizzled K-major / MN-major operand descriptor for a tile whose rows are `span` = 32, 64 or 128 bytes.  The start
+// address sits in the low 14 bits in units of 16 bytes, so moving the operand by x bytes is adding x / 16.
+__device__ inline unsigned long long tca_desc(unsigned saddr, int span) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((saddr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)(((unsigned)(8 * span) >> 4) & 0x3FFF) << 16;   // leading byte offset (one block: unused)
+  d |= (unsigned long long)(((unsigned)(8 * span) >> 4) & 0x3FFF) << 32;   // 8 rows further
+  d |= (unsigned long long)1 << 46;
+  d |= (unsigned long long)(span == 128 ? 2 : span == 64 ? 4 : 6) << 61;
+  return d;
+}
+
+template <int D>
+__global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams p) {
+  constexpr int SPAN = 2 * D;                 // bytes per tile row = swizzle span
+  constexpr int Q_BYTES = 128 * SPAN;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bars[12 + 8];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_flag;
+  unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
+  const int kv_bytes = p.kv_rows * SPAN;
+  const int qk_bytes = Q_BYTES + kv_bytes;
+  unsigned char* sQK = smem;                                      // [nqk][Q | K]
+  unsigned char* sV = sQK + p.nqk * qk_bytes;                     // [nv][V]
+  unsigned char* sOnes = sV + p.nv * kv_bytes;                    // 16 x 16 ones (512 bytes)
+  float* xmax = reinterpret_cast<float*>(sOnes + 512);            // [2 groups][2 parities][2 halves][128]
+  unsigned char* sBias = reinterpret_cast<unsigned char*>(xmax) + 2 * 2 * 2 * 128 * 4;   // [2 tiles][128][stride]
+  unsigned long long* qkfull = bars;          // [3]
+  unsigned long long* qkempty = bars + 3;     // [3] the score MMAs that read the stage are done
+  unsigned long long* vfull = bars + 6;       // [3]
+  unsigned long long* vempty = bars + 9;      // [3] the P V MMAs that read the stage are done
+  unsigned long long* sfull = bars + 12;      // [2] scores of the group's item are in TMEM
+  unsigned long long* sempty = bars + 14;     // [2] the group has read its output: buffer free
+  unsigned long long* pfull = bars + 16;      // [2] P written
+  unsigned long long* ofull = bars + 18;      // [2] P V and the row sums are complete
+
+  const BatchMeta& m = p.m;
+  const int H = p.H, Hd = H * D;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < 12; ++s) mbar_init(&bars[s], 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sfull[b], 1);
+      mbar_init(&sempty[b], 8);
+      mbar_init(&pfull[b], 8);
+      mbar_init(&ofull[b], 1);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&tmem_base_s, 512);
+  for (int idx = threadIdx.x; idx < 128; idx += TCA_THREADS) reinterpret_cast<unsigned*>(sOnes)[idx] = 0x3F803F80u;
+  fence_proxy_async_smem();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem_base = tmem_base_s;
+  AbortCtx ab{p.status, &abort_flag};
+  const float sc2 = rsqrtf((float)D) * TCA_LOG2E;
+  const bool has_bias = p.bias != nullptr;
+
+  const long long total = p.item_off[m.B];
+  long long r = total * blockIdx.x / gridDim.x;
+  const long long r_end = total * (blockIdx.x + 1) / gridDim.x;
+  unsigned it0 = 0;                           // items this CTA has finished (drives every ring position / parity)
+
+  while (r < r_end) {
+    // ------------------------------------------------------------ segment: items of one (s, h)
+    int s = 0;
+    while (s + 1 < m.B && r >= p.item_off[s + 1]) ++s;
+    const int N = m.N[s], ld = round_up8(N), Nk = (N + 15) & ~15;
+    const int njb = (N + 127) / 128;
+    const unsigned rem0 = (unsigned)(r - p.item_off[s]);           // ((h N + i) njb + jb)
+    const int h = (int)(rem0 / (unsigned)(N * njb));
+    const unsigned in_head0 = rem0 - (unsigned)h * (unsigned)(N * njb);   // i njb + jb of the first item
+    const long long left = (long long)N * njb - in_head0;
+    const int cnt = (int)(left < r_end - r ? left : r_end - r);
+    const int bstride = tca_bias_stride(N);
+    const __nv_bfloat16* bias_h = has_bias ? p.bias + (long long)H * m.cm_off[s] + (long long)h * N * ld : nullptr;
+    const long long row_base = m.pair_off[s] - p.row0;            // packed row of (i = 0, j = 0) relative to the maps
+    const int nb = (N + 31) / 32;                                  // 32-row boxes of K (and V)
+    const int ng = Nk / 16;                                        // 16-key granules
+
+    if (has_bias && warp >= 3) {
+      const int chunks = ld / 8;
+      for (int idx = threadIdx.x - 96; idx < njb * 128 * chunks; idx += 512) {
+        const int rr = idx / chunks, c = idx - rr * chunks;        // rr = query j
+        const bool ok = rr < N;
+        tca_cp_async16(sBias + (rr >> 7) * p.bias_tile_bytes + (rr & 127) * bstride + c * 16,
+                       bias_h + (long long)(ok ? rr : 0) * ld + c * 8, ok);
+      }
+      asm volatile("cp.async.wait_all;\n" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+      // -------------------------------------------------------------- Q | K producer
+      unsigned st = it0 % (unsigned)p.nqk, k = it0 / (unsigned)p.nqk;
+      for (int n = 0; n < cnt; ++n) {
+        const unsigned ih = in_head0 + n;
+        const int i = (int)(ih / (unsigned)njb), jb = (int)(ih - (unsigned)i * njb);
+        const int base = (int)(row_base + (long long)i * N);
+        unsigned char* stg = sQK + st * qk_bytes;
+        if (lane == 0) {
+          mbar_wait(&qkempty[st], (k & 1) ^ 1, ab);
+          mbar_expect_tx(&qkfull[st], Q_BYTES + nb * 32 * SPAN);
+        }
+        __syncwarp();
+        if (lane == 0) tma_load_2d(stg, &p.qmap, &qkfull[st], h * D, base + jb * 128);
+        else if (lane <= nb) tma_load_2d(stg + Q_BYTES + (lane - 1) * 32 * SPAN, &p.kmap, &qkfull[st], h * D, base + (lane - 1) * 32);
+        if (++st == (unsigned)p.nqk) { st = 0; ++k; }
+      }
+    } else if (warp == 2) {
+      // -------------------------------------------------------------- V producer
+      unsigned st = it0 % (unsigned)p.nv, k = it0 / (unsigned)p.nv;
+      for (int n = 0; n < cnt; ++n) {
+        const unsigned ih = in_head0 + n;
+        const int i = (int)(ih / (unsigned)njb);
+        const int base = (int)(row_base + (long long)i * N);
+        if (lane == 0) {
+          mbar_wait(&vempty[st], (k & 1) ^ 1, ab);
+          mbar_expect_tx(&vfull[st], nb * 32 * SPAN);
+        }
+        __syncwarp();
+        if (lane < nb) tma_load_2d(sV + st * kv_bytes + lane * 32 * SPAN, &p.vmap, &vfull[st], h * D, base + lane * 32);
+        if (++st == (unsigned)p.nv) { st = 0; ++k; }
+      }
+    } else if (warp == 1) {
+      // -------------------------------------------------------------- MMA issuer (whole warp, one elected lane issues)
+      const unsigned idesc_s = idesc_f16(128, Nk, 0, 0, FMT_BF16, FMT_BF16);
+      const unsigned idesc_o = idesc_f16(128, D, 0, 1, FMT_BF16, FMT_BF16);     // B = V is MN-major
+      const unsigned idesc_l = idesc_f16(128, 16, 0, 0, FMT_BF16, FMT_BF16);
+      const unsigned long long ones_desc = desc_kmajor_nosw(smem_u32(sOnes), 256, 128);
+      unsigned sq = it0 % (unsigned)p.nqk, kq = it0 / (unsigned)p.nqk;           // ring position of the next score item
+      unsigned sv = it0 % (unsigned)p.nv, kv = it0 / (unsigned)p.nv;             // ... of the next P V item
+      for (int n = 0; n <= cnt; ++n) {
+        if (n < cnt) {
+          const unsigned it = it0 + n, b = it & 1, u = it >> 1;
+          mbar_wait(&qkfull[sq], kq & 1, ab);
+          mbar_wait(&sempty[b], (u & 1) ^ 1, ab);
+          tc_fence_after();
+          const unsigned q_addr = smem_u32(sQK + sq * qk_bytes);
+          const unsigned long long qd = tca_desc(q_addr, SPAN), kd = tca_desc(q_addr + Q_BYTES, SPAN);
+          if (elect_one()) {
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) umma_bf16(tmem_base + b * 256, qd + ks * 2, kd + ks * 2, idesc_s, ks);
+            tc_commit(&sfull[b]);
+            tc_commit(&qkempty[sq]);
+          }
+          __syncwarp();
+          if (++sq == (unsigned)p.nqk) { sq = 0; ++kq; }
+        }
+        if (n >= 1) {
+          const unsigned it = it0 + n - 1, b = it & 1, u = it >> 1;
+          mbar_wait(&vfull[sv], kv & 1, ab);
+          mbar_wait(&pfull[b], u & 1, ab);
+          tc_fence_after();
+          const unsigned long long vd = tca_desc(smem_u32(sV + sv * kv_bytes), SPAN);
+          const unsigned a_p = tmem_base + b * 256, d_o = a_p + TCA_O_COL, d_l = a_p + TCA_L_COL;
+#pragma unroll
+          for (int kk = 0; kk < TCA_NMAX / 16; ++kk) {
+            if (kk < ng) {
+              const unsigned a_kk = a_p + kk * 16 + (kk & 1) * 8;
+              if (elect_one()) {
+                umma_ts(d_o, a_kk, vd + kk * SPAN, idesc_o, kk);     // 16 rows of V further: 16 SPAN bytes
+                umma_ts(d_l, a_kk, ones_desc, idesc_l, kk);
+              }
+            }
+          }
+          if (elect_one()) {
+            tc_commit(&ofull[b]);
+            tc_commit(&vempty[sv]);
+          }
+          __syncwarp();
+          if (++sv == (unsigned)p.nv) { sv = 0; ++kv; }
+        }
+      }
+    } else {
+      // -------------------------------------------------------------- softmax groups
+      const int sw = warp - 3, wg = sw >> 3, hf = (sw >> 2) & 1, quarter = warp & 3;
+      const int row = quarter * 32 + lane;                          // query inside the 128-block = TMEM lane
+      const unsigned t_row = tmem_base + ((unsigned)(quarter * 32) << 16) + wg * 256;
+      for (int n = (int)((wg ^ it0) & 1); n < cnt; n += 2) {
+        const unsigned it = it0 + n, u = it >> 1;
+        const unsigned ih = in_head0 + n;
+        const int i = (int)(ih / (unsigned)njb), jb = (int)(ih - (unsigned)i * njb);
+        const int j = jb * 128 + row;
+        const bool warp_live = jb * 128 + quarter * 32 < N;        // this warp owns at least one real query
+        const unsigned char* brow = sBias + jb * p.bias_tile_bytes + row * bstride;
+        float* xm = xmax + ((wg * 2 + (u & 1)) * 2) * 128;
+        unsigned ra[16], rb[16];
+        mbar_wait(&sfull[wg], u & 1, ab);
+        tc_fence_after();
+        // ---- pass 1: biased scores and row maximum over granules hf, hf + 2, ...; the TMEM and bias loads of the
+        // next granule are in flight while one is processed
+        float mx = -INFINITY;
+        if (warp_live) {
+          uint4 ba[2], bb[2];
+          auto fetch = [&](int g, unsigned (&rr)[16], uint4 (&bv)[2]) {
+            tmem_ld16(t_row + g * 16, rr);
+            if (has_bias) {
+              bv[0] = *reinterpret_cast<const uint4*>(brow + g * 32);
+              bv[1] = *reinterpret_cast<const uint4*>(brow + g * 32 + 16);
+            } else {
+              bv[0] = bv[1] = make_uint4(0, 0, 0, 0);
+            }
+          };
+          auto pass1 = [&](int g, unsigned (&rr)[16], const uint4 (&bv)[2]) {
+            const unsigned bw[8] = {bv[0].x, bv[0].y, bv[0].z, bv[0].w, bv[1].x, bv[1].y, bv[1].z, bv[1].w};
+            float sv[16];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              sv[2 * e] = __uint_as_float(rr[2 * e]) + __uint_as_float(bw[e] << 16);
+              sv[2 * e + 1] = __uint_as_float(rr[2 * e + 1]) + __uint_as_float(bw[e] & 0xffff0000u);
+            }
+            if (g * 16 + 16 > N) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e)
+                if (g * 16 + e >= N) sv[e] = -INFINITY;
+            }
+            float m4[4] = {sv[0], sv[1], sv[2], sv[3]};
+#pragma unroll
+            for (int e = 4; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], sv[e]);
+            mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+#pragma unroll
+            for (int e = 0; e < 16; ++e) rr[e] = __float_as_uint(sv[e]);
+            tmem_st16(t_row + g * 16, rr);
+          };
+          if (hf < ng) fetch(hf, ra, ba);
+#pragma unroll
+          for (int gi = 0; gi < 8; gi += 2) {
+            const int g0 = hf + 2 * gi, g1 = g0 + 2, g2 = g0 + 4;
+            if (g0 < ng) {
+              tmem_ld_wait16(ra);
+              const uint4 cur[2] = {ba[0], ba[1]};
+              if (g1 < ng) fetch(g1, rb, bb);
+              pass1(g0, ra, cur);
+            }
+            if (g1 < ng) {
+              tmem_ld_wait16(rb);
+              const uint4 cur[2] = {bb[0], bb[1]};
+              if (g2 < ng) fetch(g2, ra, ba);
+              pass1(g1, rb, cur);
+            }
+          }
+          tmem_st_wait();
+        }
+        xm[hf * 128 + row] = mx;
+        named_bar_sync(1 + wg, 256);
+        mx = fmaxf(mx, xm[(hf ^ 1) * 128 + row]);
+        // ---- pass 2: weights as packed bf16 pairs, written over the first (even granules) or second (odd granules)
+        // half of the granule's own score columns, which only this thread reads
+        if (warp_live) {
+          const float ms = -mx * sc2;
+          auto pass2 = [&](int g, const unsigned (&rr)[16]) {
+            unsigned pk[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              pk[e] = tca_exp2_bf16x2(fmaf(__uint_as_float(rr[2 * e]), sc2, ms), fmaf(__uint_as_float(rr[2 * e + 1]), sc2, ms));
+            tmem_st8(t_row + g * 16 + (g & 1) * 8, pk);
+          };
+          if (hf < ng) tmem_ld16(t_row + hf * 16, ra);
+#pragma unroll
+          for (int gi = 0; gi < 8; gi += 2) {
+            const int g0 = hf + 2 * gi, g1 = g0 + 2, g2 = g0 + 4;
+            if (g0 < ng) {
+              tmem_ld_wait16(ra);
+              if (g1 < ng) tmem_ld16(t_row + g1 * 16, rb);
+              pass2(g0, ra);
+            }
+            if (g1 < ng) {
+              tmem_ld_wait16(rb);
+              if (g2 < ng) tmem_ld16(t_row + g2 * 16, ra);
+              pass2(g1, rb);
+            }
+          }
+          tmem_st_wait();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&pfull[wg]);
+        // ---- output: O / l
+        mbar_wait(&ofull[wg], u & 1, ab);
+        tc_fence_after();
+        if (warp_live && (D >= 32 || hf == 0)) {
+          constexpr int CPT = D >= 32 ? D / 2 : D;                 // output channels per thread (16)
+          unsigned lv;
+          tmem_ld16(t_row + TCA_O_COL + hf * CPT, ra);
+          tmem_ld1(t_row + TCA_L_COL, lv);
+          tmem_ld_wait16_1(ra, lv);
+          const float inv = 1.0f / __uint_as_float(lv);
+          if (j < N) {
+            __nv_bfloat16* op = p.o + (p.row0 + row_base + (long long)i * N + j) * Hd + h * D + hf * CPT;
+            unsigned w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(ra[2 * e]) * inv, __uint_as_float(ra[2 * e + 1]) * inv);
+              w[e] = *reinterpret_cast<unsigned*>(&t2);
+            }
+            *reinterpret_cast<uint4*>(op) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(op + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sempty[wg]);
+      }
+    }
+    it0 += (unsigned)cnt;
+    r += cnt;
+    __syncthreads();   // every role has finished the segment: the bias tiles may be replaced
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+static size_t tca_smem_bytes(int D, int n_max, bool has_bias, int nqk, int nv, int* kv_rows, int* tile_bytes) {
+  const int rows = (n_max + 31) & ~31;
+  *kv_rows = rows;
+  *tile_bytes = has_bias ? 128 * tca_bias_stride(n_max) : 0;
+  const int njb = (n_max + 127) / 128;
+  return (size_t)nqk * (128 * 2 * D + rows * 2 * D) + (size_t)nv * rows * 2 * D + 512 + 2 * 2 * 2 * 128 * 4 +
+         (size_t)njb * *tile_bytes + 64 + 1024;
+}
+
+template <int D>
+static nt_status launch_attn_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                const __nv_bfloat16* bias, __nv_bfloat16* o, int H, const BatchMeta& m, int n_max,
+                                int* status, cudaStream_t st) {
+  AttnTcParams p;
+  memset(&p, 0, sizeof(p));
+  p.m = m;
+  p.bias = bias;
+  p.o = o;
+  p.H = H;
+  p.n_max = n_max;
+  p.status = status;
+  p.row0 = m.pair_off[0];
+  const long long rows = m.pair_off[m.B] - p.row0;
+  if (rows <= 0) return NT_OK;
+  if (rows > 0x7FFFFF00ll) return NT_ERR_UNSUPPORTED;
+  int longest = 0;
+  p.item_off[0] = 0;
+  for (int s = 0; s < m.B; ++s) {
+    const int N = m.N[s];
+    const bool take = N >= 1 && N <= n_max;
+    if (take && N > longest) longest = N;
+    p.item_off[s + 1] = p.item_off[s] + (take ? (long long)N * H * ((N + 127) / 128) : 0);
+  }
+  const long long total = p.item_off[m.B];
+  if (total == 0) return NT_OK;
+  const size_t limit = 232448;
+  size_t smem = 0;
+  const int tries[3][2] = {{3, 3}, {3, 2}, {2, 2}};
+  for (int t = 0; t < 3; ++t) {
+    p.nqk = tries[t][0];
+    p.nv = tries[t][1];
+    smem = tca_smem_bytes(D, longest, bias != nullptr, p.nqk, p.nv, &p.kv_rows, &p.bias_tile_bytes);
+    if (smem <= limit) break;
+  }
+  if (smem > limit) return NT_ERR_UNSUPPORTED;
+  const int Hd = H * D;
+  {
+    const unsigned long long dims[2] = {(unsigned long long)Hd, (unsigned long long)rows};
+    const unsigned long long strides[1] = {(unsigned long long)Hd * 2};
+    const unsigned qbox[2] = {(unsigned)D, 128}, kbox[2] = {(unsigned)D, 32};
+    if (!make_tmap_16bit(&p.qmap, q + p.row0 * Hd, 2, dims, strides, qbox, 2 * D)) return cuda_fail("attn tc q map");
+    if (!make_tmap_16bit(&p.kmap, k + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn tc k map");
+    if (!make_tmap_16bit(&p.vmap, v + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn tc v map");
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit - 1024) != cudaSuccess)
+      return cuda_fail("attention tc smem attribute");
+    attr_set = true;
+  }
+  const unsigned grid = (unsigned)(total < 148 ? total : 148);
+  {
+    LaunchScope ls("attn_core", st);
+    attn_tc_kernel<D><<<grid, TCA_THREADS, smem, st>>>(p);
+  }
+  return cuda_ok("attention tc launch");
+}
+
+int fast_attn_tc_max_n(int d, bool has_bias) {
+  if (d != 16 && d != 32) return 0;
+  int kv_rows, tile;
+  int n = TCA_NMAX;
+  while (n > 0 && tca_smem_bytes(d, n, has_bias, 2, 2, &kv_rows, &tile) > 232448 - 1024) n -= 8;
+  return n;
+}
+
+nt_status fast_attn_core_tc(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
+                            const BatchMeta& m, int n_max, int* status, cudaStream_t st) {
+  const __nv_bfloat16* qq = (const __nv_bfloat16*)q;
+  const __nv_bfloat16* kk = (const __nv_bfloat16*)k;
+  const __nv_bfloat16* vv = (const __nv_bfloat16*)v;
+  const __nv_bfloat16* bb = (const __nv_bfloat16*)bias;
+  __nv_bfloat16* oo = (__nv_bfloat16*)o;
+  if (d == 16) return launch_attn_tc<16>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+  if (d == 32) return launch_attn_tc<32>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+  return NT_ERR_UNSUPPORTED;
+}
+
+}  // namespace ntp

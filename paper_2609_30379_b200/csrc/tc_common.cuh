@@ -1,6 +1,6 @@
 // sm_100a building blocks for the tensor-core kernels: mbarrier with bounded waits, TMA tiled
 // loads / stores, tcgen05 MMA with shared-memory operand descriptors, TMEM allocation and loads.
-// Every wait has an iteration limit; on expiry the kernel records NT_ERR_TIMEOUT in the status
+// Every wait is bounded (a probe count and about a second of SM clocks); on expiry the kernel records NT_ERR_TIMEOUT in the status
 // word, raises a CTA-wide abort flag (later waits give up after a short spin) and still runs to
 // its normal end, so TMEM is released and the context stays usable.
 #pragma once
@@ -26,8 +26,9 @@ bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigne
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------- device helpers
-constexpr unsigned WAIT_LIMIT = 1u << 22;        // polls before a wait gives up (~ tens of ms)
-constexpr unsigned WAIT_LIMIT_ABORTED = 1u << 10;
+constexpr unsigned WAIT_PROBES = 1u << 22;            // probes before a wait gives up, whatever the clock says
+constexpr long long WAIT_CLOCKS = 1ll << 31;          // SM clocks before a wait gives up (about a second)
+constexpr long long WAIT_CLOCKS_ABORTED = 1ll << 14;  // once the CTA has given up, later waits return quickly
 
 struct AbortCtx {
   int* status;            // global status word (nullable)
@@ -46,22 +47,25 @@ __device__ inline void mbar_expect_tx(void* bar, unsigned bytes) {
 __device__ inline void mbar_arrive(void* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ inline bool mbar_try(void* bar, unsigned parity) {
+// One probe of the barrier; the hardware may park the warp for up to `suspend_ns` before it answers, so a waiting
+// role does not spend issue slots on polling.
+__device__ inline bool mbar_try(void* bar, unsigned parity, unsigned suspend_ns) {
   unsigned ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns) : "memory");
   return ok != 0;
 }
-// bounded wait; returns false (after flagging) if the limit was reached
+// bounded wait (by elapsed SM clocks); returns false (after flagging) if the limit was reached
 __device__ inline bool mbar_wait(void* bar, unsigned parity, const AbortCtx& ab) {
-  const unsigned limit = *ab.flag ? WAIT_LIMIT_ABORTED : WAIT_LIMIT;
-  for (unsigned it = 0; it < limit; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if (it >= 4) __nanosleep(40);          // waiting roles should not steal issue slots from working warps
-    if ((it & 1023u) == 1023u && *ab.flag) break;
+  if (mbar_try(bar, parity, 0)) return true;
+  const long long t0 = clock64();
+  const long long limit = *ab.flag ? WAIT_CLOCKS_ABORTED : WAIT_CLOCKS;
+  for (unsigned it = 0; it < WAIT_PROBES; ++it) {
+    if (mbar_try(bar, parity, 20000)) return true;
+    if (clock64() - t0 > limit || *ab.flag) break;
   }
   if (!*ab.flag) {
     *ab.flag = 1;
@@ -136,6 +140,44 @@ __device__ inline void tmem_ld16(unsigned taddr, unsigned (&r)[16]) {
       : "r"(taddr) : "memory");
 }
 
+__device__ inline void tmem_ld1(unsigned taddr, unsigned& r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n" : "=r"(r) : "r"(taddr) : "memory");
+}
+// registers -> TMEM: thread t writes row (lane base + t), 16 or 8 consecutive columns
+__device__ inline void tmem_st16(unsigned taddr, const unsigned (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ inline void tmem_st8(unsigned taddr, const unsigned (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};\n"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ inline void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem]: the A tile (128 rows x 16 elements, two 16-bit elements per column) is read from TMEM
+__device__ inline void umma_ts(unsigned d_tmem, unsigned a_tmem, unsigned long long bdesc, unsigned idesc,
+                               unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// waits for the TMEM loads in flight; the destination registers pass through the statement so that no use of them
+// can be scheduled ahead of the wait
+__device__ inline void tmem_ld_wait16(unsigned (&a)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(a[8]),
+                 "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15])
+               :: "memory");
+}
+__device__ inline void tmem_ld_wait16_1(unsigned (&a)[16], unsigned& b) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(a[8]),
+                 "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]), "+r"(b)
+               :: "memory");
+}
 // wait for the TMEM loads in flight; the two register sets are passed through the statement so that no use of
 // them can be scheduled ahead of the wait
 __device__ inline void tmem_ld_wait2(unsigned (&a)[16], unsigned (&b)[16]) {
@@ -197,6 +239,15 @@ __device__ inline void umma_bf16(unsigned d_tmem, unsigned long long adesc, unsi
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// true in exactly one lane of a converged warp.  The MMA issuer runs its loop with the whole warp and puts only
+// the tcgen05 instructions under this predicate: descriptors and addresses then stay warp-uniform, which keeps
+// the cost of issuing one MMA at a few instructions.
+__device__ inline bool elect_one() {
+  unsigned pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.b32 %0, 1, 0, p;\n\t}\n" : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ inline void named_bar_sync(int id, int nthreads) {
