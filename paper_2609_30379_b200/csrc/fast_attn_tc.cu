@@ -2,22 +2,25 @@
 // (N <= 224, pair order, head dim 16 or 32).
 //
 // Work item: one attention row (s, i), one head h, one block of 128 queries j.  The scores of the
-// item, S' = Q K^T (M = 128 queries, N = round_up(N_s, 16) keys, K = d), are one MMA group into a
-// 256-column TMEM buffer, so the softmax needs no running rescale:
-//   pass 1  two threads per query read their halves of the row from TMEM, add the pair bias
-//           (resident in shared memory for both query blocks of the (s, h) being processed, stored
-//           times sqrt(d)), take the row maximum and write the biased scores back;
-//   pass 2  p = exp2((s - max) log2(e) / sqrt(d)) as packed bf16 pairs, each 16-key granule written over
-//           half of its own score columns, from where the second MMA group takes P as its
-//           TMEM-resident A operand: O = P V (N = d) and the row sums l = P 1 (N = 16, a tile of
-//           ones), so numerator and denominator see the same rounded weights;
+// item are one MMA group into a 224-column TMEM accumulator (M = 128 queries, N = round_up(N_s, 16)
+// keys): S' = Q K^T (K = d) plus the pair bias, which enters through the tensor cores as well: the
+// bias tile of the (s, h, j block), resident in shared memory and stored times sqrt(d), is the
+// MN-major B operand of a product whose A operand is the 128 x 128 identity (1.0 * bias is exact in
+// the float accumulator; the identity is a 16 x 16 block sliding over a band of zeros).  With the
+// whole row in TMEM the softmax needs no running rescale:
+//   pass 1  two threads per query read their halves of the row and take the maximum;
+//   pass 2  p = exp2((s - max) log2(e) / sqrt(d)), summed in float and written as packed bf16 pairs
+//           over half of each 16-key granule's own score columns, from where the second MMA group
+//           takes P as its TMEM-resident A operand: O = P V (N = d) into 32 columns of its own;
 //   output  O / l, 16 channels per thread, stored row-major.
+// The exponentials are the floor of this kernel: an SM retires 16 per clock.
 // Roles: warp 0 streams Q | K and warp 2 streams V of each item with TMA (32-row boxes, swizzle span =
-// 2 d bytes) through two rings (a Q | K stage is free again as soon as the scores are computed), one
-// thread of warp 1 issues the MMAs (the scores of item n + 1 before P V of item n), warps 3-10 and
-// 11-18 are two softmax groups that own one TMEM buffer each and take alternate items.  Each CTA walks a contiguous range of the items ordered (s, h, i, j block), so the
-// two query blocks of a row are neighbours (their K / V come from L2 the second time) and the bias
-// tiles are reloaded only when (s, h) changes.
+// 2 d bytes) through two rings (a Q | K stage is free again as soon as the scores are computed), warp 1
+// issues the MMAs (converged, one elected lane; the scores of item n + 1 before P V of item n), warps
+// 3-10 and 11-18 are two softmax groups that own one TMEM buffer each and take alternate items.  Each
+// CTA walks a contiguous range of the items ordered (s, h, i, j block), so the two query blocks of a
+// row are neighbours (their K / V come from L2 the second time) and the bias tiles are reloaded only
+// when (s, h) changes.
 #include <cstring>
 
 #include "fast.cuh"
@@ -28,7 +31,7 @@ namespace ntp {
 constexpr int TCA_THREADS = 96 + 512;
 constexpr int TCA_NMAX = 224;      // keys per item: 224 score columns + 32 output columns = one 256-column TMEM buffer
 constexpr int TCA_O_COL = 224;     // output accumulator (up to 32 columns)
-constexpr int TCA_L_COL = 8;       // row sums (16 columns): the gap between the weights of granules 0 and 1
+constexpr int TCA_IDENT_BYTES = 31 * 256;   // identity band: 31 groups of 8 rows x 16 columns
 constexpr float TCA_LOG2E = 1.4426950408889634f;
 
 struct AttnTcParams {
@@ -45,21 +48,20 @@ struct AttnTcParams {
   int* status;
 };
 
-__host__ __device__ inline int tca_bias_stride(int N) {   // bytes per resident bias row: an odd multiple of 16
-  int b = round_up8(N) * 2;
-  return (b / 16) % 2 == 0 ? b + 16 : b;
-}
-
 __device__ inline void tca_cp_async16(void* smem, const void* gmem, bool valid) {
   const unsigned sa = (unsigned)__cvta_generic_to_shared(smem);
   const int sz = valid ? 16 : 0;
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(sa), "l"(gmem), "r"(sz));
 }
 
-__device__ inline unsigned tca_exp2_bf16x2(float lo, float hi) {
-  unsigned x, y;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(x) : "f"(hi), "f"(lo));
-  asm("ex2.approx.ftz.bf16x2 %0, %1;\n" : "=r"(y) : "r"(x));
+__device__ inline float tca_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ inline unsigned tca_pack(float lo, float hi) {
+  unsigned y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(y) : "f"(hi), "f"(lo));
   return y;
 }
 
@@ -88,17 +90,17 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
   const int qk_bytes = Q_BYTES + kv_bytes;
   unsigned char* sQK = smem;                                      // [nqk][Q | K]
   unsigned char* sV = sQK + p.nqk * qk_bytes;                     // [nv][V]
-  unsigned char* sOnes = sV + p.nv * kv_bytes;                    // 16 x 16 ones (512 bytes)
-  float* xmax = reinterpret_cast<float*>(sOnes + 512);            // [2 groups][2 parities][2 halves][128]
-  unsigned char* sBias = reinterpret_cast<unsigned char*>(xmax) + 2 * 2 * 2 * 128 * 4;   // [2 tiles][128][stride]
+  unsigned char* sIdent = sV + p.nv * kv_bytes;                   // identity band (see below)
+  float* xch = reinterpret_cast<float*>(sIdent + TCA_IDENT_BYTES + 256);   // [2 groups][2 parities][max | sum][2 halves][128]
+  unsigned char* sBias = reinterpret_cast<unsigned char*>(xch) + 2 * 2 * 2 * 2 * 128 * 4;   // [2 tiles][keys / 8][128 queries][8 keys]
   unsigned long long* qkfull = bars;          // [3]
   unsigned long long* qkempty = bars + 3;     // [3] the score MMAs that read the stage are done
   unsigned long long* vfull = bars + 6;       // [3]
   unsigned long long* vempty = bars + 9;      // [3] the P V MMAs that read the stage are done
   unsigned long long* sfull = bars + 12;      // [2] scores of the group's item are in TMEM
-  unsigned long long* sempty = bars + 14;     // [2] the group has read its output: buffer free
+  unsigned long long* sempty = bars + 14;     // [2] P V has consumed the weights: the score columns are free
   unsigned long long* pfull = bars + 16;      // [2] P written
-  unsigned long long* ofull = bars + 18;      // [2] P V and the row sums are complete
+  unsigned long long* ofull = bars + 18;      // [2] P V complete
 
   const BatchMeta& m = p.m;
   const int H = p.H, Hd = H * D;
@@ -108,14 +110,26 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     for (int s = 0; s < 12; ++s) mbar_init(&bars[s], 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sfull[b], 1);
-      mbar_init(&sempty[b], 8);
+      mbar_init(&sempty[b], 1);
       mbar_init(&pfull[b], 8);
       mbar_init(&ofull[b], 1);
     }
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
-  for (int idx = threadIdx.x; idx < 128; idx += TCA_THREADS) reinterpret_cast<unsigned*>(sOnes)[idx] = 0x3F803F80u;
+  // Identity band, K-major without swizzle: 31 groups of 8 rows; a group is two 128-byte core matrices (columns
+  // 0-7 and 8-15), a row is 16 bytes of one.  Groups 15 and 16 hold the 16 x 16 identity, the rest is zero.  The A
+  // operand of bias K step kk (queries 16 kk .. 16 kk + 15) starts at group 15 - 2 kk, so that its rows
+  // 16 kk .. 16 kk + 15 fall on the identity and all others on zeros.
+  for (int idx = threadIdx.x; idx < TCA_IDENT_BYTES / 4; idx += TCA_THREADS) {
+    const int byte = idx * 4, grp = byte >> 8, chunk = (byte >> 7) & 1, r = (byte >> 4) & 7, c2 = (byte >> 2) & 3;
+    unsigned w = 0;
+    if (grp == 15 + chunk) {                     // group 15: rows 0-7 meet columns 0-7; group 16: rows 8-15 meet columns 8-15
+      if (r == 2 * c2) w = 0x00003F80u;
+      else if (r == 2 * c2 + 1) w = 0x3F800000u;
+    }
+    reinterpret_cast<unsigned*>(sIdent)[idx] = w;
+  }
   fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
@@ -141,21 +155,32 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     const unsigned in_head0 = rem0 - (unsigned)h * (unsigned)(N * njb);   // i njb + jb of the first item
     const long long left = (long long)N * njb - in_head0;
     const int cnt = (int)(left < r_end - r ? left : r_end - r);
-    const int bstride = tca_bias_stride(N);
     const __nv_bfloat16* bias_h = has_bias ? p.bias + (long long)H * m.cm_off[s] + (long long)h * N * ld : nullptr;
     const long long row_base = m.pair_off[s] - p.row0;            // packed row of (i = 0, j = 0) relative to the maps
     const int nb = (N + 31) / 32;                                  // 32-row boxes of K (and V)
     const int ng = Nk / 16;                                        // 16-key granules
 
-    if (has_bias && warp >= 3) {
-      const int chunks = ld / 8;
+    if (warp >= 3) {
+      // bias tile of query block t: element (query q, key k) at t * tile + (k / 8) * 2048 + q * 16 + (k % 8) * 2,
+      // the MN-major layout without swizzle (8 keys x 8 queries per 128-byte core matrix).  Key columns N .. Nk - 1
+      // (rows of K that belong to other pair rows) get a large negative bias, so their weights come out as exact
+      // zeros and neither softmax pass needs a mask.
+      const int chunks = Nk / 8;
       for (int idx = threadIdx.x - 96; idx < njb * 128 * chunks; idx += 512) {
-        const int rr = idx / chunks, c = idx - rr * chunks;        // rr = query j
-        const bool ok = rr < N;
-        tca_cp_async16(sBias + (rr >> 7) * p.bias_tile_bytes + (rr & 127) * bstride + c * 16,
-                       bias_h + (long long)(ok ? rr : 0) * ld + c * 8, ok);
+        const int c = idx % chunks, q = idx / chunks;
+        const bool ok = has_bias && q < N && c * 8 < ld;
+        tca_cp_async16(sBias + (q >> 7) * p.bias_tile_bytes + c * 2048 + (q & 127) * 16,
+                       ok ? bias_h + (long long)q * ld + c * 8 : p.o, ok);
       }
       asm volatile("cp.async.wait_all;\n" ::: "memory");
+      named_bar_sync(3, 512);
+      const int tail = Nk - N;                                     // 0 .. 15 masked key columns
+      for (int idx = threadIdx.x - 96; idx < njb * 128 * tail; idx += 512) {
+        const int q = idx / tail, k = N + idx - q * tail;
+        *reinterpret_cast<unsigned short*>(sBias + (q >> 7) * p.bias_tile_bytes + (k >> 3) * 2048 + (q & 127) * 16 + (k & 7) * 2) =
+            0xC6EAu;                                               // bf16 -29952
+      }
+      fence_proxy_async_smem();
     }
     __syncthreads();
 
@@ -194,22 +219,31 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     } else if (warp == 1) {
       // -------------------------------------------------------------- MMA issuer (whole warp, one elected lane issues)
       const unsigned idesc_s = idesc_f16(128, Nk, 0, 0, FMT_BF16, FMT_BF16);
-      const unsigned idesc_o = idesc_f16(128, D, 0, 1, FMT_BF16, FMT_BF16);     // B = V is MN-major
-      const unsigned idesc_l = idesc_f16(128, 16, 0, 0, FMT_BF16, FMT_BF16);
-      const unsigned long long ones_desc = desc_kmajor_nosw(smem_u32(sOnes), 256, 128);
+      const unsigned idesc_b = idesc_f16(128, Nk, 0, 1, FMT_BF16, FMT_BF16);     // B = bias tile, MN-major
+      const unsigned idesc_o = idesc_f16(128, D, 0, 1, FMT_BF16, FMT_BF16);      // B = V, MN-major
+      // A of bias K step kk: the band from group 15 - 2 kk on (256 bytes per group; 128 bytes between the column halves)
+      const unsigned long long ident0 = desc_kmajor_nosw(smem_u32(sIdent) + 15 * 256, 128, 256);
       unsigned sq = it0 % (unsigned)p.nqk, kq = it0 / (unsigned)p.nqk;           // ring position of the next score item
       unsigned sv = it0 % (unsigned)p.nv, kv = it0 / (unsigned)p.nv;             // ... of the next P V item
       for (int n = 0; n <= cnt; ++n) {
         if (n < cnt) {
           const unsigned it = it0 + n, b = it & 1, u = it >> 1;
+          const unsigned ih = in_head0 + n;
+          const int jb = (int)(ih % (unsigned)njb);
+          const int nbk = (min(128, N - jb * 128) + 15) >> 4;                    // bias K steps: 16 queries each
           mbar_wait(&qkfull[sq], kq & 1, ab);
           mbar_wait(&sempty[b], (u & 1) ^ 1, ab);
           tc_fence_after();
           const unsigned q_addr = smem_u32(sQK + sq * qk_bytes);
           const unsigned long long qd = tca_desc(q_addr, SPAN), kd = tca_desc(q_addr + Q_BYTES, SPAN);
+          // bias tile as B: 8 keys further = 2048 bytes (stride field), 8 queries further = 128 bytes (leading field)
+          const unsigned long long bd = desc_kmajor_nosw(smem_u32(sBias + jb * p.bias_tile_bytes), 128, 2048);
           if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) umma_bf16(tmem_base + b * 256, qd + ks * 2, kd + ks * 2, idesc_s, ks);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+              if (kk < nbk) umma_bf16(tmem_base + b * 256, ident0 - kk * 32, bd + kk * 16, idesc_b, 1);
             tc_commit(&sfull[b]);
             tc_commit(&qkempty[sq]);
           }
@@ -222,19 +256,14 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
           mbar_wait(&pfull[b], u & 1, ab);
           tc_fence_after();
           const unsigned long long vd = tca_desc(smem_u32(sV + sv * kv_bytes), SPAN);
-          const unsigned a_p = tmem_base + b * 256, d_o = a_p + TCA_O_COL, d_l = a_p + TCA_L_COL;
+          const unsigned a_p = tmem_base + b * 256, d_o = a_p + TCA_O_COL;
 #pragma unroll
-          for (int kk = 0; kk < TCA_NMAX / 16; ++kk) {
-            if (kk < ng) {
-              const unsigned a_kk = a_p + kk * 16 + (kk & 1) * 8;
-              if (elect_one()) {
-                umma_ts(d_o, a_kk, vd + kk * SPAN, idesc_o, kk);     // 16 rows of V further: 16 SPAN bytes
-                umma_ts(d_l, a_kk, ones_desc, idesc_l, kk);
-              }
-            }
-          }
+          for (int kk = 0; kk < TCA_NMAX / 16; ++kk)
+            if (kk < ng && elect_one())
+              umma_ts(d_o, a_p + kk * 16 + (kk & 1) * 8, vd + kk * SPAN, idesc_o, kk);   // 16 rows of V further: 16 SPAN bytes
           if (elect_one()) {
             tc_commit(&ofull[b]);
+            tc_commit(&sempty[b]);
             tc_commit(&vempty[sv]);
           }
           __syncwarp();
@@ -252,124 +281,109 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
         const int i = (int)(ih / (unsigned)njb), jb = (int)(ih - (unsigned)i * njb);
         const int j = jb * 128 + row;
         const bool warp_live = jb * 128 + quarter * 32 < N;        // this warp owns at least one real query
-        const unsigned char* brow = sBias + jb * p.bias_tile_bytes + row * bstride;
-        float* xm = xmax + ((wg * 2 + (u & 1)) * 2) * 128;
+        float* xm = xch + (wg * 2 + (u & 1)) * 4 * 128;             // [max | sum][2 halves][128]
         unsigned ra[16], rb[16];
-        mbar_wait(&sfull[wg], u & 1, ab);
+        // one warp of the group watches the mbarrier, the others park in the named barrier
+        if ((sw & 7) == 0) mbar_wait(&sfull[wg], u & 1, ab);
+        named_bar_sync(1 + wg, 256);
         tc_fence_after();
-        // ---- pass 1: biased scores and row maximum over granules hf, hf + 2, ...; the TMEM and bias loads of the
-        // next granule are in flight while one is processed
+        // Each thread owns a contiguous half of the row: granules [gb, ge), read 32 columns at a time where a pair
+        // of granules starts on an even index, 16 otherwise.
+        const int gh = (ng + 1) >> 1, gb = hf ? gh : 0, ge = hf ? ng : gh;
+        // ---- pass 1: row maximum
         float mx = -INFINITY;
         if (warp_live) {
-          uint4 ba[2], bb[2];
-          auto fetch = [&](int g, unsigned (&rr)[16], uint4 (&bv)[2]) {
-            tmem_ld16(t_row + g * 16, rr);
-            if (has_bias) {
-              bv[0] = *reinterpret_cast<const uint4*>(brow + g * 32);
-              bv[1] = *reinterpret_cast<const uint4*>(brow + g * 32 + 16);
-            } else {
-              bv[0] = bv[1] = make_uint4(0, 0, 0, 0);
-            }
-          };
-          auto pass1 = [&](int g, unsigned (&rr)[16], const uint4 (&bv)[2]) {
-            const unsigned bw[8] = {bv[0].x, bv[0].y, bv[0].z, bv[0].w, bv[1].x, bv[1].y, bv[1].z, bv[1].w};
-            float sv[16];
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          int g = gb;
+          if ((g & 1) && g < ge) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld_wait16(ra);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              sv[2 * e] = __uint_as_float(rr[2 * e]) + __uint_as_float(bw[e] << 16);
-              sv[2 * e + 1] = __uint_as_float(rr[2 * e + 1]) + __uint_as_float(bw[e] & 0xffff0000u);
-            }
-            if (g * 16 + 16 > N) {
-#pragma unroll
-              for (int e = 0; e < 16; ++e)
-                if (g * 16 + e >= N) sv[e] = -INFINITY;
-            }
-            float m4[4] = {sv[0], sv[1], sv[2], sv[3]};
-#pragma unroll
-            for (int e = 4; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], sv[e]);
-            mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-#pragma unroll
-            for (int e = 0; e < 16; ++e) rr[e] = __float_as_uint(sv[e]);
-            tmem_st16(t_row + g * 16, rr);
-          };
-          if (hf < ng) fetch(hf, ra, ba);
-#pragma unroll
-          for (int gi = 0; gi < 8; gi += 2) {
-            const int g0 = hf + 2 * gi, g1 = g0 + 2, g2 = g0 + 4;
-            if (g0 < ng) {
-              tmem_ld_wait16(ra);
-              const uint4 cur[2] = {ba[0], ba[1]};
-              if (g1 < ng) fetch(g1, rb, bb);
-              pass1(g0, ra, cur);
-            }
-            if (g1 < ng) {
-              tmem_ld_wait16(rb);
-              const uint4 cur[2] = {bb[0], bb[1]};
-              if (g2 < ng) fetch(g2, ra, ba);
-              pass1(g1, rb, cur);
-            }
+            for (int e = 0; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(ra[e]));
+            ++g;
           }
-          tmem_st_wait();
+#pragma unroll 1
+          for (; g + 2 <= ge; g += 2) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld16(t_row + g * 16 + 16, rb);
+            tmem_ld_wait2(ra, rb);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], fmaxf(__uint_as_float(ra[e]), __uint_as_float(rb[e])));
+          }
+          if (g < ge) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld_wait16(ra);
+#pragma unroll
+            for (int e = 0; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(ra[e]));
+          }
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
         xm[hf * 128 + row] = mx;
         named_bar_sync(1 + wg, 256);
         mx = fmaxf(mx, xm[(hf ^ 1) * 128 + row]);
-        // ---- pass 2: weights as packed bf16 pairs, written over the first (even granules) or second (odd granules)
-        // half of the granule's own score columns, which only this thread reads
+        // ---- pass 2: weights, their sum, and P as packed bf16 pairs written over the first (even granules) or
+        // second (odd granules) half of the granule's own score columns, which only this thread reads
+        float lsum = 0.f;
         if (warp_live) {
           const float ms = -mx * sc2;
-          auto pass2 = [&](int g, const unsigned (&rr)[16]) {
+          float l4[4] = {0.f, 0.f, 0.f, 0.f};
+          auto pass2 = [&](int gg, const unsigned (&rr)[16]) {
+            float pv[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) pv[e] = tca_exp2(fmaf(__uint_as_float(rr[e]), sc2, ms));
             unsigned pk[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              pk[e] = tca_exp2_bf16x2(fmaf(__uint_as_float(rr[2 * e]), sc2, ms), fmaf(__uint_as_float(rr[2 * e + 1]), sc2, ms));
-            tmem_st8(t_row + g * 16 + (g & 1) * 8, pk);
+            for (int e = 0; e < 8; ++e) {
+              l4[e & 3] += pv[2 * e] + pv[2 * e + 1];
+              pk[e] = tca_pack(pv[2 * e], pv[2 * e + 1]);
+            }
+            tmem_st8(t_row + gg * 16 + (gg & 1) * 8, pk);
           };
-          if (hf < ng) tmem_ld16(t_row + hf * 16, ra);
-#pragma unroll
-          for (int gi = 0; gi < 8; gi += 2) {
-            const int g0 = hf + 2 * gi, g1 = g0 + 2, g2 = g0 + 4;
-            if (g0 < ng) {
-              tmem_ld_wait16(ra);
-              if (g1 < ng) tmem_ld16(t_row + g1 * 16, rb);
-              pass2(g0, ra);
-            }
-            if (g1 < ng) {
-              tmem_ld_wait16(rb);
-              if (g2 < ng) tmem_ld16(t_row + g2 * 16, ra);
-              pass2(g1, rb);
-            }
+          int g = gb;
+          if ((g & 1) && g < ge) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld_wait16(ra);
+            pass2(g, ra);
+            ++g;
           }
+#pragma unroll 1
+          for (; g + 2 <= ge; g += 2) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld16(t_row + g * 16 + 16, rb);
+            tmem_ld_wait2(ra, rb);
+            pass2(g, ra);
+            pass2(g + 1, rb);
+          }
+          if (g < ge) {
+            tmem_ld16(t_row + g * 16, ra);
+            tmem_ld_wait16(ra);
+            pass2(g, ra);
+          }
+          lsum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
           tmem_st_wait();
         }
+        xm[256 + hf * 128 + row] = lsum;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&pfull[wg]);
         // ---- output: O / l
-        mbar_wait(&ofull[wg], u & 1, ab);
+        if ((sw & 7) == 0) mbar_wait(&ofull[wg], u & 1, ab);
+        named_bar_sync(1 + wg, 256);                               // also: the partner's half of the row sum is visible
         tc_fence_after();
         if (warp_live && (D >= 32 || hf == 0)) {
           constexpr int CPT = D >= 32 ? D / 2 : D;                 // output channels per thread (16)
-          unsigned lv;
           tmem_ld16(t_row + TCA_O_COL + hf * CPT, ra);
-          tmem_ld1(t_row + TCA_L_COL, lv);
-          tmem_ld_wait16_1(ra, lv);
-          const float inv = 1.0f / __uint_as_float(lv);
+          const float inv = 1.0f / (xm[256 + row] + xm[256 + 128 + row]);
+          tmem_ld_wait16(ra);
           if (j < N) {
             __nv_bfloat16* op = p.o + (p.row0 + row_base + (long long)i * N + j) * Hd + h * D + hf * CPT;
             unsigned w[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(ra[2 * e]) * inv, __uint_as_float(ra[2 * e + 1]) * inv);
-              w[e] = *reinterpret_cast<unsigned*>(&t2);
-            }
+            for (int e = 0; e < 8; ++e) w[e] = tca_pack(__uint_as_float(ra[2 * e]) * inv, __uint_as_float(ra[2 * e + 1]) * inv);
             *reinterpret_cast<uint4*>(op) = make_uint4(w[0], w[1], w[2], w[3]);
             *reinterpret_cast<uint4*>(op + 8) = make_uint4(w[4], w[5], w[6], w[7]);
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sempty[wg]);
       }
     }
     it0 += (unsigned)cnt;
@@ -385,10 +399,10 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
 static size_t tca_smem_bytes(int D, int n_max, bool has_bias, int nqk, int nv, int* kv_rows, int* tile_bytes) {
   const int rows = (n_max + 31) & ~31;
   *kv_rows = rows;
-  *tile_bytes = has_bias ? 128 * tca_bias_stride(n_max) : 0;
+  *tile_bytes = has_bias ? ((n_max + 15) & ~15) / 8 * 2048 : 0;
   const int njb = (n_max + 127) / 128;
-  return (size_t)nqk * (128 * 2 * D + rows * 2 * D) + (size_t)nv * rows * 2 * D + 512 + 2 * 2 * 2 * 128 * 4 +
-         (size_t)njb * *tile_bytes + 64 + 1024;
+  return (size_t)nqk * (128 * 2 * D + rows * 2 * D) + (size_t)nv * rows * 2 * D + TCA_IDENT_BYTES + 256 +
+         2 * 2 * 2 * 2 * 128 * 4 + (size_t)njb * *tile_bytes + 1024;
 }
 
 template <int D>

@@ -47,25 +47,28 @@ __device__ inline void mbar_expect_tx(void* bar, unsigned bytes) {
 __device__ inline void mbar_arrive(void* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
 }
-// One probe of the barrier; the hardware may park the warp for up to `suspend_ns` before it answers, so a waiting
-// role does not spend issue slots on polling.
-__device__ inline bool mbar_try(void* bar, unsigned parity, unsigned suspend_ns) {
+__device__ inline bool mbar_try(void* bar, unsigned parity) {
   unsigned ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.b32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(suspend_ns) : "memory");
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// bounded wait (by elapsed SM clocks); returns false (after flagging) if the limit was reached
+// Bounded wait; returns false (after flagging) if the limit was reached.  Between probes the warp sleeps, with the
+// pause doubling up to a quarter of a microsecond, so that waiting roles leave the issue slots and the memory
+// pipeline's queue to the working warps; the abort flag and the clock are looked at every 64th probe only.
 __device__ inline bool mbar_wait(void* bar, unsigned parity, const AbortCtx& ab) {
-  if (mbar_try(bar, parity, 0)) return true;
+  if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   const long long limit = *ab.flag ? WAIT_CLOCKS_ABORTED : WAIT_CLOCKS;
+  unsigned ns = 32;
   for (unsigned it = 0; it < WAIT_PROBES; ++it) {
-    if (mbar_try(bar, parity, 20000)) return true;
-    if (clock64() - t0 > limit || *ab.flag) break;
+    if (mbar_try(bar, parity)) return true;
+    __nanosleep(ns);
+    if (ns < 256) ns <<= 1;
+    if ((it & 63u) == 63u && (clock64() - t0 > limit || *ab.flag)) break;
   }
   if (!*ab.flag) {
     *ab.flag = 1;
