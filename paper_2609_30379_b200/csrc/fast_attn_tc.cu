@@ -1,19 +1,22 @@
 // Row-wise pair-biased attention on tcgen05 for samples whose whole key range fits one accumulator
 // (N <= 224, pair order, head dim 16 or 32).
 //
-// Work item: one attention row (s, i), one head h, one block of 128 queries j.  The scores of the
-// item are one MMA group into a 224-column TMEM accumulator (M = 128 queries, N = round_up(N_s, 16)
-// keys): S' = Q K^T (K = d) plus the pair bias, which enters through the tensor cores as well: the
-// bias tile of the (s, h, j block), resident in shared memory and stored times sqrt(d), is the
-// MN-major B operand of a product whose A operand is the 128 x 128 identity (1.0 * bias is exact in
-// the float accumulator; the identity is a 16 x 16 block sliding over a band of zeros).  With the
-// whole row in TMEM the softmax needs no running rescale:
-//   pass 1  two threads per query read their halves of the row and take the maximum;
-//   pass 2  p = exp2((s - max) log2(e) / sqrt(d)), summed in float and written as packed bf16 pairs
-//           over half of each 16-key granule's own score columns, from where the second MMA group
-//           takes P as its TMEM-resident A operand: O = P V (N = d) into 32 columns of its own;
+// Work item: one attention row (s, i), one head h, one block of 128 queries j.  The raw scores of the
+// item, Q K^T (M = 128 queries, N = round_up(N_s, 16) keys, K = d), are one MMA group into a
+// 224-column TMEM accumulator, so the softmax needs no running rescale:
+//   pass 1  two threads per query read their halves of the row and take the maximum of the raw scores;
+//           with the largest bias of the row (found once per (s, h) when the bias tile is loaded) it
+//           bounds every biased score from above, which is all the reference value of a softmax needs
+//           (the normalisation cancels it exactly);
+//   pass 2  s = raw + bias (the bias tile of the (s, h, j block) is resident in shared memory, stored
+//           times sqrt(d); key columns past N hold a large negative value so their weights are exact
+//           zeros and no pass needs a mask), p = exp2((s - bound) log2(e) / sqrt(d)), summed in float
+//           and written as packed bf16 pairs over half of each 16-key granule's own score columns,
+//           from where the second MMA group takes P as its TMEM-resident A operand: O = P V (N = d)
+//           into 32 columns of its own;
 //   output  O / l, 16 channels per thread, stored row-major.
-// The exponentials are the floor of this kernel: an SM retires 16 per clock.
+// The exponentials are the floor of this kernel (an SM retires 16 per clock); the bias addition rides
+// in their shadow on the other pipes.
 // Roles: warp 0 streams Q | K and warp 2 streams V of each item with TMA (32-row boxes, swizzle span =
 // 2 d bytes) through two rings (a Q | K stage is free again as soon as the scores are computed), warp 1
 // issues the MMAs (converged, one elected lane; the scores of item n + 1 before P V of item n), warps
@@ -31,7 +34,6 @@ namespace ntp {
 constexpr int TCA_THREADS = 96 + 512;
 constexpr int TCA_NMAX = 224;      // keys per item: 224 score columns + 32 output columns = one 256-column TMEM buffer
 constexpr int TCA_O_COL = 224;     // output accumulator (up to 32 columns)
-constexpr int TCA_IDENT_BYTES = 31 * 256;   // identity band: 31 groups of 8 rows x 16 columns
 constexpr float TCA_LOG2E = 1.4426950408889634f;
 
 struct AttnTcParams {
@@ -47,6 +49,11 @@ struct AttnTcParams {
   int n_max;                      // samples with N > n_max are left to the other kernel
   int* status;
 };
+
+__host__ __device__ inline int tca_bias_stride(int nk) {   // bytes per resident bias row: an odd multiple of 16
+  const int b = nk * 2;
+  return (b / 16) % 2 == 0 ? b + 16 : b;
+}
 
 __device__ inline void tca_cp_async16(void* smem, const void* gmem, bool valid) {
   const unsigned sa = (unsigned)__cvta_generic_to_shared(smem);
@@ -90,9 +97,8 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
   const int qk_bytes = Q_BYTES + kv_bytes;
   unsigned char* sQK = smem;                                      // [nqk][Q | K]
   unsigned char* sV = sQK + p.nqk * qk_bytes;                     // [nv][V]
-  unsigned char* sIdent = sV + p.nv * kv_bytes;                   // identity band (see below)
-  float* xch = reinterpret_cast<float*>(sIdent + TCA_IDENT_BYTES + 256);   // [2 groups][2 parities][max | sum][2 halves][128]
-  unsigned char* sBias = reinterpret_cast<unsigned char*>(xch) + 2 * 2 * 2 * 2 * 128 * 4;   // [2 tiles][keys / 8][128 queries][8 keys]
+  float* xch = reinterpret_cast<float*>(sV + p.nv * kv_bytes);    // [2 groups][2 parities][max | sum][2 halves][128]
+  unsigned char* sBias = reinterpret_cast<unsigned char*>(xch) + 2 * 2 * 2 * 2 * 128 * 4;   // [2 tiles][128 queries][stride]
   unsigned long long* qkfull = bars;          // [3]
   unsigned long long* qkempty = bars + 3;     // [3] the score MMAs that read the stage are done
   unsigned long long* vfull = bars + 6;       // [3]
@@ -117,19 +123,6 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
-  // Identity band, K-major without swizzle: 31 groups of 8 rows; a group is two 128-byte core matrices (columns
-  // 0-7 and 8-15), a row is 16 bytes of one.  Groups 15 and 16 hold the 16 x 16 identity, the rest is zero.  The A
-  // operand of bias K step kk (queries 16 kk .. 16 kk + 15) starts at group 15 - 2 kk, so that its rows
-  // 16 kk .. 16 kk + 15 fall on the identity and all others on zeros.
-  for (int idx = threadIdx.x; idx < TCA_IDENT_BYTES / 4; idx += TCA_THREADS) {
-    const int byte = idx * 4, grp = byte >> 8, chunk = (byte >> 7) & 1, r = (byte >> 4) & 7, c2 = (byte >> 2) & 3;
-    unsigned w = 0;
-    if (grp == 15 + chunk) {                     // group 15: rows 0-7 meet columns 0-7; group 16: rows 8-15 meet columns 8-15
-      if (r == 2 * c2) w = 0x00003F80u;
-      else if (r == 2 * c2 + 1) w = 0x3F800000u;
-    }
-    reinterpret_cast<unsigned*>(sIdent)[idx] = w;
-  }
   fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
@@ -160,16 +153,17 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     const int nb = (N + 31) / 32;                                  // 32-row boxes of K (and V)
     const int ng = Nk / 16;                                        // 16-key granules
 
+    const int bstride = tca_bias_stride(Nk);
+    float bmax[2] = {0.f, 0.f};                                    // largest bias of this thread's query row, per j block
     if (warp >= 3) {
-      // bias tile of query block t: element (query q, key k) at t * tile + (k / 8) * 2048 + q * 16 + (k % 8) * 2,
-      // the MN-major layout without swizzle (8 keys x 8 queries per 128-byte core matrix).  Key columns N .. Nk - 1
+      // bias tile of query block t: row-major, query q at t * tile + (q % 128) * stride.  Key columns N .. Nk - 1
       // (rows of K that belong to other pair rows) get a large negative bias, so their weights come out as exact
       // zeros and neither softmax pass needs a mask.
       const int chunks = Nk / 8;
       for (int idx = threadIdx.x - 96; idx < njb * 128 * chunks; idx += 512) {
-        const int c = idx % chunks, q = idx / chunks;
+        const int q = idx / chunks, c = idx - q * chunks;
         const bool ok = has_bias && q < N && c * 8 < ld;
-        tca_cp_async16(sBias + (q >> 7) * p.bias_tile_bytes + c * 2048 + (q & 127) * 16,
+        tca_cp_async16(sBias + (q >> 7) * p.bias_tile_bytes + (q & 127) * bstride + c * 16,
                        ok ? bias_h + (long long)q * ld + c * 8 : p.o, ok);
       }
       asm volatile("cp.async.wait_all;\n" ::: "memory");
@@ -177,10 +171,21 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
       const int tail = Nk - N;                                     // 0 .. 15 masked key columns
       for (int idx = threadIdx.x - 96; idx < njb * 128 * tail; idx += 512) {
         const int q = idx / tail, k = N + idx - q * tail;
-        *reinterpret_cast<unsigned short*>(sBias + (q >> 7) * p.bias_tile_bytes + (k >> 3) * 2048 + (q & 127) * 16 + (k & 7) * 2) =
-            0xC6EAu;                                               // bf16 -29952
+        *reinterpret_cast<unsigned short*>(sBias + (q >> 7) * p.bias_tile_bytes + (q & 127) * bstride + k * 2) = 0xC6EAu;   // bf16 -29952
       }
-      fence_proxy_async_smem();
+      named_bar_sync(3, 512);
+      const int qrow = (warp & 3) * 32 + lane;
+      for (int t = 0; t < njb; ++t) {
+        const unsigned char* br = sBias + t * p.bias_tile_bytes + qrow * bstride;
+        float mb = -INFINITY;
+        for (int c = 0; c < chunks; ++c) {
+          const uint4 v = *reinterpret_cast<const uint4*>(br + c * 16);
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) mb = fmaxf(mb, fmaxf(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u)));
+        }
+        bmax[t] = mb;
+      }
     }
     __syncthreads();
 
@@ -219,31 +224,20 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
     } else if (warp == 1) {
       // -------------------------------------------------------------- MMA issuer (whole warp, one elected lane issues)
       const unsigned idesc_s = idesc_f16(128, Nk, 0, 0, FMT_BF16, FMT_BF16);
-      const unsigned idesc_b = idesc_f16(128, Nk, 0, 1, FMT_BF16, FMT_BF16);     // B = bias tile, MN-major
       const unsigned idesc_o = idesc_f16(128, D, 0, 1, FMT_BF16, FMT_BF16);      // B = V, MN-major
-      // A of bias K step kk: the band from group 15 - 2 kk on (256 bytes per group; 128 bytes between the column halves)
-      const unsigned long long ident0 = desc_kmajor_nosw(smem_u32(sIdent) + 15 * 256, 128, 256);
       unsigned sq = it0 % (unsigned)p.nqk, kq = it0 / (unsigned)p.nqk;           // ring position of the next score item
       unsigned sv = it0 % (unsigned)p.nv, kv = it0 / (unsigned)p.nv;             // ... of the next P V item
       for (int n = 0; n <= cnt; ++n) {
         if (n < cnt) {
           const unsigned it = it0 + n, b = it & 1, u = it >> 1;
-          const unsigned ih = in_head0 + n;
-          const int jb = (int)(ih % (unsigned)njb);
-          const int nbk = (min(128, N - jb * 128) + 15) >> 4;                    // bias K steps: 16 queries each
           mbar_wait(&qkfull[sq], kq & 1, ab);
           mbar_wait(&sempty[b], (u & 1) ^ 1, ab);
           tc_fence_after();
           const unsigned q_addr = smem_u32(sQK + sq * qk_bytes);
           const unsigned long long qd = tca_desc(q_addr, SPAN), kd = tca_desc(q_addr + Q_BYTES, SPAN);
-          // bias tile as B: 8 keys further = 2048 bytes (stride field), 8 queries further = 128 bytes (leading field)
-          const unsigned long long bd = desc_kmajor_nosw(smem_u32(sBias + jb * p.bias_tile_bytes), 128, 2048);
           if (elect_one()) {
 #pragma unroll
             for (int ks = 0; ks < D / 16; ++ks) umma_bf16(tmem_base + b * 256, qd + ks * 2, kd + ks * 2, idesc_s, ks);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              if (kk < nbk) umma_bf16(tmem_base + b * 256, ident0 - kk * 32, bd + kk * 16, idesc_b, 1);
             tc_commit(&sfull[b]);
             tc_commit(&qkempty[sq]);
           }
@@ -320,17 +314,23 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
         }
         xm[hf * 128 + row] = mx;
         named_bar_sync(1 + wg, 256);
-        mx = fmaxf(mx, xm[(hf ^ 1) * 128 + row]);
+        mx = fmaxf(mx, xm[(hf ^ 1) * 128 + row]) + (jb ? bmax[1] : bmax[0]);       // upper bound of the biased scores of the row
         // ---- pass 2: weights, their sum, and P as packed bf16 pairs written over the first (even granules) or
         // second (odd granules) half of the granule's own score columns, which only this thread reads
         float lsum = 0.f;
         if (warp_live) {
           const float ms = -mx * sc2;
           float l4[4] = {0.f, 0.f, 0.f, 0.f};
+          const unsigned char* brow = sBias + jb * p.bias_tile_bytes + row * bstride;
           auto pass2 = [&](int gg, const unsigned (&rr)[16]) {
+            const uint4 b0 = *reinterpret_cast<const uint4*>(brow + gg * 32), b1 = *reinterpret_cast<const uint4*>(brow + gg * 32 + 16);
+            const unsigned bw[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
             float pv[16];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) pv[e] = tca_exp2(fmaf(__uint_as_float(rr[e]), sc2, ms));
+            for (int e = 0; e < 8; ++e) {
+              pv[2 * e] = tca_exp2(fmaf(__uint_as_float(rr[2 * e]) + __uint_as_float(bw[e] << 16), sc2, ms));
+              pv[2 * e + 1] = tca_exp2(fmaf(__uint_as_float(rr[2 * e + 1]) + __uint_as_float(bw[e] & 0xffff0000u), sc2, ms));
+            }
             unsigned pk[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -399,10 +399,10 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
 static size_t tca_smem_bytes(int D, int n_max, bool has_bias, int nqk, int nv, int* kv_rows, int* tile_bytes) {
   const int rows = (n_max + 31) & ~31;
   *kv_rows = rows;
-  *tile_bytes = has_bias ? ((n_max + 15) & ~15) / 8 * 2048 : 0;
+  *tile_bytes = 128 * tca_bias_stride((n_max + 15) & ~15) + 64;
   const int njb = (n_max + 127) / 128;
-  return (size_t)nqk * (128 * 2 * D + rows * 2 * D) + (size_t)nv * rows * 2 * D + TCA_IDENT_BYTES + 256 +
-         2 * 2 * 2 * 2 * 128 * 4 + (size_t)njb * *tile_bytes + 1024;
+  return (size_t)nqk * (128 * 2 * D + rows * 2 * D) + (size_t)nv * rows * 2 * D + 2 * 2 * 2 * 2 * 128 * 4 +
+         (size_t)njb * *tile_bytes + 1024;
 }
 
 template <int D>

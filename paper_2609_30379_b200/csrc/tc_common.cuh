@@ -56,19 +56,16 @@ __device__ inline bool mbar_try(void* bar, unsigned parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait; returns false (after flagging) if the limit was reached.  Between probes the warp sleeps, with the
-// pause doubling up to a quarter of a microsecond, so that waiting roles leave the issue slots and the memory
-// pipeline's queue to the working warps; the abort flag and the clock are looked at every 64th probe only.
+// Bounded wait; returns false (after flagging) if the limit was reached.  A failing probe parks the warp in
+// hardware for a few microseconds at most and returns at once when the phase completes, so the loop needs no
+// sleep of its own; the abort flag and the clock are looked at every 16th probe.
 __device__ inline bool mbar_wait(void* bar, unsigned parity, const AbortCtx& ab) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   const long long limit = *ab.flag ? WAIT_CLOCKS_ABORTED : WAIT_CLOCKS;
-  unsigned ns = 32;
   for (unsigned it = 0; it < WAIT_PROBES; ++it) {
     if (mbar_try(bar, parity)) return true;
-    __nanosleep(ns);
-    if (ns < 256) ns <<= 1;
-    if ((it & 63u) == 63u && (clock64() - t0 > limit || *ab.flag)) break;
+    if ((it & 15u) == 15u && (clock64() - t0 > limit || *ab.flag)) break;
   }
   if (!*ab.flag) {
     *ab.flag = 1;
