@@ -106,33 +106,39 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
         tma_load_2d(sA + stage * a_stage + sl * a_slab, &p.zmap, &afull[stage], sl * 64, (int)(t * 128));
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp, one elected lane issues)
     mbar_wait(wfull, 0, ab);
     int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0};
-    long long unit = 0;
+    unsigned phase = 0, tph0 = 0, tph1 = 0;
+    unsigned unit = 0;
+    const unsigned long long w_desc = desc_kmajor_sw128(smem_u32(sW));
+    const unsigned w16 = (unsigned)w_slab >> 4, a16 = (unsigned)a_slab >> 4;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
-      const unsigned a_addr = smem_u32(sA + stage * a_stage);
+      const unsigned long long a_desc = desc_kmajor_sw128(smem_u32(sA + stage * a_stage));
       for (int u = 0; u < nunits; ++u, ++unit) {
-        const int buf = (int)(unit & 1);
-        mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
-        tph[buf] ^= 1;
+        const unsigned buf = unit & 1;
+        if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
+        else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
         tc_fence_after();
         const unsigned idesc = idesc_f16(128, u_n[u], 0, 0, FMT_F16, FMT_F16);   // z tile converted to fp16, folded weights fp16
         const unsigned d_tmem = tmem_base + buf * 256;
-        for (int sl = 0; sl < nslab; ++sl) {
-          const unsigned w_addr = smem_u32(sW + sl * w_slab + u_row[u] * 128);
+        const unsigned row16 = (unsigned)u_row[u] * 8;                           // 128-byte rows in units of 16 bytes
 #pragma unroll
-          for (int k4 = 0; k4 < 4; ++k4)
-            umma_bf16(d_tmem, desc_kmajor_sw128(a_addr + sl * a_slab + k4 * 32), desc_kmajor_sw128(w_addr + k4 * 32),
-                      idesc, (sl | k4) != 0);
-        }
-        tc_commit(&tfull[buf]);
+        for (int sl = 0; sl < 2; ++sl)
+          if (sl < nslab) {
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4)
+              if (elect_one())
+                umma_bf16(d_tmem, a_desc + (sl * a16 + k4 * 2), w_desc + (sl * w16 + row16 + k4 * 2), idesc, (sl | k4) != 0);
+          }
+        if (elect_one()) tc_commit(&tfull[buf]);
+        __syncwarp();
       }
-      tc_commit(&aempty[stage]);
+      if (elect_one()) tc_commit(&aempty[stage]);
+      __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {

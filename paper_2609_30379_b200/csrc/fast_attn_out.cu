@@ -97,34 +97,44 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
         tma_load_2d(st + (zslab + sl) * slab, &p.omap, &afull[stage], sl * 64, (int)(t * 128));
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp, one elected lane issues)
     mbar_wait(wfull, 0, ab);
     int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0}, gph[2] = {0, 0};
-    long long n = 0;
+    unsigned phase = 0, tph0 = 0, tph1 = 0, gph0 = 0, gph1 = 0;
+    unsigned n = 0;
     const unsigned idesc_g = idesc_f16(128, Hd, 0, 0, FMT_F16, FMT_F16);    // z tile converted to fp16, folded W_g fp16
     const unsigned idesc_o = idesc_f16(128, c, 0, 0, FMT_BF16, FMT_BF16);   // gated o bf16, W_o as given (bf16)
+    const unsigned long long wg_desc = desc_kmajor_sw128(smem_u32(sWg)), wo_desc = desc_kmajor_sw128(smem_u32(sWo));
+    const unsigned slab16 = (unsigned)slab >> 4, wg16 = (unsigned)wg_slab >> 4, wo16 = (unsigned)wo_slab >> 4;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
-      const int buf = (int)(n & 1);
-      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
-      tph[buf] ^= 1;
+      const unsigned buf = n & 1;
+      if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
+      else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
-      const unsigned st = smem_u32(sSt + stage * stage_bytes);
+      const unsigned long long st_desc = desc_kmajor_sw128(smem_u32(sSt + stage * stage_bytes));
       const unsigned dg = tmem_base + buf * 256, dout = dg + Hd;
-      for (int ks = 0; ks < c / 16; ++ks)
-        umma_bf16(dg, desc_kmajor_sw128(st + (ks >> 2) * slab + (ks & 3) * 32),
-                  desc_kmajor_sw128(smem_u32(sWg) + (ks >> 2) * wg_slab + (ks & 3) * 32), idesc_g, ks != 0);
-      tc_commit(&gfull[buf]);
-      mbar_wait(&ogated[buf], gph[buf], ab);     // gated o tile written back by the epilogue warps
-      gph[buf] ^= 1;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        if (ks < c / 16 && elect_one())
+          umma_bf16(dg, st_desc + ((ks >> 2) * slab16 + (ks & 3) * 2), wg_desc + ((ks >> 2) * wg16 + (ks & 3) * 2), idesc_g, ks != 0);
+      if (elect_one()) tc_commit(&gfull[buf]);
+      __syncwarp();
+      // gated o tile written back by the epilogue warps
+      if (buf == 0) { mbar_wait(&ogated[0], gph0, ab); gph0 ^= 1; }
+      else { mbar_wait(&ogated[1], gph1, ab); gph1 ^= 1; }
       tc_fence_after();
-      for (int ks = 0; ks < Hd / 16; ++ks)
-        umma_bf16(dout, desc_kmajor_sw128(st + (zslab + (ks >> 2)) * slab + (ks & 3) * 32),
-                  desc_kmajor_sw128(smem_u32(sWo) + (ks >> 2) * wo_slab + (ks & 3) * 32), idesc_o, ks != 0);
-      tc_commit(&ofull[buf]);
-      tc_commit(&aempty[stage]);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        if (ks < Hd / 16 && elect_one())
+          umma_bf16(dout, st_desc + ((zslab + (ks >> 2)) * slab16 + (ks & 3) * 2), wo_desc + ((ks >> 2) * wo16 + (ks & 3) * 2),
+                    idesc_o, ks != 0);
+      if (elect_one()) {
+        tc_commit(&ofull[buf]);
+        tc_commit(&aempty[stage]);
+      }
+      __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {

@@ -95,19 +95,19 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
         if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
       }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp, one elected lane issues)
     int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0};
-    long long n = 0;
+    unsigned phase = 0, tph0 = 0, tph1 = 0;
+    unsigned n = 0;
     for (long long job = blockIdx.x; job < njobs; job += gridDim.x, ++n) {
       int s, c, i0, j0, Nt;
       contract_decode(p, job, s, c, i0, j0, Nt);
       const int N = p.N[s];
       const int nkc = (N + 63) / 64;
-      const int buf = (int)(n & 1);
-      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
-      tph[buf] ^= 1;
+      const unsigned buf = n & 1;
+      if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
+      else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
       tc_fence_after();
       const unsigned idesc = idesc_f16(128, Nt, 0, 0, FMT_F16, FMT_F16);   // a, b are fp16
       const unsigned d_tmem = tmem_base + buf * 256;
@@ -115,15 +115,17 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
         mbar_wait(&full[stage], phase, ab);
         tc_fence_after();
         const unsigned a_addr = smem_u32(smem + stage * CT_STAGE_BYTES);
-        const unsigned b_addr = a_addr + CT_A_BYTES;
+        const unsigned long long a_desc = desc_kmajor_sw128(a_addr), b_desc = desc_kmajor_sw128(a_addr + CT_A_BYTES);
         const int ksteps = min(4, (N - kc * 64 + 15) / 16);
-        for (int k4 = 0; k4 < ksteps; ++k4)
-          umma_bf16(d_tmem, desc_kmajor_sw128(a_addr + k4 * 32), desc_kmajor_sw128(b_addr + k4 * 32), idesc,
-                    (kc | k4) != 0);
-        tc_commit(&empty[stage]);
+#pragma unroll
+        for (int k4 = 0; k4 < 4; ++k4)
+          if (k4 < ksteps && elect_one()) umma_bf16(d_tmem, a_desc + k4 * 2, b_desc + k4 * 2, idesc, (kc | k4) != 0);
+        if (elect_one()) tc_commit(&empty[stage]);
+        __syncwarp();
         if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
       }
-      tc_commit(&tfull[buf]);
+      if (elect_one()) tc_commit(&tfull[buf]);
+      __syncwarp();
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ epilogue

@@ -154,41 +154,49 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
                       sl * 64, jc, i, 0);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp runs the loop and
+    // one elected lane issues, with descriptors derived from per-CTA bases by adding constants
     mbar_wait(wfull, 0, ab);
     int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0};
-    long long unit = 0;
+    unsigned phase = 0, tph0 = 0, tph1 = 0;
+    unsigned unit = 0;
     const unsigned idesc = idesc_f16(128, 128, 0, 0, FMT_F16, FMT_F16);   // M = 128 channels, N = 128 positions
+    const unsigned long long w_desc = desc_kmajor_sw128(smem_u32(sW));
+    const unsigned long long wx_desc = desc_kmajor_nosw(smem_u32(sWx), wx_region, 128);
+    const unsigned w_slab16 = (unsigned)w_slab_bytes >> 4, z_slab16 = (unsigned)z_slab_bytes >> 4;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
-      const unsigned z_addr = smem_u32(sZ + stage * z_stage_bytes);
-      const unsigned zx_desc_addr = smem_u32(sZx + stage * 2 * zx_region);
+      const unsigned long long z_desc = desc_kmajor_sw128(smem_u32(sZ + stage * z_stage_bytes));
+      const unsigned long long zx_desc = desc_kmajor_nosw(smem_u32(sZx + stage * 2 * zx_region), zx_region, 128);
       for (int u = 0; u < nunits; ++u, ++unit) {
-        const int buf = (int)(unit & 1);
-        mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
-        tph[buf] ^= 1;
+        const unsigned buf = unit & 1;
+        if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
+        else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
         tc_fence_after();
 #pragma unroll
         for (int part = 0; part < 2; ++part) {                 // 0 = gate rows, 1 = value rows
-          const int row0 = u * 256 + part * 128;
+          const unsigned row16 = (unsigned)(u * 256 + part * 128) * 8;        // row offset in units of 16 bytes (128-byte rows)
           const unsigned d_tmem = tmem_base + buf * 256 + part * 128;
-          for (int sl = 0; sl < nslab; ++sl) {
-            const unsigned w_addr = smem_u32(sW + sl * w_slab_bytes + row0 * 128);
 #pragma unroll
-            for (int k4 = 0; k4 < 4; ++k4)
-              umma_bf16(d_tmem, desc_kmajor_sw128(w_addr + k4 * 32), desc_kmajor_sw128(z_addr + sl * z_slab_bytes + k4 * 32),
-                        idesc, (sl | k4) != 0);
+          for (int sl = 0; sl < 2; ++sl) {
+            if (sl < nslab) {
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4)
+                if (elect_one())
+                  umma_bf16(d_tmem, w_desc + (sl * w_slab16 + row16 + k4 * 2), z_desc + (sl * z_slab16 + k4 * 2), idesc,
+                            (sl | k4) != 0);
+            }
           }
-          // augmentation K step: c1 / c0 columns against the (-mean rstd, 1) columns
-          umma_bf16(d_tmem, desc_kmajor_nosw(smem_u32(sWx + row0 * 16), wx_region, 128),
-                    desc_kmajor_nosw(zx_desc_addr, zx_region, 128), idesc, 1);
+          // augmentation K step: c1 / c0 columns against the (-mean rstd, 1) columns (16-byte rows)
+          if (elect_one()) umma_bf16(d_tmem, wx_desc + (unsigned)(u * 256 + part * 128), zx_desc, idesc, 1);
         }
-        tc_commit(&tfull[buf]);
+        if (elect_one()) tc_commit(&tfull[buf]);
+        __syncwarp();
       }
-      tc_commit(&aempty[stage]);
+      if (elect_one()) tc_commit(&aempty[stage]);
+      __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < TI_EPI_WARP0) {

@@ -126,34 +126,39 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (whole warp, one elected lane issues)
     mbar_wait(wfull, 0, ab);
     int stage = 0;
-    unsigned phase = 0, tph[2] = {0, 0};
-    long long n = 0;
+    unsigned phase = 0, tph0 = 0, tph1 = 0;
+    unsigned n = 0;
     const unsigned idesc_t = idesc_f16(128, c_z, 1, 0, FMT_F16, FMT_F16);   // A = t (fp16, MN-major), W_o' fp16
     const unsigned idesc_z = idesc_f16(128, c_z, 0, 0, FMT_F16, FMT_F16);   // A = z tile converted to fp16, W_g' fp16
+    const unsigned long long wo_desc = desc_kmajor_sw128(smem_u32(sWo)), wg_desc = desc_kmajor_sw128(smem_u32(sWg));
+    const unsigned wo16 = (unsigned)wo_slab >> 4, wg16 = (unsigned)wg_slab >> 4, z16 = (unsigned)z_slab >> 4;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
-      const int buf = (int)(n & 1);
-      mbar_wait(&tempty[buf], tph[buf] ^ 1, ab);
-      tph[buf] ^= 1;
+      const unsigned buf = n & 1;
+      if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
+      else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned st = smem_u32(sSt + stage * stage_bytes);
       const unsigned d1 = tmem_base + buf * 256, d2 = d1 + c_z;
-      for (int ks = 0; ks < c_h / 16; ++ks) {                // K = channels of t, 16 per step
-        const unsigned long long ad = desc_mnmajor_sw128(st + ks * 2048, t_chunk, 1024);
-        const unsigned long long bd = desc_kmajor_sw128(smem_u32(sWo) + (ks >> 2) * wo_slab + (ks & 3) * 32);
-        umma_bf16(d1, ad, bd, idesc_t, ks != 0);
+      const unsigned long long t_desc = desc_mnmajor_sw128(st, t_chunk, 1024);
+      const unsigned long long z_desc = desc_kmajor_sw128(st + 2 * t_chunk);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)                       // K = channels of t, 16 per step (2048 bytes of the MN-major tile)
+        if (ks < c_h / 16 && elect_one())
+          umma_bf16(d1, t_desc + ks * 128, wo_desc + ((ks >> 2) * wo16 + (ks & 3) * 2), idesc_t, ks != 0);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        if (ks < c_z / 16 && elect_one())
+          umma_bf16(d2, z_desc + ((ks >> 2) * z16 + (ks & 3) * 2), wg_desc + ((ks >> 2) * wg16 + (ks & 3) * 2), idesc_z, ks != 0);
+      if (elect_one()) {
+        tc_commit(&tfull[buf]);
+        tc_commit(&aempty[stage]);
       }
-      for (int ks = 0; ks < c_z / 16; ++ks) {
-        const unsigned long long ad = desc_kmajor_sw128(st + 2 * t_chunk + (ks >> 2) * z_slab + (ks & 3) * 32);
-        const unsigned long long bd = desc_kmajor_sw128(smem_u32(sWg) + (ks >> 2) * wg_slab + (ks & 3) * 32);
-        umma_bf16(d2, ad, bd, idesc_z, ks != 0);
-      }
-      tc_commit(&tfull[buf]);
-      tc_commit(&aempty[stage]);
+      __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {
