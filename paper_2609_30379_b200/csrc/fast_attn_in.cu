@@ -15,7 +15,9 @@
 
 namespace ntp {
 
-constexpr int AI_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps, 8 epilogue warps
+constexpr int AI_CONV_WARPS = 8;
+constexpr int AI_EPI_WARP0 = 2 + AI_CONV_WARPS;
+constexpr int AI_THREADS = 64 + 32 * AI_CONV_WARPS + 256;   // producer, MMA, 8 converter warps, 8 epilogue warps
 constexpr int AI_MAXB = 16;
 
 struct AttnInParams {
@@ -29,7 +31,8 @@ struct AttnInParams {
   int B, c, H, Hd;
   long long rows;                // positions in the group
   float eps;
-  const float2* c01;             // [3 Hd + 16]
+  CUtensorMap xmap;              // augmentation columns {8, 2 * aug_rows}, box {8, 16}, no swizzle
+  int aug_rows;
   __nv_bfloat16* bias;           // nullable
   int* status;
 };
@@ -37,7 +40,6 @@ struct AttnInParams {
 __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_constant__ AttnInParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[11];
-  __shared__ float2 sStats[2][128];        // per stage: (mean, rstd) of every tile row
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -48,10 +50,13 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
   const int a_slab = 128 * 128;
   const int a_stage = nslab * a_slab;
   const int npanel = Hd / 64 > 0 ? Hd / 64 : 1;
+  const int wx_region = wrows * 16;                      // one 8-column region of the weight augmentation
+  const int zx_region = 128 * 16;                        // one 8-column region of the activation augmentation
   unsigned char* sW = smem;
   unsigned char* sA = sW + nslab * w_slab;               // 2 stages
   unsigned char* sOut = sA + 2 * a_stage;                // npanel panels of [128][64]
-  float2* sC = reinterpret_cast<float2*>(sOut + npanel * a_slab);
+  unsigned char* sWx = sOut + npanel * a_slab;           // [2 regions][wrows][8] fp16, no swizzle
+  unsigned char* sAx = sWx + 2 * wx_region;              // 2 stages x [2 regions][128][8] fp16
   unsigned long long* afull = bars;
   unsigned long long* aempty = bars + 2;
   unsigned long long* tfull = bars + 4;
@@ -64,16 +69,21 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
     abort_flag = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(&afull[s], 1);
-      mbar_init(&aempty[s], 1 + 8);
+      mbar_init(&aempty[s], 1);
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
-      mbar_init(&aconv[s], 4);
+      mbar_init(&aconv[s], AI_CONV_WARPS);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
-  for (int n = threadIdx.x; n < wrows; n += AI_THREADS) sC[n] = p.c01[n];
+  // the second 8-column region of the activation augmentation is always zero
+  for (int idx = threadIdx.x; idx < 2 * zx_region / 16; idx += AI_THREADS) {
+    const int st = idx / (zx_region / 16), r = idx % (zx_region / 16);
+    *reinterpret_cast<uint4*>(sAx + st * 2 * zx_region + zx_region + r * 16) = make_uint4(0, 0, 0, 0);
+  }
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -87,7 +97,10 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ producer
-    mbar_expect_tx(wfull, nslab * w_slab);
+    mbar_expect_tx(wfull, nslab * w_slab + 2 * wx_region);
+    for (int reg = 0; reg < 2; ++reg)
+      for (int r16 = 0; r16 < wrows; r16 += 16)
+        tma_load_2d(sWx + reg * wx_region + r16 * 16, &p.xmap, wfull, 0, reg * p.aug_rows + r16);
     for (int sl = 0; sl < nslab; ++sl) {
       for (int rb = 0; rb < 3 * Hd / 128; ++rb)
         tma_load_2d(sW + sl * w_slab + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
@@ -114,10 +127,12 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
     unsigned unit = 0;
     const unsigned long long w_desc = desc_kmajor_sw128(smem_u32(sW));
     const unsigned w16 = (unsigned)w_slab >> 4, a16 = (unsigned)a_slab >> 4;
+    const unsigned long long wx_desc = desc_kmajor_nosw(smem_u32(sWx), wx_region, 128);
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned long long a_desc = desc_kmajor_sw128(smem_u32(sA + stage * a_stage));
+      const unsigned long long ax_desc = desc_kmajor_nosw(smem_u32(sAx + stage * 2 * zx_region), zx_region, 128);
       for (int u = 0; u < nunits; ++u, ++unit) {
         const unsigned buf = unit & 1;
         if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
@@ -134,6 +149,8 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
               if (elect_one())
                 umma_bf16(d_tmem, a_desc + (sl * a16 + k4 * 2), w_desc + (sl * w16 + row16 + k4 * 2), idesc, (sl | k4) != 0);
           }
+        // augmentation K step: (-mean rstd, 1) columns against the c1 / c0 columns (16-byte rows)
+        if (elect_one()) umma_bf16(d_tmem, ax_desc, wx_desc + (unsigned)u_row[u], idesc, 1);
         if (elect_one()) tc_commit(&tfull[buf]);
         __syncwarp();
       }
@@ -141,39 +158,33 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
       __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
-    const int row = (warp - 2) * 32 + lane;
+  } else if (warp >= 2 && warp < AI_EPI_WARP0) {
+    // ------------------------------------------------------------------ converters (8 warps, two threads per row):
+    // the tile becomes fp16 scaled by the row's rstd, with the augmentation columns that complete the LayerNorm
+    const int row = (warp - 2) * 16 + (lane >> 1), hf = lane & 1;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
-      float sum, sq;
-      convert_row_bf16_to_f16(sA + stage * a_stage, nslab, a_slab, row, sum, sq);
-      const float mean = sum / (float)c;
-      sStats[stage][row] = make_float2(mean, rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps));
+      convert_row_ln_fp16(sA + stage * a_stage, nslab, a_slab, sAx + stage * 2 * zx_region + row * 16, row, hf, c, p.eps);
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&aconv[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-  } else if (warp >= 6) {
-    // ------------------------------------------------------------------ epilogue (8 warps)
+  } else if (warp >= AI_EPI_WARP0) {
+    // ------------------------------------------------------------------ epilogue (8 warps): the accumulators already hold
+    // the normalised projections
     const int quarter = warp & 3;
-    const int half = (warp - 6) >> 2;
+    const int half = (warp - AI_EPI_WARP0) >> 2;
     const int row = quarter * 32 + lane;
-    const int ep_tid = threadIdx.x - 192;
+    const int ep_tid = threadIdx.x - 32 * AI_EPI_WARP0;
     const int cpw = Hd / 2;                         // channels of one output handled by this warp
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long unit = 0;
     bool store_pending = false;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&aconv[stage], phase, ab);          // statistics of this tile are published
-      const float2 stt = sStats[stage][row];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&aempty[stage]);
-      const float mean = stt.x, rstd = stt.y;
       for (int u = 0; u < nunits; ++u, ++unit) {
         const int buf = (int)(unit & 1);
         mbar_wait(&tfull[buf], tph[buf], ab);
@@ -188,7 +199,6 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
               if (ep_tid == 0) tma_store_wait_read0();
               named_bar_sync(1, 256);
             }
-            const float2* cc = sC + o * Hd;
             for (int c0 = half * cpw; c0 < (half + 1) * cpw; c0 += 32) {
               unsigned r[32];
               tmem_ld32(taddr + oi * Hd + c0, r);
@@ -200,10 +210,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                   const int n0 = ch * 8 + e * 2;
-                  const float2 k0 = cc[c0 + n0], k1 = cc[c0 + n0 + 1];
-                  const float x0 = fmaf(rstd, __uint_as_float(r[n0]) - mean * k0.y, k0.x);
-                  const float x1 = fmaf(rstd, __uint_as_float(r[n0 + 1]) - mean * k1.y, k1.x);
-                  __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+                  __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(r[n0]), __uint_as_float(r[n0 + 1]));
                   w[e] = *reinterpret_cast<unsigned*>(&hh);
                 }
                 *reinterpret_cast<uint4*>(panel + sw128_off(row, ((c0 & 63) >> 3) + ch)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -231,11 +238,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
             const unsigned rr = (unsigned)(P - p.pair_off[s]);      // N^2 < 2^32 (N < 2^16 for this path)
             const unsigned i = rr / (unsigned)N, j = rr - i * (unsigned)N;
             __nv_bfloat16* bp = p.bias + (long long)p.H * p.cm_off[s] + (long long)i * ld + j;
-            const float2* cc = sC + 3 * Hd;
-            for (int h = 0; h < p.H; ++h) {
-              const float x = fmaf(rstd, __uint_as_float(r[h]) - mean * cc[h].y, cc[h].x);
-              bp[(long long)h * N * ld] = __float2bfloat16_rn(x);
-            }
+            for (int h = 0; h < p.H; ++h) bp[(long long)h * N * ld] = __float2bfloat16_rn(__uint_as_float(r[h]));
           }
         }
         tc_fence_before();
@@ -262,11 +265,10 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
   const int Hd = H * d;
   const int wrows = 3 * Hd + 16;
   const void* wprime = ap.w;
-  const float2* c01 = (const float2*)ap.c01;
   const int nslab = c / 64;
   const int npanel = Hd / 64;
   const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)nslab * 128 * 128 + (size_t)npanel * 128 * 128 +
-                      (size_t)wrows * 8 + 1024;
+                      2 * (size_t)wrows * 16 + 2 * 2 * (size_t)128 * 16 + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -281,7 +283,7 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
     p.H = H;
     p.Hd = Hd;
     p.eps = eps;
-    p.c01 = c01;
+    p.aug_rows = ap.aug_rows;
     p.bias = (__nv_bfloat16*)bias;
     p.status = status;
     const long long P0 = m.pair_off[g0];
@@ -303,6 +305,10 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
         return cuda_fail("attn_in z map");
       const unsigned long long wdims[2] = {(unsigned long long)c, (unsigned long long)wrows};
       if (!make_tmap_bf16(&p.wmap, wprime, 2, wdims, strides, box)) return cuda_fail("attn_in w map");
+      const unsigned long long xdims[2] = {8, (unsigned long long)2 * ap.aug_rows};
+      const unsigned long long xstr[1] = {16};
+      const unsigned xbox[2] = {8, 16};
+      if (!make_tmap_16bit(&p.xmap, ap.aug, 2, xdims, xstr, xbox, 0)) return cuda_fail("attn_in augmentation map");
       const unsigned bbox[2] = {64, 16};
       if (!make_tmap_bf16(&p.wbmap, wprime, 2, wdims, strides, bbox)) return cuda_fail("attn_in wb map");
       const unsigned long long odims[2] = {(unsigned long long)Hd, (unsigned long long)p.rows};

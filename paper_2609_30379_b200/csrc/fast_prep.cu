@@ -134,11 +134,14 @@ nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* pr
   p += align_up((size_t)rows * c * 2, 256);
   out.c01 = p;
   out.c01g = p + (size_t)(3 * Hd + 16) * sizeof(float2);
+  p += align_up((size_t)rows * sizeof(float2), 256);
+  out.aug = p;                          // [2][rows][8] fp16
+  out.aug_rows = rows;
   PrepArgs a{};
   const void* s0[6] = {W->W_q, W->W_k, W->W_v, W->W_b, nullptr, W->W_g};
   const int r0[6] = {Hd, Hd, Hd, W->W_b ? H : 0, W->W_b ? 16 - H : 16, W->W_g ? Hd : 0};
   const float sc[6] = {1.f, 1.f, 1.f, sqrtf((float)d), 1.f, 1.f};   // bias rows times sqrt(d)
-  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01, sc);
+  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01, sc, out.aug);
   return run_prep(a, st);
 }
 

@@ -171,13 +171,15 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       mbar_wait(&afull[stage], phase, ab);
       unsigned char* st = sSt + stage * stage_bytes;
       // statistics of t over channels: a column of the MN-major fp16 tile
-      float ts = 0.f, tq = 0.f;
+      float ts4[4] = {0.f, 0.f, 0.f, 0.f}, tq4[4] = {0.f, 0.f, 0.f, 0.f};   // independent chains, loads hoisted by the unroll
       const unsigned char* tcol = st + q * t_chunk + (pos & 7) * 2;
+#pragma unroll 16
       for (int c = 0; c < c_h; ++c) {
         const float v = __half2float(*reinterpret_cast<const __half*>(tcol + c * 128 + (((pos >> 3) ^ (c & 7)) << 4)));
-        ts += v;
-        tq = fmaf(v, v, tq);
+        ts4[c & 3] += v;
+        tq4[c & 3] = fmaf(v, v, tq4[c & 3]);
       }
+      const float ts = (ts4[0] + ts4[1]) + (ts4[2] + ts4[3]), tq = (tq4[0] + tq4[1]) + (tq4[2] + tq4[3]);
       // t arrives scaled by 1 / N_s (see the contraction); LayerNorm is scale-free once eps is scaled alike
       float eps_t = p.eps;
       {

@@ -278,25 +278,86 @@ __device__ inline unsigned sw128_off(int row, int chunk) { return row * 128 + ((
 // tile made of `nslab` 64-column slabs and returns the row's sum and sum of squares.
 __device__ inline void convert_row_bf16_to_f16(unsigned char* tile, int nslab, int slab_bytes, int row, float& sum,
                                                float& sq) {
-  sum = 0.f;
-  sq = 0.f;
+  float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};   // four independent chains instead of one
   for (int sl = 0; sl < nslab; ++sl) {
+    uint4 v[8];
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) v[ch] = *reinterpret_cast<const uint4*>(tile + sl * slab_bytes + sw128_off(row, ch));
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
-      uint4* ptr = reinterpret_cast<uint4*>(tile + sl * slab_bytes + sw128_off(row, ch));
-      const uint4 v = *ptr;
-      unsigned w[4] = {v.x, v.y, v.z, v.w};
+      unsigned w[4] = {v[ch].x, v[ch].y, v[ch].z, v[ch].w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-        sum += lo + hi;
-        sq = fmaf(lo, lo, sq);
-        sq = fmaf(hi, hi, sq);
+        s4[e] += lo + hi;
+        q4[e] = fmaf(lo, lo, q4[e]);
+        q4[e] = fmaf(hi, hi, q4[e]);
         __half2 h = __floats2half2_rn(lo, hi);
         w[e] = *reinterpret_cast<unsigned*>(&h);
       }
-      *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(tile + sl * slab_bytes + sw128_off(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
+  }
+  sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+  sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+}
+
+// LayerNorm folded into the MMA, activation side.  Two threads per tile row (hf = 0 / 1), each owning four of the
+// eight 16-byte chunks of every 64-channel slab of a K-major 128-byte-swizzled bf16 tile: the row is rewritten in
+// place as fp16 scaled by its rstd, and hf = 0 writes the row's augmentation columns (m_hi, m_lo, m_hi, 1, 1, 0, 0, 0),
+// m = -mean * rstd, to `aug_row` (16 bytes of a K-major no-swizzle region).  Against weight columns
+// (c1_hi, c1_hi, c1_lo, c0_hi, c0_lo) one more K step then adds m * c1 + c0, so the accumulator holds LN(z) W^T.
+// The two threads of a row must be neighbouring lanes of a converged warp.
+__device__ inline void convert_row_ln_fp16(unsigned char* tile, int nslab, int slab_bytes, unsigned char* aug_row, int row,
+                                           int hf, int c, float eps) {
+  uint4 raw[2][4];
+#pragma unroll
+  for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      raw[sl][j] = sl < nslab ? *reinterpret_cast<const uint4*>(tile + sl * slab_bytes + sw128_off(row, hf * 4 + j))
+                              : make_uint4(0, 0, 0, 0);
+  float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};   // four independent chains
+#pragma unroll
+  for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const unsigned w[4] = {raw[sl][j].x, raw[sl][j].y, raw[sl][j].z, raw[sl][j].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+        s4[e] += lo + hi;
+        q4[e] = fmaf(lo, lo, q4[e]);
+        q4[e] = fmaf(hi, hi, q4[e]);
+      }
+    }
+  float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]), sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+  const float mean = sum / (float)c;
+  const float rstd = rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + eps);
+#pragma unroll
+  for (int sl = 0; sl < 2; ++sl)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (sl < nslab) {
+        unsigned w[4] = {raw[sl][j].x, raw[sl][j].y, raw[sl][j].z, raw[sl][j].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h = __floats2half2_rn(__uint_as_float(w[e] << 16) * rstd, __uint_as_float(w[e] & 0xffff0000u) * rstd);
+          w[e] = *reinterpret_cast<unsigned*>(&h);
+        }
+        *reinterpret_cast<uint4*>(tile + sl * slab_bytes + sw128_off(row, hf * 4 + j)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  if (hf == 0) {
+    const float mm = -mean * rstd;
+    const __half mh = __float2half_rn(mm), ml = __float2half_rn(mm - __half2float(mh));
+    const __half one = __float2half_rn(1.0f), zero = __float2half_rn(0.0f);
+    __half2 p0 = __halves2half2(mh, ml), p1 = __halves2half2(mh, one), p2 = __halves2half2(one, zero),
+            p3 = __halves2half2(zero, zero);
+    *reinterpret_cast<uint4*>(aug_row) = make_uint4(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1),
+                                                    *reinterpret_cast<unsigned*>(&p2), *reinterpret_cast<unsigned*>(&p3));
   }
 }
 
