@@ -4,8 +4,12 @@
 // positions of one pair row is, per channel, 128 contiguous bytes: exactly the MN-major operand
 // form of the MMA (positions are M, channels are K).  The output gate is recomputed here from z
 // instead of being stored by the input projection, which saves one write and one read of a
-// [T2, c_z] buffer.  Both LayerNorms are folded into the weights (see fast_tri_in.cu); the row
-// statistics come from the shared-memory tiles.
+// [T2, c_z] buffer.  Both LayerNorms are folded into the weights (see fast_tri_in.cu) and their mean
+// terms into the MMA: one more K step multiplies (-mean_hi, -mean_lo, -mean_hi) per position with
+// (c1_hi, c1_hi, c1_lo) per output channel, so the epilogue is left with
+//   o / 2 = (rstd_t / 2) acc_o + c0_o / 2,  g / 2 = (rstd_z / 2) acc_g + c0_g / 2,
+//   z += (tanh(g / 2) + 1) (o / 2).
+// The row statistics come from the shared-memory tiles; z stays an exact fp16 copy of the bf16 state.
 //
 // A tile is two 64-position chunks (s, i, j0).  Per tile the producer brings the t chunk
 // [c_h][64] and the z chunk [64][c_z]; the MMA warp issues t^T W_o'^T and z W_g'^T into one TMEM
@@ -26,6 +30,8 @@ struct TriOutParams {
   CUtensorMap tmap[TO_MAXB];     // {N (j), N (i), c_h, 1}, box {64, 1, c_h, 1}
   CUtensorMap womap;             // {c_h, c_z}, box {64, c_z}
   CUtensorMap wgmap;             // {c_z, c_z}, box {64, c_z}
+  CUtensorMap wgxmap, woxmap;    // augmentation columns of W_g / W_o: {8, rows}, box {8, 64}, no swizzle
+  int wgx_row0, wgx_rows, wox_rows;   // first row of W_g in its table; rows per region of each table
   long long chunk_off[TO_MAXB + 1];
   int N[TO_MAXB];
   int B, c_z, c_h;
@@ -47,16 +53,16 @@ __device__ inline bool to_decode(const TriOutParams& p, long long q, int& s, int
   return true;
 }
 
-__device__ inline float sigmoid_fast2(float x) {
+__device__ inline float to_tanh(float x) {
   float t;
-  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(0.5f * x));
-  return fmaf(0.5f, t, 0.5f);
+  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(x));
+  return t;
 }
 
 __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_constant__ TriOutParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[11];
-  __shared__ float4 sStats[2][128];      // per stage and tile row: (t mean, t rstd, z mean, z rstd)
+  __shared__ float2 sStats[2][128];        // per stage and position: (rstd_t / 2, rstd_z / 2)
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -70,8 +76,13 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   unsigned char* sWo = smem;
   unsigned char* sWg = sWo + wo_bytes;
   unsigned char* sSt = sWg + wg_bytes;                       // 2 stages: t chunks then z slabs
-  float2* sCo = reinterpret_cast<float2*>(sSt + 2 * stage_bytes);
-  float2* sCg = sCo + c_z;
+  float* sCo = reinterpret_cast<float*>(sSt + 2 * stage_bytes);   // c0 of W_o / 2 per channel
+  float* sCg = sCo + c_z;                                         // c0 of W_g / 2
+  const int wx_region = c_z * 16;                                 // one 8-column region of a weight augmentation
+  unsigned char* sWox = reinterpret_cast<unsigned char*>(sCg + c_z);   // [2 regions][c_z][8] fp16, K-major no swizzle
+  unsigned char* sWgx = sWox + 2 * wx_region;
+  unsigned char* sZx = sWgx + 2 * wx_region;                      // 2 stages x [2 regions][128 positions][8] fp16 (K-major)
+  unsigned char* sTx = sZx + 2 * 2 * 2048;                        // 2 stages x [2 k groups][16 position groups][8 k][8 positions] (MN-major)
   unsigned long long* afull = bars;
   unsigned long long* aempty = bars + 2;
   unsigned long long* tfull = bars + 4;
@@ -94,9 +105,13 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
   for (int n = threadIdx.x; n < c_z; n += TO_THREADS) {
-    sCo[n] = p.c01o[n];
-    sCg[n] = p.c01g[n];
+    sCo[n] = 0.5f * p.c01o[n].x;
+    sCg[n] = 0.5f * p.c01g[n].x;
   }
+  // activation augmentation tiles start as zeros; the converters fill the three mean columns of every position
+  for (int idx = threadIdx.x; idx < 2 * (2 * 2048 + 4096) / 16; idx += TO_THREADS)
+    *reinterpret_cast<uint4*>(sZx + idx * 16) = make_uint4(0, 0, 0, 0);
+  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -107,7 +122,12 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
 
   if (warp == 0 && lane == 0) {
     // ------------------------------------------------------------------ producer
-    mbar_expect_tx(wfull, wo_bytes + wg_bytes);
+    mbar_expect_tx(wfull, wo_bytes + wg_bytes + 4 * wx_region);
+    for (int reg = 0; reg < 2; ++reg)
+      for (int r = 0; r < c_z; r += 64) {
+        tma_load_2d(sWox + reg * wx_region + r * 16, &p.woxmap, wfull, 0, reg * p.wox_rows + r);
+        tma_load_2d(sWgx + reg * wx_region + r * 16, &p.wgxmap, wfull, 0, reg * p.wgx_rows + p.wgx_row0 + r);
+      }
     for (int sl = 0; sl < hslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
     for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
     int stage = 0;
@@ -136,6 +156,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     const unsigned idesc_z = idesc_f16(128, c_z, 0, 0, FMT_F16, FMT_F16);   // A = z tile converted to fp16, W_g' fp16
     const unsigned long long wo_desc = desc_kmajor_sw128(smem_u32(sWo)), wg_desc = desc_kmajor_sw128(smem_u32(sWg));
     const unsigned wo16 = (unsigned)wo_slab >> 4, wg16 = (unsigned)wg_slab >> 4, z16 = (unsigned)z_slab >> 4;
+    const unsigned long long wox_desc = desc_kmajor_nosw(smem_u32(sWox), wx_region, 128);
+    const unsigned long long wgx_desc = desc_kmajor_nosw(smem_u32(sWgx), wx_region, 128);
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const unsigned buf = n & 1;
       if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
@@ -154,7 +176,11 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       for (int ks = 0; ks < 8; ++ks)
         if (ks < c_z / 16 && elect_one())
           umma_bf16(d2, z_desc + ((ks >> 2) * z16 + (ks & 3) * 2), wg_desc + ((ks >> 2) * wg16 + (ks & 3) * 2), idesc_z, ks != 0);
+      // augmentation K steps: the mean terms of both LayerNorms.  t side: MN-major without swizzle (8 positions
+      // further = 128 bytes, 8 k further = 2048); z side: K-major without swizzle (8 k further = 2048, 8 rows = 128).
       if (elect_one()) {
+        umma_bf16(d1, desc_kmajor_nosw(smem_u32(sTx + stage * 4096), 2048, 128), wox_desc, idesc_t, 1);
+        umma_bf16(d2, desc_kmajor_nosw(smem_u32(sZx + stage * 4096), 2048, 128), wgx_desc, idesc_z, 1);
         tc_commit(&tfull[buf]);
         tc_commit(&aempty[stage]);
       }
@@ -193,7 +219,18 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       convert_row_bf16_to_f16(st + 2 * t_chunk, zslab, z_slab, row, zs, zq);
       const float zmean = zs / (float)c_z;
       const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
-      sStats[stage][row] = make_float4(tmean, trstd, zmean, zrstd);
+      sStats[stage][row] = make_float2(0.5f * trstd, 0.5f * zrstd);
+      {
+        const __half th = __float2half_rn(-tmean), tl = __float2half_rn(-tmean - __half2float(th));
+        const __half zh = __float2half_rn(-zmean), zl = __float2half_rn(-zmean - __half2float(zh));
+        // t side: element (position, k) at (position / 8) * 128 + k * 16 + (position % 8) * 2
+        __half* tx = reinterpret_cast<__half*>(sTx + stage * 4096 + (row >> 3) * 128 + (row & 7) * 2);
+        tx[0] = th; tx[8] = tl; tx[16] = th;
+        // z side: row's 16 bytes (k = 0 .. 7)
+        __half2 p0 = __halves2half2(zh, zl), p1 = __halves2half2(zh, __float2half_rn(0.f));
+        *reinterpret_cast<uint2*>(sZx + stage * 4096 + row * 16) =
+            make_uint2(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1));
+      }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&aconv[stage]);
@@ -215,8 +252,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       mbar_wait(&tfull[buf], tph[buf], ab);         // MMAs done, hence the statistics are published too
       tph[buf] ^= 1;
       tc_fence_after();
-      const float4 stt = sStats[stage][row];
-      const float tmean = stt.x, trstd = stt.y, zmean = stt.z, zrstd = stt.w;
+      const float2 stt = sStats[stage][row];
+      const float trh = stt.x, zrh = stt.y;
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       for (int c0 = half * (c_z / 2); c0 < (half + 1) * (c_z / 2); c0 += 32) {
         unsigned r1[32], r2[32];
@@ -231,19 +268,18 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
           uint4 v = *ptr;
           unsigned w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
+          const float4 co0 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8), co1 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8 + 4);
+          const float4 cg0 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8), cg1 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8 + 4);
+          const float ko[8] = {co0.x, co0.y, co0.z, co0.w, co1.x, co1.y, co1.z, co1.w};
+          const float kg[8] = {cg0.x, cg0.y, cg0.z, cg0.w, cg1.x, cg1.y, cg1.z, cg1.w};
+#pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            float out[2];
-#pragma unroll
-            for (int h2 = 0; h2 < 2; ++h2) {
-              const float2 ko = sCo[c0 + n0 + h2], kg = sCg[c0 + n0 + h2];
-              const float o = fmaf(trstd, __uint_as_float(r1[n0 + h2]) - tmean * ko.y, ko.x);
-              const float g = sigmoid_fast2(fmaf(zrstd, __uint_as_float(r2[n0 + h2]) - zmean * kg.y, kg.x));
-              const float2 zo = unpack_h2(w[e]);       // the z tile holds fp16 after conversion
-              const float zold = h2 == 0 ? zo.x : zo.y;
-              out[h2] = fmaf(g, o, zold);
-            }
-            __nv_bfloat162 hh = __floats2bfloat162_rn(out[0], out[1]);
+            const float2 zo = unpack_h2(w[e]);         // the z tile holds fp16 after conversion
+            const float oh0 = fmaf(trh, __uint_as_float(r1[n0]), ko[e * 2]), oh1 = fmaf(trh, __uint_as_float(r1[n0 + 1]), ko[e * 2 + 1]);
+            const float t0 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0]), kg[e * 2]));
+            const float t1 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0 + 1]), kg[e * 2 + 1]));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(fmaf(oh0, t0, oh0) + zo.x, fmaf(oh1, t1, oh1) + zo.y);
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);
@@ -286,7 +322,8 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
   const float2* c01g = (const float2*)tp.c01g;
   const int zslab = c_z / 64, hslab = c_h / 64;
   const size_t smem = (size_t)hslab * c_z * 128 + (size_t)zslab * c_z * 128 +
-                      2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 2 * c_z * 8 + 1024;
+                      2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 2 * c_z * 4 + 4 * (size_t)c_z * 16 +
+                      2 * (2 * 2048 + 4096) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(tri_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -311,6 +348,14 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
       const unsigned long long dims2[2] = {(unsigned long long)c_z, (unsigned long long)c_z};
       const unsigned long long strides2[1] = {(unsigned long long)c_z * 2};
       if (!make_tmap_bf16(&p.wgmap, wg, 2, dims2, strides2, box)) return cuda_fail("tri_out W_g map");
+      const unsigned long long xstr[1] = {16};
+      const unsigned xbox[2] = {8, 64};
+      const unsigned long long gdims[2] = {8, (unsigned long long)2 * tp.aug1_rows}, odims[2] = {8, (unsigned long long)2 * c_z};
+      if (!make_tmap_16bit(&p.wgxmap, tp.aug1, 2, gdims, xstr, xbox, 0)) return cuda_fail("tri_out W_g augmentation map");
+      if (!make_tmap_16bit(&p.woxmap, tp.augo, 2, odims, xstr, xbox, 0)) return cuda_fail("tri_out W_o augmentation map");
+      p.wgx_row0 = 4 * c_h;
+      p.wgx_rows = tp.aug1_rows;
+      p.wox_rows = c_z;
     }
     p.chunk_off[0] = 0;
     for (int l = 0; l < TO_MAXB; ++l) {
