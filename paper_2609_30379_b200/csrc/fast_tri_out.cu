@@ -26,7 +26,7 @@ constexpr int TO_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps
 constexpr int TO_MAXB = 12;
 
 struct TriOutParams {
-  CUtensorMap zmap[TO_MAXB];     // {c_z, N (j), N (i), 1}, box {64, 64, 1, 1}
+  CUtensorMap zmap[TO_MAXB];     // {c_z, N (j), N (i), 1}, box {64, 32, 1, 1}
   CUtensorMap tmap[TO_MAXB];     // {N (j), N (i), c_h, 1}, box {64, 1, c_h, 1}
   CUtensorMap womap;             // {c_h, c_z}, box {64, c_z}
   CUtensorMap wgmap;             // {c_z, c_z}, box {64, c_z}
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     abort_flag = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(&afull[s], 1);
-      mbar_init(&aempty[s], 2);            // MMA commit + the storing epilogue thread
+      mbar_init(&aempty[s], 1 + 4 * (p.c_z / 64));   // MMA commit + the storing epilogue lanes
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
       mbar_init(&aconv[s], 4);
@@ -120,29 +120,36 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   const long long nchunks = p.chunk_off[p.B];
   const long long ntiles = (nchunks + 1) / 2;
 
-  if (warp == 0 && lane == 0) {
-    // ------------------------------------------------------------------ producer
-    mbar_expect_tx(wfull, wo_bytes + wg_bytes + 4 * wx_region);
-    for (int reg = 0; reg < 2; ++reg)
-      for (int r = 0; r < c_z; r += 64) {
-        tma_load_2d(sWox + reg * wx_region + r * 16, &p.woxmap, wfull, 0, reg * p.wox_rows + r);
-        tma_load_2d(sWgx + reg * wx_region + r * 16, &p.wgxmap, wfull, 0, reg * p.wgx_rows + p.wgx_row0 + r);
-      }
-    for (int sl = 0; sl < hslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
-    for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (lane q decodes and loads chunk q)
+    if (lane == 0) {
+      mbar_expect_tx(wfull, wo_bytes + wg_bytes + 4 * wx_region);
+      for (int reg = 0; reg < 2; ++reg)
+        for (int r = 0; r < c_z; r += 64) {
+          tma_load_2d(sWox + reg * wx_region + r * 16, &p.woxmap, wfull, 0, reg * p.wox_rows + r);
+          tma_load_2d(sWgx + reg * wx_region + r * 16, &p.wgxmap, wfull, 0, reg * p.wgx_rows + p.wgx_row0 + r);
+        }
+      for (int sl = 0; sl < hslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
+      for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
+    }
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&aempty[stage], phase ^ 1, ab);
-      const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
-      mbar_expect_tx(&afull[stage], nvalid * (t_chunk + zslab * 64 * 128));
-      unsigned char* st = sSt + stage * stage_bytes;
-      for (int q = 0; q < nvalid; ++q) {
-        int s, i, j0;
-        to_decode(p, 2 * t + q, s, i, j0);
-        tma_load_4d(st + q * t_chunk, &p.tmap[s], &afull[stage], j0, i, 0, 0);
+      int s = 0, i = 0, j0 = 0;
+      const bool valid = lane < 2 && to_decode(p, 2 * t + lane, s, i, j0);
+      if (lane == 0) {
+        const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
+        mbar_wait(&aempty[stage], phase ^ 1, ab);
+        mbar_expect_tx(&afull[stage], nvalid * (t_chunk + zslab * 64 * 128));
+      }
+      __syncwarp();
+      if (valid) {
+        unsigned char* st = sSt + stage * stage_bytes;
+        tma_load_4d(st + lane * t_chunk, &p.tmap[s], &afull[stage], j0, i, 0, 0);
         for (int sl = 0; sl < zslab; ++sl)
-          tma_load_4d(st + 2 * t_chunk + sl * z_slab + q * 64 * 128, &p.zmap[s], &afull[stage], sl * 64, j0, i, 0);
+          for (int sub = 0; sub < 2; ++sub)      // 32-position boxes (the size the epilogue warps store)
+            tma_load_4d(st + 2 * t_chunk + sl * z_slab + (lane * 64 + sub * 32) * 128, &p.zmap[s], &afull[stage], sl * 64,
+                        j0 + sub * 32, i, 0);
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
@@ -190,22 +197,56 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   } else if (warp >= 2 && warp < 6) {
     // ------------------------------------------------------------------ converters (4 warps, one position per thread)
     const int row = (warp - 2) * 32 + lane;
-    const int q = row >> 6, pos = row & 63;
+    const int q = row >> 6;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
       unsigned char* st = sSt + stage * stage_bytes;
-      // statistics of t over channels: a column of the MN-major fp16 tile
-      float ts4[4] = {0.f, 0.f, 0.f, 0.f}, tq4[4] = {0.f, 0.f, 0.f, 0.f};   // independent chains, loads hoisted by the unroll
-      const unsigned char* tcol = st + q * t_chunk + (pos & 7) * 2;
-#pragma unroll 16
-      for (int c = 0; c < c_h; ++c) {
-        const float v = __half2float(*reinterpret_cast<const __half*>(tcol + c * 128 + (((pos >> 3) ^ (c & 7)) << 4)));
-        ts4[c & 3] += v;
-        tq4[c & 3] = fmaf(v, v, tq4[c & 3]);
+      // Statistics of t over channels (columns of the MN-major fp16 tile).  Eight lanes share a group of eight
+      // positions: lane cg sums channels cg, cg + 8, ... with 16-byte loads (8 positions each), then a
+      // reduce-scatter over the eight lanes leaves every lane with the two sums of one position -- its own row.
+      float ts, tq;
+      {
+        const int cg = lane & 7, pgl = ((warp - 2) * 4 + (lane >> 3)) & 7;      // position group inside the 64-position chunk
+        float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, q8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        const unsigned char* tb = st + q * t_chunk + cg * 128 + ((pgl ^ cg) << 4);   // channel c = cc * 8 + cg: c & 7 = cg
+#pragma unroll 4
+        for (int cc = 0; cc < c_h / 8; ++cc) {
+          const uint4 v = *reinterpret_cast<const uint4*>(tb + cc * 1024);
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = unpack_h2(w[e]);
+            a8[2 * e] += f.x; a8[2 * e + 1] += f.y;
+            q8[2 * e] = fmaf(f.x, f.x, q8[2 * e]); q8[2 * e + 1] = fmaf(f.y, f.y, q8[2 * e + 1]);
+          }
+        }
+        // reduce-scatter: after the step with lane bit b, a lane keeps the half of the positions whose bit b equals its own
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool up = cg & 4;
+          const float sa = up ? a8[e] : a8[e + 4], sq_ = up ? q8[e] : q8[e + 4];
+          const float ka = up ? a8[e + 4] : a8[e], kq = up ? q8[e + 4] : q8[e];
+          a8[e] = ka + __shfl_xor_sync(0xffffffffu, sa, 4);
+          q8[e] = kq + __shfl_xor_sync(0xffffffffu, sq_, 4);
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const bool up = cg & 2;
+          const float sa = up ? a8[e] : a8[e + 2], sq_ = up ? q8[e] : q8[e + 2];
+          const float ka = up ? a8[e + 2] : a8[e], kq = up ? q8[e + 2] : q8[e];
+          a8[e] = ka + __shfl_xor_sync(0xffffffffu, sa, 2);
+          q8[e] = kq + __shfl_xor_sync(0xffffffffu, sq_, 2);
+        }
+        {
+          const bool up = cg & 1;
+          const float sa = up ? a8[0] : a8[1], sq_ = up ? q8[0] : q8[1];
+          const float ka = up ? a8[1] : a8[0], kq = up ? q8[1] : q8[0];
+          ts = ka + __shfl_xor_sync(0xffffffffu, sa, 1);
+          tq = kq + __shfl_xor_sync(0xffffffffu, sq_, 1);
+        }
       }
-      const float ts = (ts4[0] + ts4[1]) + (ts4[2] + ts4[3]), tq = (tq4[0] + tq4[1]) + (tq4[2] + tq4[3]);
       // t arrives scaled by 1 / N_s (see the contraction); LayerNorm is scale-free once eps is scaled alike
       float eps_t = p.eps;
       {
@@ -241,7 +282,6 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     const int quarter = warp & 3;
     const int half = (warp - 6) >> 2;
     const int row = quarter * 32 + lane;           // position inside the tile
-    const int ep_tid = threadIdx.x - 192;
     int stage = 0;
     unsigned phase = 0, tph[2] = {0, 0};
     long long n = 0;
@@ -267,7 +307,6 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
           uint4* ptr = reinterpret_cast<uint4*>(zp + sw128_off(row, chunk16));
           uint4 v = *ptr;
           unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
           const float4 co0 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8), co1 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8 + 4);
           const float4 cg0 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8), cg1 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8 + 4);
           const float ko[8] = {co0.x, co0.y, co0.z, co0.w, co1.x, co1.y, co1.z, co1.w};
@@ -288,23 +327,24 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[buf]);
+      // every warp stores its own 32 positions x 64 channels as soon as it has written them (c_z = 64: the two
+      // warps of a lane quarter share the slab and meet at a barrier of their own)
       fence_proxy_async_smem();
-      named_bar_sync(1, 256);
-      if (ep_tid == 0) {
-        const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
-        for (int qq = 0; qq < nvalid; ++qq) {
-          int s, i, j0;
-          to_decode(p, 2 * t + qq, s, i, j0);
-          for (int sl = 0; sl < zslab; ++sl)
-            tma_store_4d(&p.zmap[s], zrow + sl * z_slab + qq * 64 * 128, sl * 64, j0, i, 0);
-        }
+      if (zslab == 1) named_bar_sync(2 + quarter, 64);
+      else __syncwarp();
+      if (lane == 0 && (zslab == 2 || half == 0)) {
+        const int qq = quarter >> 1, sub = quarter & 1;
+        int s, i, j0;
+        if (to_decode(p, 2 * t + qq, s, i, j0) && j0 + sub * 32 < p.N[s])
+          tma_store_4d(&p.zmap[s], zrow + (zslab == 2 ? half : 0) * z_slab + (qq * 64 + sub * 32) * 128, (zslab == 2 ? half : 0) * 64,
+                       j0 + sub * 32, i, 0);
         tma_store_commit();
         tma_store_wait_read0();
         mbar_arrive(&aempty[stage]);
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-    if (ep_tid == 0) tma_store_wait_all0();
+    if (lane == 0) tma_store_wait_all0();
   }
   tc_fence_before();
   __syncthreads();
@@ -368,7 +408,7 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
           const unsigned long long dims[4] = {(unsigned long long)c_z, (unsigned long long)N, (unsigned long long)N, 1};
           const unsigned long long strides[3] = {(unsigned long long)c_z * 2, (unsigned long long)N * c_z * 2,
                                                  (unsigned long long)N * N * c_z * 2};
-          const unsigned box[4] = {64, 64, 1, 1};
+          const unsigned box[4] = {64, 32, 1, 1};
           const char* base = (const char*)z + (size_t)m.pair_off[g0 + l] * c_z * 2;
           if (!make_tmap_bf16(&p.zmap[l], base, 4, dims, strides, box)) return cuda_fail("tri_out z map");
         }
