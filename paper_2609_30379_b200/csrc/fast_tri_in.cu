@@ -29,10 +29,11 @@ constexpr int TI_CH = 32;                       // positions per chunk
 constexpr int TI_CONV_WARPS = 8;
 constexpr int TI_EPI_WARP0 = 2 + TI_CONV_WARPS; // first epilogue warp (a multiple of 4 plus 2: see the lane quarters below)
 constexpr int TI_THREADS = 64 + 32 * TI_CONV_WARPS + 256;   // producer warp, MMA warp, converter warps, 8 epilogue warps
-constexpr int TI_MAXB = 16;
+constexpr int TI_MAXB = 12;
 
 struct TriInParams {
   CUtensorMap zmap[TI_MAXB];               // {c_z, N (k), N (i), 1}, box {64, 32, 1, 1}
+  CUtensorMap omap[TI_MAXB];               // outputs {ld (k), N (i), c_h, 2 (a | b)}, box {16, 1, 32, 1}, no swizzle
   CUtensorMap wmap;                        // {c_z, 4 c_h}, box {64, 128}
   CUtensorMap xmap;                        // augmentation columns {8, 2 * aug_rows}, box {8, 256}, no swizzle
   long long chunk_off[TI_MAXB + 1];
@@ -40,8 +41,6 @@ struct TriInParams {
   int N[TI_MAXB];
   int B, c_z, c_h, aug_rows;
   float eps;
-  __half* a;
-  __half* b;
   int* status;
 };
 
@@ -84,6 +83,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   unsigned char* sWx = sW + w_bytes;               // [2 regions][wrows][8] fp16, no swizzle
   unsigned char* sZ = sWx + 2 * wx_region;         // 2 stages of the z tile
   unsigned char* sZx = sZ + 2 * z_stage_bytes;     // 2 stages x [2 regions][128][8] fp16
+  unsigned char* sOut = sZx + 2 * 2 * zx_region;   // per epilogue warp: [32 channels][16 positions] fp16 staged for a TMA store
   unsigned long long* afull = bars;        // [2] TMA landed
   unsigned long long* aempty = bars + 2;   // [2] MMAs that read the stage are done
   unsigned long long* tfull = bars + 4;    // [2] accumulator buffer ready
@@ -269,7 +269,6 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     // ------------------------------------------------------------------ epilogue (8 warps)
     const int quarter = warp & 3;                  // TMEM lane quarter = 32 output channels
     const int half = (warp - TI_EPI_WARP0) >> 2;   // which two of the tile's four chunks this warp stores
-    const int lane_ch = quarter * 32 + lane;       // accumulator row
     const __half2 hmax2 = __float2half2_rn(65504.f), hmin2 = __float2half2_rn(-65504.f);
     unsigned tph[2] = {0, 0};
     long long unit = 0;
@@ -281,10 +280,13 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         tph[buf] ^= 1;
         tc_fence_after();
         // c_h = 128: unit 0 -> a, unit 1 -> b, channel = accumulator row; c_h = 64: rows 0-63 -> a, 64-127 -> b
-        const int ch = c_h == 128 ? lane_ch : (lane_ch & 63);
-        __half* obase = (c_h == 128 ? (u == 0) : (lane_ch < 64)) ? p.a : p.b;
+        const int which = c_h == 128 ? u : (quarter >> 1);
+        const int ch0 = c_h == 128 ? quarter * 32 : (quarter & 1) * 32;          // first channel of this warp
+        unsigned char* stg = sOut + (warp - TI_EPI_WARP0) * 1024;
         const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256 + half * 64;
-        // four steps of 16 positions; the TMEM loads of step k + 1 are in flight while step k is computed
+        // four steps of 16 positions; the TMEM loads of step k + 1 are in flight while step k is computed.  A step's
+        // 32 channels x 16 positions go through a 1 KB staging tile and out with one TMA store (runs of 32 bytes per
+        // channel row, clipped at the row end), which keeps the scattered writes off the load / store units.
         unsigned rg[2][16], rv[2][16];
         tmem_ld16(taddr, rg[0]);
         tmem_ld16(taddr + 128, rv[0]);
@@ -296,27 +298,28 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
             tmem_ld16(taddr + 128 + (k + 1) * 16, rv[(k + 1) & 1]);
           }
           const int4 info = tinfo[tn & 7][half * 2 + (k >> 1)];
-          if (info.w) {
-            const int s = info.x, i = info.y, jc = info.z + (k & 1) * 16;
-            const int N = p.N[s], ld = round_up8(N);
-            __half* outp = obase + (long long)c_h * p.cm_off[s] + (long long)ch * N * ld + (long long)i * ld + jc;
+          unsigned w[8];
 #pragma unroll
-            for (int vec = 0; vec < 2; ++vec) {
-              unsigned w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int n0 = vec * 8 + e * 2;
-                // the gate and value weight rows were folded times 1/2, so with g' = g / 2, v' = v / 2:
-                // sigmoid(g) * v = (tanh(g') + 1) * v' = fma(v', tanh(g'), v')
-                const float h0 = __uint_as_float(rv[k & 1][n0]), h1 = __uint_as_float(rv[k & 1][n0 + 1]);
-                const float v0 = fmaf(h0, tanh_fast(__uint_as_float(rg[k & 1][n0])), h0);
-                const float v1 = fmaf(h1, tanh_fast(__uint_as_float(rg[k & 1][n0 + 1])), h1);
-                __half2 h = __floats2half2_rn(v0, v1);          // overflow gives inf, clamped below
-                h = __hmax2(__hmin2(h, hmax2), hmin2);
-                w[e] = *reinterpret_cast<unsigned*>(&h);
-              }
-              if (jc + vec * 8 < ld) *reinterpret_cast<uint4*>(outp + vec * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
+          for (int e = 0; e < 8; ++e) {
+            // the gate and value weight rows were folded times 1/2, so with g' = g / 2, v' = v / 2:
+            // sigmoid(g) * v = (tanh(g') + 1) * v' = fma(v', tanh(g'), v')
+            const float h0 = __uint_as_float(rv[k & 1][2 * e]), h1 = __uint_as_float(rv[k & 1][2 * e + 1]);
+            const float v0 = fmaf(h0, tanh_fast(__uint_as_float(rg[k & 1][2 * e])), h0);
+            const float v1 = fmaf(h1, tanh_fast(__uint_as_float(rg[k & 1][2 * e + 1])), h1);
+            __half2 h = __floats2half2_rn(v0, v1);          // overflow gives inf, clamped below
+            h = __hmax2(__hmin2(h, hmax2), hmin2);
+            w[e] = *reinterpret_cast<unsigned*>(&h);
+          }
+          if (lane == 0) tma_store_wait_read0();            // the previous step's store has read the staging tile
+          __syncwarp();
+          *reinterpret_cast<uint4*>(stg + lane * 32) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(stg + lane * 32 + 16) = make_uint4(w[4], w[5], w[6], w[7]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0 && info.w) {
+            const int jc = info.z + (k & 1) * 16;
+            if (jc < round_up8(p.N[info.x])) tma_store_4d(&p.omap[info.x], stg, jc, info.y, ch0, which);
+            tma_store_commit();
           }
         }
         tc_fence_before();
@@ -324,6 +327,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         if (lane == 0) mbar_arrive(&tempty[buf]);
       }
     }
+    if (lane == 0) tma_store_wait_all0();
   }
   tc_fence_before();
   __syncthreads();
@@ -338,10 +342,11 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
   const int nslab = c_z / 64;
   const int wrows = 4 * c_h;
   const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)wrows * 16 + 2 * (size_t)nslab * 128 * 128 +
-                      2 * 2 * (size_t)128 * 16 + 1024;
+                      2 * 2 * (size_t)128 * 16 + 8 * 1024 + 1024;
+  if (((const char*)b - (const char*)a) % 16 != 0 || b <= a) return NT_ERR_UNSUPPORTED;   // a | b form one 4-D tensor
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(tri_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(tri_in_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 231424) != cudaSuccess)
       return cuda_fail("tri_in smem attribute");
     attr_set = true;
   }
@@ -353,8 +358,6 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
     p.c_h = c_h;
     p.aug_rows = tp.aug1_rows;
     p.eps = eps;
-    p.a = (__half*)a;
-    p.b = (__half*)b;
     p.status = status;
     {
       const unsigned long long dims[2] = {(unsigned long long)c_z, (unsigned long long)wrows};
@@ -379,6 +382,13 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
         const unsigned box[4] = {64, TI_CH, 1, 1};
         const char* base = (const char*)z + (size_t)m.pair_off[g0 + l] * c_z * 2;
         if (!make_tmap_bf16(&p.zmap[l], base, 4, dims, strides, box)) return cuda_fail("tri_in z map");
+        const int ld = round_up8(N);
+        const unsigned long long odims[4] = {(unsigned long long)ld, (unsigned long long)N, (unsigned long long)c_h, 2};
+        const unsigned long long ostr[3] = {(unsigned long long)ld * 2, (unsigned long long)N * ld * 2,
+                                            (unsigned long long)((const char*)b - (const char*)a)};
+        const unsigned obox[4] = {16, 1, 32, 1};
+        const char* obase = (const char*)a + (size_t)c_h * m.cm_off[g0 + l] * 2;
+        if (!make_tmap_16bit(&p.omap[l], obase, 4, odims, ostr, obox, 0)) return cuda_fail("tri_in output map");
       }
     }
     const long long ntiles = (p.chunk_off[p.B] + 3) / 4;
