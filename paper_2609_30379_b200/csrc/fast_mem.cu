@@ -272,6 +272,74 @@ __global__ void __launch_bounds__(256) token_gemm_kernel(TokGemmArgs a) {
     }
 }
 
+// Tensor-core version (mma.sync m16n8k16, bf16 in, float accumulate) for 64 x 64 output tiles: the token-side GEMMs
+// have only a few thousand rows, so one small CTA tile per SM and a whole-K shared-memory panel is all they need.
+// Eight warps: warp w owns rows (w & 3) * 16 .. + 16 and columns (w >> 2) * 32 .. + 32 of the tile.
+__device__ inline void tg_ldsm_x4(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, const void* p) {
+  const unsigned a = (unsigned)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(a));
+}
+__device__ inline void tg_mma(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(256) token_gemm_mma_kernel(TokGemmArgs a) {
+  extern __shared__ __align__(16) unsigned char tg_smem[];
+  const int K = a.K, ldk = K + 8;                      // row pitch 16 bytes off a multiple of 128: conflict-free ldmatrix
+  __nv_bfloat16* As = reinterpret_cast<__nv_bfloat16*>(tg_smem);
+  __nv_bfloat16* Ws = As + 64 * ldk;
+  const long long r0 = (long long)blockIdx.x * 64;
+  int n0 = blockIdx.y * 64, which = 0;
+  if (n0 >= a.N[0]) { n0 -= a.N[0]; which = 1; }
+  const __nv_bfloat16* W = a.W[which];
+  const int N = a.N[which];
+  const int t = threadIdx.x, kv = K / 8;
+  // both panels with asynchronous 16-byte copies: every load of the CTA is in flight at once
+  for (int idx = t; idx < 64 * kv; idx += 256) {
+    const int r = idx / kv, c = idx - r * kv;
+    const bool ok = r0 + r < a.rows;
+    const unsigned da = (unsigned)__cvta_generic_to_shared(As + r * ldk + c * 8), dw = (unsigned)__cvta_generic_to_shared(Ws + r * ldk + c * 8);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(da), "l"(a.A + (ok ? r0 + r : 0) * K + c * 8), "r"(ok ? 16 : 0));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dw), "l"(W + (long long)(n0 + r) * K + c * 8));
+  }
+  asm volatile("cp.async.wait_all;\n" ::: "memory");
+  __syncthreads();
+  const int warp = t >> 5, lane = t & 31;
+  const int wr = (warp & 3) * 16, wc = (warp >> 2) * 32;
+  float acc[4][4] = {};
+  const __nv_bfloat16* ap = As + (wr + (lane & 7) + ((lane >> 3) & 1) * 8) * ldk + (lane >> 4) * 8;
+  const __nv_bfloat16* wp = Ws + (wc + (lane & 7) + (lane >> 4) * 8) * ldk + ((lane >> 3) & 1) * 8;
+  for (int k = 0; k < K; k += 16) {
+    unsigned af[4], b[4], d[4];
+    tg_ldsm_x4(af[0], af[1], af[2], af[3], ap + k);
+    tg_ldsm_x4(b[0], b[1], b[2], b[3], wp + k);
+    tg_ldsm_x4(d[0], d[1], d[2], d[3], wp + 16 * ldk + k);
+    tg_mma(acc[0], af, b[0], b[1]);
+    tg_mma(acc[1], af, b[2], b[3]);
+    tg_mma(acc[2], af, d[0], d[1]);
+    tg_mma(acc[3], af, d[2], d[3]);
+  }
+  const int g = lane >> 2, tq = lane & 3;
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      const long long r = r0 + wr + g + hh * 8;
+      const int n = n0 + wc + nt * 8 + 2 * tq;
+      if (r >= a.rows) continue;
+      const float x0 = acc[nt][hh * 2], x1 = acc[nt][hh * 2 + 1];
+      if (a.out_f32) {
+        *reinterpret_cast<float2*>(reinterpret_cast<float*>(a.out[which]) + r * N + n) = make_float2(x0, x1);
+      } else {
+        __nv_bfloat162* o = reinterpret_cast<__nv_bfloat162*>(reinterpret_cast<__nv_bfloat16*>(a.out[which]) + r * N + n);
+        float2 base = make_float2(0.f, 0.f);
+        if (a.accumulate) base = __bfloat1622float2(*o);
+        *o = __floats2bfloat162_rn(base.x + x0, base.y + x1);
+      }
+    }
+}
+
 bool fast_token_gemm_supported(int K, int N0, int N1) {
   return K % 8 == 0 && K >= 8 && K <= 1024 && N0 % 32 == 0 && N1 % 32 == 0;
 }
@@ -291,6 +359,25 @@ nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, 
   a.out[1] = out1;
   a.out_f32 = out_f32;
   a.accumulate = accumulate;
+  if (K % 16 == 0 && N0 % 64 == 0 && N1 % 64 == 0) {
+    const size_t smem64 = (size_t)2 * 64 * (K + 8) * 2;
+    static bool attr64 = false;
+    if (!attr64) {
+      if (cudaFuncSetAttribute(token_gemm_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+        return cuda_fail("token gemm smem attribute");
+      attr64 = true;
+    }
+    if (smem64 <= 200 * 1024) {
+      const long long bx64 = (rows + 63) / 64;
+      if (bx64 > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+      dim3 grid64((unsigned)bx64, (unsigned)((N0 + N1) / 64));
+      {
+        LaunchScope ls(name, st);
+        token_gemm_mma_kernel<<<grid64, 256, smem64, st>>>(a);
+      }
+      return cuda_ok(name);
+    }
+  }
   const size_t smem = (size_t)2 * 32 * (K + 8) * 2;
   static size_t attr = 0;
   if (smem > 48 * 1024 && smem > attr) {
