@@ -118,9 +118,10 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
 
 // ------------------------------------------------------------------------------------------
 // segmented mean / sum over contiguous row groups, bf16 in, float accumulate, bf16 out.
-// One block per group; VL = C / 8 lanes cover a row with 16-byte loads, 256 / VL rows in flight.
+// One block per group; VL = C / 8 lanes cover a row with 16-byte loads, 128 / VL rows in flight (small blocks: all
+// groups of a typical batch are resident at once, so there is no second, partly filled wave).
 // ------------------------------------------------------------------------------------------
-constexpr int SR_THREADS = 256;
+constexpr int SR_THREADS = 128;
 constexpr int SR_UNROLL = 4;
 
 __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const __nv_bfloat16* __restrict__ v,
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const _
   }
 }
 
-bool fast_segment_reduce_supported(int C) { return C % 8 == 0 && C >= 8 && C <= 2048; }
+bool fast_segment_reduce_supported(int C) { return C % 8 == 0 && C >= 8 && C <= 8 * SR_THREADS; }
 
 nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,
                               cudaStream_t st) {
