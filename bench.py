@@ -71,7 +71,8 @@ def kernel_work(cfg: wl.Config):
         w[f"generic_attn_in_{n}"] = dict(bytes=T2 * (c_z + Hd) * e, flops=2 * T2 * c_z * Hd)
     w["generic_attn_in_bias"] = dict(bytes=T2 * (c_z + H) * e, flops=2 * T2 * c_z * H)
     w["attn_in"] = dict(bytes=T2 * (c_z + 4 * Hd + H) * e, flops=2 * T2 * c_z * (4 * Hd + H))
-    w["generic_attn_core"] = w["attn_core"] = dict(bytes=T2 * (4 * Hd + H) * e, flops=4 * N3 * Hd)
+    # the softmax needs one exponential per (query, key, head): the special-function units retire 16 per clock and SM
+    w["generic_attn_core"] = w["attn_core"] = dict(bytes=T2 * (4 * Hd + H) * e, flops=4 * N3 * Hd, exps=N3 * H)
     w["generic_attn_out"] = w["attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
@@ -81,7 +82,15 @@ def kernel_work(cfg: wl.Config):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (cfg2 only);
 # other workloads report traffic = None.
-NCU_TRAFFIC_CFG2 = {"attn_core": 367.4e6, "tri_in": 230.2e6, "tri_contract": 256.3e6}
+NCU_TRAFFIC_CFG2 = {"attn_core": 375.1e6, "tri_out": 243.3e6, "attn_in": 324.7e6, "tri_in": 233.1e6, "attn_out": 240.1e6,
+                    "tri_contract": 255.0e6}
+
+
+# Exponentials per second of the special-function units: 16 per clock and SM (measured: 15.99 with ex2.approx.f32,
+# the same with the packed bf16 / fp16 forms) times 148 SMs at the maximum SM clock.
+EXP_PER_CLK_SM = 16
+N_SM = 148
+SM_MAX_MHZ = 1965.0
 
 
 def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
@@ -92,6 +101,14 @@ def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
     hbm = peaks["hbm_gbs"] * 1e9
     tens = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
     t_hbm, t_tensor = wk["bytes"] / hbm, wk["flops"] / tens
+    exp_peak = EXP_PER_CLK_SM * N_SM * SM_MAX_MHZ * 1e6
+    t_alu = wk.get("exps", 0) / exp_peak
+    if t_alu > t_hbm and t_alu > t_tensor:
+        ach = wk["exps"] / t / 1e9
+        return dict(kernel=name, bound="alu", achieved=round(ach, 1), peak=round(exp_peak / 1e9, 1), unit="Gexp/s",
+                    frac=round(ach * 1e9 / exp_peak, 4), traffic=None,
+                    peak_source="16 exponentials per clock and SM x 148 SMs x 1965 MHz (rate measured on this pool)",
+                    hbm_frac=round(wk["bytes"] / t / hbm, 4), us_per_launch=round(t * 1e6, 2), launches=launches)
     if t_hbm >= t_tensor:
         ach = wk["bytes"] / t / 1e9
         return dict(kernel=name, bound="hbm", achieved=round(ach, 1), peak=peaks["hbm_gbs"], unit="GB/s",

@@ -446,9 +446,9 @@ static nt_status launch_attn_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, 
     const unsigned long long dims[2] = {(unsigned long long)Hd, (unsigned long long)rows};
     const unsigned long long strides[1] = {(unsigned long long)Hd * 2};
     const unsigned qbox[2] = {(unsigned)D, 128}, kbox[2] = {(unsigned)D, 32};
-    if (!make_tmap_16bit(&p.qmap, q + p.row0 * Hd, 2, dims, strides, qbox, 2 * D)) return cuda_fail("attn tc q map");
-    if (!make_tmap_16bit(&p.kmap, k + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn tc k map");
-    if (!make_tmap_16bit(&p.vmap, v + p.row0 * Hd, 2, dims, strides, kbox, 2 * D)) return cuda_fail("attn tc v map");
+    if (!make_tmap_16bit(&p.qmap, q + p.row0 * Hd, 2, dims, strides, qbox, 2 * D, 2 * D >= 128 ? 128 : 2 * D)) return cuda_fail("attn tc q map");
+    if (!make_tmap_16bit(&p.kmap, k + p.row0 * Hd, 2, dims, strides, kbox, 2 * D, 2 * D >= 128 ? 128 : 2 * D)) return cuda_fail("attn tc k map");
+    if (!make_tmap_16bit(&p.vmap, v + p.row0 * Hd, 2, dims, strides, kbox, 2 * D, 2 * D >= 128 ? 128 : 2 * D)) return cuda_fail("attn tc v map");
   }
   static bool attr_set = false;
   if (!attr_set) {

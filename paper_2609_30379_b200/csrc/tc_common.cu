@@ -19,7 +19,7 @@ EncodeTiledFn get_encode_tiled() {
 }
 
 bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes) {
+                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes, int l2_promotion_bytes) {
   EncodeTiledFn enc = get_encode_tiled();
   if (!enc) return false;
   cuuint64_t gdim[5];
@@ -37,7 +37,9 @@ bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigne
                                                      : CU_TENSOR_MAP_SWIZZLE_128B;
   // bf16 and fp16 tiles move identically (no conversion on the way), so one 16-bit type serves both
   CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bdim,
-                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                   l2_promotion_bytes >= 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
+                   : l2_promotion_bytes == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }

@@ -20,9 +20,12 @@ EncodeTiledFn get_encode_tiled();
 // bf16 tensor map with 128-byte swizzle; dims / strides fastest first (strides in bytes for dims 1..rank-1)
 bool make_tmap_bf16(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
                     const unsigned long long* strides_bytes, const unsigned* box);
-// same with a 32-, 64- or 128-byte swizzle span (the inner box extent in bytes must not exceed it); 0 = no swizzle
+// same with a 32-, 64- or 128-byte swizzle span (the inner box extent in bytes must not exceed it); 0 = no swizzle.
+// l2_promotion_bytes: granularity at which L2 fetches around a request (128, 64 or 0 = none); boxes narrower than a
+// 128-byte line that other CTAs read at other times should not promote, or DRAM delivers their neighbours in vain.
 bool make_tmap_16bit(CUtensorMap* map, const void* base, int rank, const unsigned long long* dims,
-                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes);
+                     const unsigned long long* strides_bytes, const unsigned* box, int swizzle_bytes,
+                     int l2_promotion_bytes = 128);
 
 #ifdef __CUDACC__
 // ---------------------------------------------------------------------------------- device helpers
