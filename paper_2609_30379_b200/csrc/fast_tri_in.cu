@@ -33,7 +33,7 @@ constexpr int TI_MAXB = 12;
 
 struct TriInParams {
   CUtensorMap zmap[TI_MAXB];               // {c_z, N (k), N (i), 1}, box {64, 32, 1, 1}
-  CUtensorMap omap[TI_MAXB];               // outputs {ld (k), N (i), c_h, 2 (a | b)}, box {16, 1, 32, 1}, no swizzle
+  CUtensorMap omap[TI_MAXB];               // outputs {ld (k), N (i), c_h, 2 (a | b)}, box {32, 1, 32, 1}, 64-byte swizzle
   CUtensorMap wmap;                        // {c_z, 4 c_h}, box {64, 128}
   CUtensorMap xmap;                        // augmentation columns {8, 2 * aug_rows}, box {8, 256}, no swizzle
   long long chunk_off[TI_MAXB + 1];
@@ -80,10 +80,11 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   const int z_stage_bytes = nslab * z_slab_bytes;
   const int zx_region = 128 * 16;                  // one 8-column region of the activation augmentation
   unsigned char* sW = smem;
-  unsigned char* sWx = sW + w_bytes;               // [2 regions][wrows][8] fp16, no swizzle
-  unsigned char* sZ = sWx + 2 * wx_region;         // 2 stages of the z tile
-  unsigned char* sZx = sZ + 2 * z_stage_bytes;     // 2 stages x [2 regions][128][8] fp16
-  unsigned char* sOut = sZx + 2 * 2 * zx_region;   // per epilogue warp: [32 channels][16 positions] fp16 staged for a TMA store
+  unsigned char* sWx = sW + w_bytes;               // [wrows][8] fp16, no swizzle: augmentation columns 0-7 of the weights
+  unsigned char* sZ = sWx + wx_region;             // 2 stages of the z tile
+  unsigned char* sZx = sZ + 2 * z_stage_bytes;     // 2 stages x [128][8] fp16: augmentation columns 0-7 of the activations
+  unsigned char* sZero = sZx + 2 * zx_region;      // [128][8] zeros: augmentation columns 8-15 of either operand
+  unsigned char* sOut = sZero + zx_region;         // per epilogue warp: 2 x [32 channels][16 positions] fp16 staged for TMA stores
   unsigned long long* afull = bars;        // [2] TMA landed
   unsigned long long* aempty = bars + 2;   // [2] MMAs that read the stage are done
   unsigned long long* tfull = bars + 4;    // [2] accumulator buffer ready
@@ -106,10 +107,8 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
   // the second 8-column region of the activation augmentation is always zero
-  for (int idx = threadIdx.x; idx < 2 * zx_region / 16; idx += TI_THREADS) {
-    const int st = idx / (zx_region / 16), r = idx % (zx_region / 16);
-    *reinterpret_cast<uint4*>(sZx + st * 2 * zx_region + zx_region + r * 16) = make_uint4(0, 0, 0, 0);
-  }
+  for (int idx = threadIdx.x; idx < zx_region / 16; idx += TI_THREADS)
+    *reinterpret_cast<uint4*>(sZero + idx * 16) = make_uint4(0, 0, 0, 0);
   fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
@@ -123,13 +122,11 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (lane q decodes and loads chunk q)
     if (lane == 0) {
-      mbar_expect_tx(wfull, w_bytes + 2 * wx_region);
+      mbar_expect_tx(wfull, w_bytes + wx_region);
       for (int sl = 0; sl < nslab; ++sl)
         for (int rb = 0; rb < wrows / 128; ++rb)
           tma_load_2d(sW + sl * w_slab_bytes + rb * 128 * 128, &p.wmap, wfull, sl * 64, rb * 128);
-      for (int reg = 0; reg < 2; ++reg)
-        for (int rb = 0; rb < wrows / 256; ++rb)
-          tma_load_2d(sWx + reg * wx_region + rb * 256 * 16, &p.xmap, wfull, 0, reg * p.aug_rows + rb * 256);
+      for (int rb = 0; rb < wrows / 256; ++rb) tma_load_2d(sWx + rb * 256 * 16, &p.xmap, wfull, 0, rb * 256);
     }
     int stage = 0, tn = 0;
     unsigned phase = 0;
@@ -163,13 +160,14 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     unsigned unit = 0;
     const unsigned idesc = idesc_f16(128, 128, 0, 0, FMT_F16, FMT_F16);   // M = 128 channels, N = 128 positions
     const unsigned long long w_desc = desc_kmajor_sw128(smem_u32(sW));
-    const unsigned long long wx_desc = desc_kmajor_nosw(smem_u32(sWx), wx_region, 128);
+    const unsigned wx_addr = smem_u32(sWx), zero_addr = smem_u32(sZero);   // columns 8-15 of both operands: the zero region
     const unsigned w_slab16 = (unsigned)w_slab_bytes >> 4, z_slab16 = (unsigned)z_slab_bytes >> 4;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&aconv[stage], phase, ab);
       tc_fence_after();
       const unsigned long long z_desc = desc_kmajor_sw128(smem_u32(sZ + stage * z_stage_bytes));
-      const unsigned long long zx_desc = desc_kmajor_nosw(smem_u32(sZx + stage * 2 * zx_region), zx_region, 128);
+      const unsigned zx_addr = smem_u32(sZx + stage * zx_region);
+      const unsigned long long zx_desc = desc_kmajor_nosw(zx_addr, zero_addr - zx_addr, 128);
       for (int u = 0; u < nunits; ++u, ++unit) {
         const unsigned buf = unit & 1;
         if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
@@ -190,7 +188,8 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
             }
           }
           // augmentation K step: c1 / c0 columns against the (-mean rstd, 1) columns (16-byte rows)
-          if (elect_one()) umma_bf16(d_tmem, wx_desc + (unsigned)(u * 256 + part * 128), zx_desc, idesc, 1);
+          const unsigned wxa = wx_addr + (unsigned)(u * 256 + part * 128) * 16;
+          if (elect_one()) umma_bf16(d_tmem, desc_kmajor_nosw(wxa, zero_addr - wxa, 128), zx_desc, idesc, 1);
         }
         if (elect_one()) tc_commit(&tfull[buf]);
         __syncwarp();
@@ -256,7 +255,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         const __half one = __float2half_rn(1.0f), zero = __float2half_rn(0.0f);
         __half2 p0 = __halves2half2(mh, ml), p1 = __halves2half2(mh, one), p2 = __halves2half2(one, zero),
                 p3 = __halves2half2(zero, zero);
-        *reinterpret_cast<uint4*>(sZx + stage * 2 * zx_region + row * 16) =
+        *reinterpret_cast<uint4*>(sZx + stage * zx_region + row * 16) =
             make_uint4(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1),
                        *reinterpret_cast<unsigned*>(&p2), *reinterpret_cast<unsigned*>(&p3));
       }
@@ -282,7 +281,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
         // c_h = 128: unit 0 -> a, unit 1 -> b, channel = accumulator row; c_h = 64: rows 0-63 -> a, 64-127 -> b
         const int which = c_h == 128 ? u : (quarter >> 1);
         const int ch0 = c_h == 128 ? quarter * 32 : (quarter & 1) * 32;          // first channel of this warp
-        unsigned char* stg = sOut + (warp - TI_EPI_WARP0) * 1024;
+        unsigned char* stg0 = sOut + (warp - TI_EPI_WARP0) * 2048;
         const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256 + half * 64;
         // four steps of 16 positions; the TMEM loads of step k + 1 are in flight while step k is computed.  A step's
         // 32 channels x 16 positions go through a 1 KB staging tile and out with one TMA store (runs of 32 bytes per
@@ -310,16 +309,25 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
             h = __hmax2(__hmin2(h, hmax2), hmin2);
             w[e] = *reinterpret_cast<unsigned*>(&h);
           }
-          if (lane == 0) tma_store_wait_read0();            // the previous step's store has read the staging tile
-          __syncwarp();
-          *reinterpret_cast<uint4*>(stg + lane * 32) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(stg + lane * 32 + 16) = make_uint4(w[4], w[5], w[6], w[7]);
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0 && info.w) {
-            const int jc = info.z + (k & 1) * 16;
-            if (jc < round_up8(p.N[info.x])) tma_store_4d(&p.omap[info.x], stg, jc, info.y, ch0, which);
-            tma_store_commit();
+          // a chunk (two steps, 32 positions) is staged as 32 channel rows of 64 bytes and leaves with one TMA store:
+          // the store engine's cost is per row, so rows should be as long as the tile geometry allows
+          if ((k & 1) == 0) {
+            if (lane == 0) tma_store_wait_read0();          // the previous chunk's store has read the staging tile
+            __syncwarp();
+          }
+          // 64-byte swizzle of the store map: the 16-byte pieces of a row are XOR-ed with the row's bits 1-2, so eight
+          // lanes cover all banks
+          unsigned char* rowp = stg0 + lane * 64;
+          const int sw = (lane >> 1) & 3;
+          *reinterpret_cast<uint4*>(rowp + ((((k & 1) * 2) ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(rowp + ((((k & 1) * 2 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+          if (k & 1) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && info.w) {
+              if (info.z < round_up8(p.N[info.x])) tma_store_4d(&p.omap[info.x], stg0, info.z, info.y, ch0, which);
+              tma_store_commit();
+            }
           }
         }
         tc_fence_before();
@@ -341,8 +349,8 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
                       const BatchMeta& m, int* status, cudaStream_t st) {
   const int nslab = c_z / 64;
   const int wrows = 4 * c_h;
-  const size_t smem = (size_t)nslab * wrows * 128 + 2 * (size_t)wrows * 16 + 2 * (size_t)nslab * 128 * 128 +
-                      2 * 2 * (size_t)128 * 16 + 8 * 1024 + 1024;
+  const size_t smem = (size_t)nslab * wrows * 128 + (size_t)wrows * 16 + 2 * (size_t)nslab * 128 * 128 +
+                      3 * (size_t)128 * 16 + 16 * 1024 + 1024;
   if (((const char*)b - (const char*)a) % 16 != 0 || b <= a) return NT_ERR_UNSUPPORTED;   // a | b form one 4-D tensor
   static bool attr_set = false;
   if (!attr_set) {
@@ -386,9 +394,9 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
         const unsigned long long odims[4] = {(unsigned long long)ld, (unsigned long long)N, (unsigned long long)c_h, 2};
         const unsigned long long ostr[3] = {(unsigned long long)ld * 2, (unsigned long long)N * ld * 2,
                                             (unsigned long long)((const char*)b - (const char*)a)};
-        const unsigned obox[4] = {16, 1, 32, 1};
+        const unsigned obox[4] = {32, 1, 32, 1};
         const char* obase = (const char*)a + (size_t)c_h * m.cm_off[g0 + l] * 2;
-        if (!make_tmap_16bit(&p.omap[l], obase, 4, odims, ostr, obox, 0)) return cuda_fail("tri_in output map");
+        if (!make_tmap_16bit(&p.omap[l], obase, 4, odims, ostr, obox, 64)) return cuda_fail("tri_in output map");
       }
     }
     const long long ntiles = (p.chunk_off[p.B] + 3) / 4;
