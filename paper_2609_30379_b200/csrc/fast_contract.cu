@@ -6,7 +6,8 @@
 // (sample, channel, 128-row block of i, up-to-256-column block of j) taken from the host lengths:
 //   warp 0   TMA producer: 64-wide k slabs of the a rows and b rows into a 3-stage ring
 //   warp 1   MMA issuer: 128 x Nt x 16 tcgen05.mma steps, accumulating into one of two TMEM buffers
-//   warps 2-5 epilogue: TMEM -> registers -> bf16 -> swizzled staging tile -> TMA store into t
+//   warps 2-9 epilogue (two per TMEM lane quarter, alternate 64-column groups): TMEM -> registers -> fp16 ->
+//            swizzled staging tile -> TMA store into t
 // One 4-D tensor map per sample {k, i, channel, which of a/b/t} serves loads and stores; rows and
 // columns past N are zero-filled on load and clipped on store, so no padded tile is ever moved.
 #include <cstring>
@@ -22,7 +23,7 @@ constexpr int CT_B_BYTES = 256 * 128;
 constexpr int CT_STAGE_BYTES = CT_A_BYTES + CT_B_BYTES;
 constexpr int CT_STAGING_BYTES = 4 * CT_A_BYTES; // 128 x 256 bf16 in four swizzled 64-column panels
 constexpr int CT_SMEM = CT_STAGES * CT_STAGE_BYTES + CT_STAGING_BYTES + 1024;
-constexpr int CT_THREADS = 192;
+constexpr int CT_THREADS = 64 + 256;          // producer, MMA issuer, 8 epilogue warps
 constexpr int TMA_MAXB = 16;
 
 struct ContractParams {
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < CT_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 4); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 8); }
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
@@ -129,9 +130,15 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
     }
   } else if (warp >= 2) {
     // ------------------------------------------------------------------ epilogue
-    const int quarter = warp & 3;
+    const int quarter = warp & 3, half = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
     const int ep_tid = threadIdx.x - 64;
+    const __half2 hmax2 = __float2half2_rn(65504.f), hmin2 = __float2half2_rn(-65504.f);
+    auto pk = [&](unsigned lo, unsigned hi, float sc) {     // scale, round to fp16, clamp into its finite range
+      __half2 h = __floats2half2_rn(__uint_as_float(lo) * sc, __uint_as_float(hi) * sc);
+      h = __hmax2(__hmin2(h, hmax2), hmin2);
+      return *reinterpret_cast<unsigned*>(&h);
+    };
     unsigned tph[2] = {0, 0};
     long long n = 0;
     for (long long job = blockIdx.x; job < njobs; job += gridDim.x, ++n) {
@@ -143,12 +150,12 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       tc_fence_after();
       if (n > 0) {                          // staging tile still being read by the previous store?
         if (ep_tid == 0) tma_store_wait_read0();
-        named_bar_sync(1, 128);
+        named_bar_sync(1, 256);
       }
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       const int ncg = (Nt + 63) / 64;
       const float tscale = 1.0f / (float)p.N[s];   // t is stored as t / N in fp16; the following LayerNorm is scale-free
-      for (int cg = 0; cg < ncg; ++cg) {
+      for (int cg = half; cg < ncg; cg += 2) {
         unsigned r0[32], r1[32];
         tmem_ld32(taddr + cg * 64, r0);
         tmem_ld32(taddr + cg * 64 + 32, r1);
@@ -157,19 +164,19 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint4 v;
-          v.x = pack2h(r0[ch * 8 + 0], r0[ch * 8 + 1], tscale);
-          v.y = pack2h(r0[ch * 8 + 2], r0[ch * 8 + 3], tscale);
-          v.z = pack2h(r0[ch * 8 + 4], r0[ch * 8 + 5], tscale);
-          v.w = pack2h(r0[ch * 8 + 6], r0[ch * 8 + 7], tscale);
+          v.x = pk(r0[ch * 8 + 0], r0[ch * 8 + 1], tscale);
+          v.y = pk(r0[ch * 8 + 2], r0[ch * 8 + 3], tscale);
+          v.z = pk(r0[ch * 8 + 4], r0[ch * 8 + 5], tscale);
+          v.w = pk(r0[ch * 8 + 6], r0[ch * 8 + 7], tscale);
           *reinterpret_cast<uint4*>(panel + sw128_off(row, ch)) = v;
         }
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           uint4 v;
-          v.x = pack2h(r1[ch * 8 + 0], r1[ch * 8 + 1], tscale);
-          v.y = pack2h(r1[ch * 8 + 2], r1[ch * 8 + 3], tscale);
-          v.z = pack2h(r1[ch * 8 + 4], r1[ch * 8 + 5], tscale);
-          v.w = pack2h(r1[ch * 8 + 6], r1[ch * 8 + 7], tscale);
+          v.x = pk(r1[ch * 8 + 0], r1[ch * 8 + 1], tscale);
+          v.y = pk(r1[ch * 8 + 2], r1[ch * 8 + 3], tscale);
+          v.z = pk(r1[ch * 8 + 4], r1[ch * 8 + 5], tscale);
+          v.w = pk(r1[ch * 8 + 6], r1[ch * 8 + 7], tscale);
           *reinterpret_cast<uint4*>(panel + sw128_off(row, 4 + ch)) = v;
         }
       }
@@ -177,7 +184,7 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[buf]);
       fence_proxy_async_smem();
-      named_bar_sync(1, 128);
+      named_bar_sync(1, 256);
       if (ep_tid == 0) {
         for (int cg = 0; cg < ncg; ++cg)
           tma_store_4d(&p.maps[s], staging + cg * CT_A_BYTES, j0 + cg * 64, i0, c, 2);
