@@ -93,11 +93,12 @@ N_SM = 148
 SM_MAX_MHZ = 1965.0
 
 
-def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
+def roofline_entry(name, total_ms, launches, calls, work, peaks, peak_kind):
+    """`work` is per library call; a call may split a long batch over several launches, so time is per call too."""
     if name not in work or launches == 0:
         return None
     wk = work[name]
-    t = total_ms / launches * 1e-3
+    t = total_ms / calls * 1e-3
     hbm = peaks["hbm_gbs"] * 1e9
     tens = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12
     t_hbm, t_tensor = wk["bytes"] / hbm, wk["flops"] / tens
@@ -108,17 +109,17 @@ def roofline_entry(name, total_ms, launches, work, peaks, peak_kind):
         return dict(kernel=name, bound="alu", achieved=round(ach, 1), peak=round(exp_peak / 1e9, 1), unit="Gexp/s",
                     frac=round(ach * 1e9 / exp_peak, 4), traffic=None,
                     peak_source="16 exponentials per clock and SM x 148 SMs x 1965 MHz (rate measured on this pool)",
-                    hbm_frac=round(wk["bytes"] / t / hbm, 4), us_per_launch=round(t * 1e6, 2), launches=launches)
+                    hbm_frac=round(wk["bytes"] / t / hbm, 4), us_per_call=round(t * 1e6, 2), launches=launches)
     if t_hbm >= t_tensor:
         ach = wk["bytes"] / t / 1e9
         return dict(kernel=name, bound="hbm", achieved=round(ach, 1), peak=peaks["hbm_gbs"], unit="GB/s",
                     frac=round(ach / peaks["hbm_gbs"], 4), traffic=None, peak_source=f"of {peak_kind}",
-                    us_per_launch=round(t * 1e6, 2), launches=launches)
+                    us_per_call=round(t * 1e6, 2), launches=launches)
     ach = wk["flops"] / t / 1e12
     pk = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     return dict(kernel=name, bound="tensor", achieved=round(ach, 2), peak=pk, unit="TFLOP/s",
                 frac=round(ach / pk, 4), traffic=None, peak_source=f"of {peak_kind} (sustained)",
-                us_per_launch=round(t * 1e6, 2), launches=launches)
+                us_per_call=round(t * 1e6, 2), launches=launches)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -326,7 +327,8 @@ def main():
     work = kernel_work(cfg)
     kernels = {k: dict(ms_per_step=round(v[0] / steps, 4), launches_per_step=v[1] / steps, share=round(v[0] / tot_prof, 4))
                for k, v in sorted(prof.items(), key=lambda kv: -kv[1][0])}
-    roofs = {k: roofline_entry(k, v[0], v[1], work, peaks, peak_kind) for k, v in prof.items()}
+    calls = steps * cfg.blocks          # every kernel family of the table runs once per block (in one or more launches)
+    roofs = {k: roofline_entry(k, v[0], v[1], calls, work, peaks, peak_kind) for k, v in prof.items()}
     roofs = {k: r for k, r in roofs.items() if r}
     for k in kernels:
         if k in roofs:

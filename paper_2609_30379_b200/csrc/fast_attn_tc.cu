@@ -320,22 +320,22 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
         float lsum = 0.f;
         if (warp_live) {
           const float ms = -mx * sc2;
-          float l4[4] = {0.f, 0.f, 0.f, 0.f};
+          // packed float pairs (add / fma on two floats per instruction) for everything around the exponentials
+          float2 l2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          const float2 sc22 = make_float2(sc2, sc2), ms2 = make_float2(ms, ms);
           const unsigned char* brow = sBias + jb * p.bias_tile_bytes + row * bstride;
           auto pass2 = [&](int gg, const unsigned (&rr)[16]) {
             const uint4 b0 = *reinterpret_cast<const uint4*>(brow + gg * 32), b1 = *reinterpret_cast<const uint4*>(brow + gg * 32 + 16);
             const unsigned bw[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-            float pv[16];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              pv[2 * e] = tca_exp2(fmaf(__uint_as_float(rr[2 * e]) + __uint_as_float(bw[e] << 16), sc2, ms));
-              pv[2 * e + 1] = tca_exp2(fmaf(__uint_as_float(rr[2 * e + 1]) + __uint_as_float(bw[e] & 0xffff0000u), sc2, ms));
-            }
             unsigned pk[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-              l4[e & 3] += pv[2 * e] + pv[2 * e + 1];
-              pk[e] = tca_pack(pv[2 * e], pv[2 * e + 1]);
+              const float2 sv = make_float2(__uint_as_float(rr[2 * e]), __uint_as_float(rr[2 * e + 1]));
+              const float2 bv = make_float2(__uint_as_float(bw[e] << 16), __uint_as_float(bw[e] & 0xffff0000u));
+              const float2 x = __ffma2_rn(__fadd2_rn(sv, bv), sc22, ms2);
+              const float2 pv = make_float2(tca_exp2(x.x), tca_exp2(x.y));
+              l2[e & 1] = __fadd2_rn(l2[e & 1], pv);
+              pk[e] = tca_pack(pv.x, pv.y);
             }
             tmem_st8(t_row + gg * 16 + (gg & 1) * 8, pk);
           };
@@ -359,7 +359,7 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
             tmem_ld_wait16(ra);
             pass2(g, ra);
           }
-          lsum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
+          lsum = (l2[0].x + l2[0].y) + (l2[1].x + l2[1].y);
           tmem_st_wait();
         }
         xm[256 + hf * 128 + row] = lsum;
