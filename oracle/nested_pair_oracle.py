@@ -23,6 +23,9 @@ What each function follows:
   segment_reduce       Eq. 4 (pair reduction) and the mean of Eq. 1 line 3; App. A batch-axis
                        convention (``[1,2],[3,4]`` sums to ``[3,7]``).
   token_update         Eq. 1 line 3: ``X~ = X + g(mean_b P~[a,b,:])`` with ``g`` a bias-free projection.
+  pair_transition      Eq. 1 line 2: ``P~ = P + h(LN(P))`` with ``h`` the SwiGLU feature update named there
+                       (gate ``silu(x W_a^T)``, value ``x W_b^T``, output projection ``W_2``; expansion four in the
+                       paper's settings, App. A.1), position-wise on the packed values.
 
 Pins (tests/test_oracle_pins.py): the paper's printed (2,3) example, the ``[3,7]`` reduction,
 structural invariants, closed forms, brute-force triple loops, an independent padded-and-masked
@@ -241,6 +244,21 @@ def token_update(x, m, W_r, dtype=np.float64):
     """x' = x + m W_r^T  (the projection g of Eq. 1 line 3, bias-free)."""
     x, m, W_r = _as(dtype, x, m, W_r)
     return x + m @ W_r.T
+
+
+def silu(v):
+    return v * sigmoid(v)
+
+
+def pair_transition(z, W, eps=LN_EPS, dtype=np.float64):
+    """Eq. 1 line 2 on the packed values: z' = z + (silu(LN(z) W_a^T) * (LN(z) W_b^T)) W_2^T, position by position
+    (no sample structure enters: the update acts on the static channel tail only).  W: ln_gamma, ln_beta [c],
+    W_a, W_b [hidden, c], W_2 [c, hidden]; all projections bias-free."""
+    z = np.asarray(z, dtype=dtype)
+    Wd = {k: np.asarray(v, dtype=dtype) for k, v in W.items()}
+    zh = layer_norm(z, Wd["ln_gamma"], Wd["ln_beta"], eps)
+    h = silu(zh @ Wd["W_a"].T) * (zh @ Wd["W_b"].T)
+    return z + h @ Wd["W_2"].T
 
 
 # --------------------------------------------------------------------------------------------

@@ -277,9 +277,7 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
         const bool warp_live = jb * 128 + quarter * 32 < N;        // this warp owns at least one real query
         float* xm = xch + (wg * 2 + (u & 1)) * 4 * 128;             // [max | sum][2 halves][128]
         unsigned ra[16], rb[16];
-        // one warp of the group watches the mbarrier, the others park in the named barrier
-        if ((sw & 7) == 0) mbar_wait(&sfull[wg], u & 1, ab);
-        named_bar_sync(1 + wg, 256);
+        mbar_wait(&sfull[wg], u & 1, ab);      // a failed probe parks the warp in hardware: every warp may watch the barrier
         tc_fence_after();
         // Each thread owns a contiguous half of the row: granules [gb, ge), read 32 columns at a time where a pair
         // of granules starts on an even index, 16 otherwise.

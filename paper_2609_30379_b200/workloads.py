@@ -137,6 +137,15 @@ def make_block_weights(st: _Stream, cfg: Config) -> dict:
     return w
 
 
+def make_transition_weights(cfg: Config, block: int = 0, expansion: int = 4) -> dict:
+    """Weights of the SwiGLU pair transition of one block (hidden = expansion * c_z).  They come from a stream of
+    their own (seed + 7919 * (block + 1)), so the frozen draws of the other sub-layers are unchanged."""
+    st = _Stream(cfg.seed + 7919 * (block + 1), cfg.dtype == "bf16")
+    c, hid = cfg.c_z, expansion * cfg.c_z
+    return dict(ln_gamma=st.ln_gamma(c), ln_beta=st.ln_beta(c), W_a=st.weight(hid, c), W_b=st.weight(hid, c),
+                W_2=st.weight(c, hid))
+
+
 def make_token_weights(st: _Stream, cfg: Config) -> dict:
     """Weights of the single-ragged special case: attention over the token axis, no LN/gate/bias."""
     c, Hd = cfg.c_z, cfg.H * cfg.d

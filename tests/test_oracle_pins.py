@@ -360,3 +360,71 @@ def test_sampled_evaluators_equal_full_functions():
     full = orc.row_attn_pairbias(z, cfg.lengths, inp["blocks"][0]["attn"], cfg.H, cfg.d).reshape(7, 7, -1)
     got = orc.row_attn_pairbias_at(z.reshape(7, 7, -1), inp["blocks"][0]["attn"], cfg.H, cfg.d, pos)
     assert np.allclose(got, np.stack([full[i, j] for i, j in pos]), rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# SwiGLU pair transition (Eq. 1 line 2)
+# ---------------------------------------------------------------------------------------------
+def _transition_case(rows=11, c=8, seed=3):
+    cfg = wl.Config("tiny", "f32", (3,), c_s=6, c_z=c, c_h=4, H=2, d=4, blocks=1, seed=seed)
+    W = wl.make_transition_weights(cfg)
+    rng = np.random.default_rng(seed)
+    z = rng.standard_normal((rows, c))
+    return z, W
+
+
+def test_transition_brute_force_scalar_loops():
+    """Every output element from scalar arithmetic: mean / variance by hand, math.exp for the sigmoid."""
+    import math
+    z, W = _transition_case()
+    c, hid = z.shape[1], W["W_a"].shape[0]
+    out = orc.pair_transition(z, W)
+    for p in range(z.shape[0]):
+        mean = sum(z[p]) / c
+        var = sum((v - mean) ** 2 for v in z[p]) / c
+        zh = [(z[p, k] - mean) / math.sqrt(var + orc.LN_EPS) * float(W["ln_gamma"][k]) + float(W["ln_beta"][k]) for k in range(c)]
+        h = []
+        for n in range(hid):
+            g = sum(zh[k] * float(W["W_a"][n, k]) for k in range(c))
+            v = sum(zh[k] * float(W["W_b"][n, k]) for k in range(c))
+            h.append(g / (1.0 + math.exp(-g)) * v)
+        for m in range(c):
+            want = z[p, m] + sum(h[n] * float(W["W_2"][m, n]) for n in range(hid))
+            assert abs(out[p, m] - want) < 1e-10
+
+
+def test_transition_equals_torch_library_routines():
+    """LayerNorm, SiLU and linear maps from torch (float64) give the same update."""
+    z, W = _transition_case(rows=17, c=16, seed=5)
+    t = {k: torch.tensor(np.asarray(v, dtype=np.float64)) for k, v in W.items()}
+    zt = torch.tensor(z)
+    zh = torch.nn.functional.layer_norm(zt, (z.shape[1],), t["ln_gamma"], t["ln_beta"], orc.LN_EPS)
+    ref = zt + (torch.nn.functional.silu(zh @ t["W_a"].T) * (zh @ t["W_b"].T)) @ t["W_2"].T
+    np.testing.assert_allclose(orc.pair_transition(z, W), ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_transition_closed_forms():
+    z, W = _transition_case(rows=9, c=8, seed=11)
+    # zero output projection: the residual alone
+    W0 = dict(W, W_2=np.zeros_like(W["W_2"]))
+    np.testing.assert_array_equal(orc.pair_transition(z, W0), z)
+    # the update is linear in W_2 and odd in W_b
+    upd = orc.pair_transition(z, W) - z
+    np.testing.assert_allclose(orc.pair_transition(z, dict(W, W_2=2.0 * W["W_2"])) - z, 2.0 * upd, rtol=1e-12)
+    np.testing.assert_allclose(orc.pair_transition(z, dict(W, W_b=-W["W_b"])) - z, -upd, rtol=1e-12)
+    # LayerNorm makes the update invariant to a per-position shift and (up to eps) positive scale of z
+    np.testing.assert_allclose(orc.pair_transition(z + 3.0, W) - (z + 3.0), upd, rtol=1e-9, atol=1e-9)
+    np.testing.assert_allclose(orc.pair_transition(4.0 * z, W) - 4.0 * z, upd, rtol=1e-4, atol=1e-5)
+    # gate saturation: with W_a scaled up silu(g) -> relu(g), so the update approaches (relu(g) * v) W_2^T
+    zh = orc.layer_norm(z, W["ln_gamma"], W["ln_beta"])
+    big = dict(W, W_a=1e4 * np.asarray(W["W_a"], dtype=np.float64))
+    g = zh @ big["W_a"].T
+    want = (np.maximum(g, 0.0) * (zh @ np.asarray(W["W_b"], dtype=np.float64).T)) @ np.asarray(W["W_2"], dtype=np.float64).T
+    np.testing.assert_allclose(orc.pair_transition(z, big) - z, want, rtol=1e-6, atol=1e-6)
+
+
+def test_transition_is_position_wise():
+    """No sample structure enters: permuting the packed positions permutes the result."""
+    z, W = _transition_case(rows=13, c=8, seed=2)
+    perm = np.random.default_rng(0).permutation(z.shape[0])
+    np.testing.assert_allclose(orc.pair_transition(z[perm], W), orc.pair_transition(z, W)[perm], rtol=1e-13, atol=1e-13)
