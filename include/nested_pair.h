@@ -181,6 +181,24 @@ nt_status nt_pair_broadcast_static(const nt_layout *L, nt_dtype dt, int32_t c_s,
                                    const void *ln_gamma, const void *ln_beta, float ln_eps,
                                    void *z, nt_stream stream);
 
+/*
+ * nt_pair_transition -- the SwiGLU feature update of the pair state (Eq. 1 line 2: P~ = P + h(LN(P)), h the
+ * SwiGLU update named there; expansion four in the paper's settings, App. A.1), position-wise on packed values:
+ *   zh = LN(z);  z += (silu(zh W_a^T) * (zh W_b^T)) W_2^T.
+ *   z [rows, c] in/out (in place), row-major, dtype dt; rows = T2 for the pair state (any packed [rows, c]
+ *   buffer works: no sample structure enters).  W_a, W_b [hidden, c], W_2 [c, hidden], ln_gamma, ln_beta [c]:
+ *   device pointers of dtype dt, none may be NULL.  workspace: device scratch of at least
+ *   nt_transition_workspace_bytes(...) bytes (hidden activations of a block of rows on the generic path, folded
+ *   weights on the tensor-core path); the call allocates nothing and keeps no state.
+ *   Errors: NT_ERR_INVALID_ARG (NULL pointer, non-positive width, rows < 0), NT_ERR_UNSUPPORTED (dtype),
+ *   NT_ERR_WORKSPACE, NT_ERR_CUDA; a device-side wait that runs out reports NT_ERR_TIMEOUT in *status_d (nullable).
+ */
+typedef struct { const void *ln_gamma, *ln_beta, *W_a, *W_b, *W_2; } nt_transition_weights;
+nt_status nt_pair_transition(nt_dtype dt, int32_t c, int32_t hidden, int64_t rows,
+                             const nt_transition_weights *W, float ln_eps, void *z,
+                             void *workspace, size_t workspace_bytes, int32_t *status_d, nt_stream stream);
+size_t nt_transition_workspace_bytes(nt_dtype dt, int32_t c, int32_t hidden, int64_t rows);
+
 /* ------------------------------- auxiliaries (not among the five) ------------------------------- */
 
 /* x[T1, c_s] += m[T1, c_z] W_r^T  -- the projection g of Eq. 1 line 3 applied to the reduced

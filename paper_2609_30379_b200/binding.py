@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3:
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
 EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_row_attn_pairbias",
-           "nt_segment_reduce", "nt_token_update", "nt_workspace_bytes", "nt_status_string",
+           "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
+           "nt_workspace_bytes", "nt_status_string",
            "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
 
 
@@ -51,6 +52,10 @@ class nt_attn_weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("ln_gamma", "ln_beta", "W_q", "W_k", "W_v", "W_b", "W_g", "W_o")]
 
 
+class nt_transition_weights(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("ln_gamma", "ln_beta", "W_a", "W_b", "W_2")]
+
+
 def _load() -> C.CDLL:
     path = _build.LIB_PATH
     if not os.path.exists(path):
@@ -66,6 +71,10 @@ def _load() -> C.CDLL:
                                          f32, vp, vp, sz, vp]
     lib.nt_segment_reduce.argtypes = [i32, i32, i32, i64, i64, vp, vp, vp, vp, vp]
     lib.nt_token_update.argtypes = [i32, i32, i32, i64, vp, vp, vp, vp]
+    lib.nt_pair_transition.argtypes = [i32, i32, i32, i64, C.POINTER(nt_transition_weights), f32, vp, vp, sz, vp, vp]
+    lib.nt_pair_transition.restype = i32
+    lib.nt_transition_workspace_bytes.argtypes = [i32, i32, i32, i64]
+    lib.nt_transition_workspace_bytes.restype = sz
     lib.nt_workspace_bytes.argtypes = [i32, i32, i32, vp, i32, vp]
     lib.nt_workspace_bytes.restype = sz
     lib.nt_status_string.argtypes = [i32]
@@ -201,6 +210,19 @@ def nt_segment_reduce(op: int, splits_d, v, out, status_d=None, stream=None):
     st = lib.nt_segment_reduce(dtype_code(v.dtype), op, Cc, G, rows, _ptr(splits_d), _ptr(v) if rows else None,
                                _ptr(out), _ptr(status_d), _stream(stream))
     _check(st, "nt_segment_reduce")
+
+
+def nt_transition_workspace_bytes(dtype, c: int, hidden: int, rows: int) -> int:
+    return int(lib.nt_transition_workspace_bytes(dtype_code(dtype), c, hidden, rows))
+
+
+def nt_pair_transition(W: dict, eps: float, z, workspace, status=None, stream=None):
+    """z [rows, c] in place; W holds device tensors ln_gamma, ln_beta, W_a, W_b [hidden, c], W_2 [c, hidden]."""
+    w = nt_transition_weights(*[_ptr(W[k]) for k in ("ln_gamma", "ln_beta", "W_a", "W_b", "W_2")])
+    st = lib.nt_pair_transition(dtype_code(z.dtype), int(z.shape[1]), int(W["W_a"].shape[0]), int(z.shape[0]),
+                                C.byref(w), eps, _ptr(z), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                _ptr(status), _stream(stream))
+    _check(st, "nt_pair_transition")
 
 
 def nt_token_update(m, W_r, x, stream=None):

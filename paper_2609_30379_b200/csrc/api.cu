@@ -412,6 +412,53 @@ nt_status nt_token_update(nt_dtype dt, int32_t c_s, int32_t c_z, int64_t T1, con
   return launch_proj<__nv_bfloat16>(pa, dummy, st, "token_update");
 }
 
+// rows of the hidden activation the generic transition keeps in the workspace at a time
+static const long long TRANSITION_BLOCK_ROWS = 1 << 16;
+
+size_t nt_transition_workspace_bytes(nt_dtype dt, int32_t c, int32_t hidden, int64_t rows) {
+  if (c <= 0 || hidden <= 0 || rows <= 0) return 0;
+  const size_t e = dt == NT_F32 ? 4 : 2;
+  const long long blk = rows < TRANSITION_BLOCK_ROWS ? rows : TRANSITION_BLOCK_ROWS;
+  return align_up((size_t)blk * hidden * e, 256) + (1 << 20);
+}
+
+nt_status nt_pair_transition(nt_dtype dt, int32_t c, int32_t hidden, int64_t rows, const nt_transition_weights* W,
+                             float ln_eps, void* z, void* workspace, size_t workspace_bytes, int32_t* status_d,
+                             nt_stream stream) {
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c <= 0 || hidden <= 0 || rows < 0 || !W) return NT_ERR_INVALID_ARG;
+  if (rows == 0) return NT_OK;
+  if (!W->ln_gamma || !W->ln_beta || !W->W_a || !W->W_b || !W->W_2 || !z) return NT_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < nt_transition_workspace_bytes(dt, c, hidden, rows)) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t e = dt == NT_F32 ? 4 : 2;
+  const long long blk = rows < TRANSITION_BLOCK_ROWS ? rows : TRANSITION_BLOCK_ROWS;
+  char* hbuf = (char*)workspace;
+  char* prep = hbuf + align_up((size_t)blk * hidden * e, 256);
+  if (dt == NT_BF16 && !g_force_generic && fast_transition_supported(c, hidden))
+    return fast_transition(z, W, ln_eps, c, hidden, rows, prep, status_d, st);
+  BatchMeta dummy;
+  fill_meta(dummy, nullptr, 0, 0, 0, 0, 0);
+  for (long long r0 = 0; r0 < rows; r0 += blk) {
+    const long long n = rows - r0 < blk ? rows - r0 : blk;
+    char* zr = (char*)z + (size_t)r0 * c * e;
+    ProjArgs pa{};
+    pa.A = zr; pa.a_mode = A_ROWMAJOR; pa.row0 = 0; pa.rows = n; pa.K = c;
+    pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = ln_eps;
+    pa.W1 = W->W_a; pa.W2 = W->W_b; pa.act = ACT_SILU; pa.Nout = hidden; pa.out = hbuf; pa.out_mode = O_STORE;
+    ProjArgs po{};
+    po.A = hbuf; po.a_mode = A_ROWMAJOR; po.row0 = 0; po.rows = n; po.K = hidden;
+    po.W1 = W->W_2; po.Nout = c; po.act = ACT_NONE; po.out = zr; po.out_mode = O_ACCUM;
+    nt_status r = dt == NT_F32 ? launch_proj<float>(pa, dummy, st, "generic_transition_in")
+                               : launch_proj<__nv_bfloat16>(pa, dummy, st, "generic_transition_in");
+    if (r != NT_OK) return r;
+    r = dt == NT_F32 ? launch_proj<float>(po, dummy, st, "generic_transition_out")
+                     : launch_proj<__nv_bfloat16>(po, dummy, st, "generic_transition_out");
+    if (r != NT_OK) return r;
+  }
+  return NT_OK;
+}
+
 size_t nt_workspace_bytes(nt_op op, nt_dtype dt, nt_order order, const int64_t* lengths_h, int32_t B,
                           const int32_t* dims) {
   if (B <= 0 || !lengths_h || !dims) return 0;

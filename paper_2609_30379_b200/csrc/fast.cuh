@@ -63,4 +63,10 @@ bool fast_attn_out_supported(int c, int H, int d);
 nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
                         const BatchMeta& m, int* status, cudaStream_t st);
 
+// SwiGLU transition, fused on tcgen05: z += (silu(LN(z) W_a^T) * (LN(z) W_b^T)) W_2^T with the hidden activation
+// kept on chip.  prep: at least 1 MiB of device scratch for the folded weights.
+bool fast_transition_supported(int c, int hidden);
+nt_status fast_transition(void* z, const nt_transition_weights* W, float eps, int c, int hidden, long long rows,
+                          void* prep, int* status, cudaStream_t st);
+
 }  // namespace ntp

@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(PTHREADS) proj_kernel(ProjArgs a, BatchMeta m)
       const int n = n0 + tx * 4 + j;
       if (n >= a.Nout) continue;
       float v = acc1[i][j];
-      if (W2) v = sigmoidf_acc(v) * acc2[i][j];
+      if (W2) v = (a.act == ACT_SILU ? v * sigmoidf_acc(v) : sigmoidf_acc(v)) * acc2[i][j];
       else if (a.act == ACT_SIGMOID) v = sigmoidf_acc(v);
       if (gO) v *= Cvt<T>::ld(gO + p * a.Nout + n);
       if (a.out_mode == O_CHANNEL_MAJOR) {

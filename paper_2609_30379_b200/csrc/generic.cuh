@@ -7,7 +7,7 @@ namespace ntp {
 
 enum AMode { A_ROWMAJOR = 0, A_CHANNEL_MAJOR = 1 };
 enum OutMode { O_STORE = 0, O_ACCUM = 1, O_CHANNEL_MAJOR = 2 };
-enum Act { ACT_NONE = 0, ACT_SIGMOID = 1 };
+enum Act { ACT_NONE = 0, ACT_SIGMOID = 1, ACT_SILU = 2 };   // with W2: gate activation (0 / 1: sigmoid, 2: SiLU)
 
 // out = epilogue( prologue(A) W^T ) over the packed rows [row0, row0 + rows)
 struct ProjArgs {
@@ -20,9 +20,9 @@ struct ProjArgs {
   const void* ln_b;
   float eps;
   const void* W1;       // [Nout, K]
-  const void* W2;       // nullable: value = sigmoid(A W1^T) * (A W2^T)
+  const void* W2;       // nullable: value = gate(A W1^T) * (A W2^T), gate = sigmoid unless act == ACT_SILU
   int Nout;
-  int act;              // used when W2 == NULL
+  int act;              // activation (W2 == NULL) or gate kind (W2 != NULL)
   void* out;
   int out_mode;         // O_STORE / O_ACCUM: row-major [.., Nout]; O_CHANNEL_MAJOR: pair layout, Nout channels
   const void* gateO;    // nullable: row-major [.., Nout]; value *= gateO before store/accumulate
