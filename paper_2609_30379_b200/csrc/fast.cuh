@@ -65,6 +65,8 @@ nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep&
 
 // SwiGLU transition, fused on tcgen05: z += (silu(LN(z) W_a^T) * (LN(z) W_b^T)) W_2^T with the hidden activation
 // kept on chip.  prep: at least 1 MiB of device scratch for the folded weights.
+struct TransPrep { void *w1, *c01, *aug; int rows; };   // folded [W_a / 2; W_b] (2 hidden rows), their (c0, c1), augmentation columns
+nt_status fast_transition_prep(const nt_transition_weights* W, int c, int hidden, void* prep, TransPrep& out, cudaStream_t st);
 bool fast_transition_supported(int c, int hidden);
 nt_status fast_transition(void* z, const nt_transition_weights* W, float eps, int c, int hidden, long long rows,
                           void* prep, int* status, cudaStream_t st);

@@ -147,4 +147,22 @@ nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* pr
   return run_prep(a, st);
 }
 
+// Transition: [W_a (times 1/2: the gate goes through tanh); W_b] folded with LN (K = c).
+nt_status fast_transition_prep(const nt_transition_weights* W, int c, int hidden, void* prep, TransPrep& out, cudaStream_t st) {
+  const int rows = 2 * hidden;
+  char* p = (char*)prep;
+  out.w1 = p;
+  p += align_up((size_t)rows * c * 2, 256);
+  out.c01 = p;
+  p += align_up((size_t)rows * sizeof(float2), 256);
+  out.aug = p;                          // [2][rows][8] fp16
+  out.rows = rows;
+  PrepArgs a{};
+  const void* s0[2] = {W->W_a, W->W_b};
+  const int r0[2] = {hidden, hidden};
+  const float sc[2] = {0.5f, 1.0f};
+  add_job(a, s0, r0, 2, c, W->ln_gamma, W->ln_beta, out.w1, out.c01, sc, out.aug);
+  return run_prep(a, st);
+}
+
 }  // namespace ntp
