@@ -77,6 +77,8 @@ def kernel_work(cfg: wl.Config):
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
     w["token_update"] = dict(bytes=T1 * (c_z + 2 * c_s) * e + c_s * c_z * e, flops=2 * T1 * c_s * c_z)
+    # SwiGLU pair transition with expansion 4: read and write the state once, three GEMMs of c_z x 4 c_z per row
+    w["transition"] = w["generic_transition"] = dict(bytes=2 * T2 * c_z * e, flops=6 * T2 * c_z * 4 * c_z)
     return w
 
 
@@ -237,6 +239,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
+    ap.add_argument("--only-transition", action="store_true",
+                    help="run just the pair-transition measurement (the row after the block; for ncu captures)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-kernel timing pass, the end-to-end pass and the CPU baseline (for ncu captures)")
     args = ap.parse_args()
@@ -277,6 +281,40 @@ def main():
     def step():
         x.copy_(x0)
         return stack.forward(x)
+
+    def transition_pass(n_calls):
+        """The row after the block: nt_pair_transition on a state of the bench workload's shape (expansion 4).
+        Not part of the step or of `value`; timed per launch on the launching stream."""
+        if cfg.kind != "pair":
+            return None
+        Wt = {k: torch.from_numpy(np.ascontiguousarray(v)).to("cuda", stack.dtype)
+              for k, v in wl.make_transition_weights(cfg).items()}
+        zt = torch.randn((cfg.T2, cfg.c_z), device="cuda").to(stack.dtype)
+        hidden = 4 * cfg.c_z
+        ws = torch.empty(nt.nt_transition_workspace_bytes(stack.dtype, cfg.c_z, hidden, cfg.T2), dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            nt.nt_pair_transition(Wt, 1e-5, zt, ws)
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            nt.nt_pair_transition(Wt, 1e-5, zt, ws)
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        out = {}
+        for k, v in tp.items():
+            r = roofline_entry(k, v[0], v[1], n_calls, kernel_work(cfg), peaks_t, kind_t)
+            out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        return dict(rows=cfg.T2, c=cfg.c_z, hidden=hidden, calls=n_calls, kernels=out,
+                    note="state rewritten in place call after call (values drift; timing only)")
+
+    if args.only_transition:
+        res = transition_pass(steps)
+        if rank == 0:
+            print(json.dumps(dict(pair_transition=res)))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     def barrier():
         torch.cuda.synchronize()
@@ -339,6 +377,8 @@ def main():
     if roofline and cfg.name == "cfg2" and not args.force_generic:
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
+    next_rows = dict(pair_transition=transition_pass(steps)) if not args.force_generic else None
+
     # ---- end to end through the public API with host buffers
     x_pin = torch.from_numpy(np.ascontiguousarray(inp["x"])).to(stack.dtype).pin_memory()
     out_pin = torch.empty_like(x_pin).pin_memory()
@@ -388,7 +428,7 @@ def main():
                     kernels_path="generic" if args.force_generic else "default"),
         tokens_per_s=world * cfg.blocks * cfg.T1 * steps / (ms * 1e-3),
         peak_alloc_bytes=peak_alloc, padded_envelope_z_bytes=cfg.B * nmax * nmax * cfg.c_z * esz,
-        gpu_launches=launches, clocks=clocks, roofline=roofline, kernels=kernels, cpu_baseline=cpu,
+        gpu_launches=launches, clocks=clocks, roofline=roofline, kernels=kernels, next_rows=next_rows, cpu_baseline=cpu,
         e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                  note="host pinned tokens + lengths in, offsets rebuilt, updated tokens out; wall clock"),
     )
