@@ -17,6 +17,9 @@ What each function follows:
                        LayerNorm on the static tail (Sec. 3.3).  No activation at construction (App. A.1).
   tri_mul_out          Sec. 4.3 names the triangle multiplicative update of the Pairformer block;
                        its internals are the standard gated outgoing form (a reading; see below).
+  tri_mul_in           the second direction of the same update (contraction over the first index); pinned by a
+                       triple loop, torch einsum, and its relations to the outgoing form (transposed state, symmetric
+                       state, a == b).
   row_attn_pairbias    Sec. 3.3 "Attention through packed blocks" (segments from cumulative lengths;
                        output adopts the query structure) and Sec. 4.3 (triangle attention with a
                        pair bias); internals are a reading (see below).
@@ -176,6 +179,32 @@ def tri_mul_out(z, lengths, W, eps=LN_EPS, dtype=np.float64, return_parts=False)
     return (res, parts) if return_parts else res
 
 
+def tri_mul_in(z, lengths, W, eps=LN_EPS, dtype=np.float64, return_parts=False):
+    """Incoming triangle multiplicative update with residual, per sample (Sec. 4.3 names the triangle
+    multiplication of the Pairformer block; this is its second direction).  Same projections, gate, output
+    normalisation and residual as the outgoing update; only the contraction runs over the FIRST index:
+        t[i,j,c] = sum_k a[k,i,c] b[k,j,c]
+    """
+    z = np.asarray(z, dtype=dtype)
+    Wd = {k: np.asarray(v, dtype=dtype) for k, v in W.items()}
+    out, parts, o = [], [], 0
+    for n in (int(v) for v in lengths):
+        zs = z[o:o + n * n].reshape(n, n, z.shape[1])
+        zh = layer_norm(zs, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)
+        a = sigmoid(zh @ Wd["W_ag"].T) * (zh @ Wd["W_ap"].T)
+        b = sigmoid(zh @ Wd["W_bg"].T) * (zh @ Wd["W_bp"].T)
+        g = sigmoid(zh @ Wd["W_g"].T)
+        # per channel c the contraction is the matrix product A_c^T B_c (a batched matmul serves as the step)
+        t = np.matmul(a.transpose(2, 1, 0), b.transpose(2, 0, 1)).transpose(1, 2, 0)
+        upd = g * (layer_norm(t, Wd["ln_out_gamma"], Wd["ln_out_beta"], eps) @ Wd["W_o"].T)
+        out.append((zs + upd).reshape(n * n, z.shape[1]))
+        if return_parts:
+            parts.append(dict(a=a, b=b, g=g, t=t))
+        o += n * n
+    res = np.concatenate(out, axis=0) if out else z.copy()
+    return (res, parts) if return_parts else res
+
+
 def row_attn_pairbias(zx, lengths, W, H, d, eps=LN_EPS, order="pair", dtype=np.float64, return_parts=False):
     """Row-wise pair-biased softmax attention with residual.
 
@@ -280,6 +309,24 @@ def tri_mul_out_at(zs, W, positions, eps=LN_EPS, dtype=np.float64):
         t = (a_i * b_j).sum(axis=0)
         g = sigmoid(zi[j] @ Wd["W_g"].T)
         out.append(ri[j] + g * (layer_norm(t, Wd["ln_out_gamma"], Wd["ln_out_beta"], eps) @ Wd["W_o"].T))
+    return np.stack(out)
+
+
+def tri_mul_in_at(zs, W, positions, eps=LN_EPS, dtype=np.float64):
+    """Incoming triangle update of one sample at the listed (i, j).  ``zs`` is the sample's [n, n, c_z]
+    state (anything indexable as zs[:, i]): only columns i and j enter t[i,j,:] = sum_k a[k,i,:] b[k,j,:]."""
+    Wd = {k: np.asarray(v, dtype=dtype) for k, v in W.items()}
+    out = []
+    for (i, j) in positions:
+        ci, cj = np.asarray(zs[:, i], dtype=dtype), np.asarray(zs[:, j], dtype=dtype)   # [n, c_z] each
+        zi = layer_norm(ci, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)
+        zj = layer_norm(cj, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps)
+        a_i = sigmoid(zi @ Wd["W_ag"].T) * (zi @ Wd["W_ap"].T)               # a[k, i, :]
+        b_j = sigmoid(zj @ Wd["W_bg"].T) * (zj @ Wd["W_bp"].T)               # b[k, j, :]
+        t = (a_i * b_j).sum(axis=0)
+        zij = cj[i]                                                          # z[i, j]
+        g = sigmoid(layer_norm(zij, Wd["ln_in_gamma"], Wd["ln_in_beta"], eps) @ Wd["W_g"].T)
+        out.append(zij + g * (layer_norm(t, Wd["ln_out_gamma"], Wd["ln_out_beta"], eps) @ Wd["W_o"].T))
     return np.stack(out)
 
 

@@ -202,6 +202,91 @@ def test_trimul_full_formula_via_torch():
     assert np.allclose(got, ref, rtol=1e-11, atol=1e-11)
 
 
+def _pair_transpose(z, lengths):
+    """Packed state with every sample's (i, j) axes swapped."""
+    out, o = [], 0
+    for n in lengths:
+        out.append(z[o:o + n * n].reshape(n, n, -1).transpose(1, 0, 2).reshape(n * n, -1))
+        o += n * n
+    return np.concatenate(out, axis=0)
+
+
+def test_trimul_incoming_contraction_bruteforce():
+    cfg, inp = tiny_inputs((3, 5, 2))
+    rng = np.random.default_rng(13)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    W = inp["blocks"][0]["trimul"]
+    znew, parts = orc.tri_mul_in(z, cfg.lengths, W, return_parts=True)
+    _, parts_out = orc.tri_mul_out(z, cfg.lengths, W, return_parts=True)
+    o = 0
+    for n, p, po in zip(cfg.lengths, parts, parts_out):
+        a, b, t = p["a"], p["b"], p["t"]
+        assert np.array_equal(a, po["a"]) and np.array_equal(b, po["b"]) and np.array_equal(p["g"], po["g"])   # same projections
+        ref = np.zeros_like(t)
+        for i in range(n):
+            for j in range(n):
+                for k in range(n):
+                    ref[i, j, :] += a[k, i, :] * b[k, j, :]
+        assert np.allclose(t, ref, rtol=1e-12, atol=1e-12)
+        for c in range(cfg.c_h):                               # per channel: a library matmul A_c^T B_c
+            assert np.allclose(t[:, :, c], a[:, :, c].T @ b[:, :, c], rtol=1e-12, atol=1e-12)
+        assert not np.allclose(t, po["t"])                     # and it is not the outgoing contraction
+        # the update itself, position by position, from the brute-force t
+        zs = z[o:o + n * n].reshape(n, n, -1)
+        lnt = orc.layer_norm(ref, W["ln_out_gamma"], W["ln_out_beta"])
+        want = zs + p["g"] * (lnt @ np.asarray(W["W_o"], dtype=np.float64).T)
+        assert np.allclose(znew[o:o + n * n].reshape(n, n, -1), want, rtol=1e-11, atol=1e-11)
+        o += n * n
+    W0 = dict(W, W_o=np.zeros_like(W["W_o"]))
+    assert np.array_equal(orc.tri_mul_in(z, cfg.lengths, W0), z)
+
+
+def test_trimul_incoming_full_formula_via_torch():
+    cfg, inp = tiny_inputs((6,))
+    rng = np.random.default_rng(14)
+    z = rng.standard_normal((36, cfg.c_z))
+    W = {k: torch.from_numpy(np.asarray(v, dtype=np.float64)) for k, v in inp["blocks"][0]["trimul"].items()}
+    zt = torch.from_numpy(z).reshape(6, 6, -1)
+    F = torch.nn.functional
+    zh = F.layer_norm(zt, (cfg.c_z,), W["ln_in_gamma"], W["ln_in_beta"], 1e-5)
+    a = torch.sigmoid(F.linear(zh, W["W_ag"])) * F.linear(zh, W["W_ap"])
+    b = torch.sigmoid(F.linear(zh, W["W_bg"])) * F.linear(zh, W["W_bp"])
+    t = torch.einsum("kic,kjc->ijc", a, b)
+    upd = torch.sigmoid(F.linear(zh, W["W_g"])) * F.linear(F.layer_norm(t, (cfg.c_h,), W["ln_out_gamma"], W["ln_out_beta"], 1e-5), W["W_o"])
+    ref = (zt + upd).reshape(36, -1).numpy()
+    got = orc.tri_mul_in(z, cfg.lengths, inp["blocks"][0]["trimul"])
+    assert np.allclose(got, ref, rtol=1e-11, atol=1e-11)
+
+
+def test_trimul_incoming_relations_to_outgoing():
+    cfg, inp = tiny_inputs((4, 1, 6))
+    rng = np.random.default_rng(15)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    W = inp["blocks"][0]["trimul"]
+    zT = _pair_transpose(z, cfg.lengths)
+    # the incoming contraction of a state is the outgoing contraction of the transposed state
+    _, p_in = orc.tri_mul_in(z, cfg.lengths, W, return_parts=True)
+    _, p_out = orc.tri_mul_out(zT, cfg.lengths, W, return_parts=True)
+    for a, b in zip(p_in, p_out):
+        assert np.allclose(a["t"], b["t"], rtol=1e-12, atol=1e-12)
+    # on a symmetric state a[k,i] = a[i,k]: the two directions give the same update
+    zsym = 0.5 * (z + zT)
+    assert np.allclose(orc.tri_mul_in(zsym, cfg.lengths, W), orc.tri_mul_out(zsym, cfg.lengths, W), rtol=1e-11, atol=1e-11)
+    # with a == b the contraction is symmetric in (i, j), and then incoming(z) is the transpose of outgoing(z^T)
+    Ws = dict(W, W_bp=W["W_ap"], W_bg=W["W_ag"])
+    lhs = orc.tri_mul_in(z, cfg.lengths, Ws)
+    rhs = _pair_transpose(orc.tri_mul_out(zT, cfg.lengths, Ws), cfg.lengths)
+    assert np.allclose(lhs, rhs, rtol=1e-11, atol=1e-11)
+    # sampled evaluator equals the full function
+    n = cfg.lengths[2]
+    o = sum(m * m for m in cfg.lengths[:2])
+    zs = z[o:o + n * n].reshape(n, n, -1)
+    pos = [(0, 0), (3, 5), (5, 1), (2, 2)]
+    full = orc.tri_mul_in(zs.reshape(n * n, -1), (n,), W).reshape(n, n, -1)
+    got = orc.tri_mul_in_at(zs, W, pos)
+    assert np.allclose(got, np.stack([full[i, j] for i, j in pos]), rtol=1e-12, atol=1e-12)
+
+
 # ------------------------------------------------------------------ attention
 def test_attention_matches_library_sdpa():
     cfg, inp = tiny_inputs((4, 7, 1))
