@@ -65,6 +65,7 @@ def kernel_work(cfg: wl.Config):
     w["generic_tri_in_g"] = dict(bytes=2 * T2 * c_z * e, flops=2 * T2 * c_z * c_z)
     w["tri_in"] = dict(bytes=T2 * (c_z + 2 * c_h) * e, flops=2 * T2 * c_z * 4 * c_h)
     w["generic_tri_contract"] = w["tri_contract"] = dict(bytes=3 * T2 * c_h * e, flops=2 * N3 * c_h)
+    w["generic_tri_contract_in"] = w["tri_contract_in"] = w["tri_contract"]      # incoming direction: same work
     w["generic_tri_out"] = dict(bytes=T2 * (c_h + 3 * c_z) * e, flops=2 * T2 * c_h * c_z)
     w["tri_out"] = dict(bytes=T2 * (c_h + 2 * c_z) * e, flops=2 * T2 * (c_h + c_z) * c_z)
     for n in ("q", "k", "v", "g"):
@@ -241,6 +242,8 @@ def main():
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
     ap.add_argument("--only-transition", action="store_true",
                     help="run just the pair-transition measurement (the row after the block; for ncu captures)")
+    ap.add_argument("--only-tri-mul-in", action="store_true",
+                    help="run just the incoming-triangle-update measurement (for ncu captures)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-kernel timing pass, the end-to-end pass and the CPU baseline (for ncu captures)")
     args = ap.parse_args()
@@ -308,10 +311,33 @@ def main():
         return dict(rows=cfg.T2, c=cfg.c_z, hidden=hidden, calls=n_calls, kernels=out,
                     note="state rewritten in place call after call (values drift; timing only)")
 
-    if args.only_transition:
-        res = transition_pass(steps)
+    def tri_mul_in_pass(n_calls):
+        """The incoming direction of the triangle update (a row after the block) on the bench workload: the state the
+        first block's broadcast produces, nt_tri_mul_in timed per launch.  Not part of the step or of `value`."""
+        if cfg.kind != "pair":
+            return None
+        w0 = stack.W[0]
+        b = w0["broadcast"]
+        nt.nt_pair_broadcast(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        for _ in range(3):
+            nt.nt_tri_mul_in(stack.L, w0["trimul"], 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            nt.nt_tri_mul_in(stack.L, w0["trimul"], 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        out = {}
+        for k, v in tp.items():
+            r = roofline_entry(k, v[0], v[1], n_calls, kernel_work(cfg), peaks_t, kind_t)
+            out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
+
+    if args.only_transition or args.only_tri_mul_in:
+        res = dict(pair_transition=transition_pass(steps)) if args.only_transition else dict(tri_mul_in=tri_mul_in_pass(steps))
         if rank == 0:
-            print(json.dumps(dict(pair_transition=res)))
+            print(json.dumps(res))
         if world > 1:
             dist.destroy_process_group()
         return
@@ -377,7 +403,7 @@ def main():
     if roofline and cfg.name == "cfg2" and not args.force_generic:
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
-    next_rows = dict(pair_transition=transition_pass(steps)) if not args.force_generic else None
+    next_rows = dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps)) if not args.force_generic else None
 
     # ---- end to end through the public API with host buffers
     x_pin = torch.from_numpy(np.ascontiguousarray(inp["x"])).to(stack.dtype).pin_memory()

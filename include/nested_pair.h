@@ -127,6 +127,17 @@ nt_status nt_tri_mul_out(const nt_layout *L, nt_dtype dt, int32_t c_z, int32_t c
                          void *workspace, size_t workspace_bytes, nt_stream stream);
 
 /*
+ * nt_tri_mul_in -- incoming triangle multiplicative update: the second direction of the block's triangle
+ * multiplication (Sec. 4.3).  Same projections, gate, output normalisation, residual, weights, workspace and
+ * error behaviour as nt_tri_mul_out; only the contraction runs over the FIRST pair index:
+ *   t_s[i,j,c] = sum_k a_s[k,i,c] b_s[k,j,c];   z += g * (LN_out(t) W_o^T)      (in place)
+ *   z [T2, c_z] in/out.  Workspace size: nt_workspace_bytes (the same as for nt_tri_mul_out).
+ */
+nt_status nt_tri_mul_in(const nt_layout *L, nt_dtype dt, int32_t c_z, int32_t c_h,
+                         const nt_trimul_weights *W, float ln_eps, void *z,
+                         void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
  * nt_row_attn_pairbias -- row-wise pair-biased softmax attention over ragged N_s (Sec. 3.3
  * "Attention through packed blocks": segments from the offsets, output adopts the query
  * structure; Sec. 4.3 triangle attention, starting node).

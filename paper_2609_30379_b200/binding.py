@@ -25,8 +25,8 @@ NT_OP_PAIR_BROADCAST, NT_OP_TRI_MUL_OUT, NT_OP_ROW_ATTN, NT_OP_BLOCK = 0, 1, 2, 
 STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3: "NT_ERR_WORKSPACE",
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
-EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_row_attn_pairbias",
-           "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
+EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
+           "nt_row_attn_pairbias", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
            "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
 
@@ -67,6 +67,7 @@ def _load() -> C.CDLL:
     lib.nt_pair_broadcast.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp, sz, vp]
     lib.nt_pair_broadcast_static.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.nt_tri_mul_out.argtypes = [C.POINTER(nt_layout), i32, i32, i32, C.POINTER(nt_trimul_weights), f32, vp, vp, sz, vp]
+    lib.nt_tri_mul_in.argtypes = lib.nt_tri_mul_out.argtypes
     lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
                                          f32, vp, vp, sz, vp]
     lib.nt_segment_reduce.argtypes = [i32, i32, i32, i64, i64, vp, vp, vp, vp, vp]
@@ -87,8 +88,8 @@ def _load() -> C.CDLL:
     lib.nt_profile_begin.restype = i32
     lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
     lib.nt_profile_end.restype = i32
-    for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_row_attn_pairbias",
-                 "nt_segment_reduce", "nt_token_update"):
+    for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
+                 "nt_row_attn_pairbias", "nt_segment_reduce", "nt_token_update"):
         getattr(lib, name).restype = i32
     return lib
 
@@ -194,6 +195,15 @@ def nt_tri_mul_out(L: Layout, W: dict, ln_eps, z, workspace, stream=None):
     st = lib.nt_tri_mul_out(C.byref(L.c), dtype_code(z.dtype), c_z, c_h, C.byref(w), float(ln_eps), _ptr(z),
                             _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "nt_tri_mul_out")
+
+
+def nt_tri_mul_in(L: Layout, W: dict, ln_eps, z, workspace, stream=None):
+    """Incoming direction of the triangle update; same arguments and workspace as nt_tri_mul_out."""
+    c_h, c_z = int(W["W_ap"].shape[0]), int(W["W_ap"].shape[1])
+    w = nt_trimul_weights(*[_ptr(W[n]) for n, _ in nt_trimul_weights._fields_])
+    st = lib.nt_tri_mul_in(C.byref(L.c), dtype_code(z.dtype), c_z, c_h, C.byref(w), float(ln_eps), _ptr(z),
+                           _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_tri_mul_in")
 
 
 def nt_row_attn_pairbias(L: Layout, order: int, W: dict, H: int, d: int, ln_eps, zx, workspace, stream=None):

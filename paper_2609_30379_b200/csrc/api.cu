@@ -186,7 +186,7 @@ static nt_status pair_broadcast_impl(const nt_layout* L, const Totals& tot, int 
 
 template <typename T>
 static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z, int c_h, const nt_trimul_weights* W,
-                                 float eps, void* z, void* ws, nt_dtype dt, cudaStream_t st) {
+                                 float eps, void* z, void* ws, nt_dtype dt, cudaStream_t st, bool incoming) {
   TriWs w = carve_trimul(ws, dt, tot, c_z, c_h);
   // The tensor-core stages exchange a, b (fp16) and t (fp16, scaled by 1 / N): all three or none.
   // (the tensor-core kernels index positions inside a sample with 32 bits: N below 2^16)
@@ -224,9 +224,9 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
       if (r != NT_OK) return r;
     }
     if (tc && fast_contract_supported(c_h))
-      r = fast_contract(w.a, (size_t)((char*)w.b - (char*)w.a), c_h, m, L->status_d, st);
+      r = fast_contract(w.a, (size_t)((char*)w.b - (char*)w.a), c_h, m, L->status_d, st, incoming);
     else
-      r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st);
+      r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st, incoming);
     if (r != NT_OK) return r;
     if (tc_out) {
       r = fast_tri_out(z, w.t, tprep, eps, c_z, c_h, m, L->status_d, st);
@@ -337,8 +337,9 @@ nt_status nt_pair_broadcast(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_
                                             fast);
 }
 
-nt_status nt_tri_mul_out(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,
-                         float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+static nt_status tri_mul_entry(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,
+                               float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream,
+                               bool incoming) {
   Totals tot;
   nt_status r = check_layout(L, tot);
   if (r != NT_OK) return r;
@@ -351,8 +352,18 @@ nt_status nt_tri_mul_out(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c
   if (!z || !workspace || !aligned16(z) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
   if (workspace_bytes < carve_trimul(nullptr, dt, tot, c_z, c_h).bytes) return NT_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
-  if (dt == NT_F32) return tri_mul_generic<float>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st);
-  return tri_mul_generic<__nv_bfloat16>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st);
+  if (dt == NT_F32) return tri_mul_generic<float>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st, incoming);
+  return tri_mul_generic<__nv_bfloat16>(L, tot, c_z, c_h, W, ln_eps, z, workspace, dt, st, incoming);
+}
+
+nt_status nt_tri_mul_out(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,
+                         float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+  return tri_mul_entry(L, dt, c_z, c_h, W, ln_eps, z, workspace, workspace_bytes, stream, false);
+}
+
+nt_status nt_tri_mul_in(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,
+                        float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+  return tri_mul_entry(L, dt, c_z, c_h, W, ln_eps, z, workspace, workspace_bytes, stream, true);
 }
 
 nt_status nt_row_attn_pairbias(const nt_layout* L, nt_order order, nt_dtype dt, int32_t c, int32_t H, int32_t d,

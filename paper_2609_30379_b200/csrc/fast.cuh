@@ -31,10 +31,10 @@ nt_status fast_attn_core_tc(const void* q, const void* k, const void* v, const v
                             const BatchMeta& m, int n_max, int* status, cudaStream_t st);
 
 // triangle contraction on tcgen05: a, b, t are three equally spaced channel-major buffers
-// (b = a + stride, t = a + 2 * stride)
+// (b = a + stride, t = a + 2 * stride); incoming = contraction over the first index (sum_k a[k][i] b[k][j])
 bool fast_contract_supported(int C);
 nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
-                        cudaStream_t st);
+                        cudaStream_t st, bool incoming = false);
 
 // ---- tensor-core projections (tcgen05, LayerNorm folded into fp16 weights prepared once per call)
 struct TriPrep { void *w1, *c01_1, *wg, *c01g, *wo, *c01o, *aug1, *augo; int aug1_rows; };

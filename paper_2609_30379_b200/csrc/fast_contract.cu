@@ -10,6 +10,12 @@
 //            swizzled staging tile -> TMA store into t
 // One 4-D tensor map per sample {k, i, channel, which of a/b/t} serves loads and stores; rows and
 // columns past N are zero-filled on load and clipped on store, so no padded tile is ever moved.
+//
+// Incoming direction (IN = true): t[c][i][j] = sum_k a[c][k][i] b[c][k][j].  The contraction index is now the ROW
+// of the channel-major matrices and i / j are contiguous, so both operands are MN-major: a stage holds boxes of
+// {64 contiguous i (or j), 64 rows k} (8 KB each: 8-row groups are the 1024-byte swizzle atoms, the next 64
+// columns live one box further), a K step of 16 rows advances the start address by two atoms, and the same
+// box shape stores t in two halves per 64-column panel.  Everything else is shared.
 #include <cstring>
 
 #include "fast.cuh"
@@ -49,6 +55,7 @@ __device__ inline void contract_decode(const ContractParams& p, long long job, i
   Nt = left >= 256 ? 256 : ((left + 15) & ~15);
 }
 
+template <bool IN>
 __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __grid_constant__ ContractParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[2 * CT_STAGES + 4];
@@ -89,10 +96,18 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
         mbar_wait(&empty[stage], phase ^ 1, ab);
         unsigned char* As = smem + stage * CT_STAGE_BYTES;
         unsigned char* Bs = As + CT_A_BYTES;
-        mbar_expect_tx(&full[stage], CT_A_BYTES + (Nt > 128 ? CT_B_BYTES : CT_B_BYTES / 2));
-        tma_load_4d(As, map, &full[stage], kc * 64, i0, c, 0);
-        tma_load_4d(Bs, map, &full[stage], kc * 64, j0, c, 1);
-        if (Nt > 128) tma_load_4d(Bs + CT_B_BYTES / 2, map, &full[stage], kc * 64, j0 + 128, c, 1);
+        if (IN) {
+          const int nb = (Nt + 63) / 64;                 // 64-column boxes of b
+          mbar_expect_tx(&full[stage], CT_A_BYTES + nb * 8192);
+          tma_load_4d(As, map, &full[stage], i0, kc * 64, c, 0);
+          tma_load_4d(As + 8192, map, &full[stage], i0 + 64, kc * 64, c, 0);
+          for (int h = 0; h < nb; ++h) tma_load_4d(Bs + h * 8192, map, &full[stage], j0 + h * 64, kc * 64, c, 1);
+        } else {
+          mbar_expect_tx(&full[stage], CT_A_BYTES + (Nt > 128 ? CT_B_BYTES : CT_B_BYTES / 2));
+          tma_load_4d(As, map, &full[stage], kc * 64, i0, c, 0);
+          tma_load_4d(Bs, map, &full[stage], kc * 64, j0, c, 1);
+          if (Nt > 128) tma_load_4d(Bs + CT_B_BYTES / 2, map, &full[stage], kc * 64, j0 + 128, c, 1);
+        }
         if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
       }
     }
@@ -110,17 +125,19 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
       else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
       tc_fence_after();
-      const unsigned idesc = idesc_f16(128, Nt, 0, 0, FMT_F16, FMT_F16);   // a, b are fp16
+      const unsigned idesc = idesc_f16(128, Nt, IN ? 1 : 0, IN ? 1 : 0, FMT_F16, FMT_F16);   // a, b are fp16
       const unsigned d_tmem = tmem_base + buf * 256;
       for (int kc = 0; kc < nkc; ++kc) {
         mbar_wait(&full[stage], phase, ab);
         tc_fence_after();
         const unsigned a_addr = smem_u32(smem + stage * CT_STAGE_BYTES);
-        const unsigned long long a_desc = desc_kmajor_sw128(a_addr), b_desc = desc_kmajor_sw128(a_addr + CT_A_BYTES);
+        const unsigned long long a_desc = IN ? desc_mnmajor_sw128(a_addr, 8192, 1024) : desc_kmajor_sw128(a_addr);
+        const unsigned long long b_desc = IN ? desc_mnmajor_sw128(a_addr + CT_A_BYTES, 8192, 1024) : desc_kmajor_sw128(a_addr + CT_A_BYTES);
         const int ksteps = min(4, (N - kc * 64 + 15) / 16);
+        constexpr int KADV = IN ? 128 : 2;       // 16 further k: two 1024-byte atoms (MN-major) or 32 bytes (K-major)
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4)
-          if (k4 < ksteps && elect_one()) umma_bf16(d_tmem, a_desc + k4 * 2, b_desc + k4 * 2, idesc, (kc | k4) != 0);
+          if (k4 < ksteps && elect_one()) umma_bf16(d_tmem, a_desc + k4 * KADV, b_desc + k4 * KADV, idesc, (kc | k4) != 0);
         if (elect_one()) tc_commit(&empty[stage]);
         __syncwarp();
         if (++stage == CT_STAGES) { stage = 0; phase ^= 1; }
@@ -186,8 +203,10 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
       fence_proxy_async_smem();
       named_bar_sync(1, 256);
       if (ep_tid == 0) {
-        for (int cg = 0; cg < ncg; ++cg)
+        for (int cg = 0; cg < ncg; ++cg) {
           tma_store_4d(&p.maps[s], staging + cg * CT_A_BYTES, j0 + cg * 64, i0, c, 2);
+          if (IN && i0 + 64 < p.N[s]) tma_store_4d(&p.maps[s], staging + cg * CT_A_BYTES + 8192, j0 + cg * 64, i0 + 64, c, 2);   // box of 64 rows
+        }
         tma_store_commit();
       }
     }
@@ -202,10 +221,11 @@ __global__ void __launch_bounds__(CT_THREADS, 1) tri_contract_kernel(const __gri
 bool fast_contract_supported(int C) { return C >= 1; }
 
 nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const BatchMeta& m, int* status,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool incoming) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(tri_contract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, CT_SMEM) != cudaSuccess)
+    if (cudaFuncSetAttribute(tri_contract_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, CT_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(tri_contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, CT_SMEM) != cudaSuccess)
       return cuda_fail("shared memory attribute");
     attr_set = true;
   }
@@ -225,7 +245,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
         const unsigned long long dims[4] = {(unsigned long long)N, (unsigned long long)N, (unsigned long long)C, 3};
         const unsigned long long strides[3] = {(unsigned long long)ld * 2, (unsigned long long)N * ld * 2,
                                                (unsigned long long)buf_stride_bytes};
-        const unsigned box[4] = {64, 128, 1, 1};
+        const unsigned box[4] = {64, incoming ? 64u : 128u, 1, 1};
         const char* base = (const char*)a + (size_t)C * m.cm_off[g0 + l] * 2;
         if (!make_tmap_bf16(&p.maps[l], base, 4, dims, strides, box)) { fprintf(stderr, "libnested_pair: tensor map encode failed (%s:%d)\n", __FILE__, __LINE__); return NT_ERR_CUDA; }
       } else {
@@ -236,8 +256,9 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
     if (njobs == 0) continue;
     const unsigned grid = (unsigned)(njobs < 148 ? njobs : 148);
     {
-      LaunchScope ls("tri_contract", st);
-      tri_contract_kernel<<<grid, CT_THREADS, CT_SMEM, st>>>(p);
+      LaunchScope ls(incoming ? "tri_contract_in" : "tri_contract", st);
+      if (incoming) tri_contract_kernel<true><<<grid, CT_THREADS, CT_SMEM, st>>>(p);
+      else tri_contract_kernel<false><<<grid, CT_THREADS, CT_SMEM, st>>>(p);
     }
     if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("tensor-core kernel launch");
   }

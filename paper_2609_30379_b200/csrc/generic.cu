@@ -169,13 +169,14 @@ template nt_status launch_proj<float>(const ProjArgs&, const BatchMeta&, cudaStr
 template nt_status launch_proj<__nv_bfloat16>(const ProjArgs&, const BatchMeta&, cudaStream_t, const char*);
 
 // ------------------------------------------------------------------------------------------
-// triangle contraction  t[c][i][j] = sum_k a[c][i][k] b[c][j][k]
+// triangle contraction  t[c][i][j] = sum_k a[c][i][k] b[c][j][k]   (outgoing)
+//                       t[c][i][j] = sum_k a[c][k][i] b[c][k][j]   (incoming)
 // ------------------------------------------------------------------------------------------
 constexpr int CT = 64, CK = 16;
 
 template <typename T>
 __global__ void __launch_bounds__(256) contract_kernel(const T* __restrict__ a, const T* __restrict__ b,
-                                                      T* __restrict__ tout, int C, BatchMeta m) {
+                                                      T* __restrict__ tout, int C, BatchMeta m, int incoming) {
   __shared__ __align__(16) float As[CK][CT + 4];
   __shared__ __align__(16) float Bs[CK][CT + 4];
   long long w = blockIdx.x;
@@ -201,8 +202,10 @@ __global__ void __launch_bounds__(256) contract_kernel(const T* __restrict__ a, 
     for (int u = 0; u < 4; ++u) {
       const int rl = t >> 2, kk = (t & 3) * 4 + u, k = k0 + kk;
       const int i = i0 + rl, j = j0 + rl;
-      As[kk][rl] = (i < N && k < N) ? Cvt<T>::ld(Ap + (long long)i * ld + k) : 0.f;
-      Bs[kk][rl] = (j < N && k < N) ? Cvt<T>::ld(Bp + (long long)j * ld + k) : 0.f;
+      const long long ia = incoming ? (long long)k * ld + i : (long long)i * ld + k;
+      const long long ib = incoming ? (long long)k * ld + j : (long long)j * ld + k;
+      As[kk][rl] = (i < N && k < N) ? Cvt<T>::ld(Ap + ia) : 0.f;
+      Bs[kk][rl] = (j < N && k < N) ? Cvt<T>::ld(Bp + ib) : 0.f;
     }
     __syncthreads();
 #pragma unroll
@@ -229,7 +232,7 @@ __global__ void __launch_bounds__(256) contract_kernel(const T* __restrict__ a, 
 }
 
 template <typename T>
-nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& m, cudaStream_t st) {
+nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& m, cudaStream_t st, bool incoming) {
   long long tiles = 0;
   for (int s = 0; s < m.B; ++s) {
     long long nt = (m.N[s] + CT - 1) / CT;
@@ -238,14 +241,14 @@ nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& 
   if (tiles == 0) return NT_OK;
   if (tiles > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
   {
-    LaunchScope ls("generic_tri_contract", st);
-    contract_kernel<T><<<(unsigned)tiles, 256, 0, st>>>(a, b, t, C, m);
+    LaunchScope ls(incoming ? "generic_tri_contract_in" : "generic_tri_contract", st);
+    contract_kernel<T><<<(unsigned)tiles, 256, 0, st>>>(a, b, t, C, m, incoming ? 1 : 0);
   }
   return cuda_ok();
 }
-template nt_status launch_contract<float>(const float*, const float*, float*, int, const BatchMeta&, cudaStream_t);
+template nt_status launch_contract<float>(const float*, const float*, float*, int, const BatchMeta&, cudaStream_t, bool);
 template nt_status launch_contract<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, __nv_bfloat16*, int,
-                                                  const BatchMeta&, cudaStream_t);
+                                                  const BatchMeta&, cudaStream_t, bool);
 
 // ------------------------------------------------------------------------------------------
 // broadcast + LayerNorm (generic widths): one warp per packed position

@@ -34,7 +34,7 @@ nt_status launch_proj(const ProjArgs& a, const BatchMeta& m, cudaStream_t st, co
 
 // t[c][i][j] = sum_k a[c][i][k] b[c][j][k] on channel-major buffers with C channels
 template <typename T>
-nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& m, cudaStream_t st);
+nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& m, cudaStream_t st, bool incoming = false);
 
 // z[p,:] = LN(u[row(p)] + v[col(p)]) * gamma + beta;  u, v float [T1, c_z]
 template <typename T>
