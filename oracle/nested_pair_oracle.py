@@ -23,6 +23,9 @@ What each function follows:
   row_attn_pairbias    Sec. 3.3 "Attention through packed blocks" (segments from cumulative lengths;
                        output adopts the query structure) and Sec. 4.3 (triangle attention with a
                        pair bias); internals are a reading (see below).
+  col_attn_pairbias    the second (column-wise, "ending node") triangle attention of Sec. 4.3: the mirror image of
+                       row_attn_pairbias; pinned by the exact transposition relation to it, library attention, and
+                       scalar loops.
   segment_reduce       Eq. 4 (pair reduction) and the mean of Eq. 1 line 3; App. A batch-axis
                        convention (``[1,2],[3,4]`` sums to ``[3,7]``).
   token_update         Eq. 1 line 3: ``X~ = X + g(mean_b P~[a,b,:])`` with ``g`` a bias-free projection.
@@ -253,6 +256,49 @@ def row_attn_pairbias(zx, lengths, W, H, d, eps=LN_EPS, order="pair", dtype=np.f
     return (res, parts) if return_parts else res
 
 
+def col_attn_pairbias(z, lengths, W, H, d, eps=LN_EPS, dtype=np.float64, return_parts=False):
+    """Column-wise ("ending node") pair-biased softmax attention with residual, the second triangle attention of
+    the Pairformer block (Sec. 4.3).  For each sample, each pair COLUMN j and head h, the N positions i of the
+    column attend over the positions k of the same column:
+        zh = LN(z); q,k,v = zh W_{q,k,v}^T viewed [N,N,H,d]; bias = zh W_b^T [N,N,H]; g = sig(zh W_g^T)
+        S[j,h,i,k] = <q[i,j,h,:], k[k,j,h,:]>/sqrt(d) + bias[k,i,h];  A = softmax_k S
+        o[i,j,h,:] = sum_k A[j,h,i,k] v[k,j,h,:];  z <- z + (g * o) W_o^T
+    The bias is shared by all columns j of the sample.  (The mirror image of row_attn_pairbias: the same formulas
+    with the roles of the two pair indices exchanged.)
+    """
+    z = np.asarray(z, dtype=dtype)
+    Wd = {k: (None if v is None else np.asarray(v, dtype=dtype)) for k, v in W.items()}
+    W_b, W_g = Wd.get("W_b"), Wd.get("W_g")
+    scale = 1.0 / np.sqrt(float(d))
+    out, parts, o = [], [], 0
+    for n in (int(v) for v in lengths):
+        if n == 0:
+            continue
+        zs = z[o:o + n * n].reshape(n, n, z.shape[1])
+        zh = layer_norm(zs, Wd["ln_gamma"], Wd["ln_beta"], eps)
+        q = (zh @ Wd["W_q"].T).reshape(n, n, H, d)           # [i, j, h, :]
+        k = (zh @ Wd["W_k"].T).reshape(n, n, H, d)           # [k, j, h, :]
+        v = (zh @ Wd["W_v"].T).reshape(n, n, H, d)
+        # scores per (column j, head): Q_j K_j^T with Q_j = q[:, j], K_j = k[:, j]
+        S = np.matmul(q.transpose(1, 2, 0, 3), k.transpose(1, 2, 3, 0)) * scale      # [j, h, i, k]
+        if W_b is not None:
+            bias = zh @ W_b.T                                # [row, col, H]; the score of (i, k) takes bias[k, i]
+            S = S + bias.transpose(2, 1, 0)[None, :, :, :]
+        S = S - S.max(axis=-1, keepdims=True)
+        A = np.exp(S)
+        A = A / A.sum(axis=-1, keepdims=True)
+        ov = np.matmul(A, v.transpose(1, 2, 0, 3))           # [j, h, i, :]
+        ov = ov.transpose(2, 0, 1, 3).reshape(n, n, H * d)   # [i, j, h d]
+        if W_g is not None:
+            ov = sigmoid(zh @ W_g.T) * ov
+        out.append((zs + ov @ Wd["W_o"].T).reshape(n * n, z.shape[1]))
+        if return_parts:
+            parts.append(dict(q=q, k=k, v=v, A=A, o=ov))
+        o += n * n
+    res = np.concatenate(out, axis=0) if out else z.copy()
+    return (res, parts) if return_parts else res
+
+
 def segment_reduce(v, splits, op="mean", dtype=np.float64):
     """out[g,:] = sum (or mean) of rows splits[g] .. splits[g+1]-1 of v.  An empty segment gives
     zeros (there is nothing to average; the pair path never produces one because an empty
@@ -359,6 +405,33 @@ def row_attn_pairbias_at(zs, W, H, d, positions, eps=LN_EPS, dtype=np.float64):
 # --------------------------------------------------------------------------------------------
 # compositions
 # --------------------------------------------------------------------------------------------
+def col_attn_pairbias_at(zs, W, H, d, positions, eps=LN_EPS, dtype=np.float64):
+    """Column-wise pair-biased attention of one sample at the listed (i, j).  ``zs`` is indexable as zs[:, c]
+    (pair column c, an [n, c_z] array): query i of column j attends over the keys of column j with
+    bias[:, h] = bias[k, i, h] taken from pair column i."""
+    Wd = {k: (None if v is None else np.asarray(v, dtype=dtype)) for k, v in W.items()}
+    out = []
+    for (i, j) in positions:
+        ci, cj = np.asarray(zs[:, i], dtype=dtype), np.asarray(zs[:, j], dtype=dtype)
+        n = cj.shape[0]
+        zi = layer_norm(ci, Wd["ln_gamma"], Wd["ln_beta"], eps)               # LN(z[k, i]) over k
+        zj = layer_norm(cj, Wd["ln_gamma"], Wd["ln_beta"], eps)               # LN(z[k, j]) over k
+        q = (zj[i] @ Wd["W_q"].T).reshape(H, d)
+        k = (zj @ Wd["W_k"].T).reshape(n, H, d)
+        v = (zj @ Wd["W_v"].T).reshape(n, H, d)
+        bias = zi @ Wd["W_b"].T if Wd.get("W_b") is not None else np.zeros((n, H), dtype=dtype)   # [k, H]
+        o = np.zeros((H, d), dtype=dtype)
+        for h in range(H):
+            sc = k[:, h, :] @ q[h] / np.sqrt(float(d)) + bias[:, h]
+            w = np.exp(sc - sc.max())
+            o[h] = (w / w.sum()) @ v[:, h, :]
+        ov = o.reshape(H * d)
+        if Wd.get("W_g") is not None:
+            ov = sigmoid(zj[i] @ Wd["W_g"].T) * ov
+        out.append(cj[i] + ov @ Wd["W_o"].T)
+    return np.stack(out)
+
+
 def block_forward(x, lengths, w, H, d, eps=LN_EPS, dtype=np.float64):
     """One Pairformer-style block: broadcast+LN, outgoing triangle update, row-wise pair-biased
     attention, segmented mean over j and token update.  Returns (x', z)."""

@@ -339,6 +339,66 @@ def test_attention_special_cases():
     assert np.allclose(orc.row_attn_pairbias(zc, cfg.lengths, Wn2, cfg.H, cfg.d), base, rtol=1e-11, atol=1e-11)
 
 
+def test_col_attention_is_row_attention_of_the_transposed_state():
+    cfg, inp = tiny_inputs((4, 1, 6, 3))
+    rng = np.random.default_rng(31)
+    z = rng.standard_normal((cfg.T2, cfg.c_z))
+    W = inp["blocks"][0]["attn"]
+    zT = _pair_transpose(z, cfg.lengths)
+    lhs = orc.col_attn_pairbias(z, cfg.lengths, W, cfg.H, cfg.d)
+    rhs = _pair_transpose(orc.row_attn_pairbias(zT, cfg.lengths, W, cfg.H, cfg.d), cfg.lengths)
+    assert np.allclose(lhs, rhs, rtol=1e-11, atol=1e-11)
+    assert not np.allclose(lhs, orc.row_attn_pairbias(z, cfg.lengths, W, cfg.H, cfg.d))
+    # on a symmetric state the two attentions give transposed results of each other, hence equal updates after transposing
+    zsym = 0.5 * (z + zT)
+    a = orc.col_attn_pairbias(zsym, cfg.lengths, W, cfg.H, cfg.d)
+    b = _pair_transpose(orc.row_attn_pairbias(zsym, cfg.lengths, W, cfg.H, cfg.d), cfg.lengths)
+    assert np.allclose(a, b, rtol=1e-11, atol=1e-11)
+
+
+def test_col_attention_scalar_loops_and_library_sdpa():
+    cfg, inp = tiny_inputs((5,))
+    n, H, d = 5, cfg.H, cfg.d
+    rng = np.random.default_rng(32)
+    z = rng.standard_normal((n * n, cfg.c_z))
+    W = {k: np.asarray(v, dtype=np.float64) for k, v in inp["blocks"][0]["attn"].items()}
+    got, parts = orc.col_attn_pairbias(z, (n,), W, H, d, return_parts=True)
+    zs = z.reshape(n, n, -1)
+    zh = orc.layer_norm(zs, W["ln_gamma"], W["ln_beta"])
+    q = (zh @ W["W_q"].T).reshape(n, n, H, d)
+    k = (zh @ W["W_k"].T).reshape(n, n, H, d)
+    v = (zh @ W["W_v"].T).reshape(n, n, H, d)
+    bias = zh @ W["W_b"].T
+    g = 1.0 / (1.0 + np.exp(-(zh @ W["W_g"].T)))
+    want = np.zeros((n, n, cfg.c_z))
+    for i in range(n):
+        for j in range(n):
+            o = np.zeros((H, d))
+            for h in range(H):
+                sc = np.array([sum(q[i, j, h, e] * k[kk, j, h, e] for e in range(d)) / np.sqrt(d) + bias[kk, i, h] for kk in range(n)])
+                w = np.exp(sc - sc.max())
+                w /= w.sum()
+                for kk in range(n):
+                    o[h] += w[kk] * v[kk, j, h]
+            want[i, j] = zs[i, j] + (g[i, j] * o.reshape(-1)) @ W["W_o"].T
+    assert np.allclose(got.reshape(n, n, -1), want, rtol=1e-11, atol=1e-11)
+    # the attention weights of every (column, head) sum to one; and the core equals the library attention with an additive mask
+    assert np.allclose(parts[0]["A"].sum(-1), 1.0, rtol=1e-12)
+    F = torch.nn.functional
+    for j in range(n):
+        qt = torch.from_numpy(q[:, j].transpose(1, 0, 2))[None]              # [1, H, i, d]
+        kt = torch.from_numpy(k[:, j].transpose(1, 0, 2))[None]
+        vt = torch.from_numpy(v[:, j].transpose(1, 0, 2))[None]
+        mask = torch.from_numpy(bias.transpose(2, 1, 0).copy())[None]        # [1, H, i, k] = bias[k, i, h]
+        ref = F.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask)[0].numpy()      # [H, i, d]
+        o_col = (parts[0]["o"][:, j] / g[:, j]).reshape(n, H, d).transpose(1, 0, 2)
+        assert np.allclose(o_col, ref, rtol=1e-9, atol=1e-10)
+    # sampled evaluator equals the full function
+    pos = [(0, 0), (3, 4), (4, 1), (2, 2)]
+    at = orc.col_attn_pairbias_at(zs, W, H, d, pos)
+    assert np.allclose(at, np.stack([got.reshape(n, n, -1)[i, j] for i, j in pos]), rtol=1e-12, atol=1e-12)
+
+
 def test_token_attention_is_textbook_varlen():
     cfg = wl.Config("tok", "f32", (7, 3, 12), c_s=16, c_z=16, c_h=0, H=2, d=8, blocks=1, seed=11, kind="token")
     inp = wl.make_inputs(cfg)
