@@ -74,6 +74,7 @@ def kernel_work(cfg: wl.Config):
     w["attn_in"] = dict(bytes=T2 * (c_z + 4 * Hd + H) * e, flops=2 * T2 * c_z * (4 * Hd + H))
     # the softmax needs one exponential per (query, key, head): the special-function units retire 16 per clock and SM
     w["generic_attn_core"] = w["attn_core"] = dict(bytes=T2 * (4 * Hd + H) * e, flops=4 * N3 * Hd, exps=N3 * H)
+    w["generic_attn_core_col"] = w["attn_core_col"] = w["attn_core"]            # column-wise attention: same work
     w["generic_attn_out"] = w["attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
@@ -242,6 +243,8 @@ def main():
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
     ap.add_argument("--only-transition", action="store_true",
                     help="run just the pair-transition measurement (the row after the block; for ncu captures)")
+    ap.add_argument("--only-col-attn", action="store_true",
+                    help="run just the column-wise attention measurement (for ncu captures)")
     ap.add_argument("--only-tri-mul-in", action="store_true",
                     help="run just the incoming-triangle-update measurement (for ncu captures)")
     ap.add_argument("--no-extras", action="store_true",
@@ -334,8 +337,32 @@ def main():
             out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
         return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
 
-    if args.only_transition or args.only_tri_mul_in:
-        res = dict(pair_transition=transition_pass(steps)) if args.only_transition else dict(tri_mul_in=tri_mul_in_pass(steps))
+    def col_attn_pass(n_calls):
+        """Column-wise ("ending node") attention (a row after the block) on the state the first block's broadcast
+        produces; nt_col_attn_pairbias timed per launch.  Not part of the step or of `value`."""
+        if cfg.kind != "pair":
+            return None
+        w0 = stack.W[0]
+        b = w0["broadcast"]
+        nt.nt_pair_broadcast(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        for _ in range(3):
+            nt.nt_col_attn_pairbias(stack.L, w0["attn"], cfg.H, cfg.d, 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            nt.nt_col_attn_pairbias(stack.L, w0["attn"], cfg.H, cfg.d, 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        out = {}
+        for k, v in tp.items():
+            r = roofline_entry(k, v[0], v[1], n_calls, kernel_work(cfg), peaks_t, kind_t)
+            out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
+
+    if args.only_transition or args.only_tri_mul_in or args.only_col_attn:
+        res = (dict(pair_transition=transition_pass(steps)) if args.only_transition else
+               dict(tri_mul_in=tri_mul_in_pass(steps)) if args.only_tri_mul_in else dict(col_attn=col_attn_pass(steps)))
         if rank == 0:
             print(json.dumps(res))
         if world > 1:
@@ -403,7 +430,8 @@ def main():
     if roofline and cfg.name == "cfg2" and not args.force_generic:
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
-    next_rows = dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps)) if not args.force_generic else None
+    next_rows = (dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps), col_attn=col_attn_pass(steps))
+                 if not args.force_generic else None)
 
     # ---- end to end through the public API with host buffers
     x_pin = torch.from_numpy(np.ascontiguousarray(inp["x"])).to(stack.dtype).pin_memory()

@@ -154,6 +154,20 @@ nt_status nt_row_attn_pairbias(const nt_layout *L, nt_order order, nt_dtype dt,
                                void *workspace, size_t workspace_bytes, nt_stream stream);
 
 /*
+ * nt_col_attn_pairbias -- column-wise pair-biased softmax attention over ragged N_s: the second triangle
+ * attention of the block (Sec. 4.3, "ending node"), the mirror image of nt_row_attn_pairbias in pair order.
+ *   Attention rows are the pair COLUMNS (s, j); for each column and head h:
+ *     S[i,k] = <q_ij, k_kj>/sqrt(d) + bias[k,i,h] with bias = LN(z) W_b^T shared by all columns of the sample;
+ *     P = softmax_k S; o_ij = sum_k P[i,k] v_kj; z += (g * o) W_o^T.
+ *   z [T2, c] in/out (in place).  Same weights structure, workspace size (nt_workspace_bytes) and error behaviour
+ *   as nt_row_attn_pairbias with order = NT_ORDER_PAIR_IJC.  Keys of a column are N_s packed rows apart; nothing
+ *   is transposed in memory.
+ */
+nt_status nt_col_attn_pairbias(const nt_layout *L, nt_dtype dt, int32_t c, int32_t H, int32_t d,
+                               const nt_attn_weights *W, float ln_eps, void *z,
+                               void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
  * nt_segment_reduce -- segmented sum or mean of contiguous row groups (Eq. 4 pair reduction; the
  * mean over j of Eq. 1 line 3 divides by the group's count; App. A batch-axis convention).
  *   out[g,:] = (1/len_g or 1) * sum_{r = splits[g]}^{splits[g+1]-1} v[r,:],  empty group -> 0.

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3:
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
 EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-           "nt_row_attn_pairbias", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
+           "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
            "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
 
@@ -68,6 +68,7 @@ def _load() -> C.CDLL:
     lib.nt_pair_broadcast_static.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.nt_tri_mul_out.argtypes = [C.POINTER(nt_layout), i32, i32, i32, C.POINTER(nt_trimul_weights), f32, vp, vp, sz, vp]
     lib.nt_tri_mul_in.argtypes = lib.nt_tri_mul_out.argtypes
+    lib.nt_col_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, C.POINTER(nt_attn_weights), f32, vp, vp, sz, vp]
     lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
                                          f32, vp, vp, sz, vp]
     lib.nt_segment_reduce.argtypes = [i32, i32, i32, i64, i64, vp, vp, vp, vp, vp]
@@ -89,7 +90,7 @@ def _load() -> C.CDLL:
     lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
     lib.nt_profile_end.restype = i32
     for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-                 "nt_row_attn_pairbias", "nt_segment_reduce", "nt_token_update"):
+                 "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_segment_reduce", "nt_token_update"):
         getattr(lib, name).restype = i32
     return lib
 
@@ -213,6 +214,17 @@ def nt_row_attn_pairbias(L: Layout, order: int, W: dict, H: int, d: int, ln_eps,
                                   _ptr(zx), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                   _stream(stream))
     _check(st, "nt_row_attn_pairbias")
+
+
+def nt_col_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, z, workspace, stream=None):
+    """Column-wise ("ending node") pair-biased attention on the packed pair state; weights and workspace as for
+    nt_row_attn_pairbias in pair order."""
+    c = int(W["W_q"].shape[1])
+    w = nt_attn_weights(*[_ptr(W.get(n)) for n, _ in nt_attn_weights._fields_])
+    st = lib.nt_col_attn_pairbias(C.byref(L.c), dtype_code(z.dtype), c, H, d, C.byref(w), float(ln_eps),
+                                  _ptr(z), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _stream(stream))
+    _check(st, "nt_col_attn_pairbias")
 
 
 def nt_segment_reduce(op: int, splits_d, v, out, status_d=None, stream=None):

@@ -246,7 +246,7 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
 template <typename T>
 static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order order, int c, int H, int d,
                               const nt_attn_weights* W, float eps, void* zx, void* ws, nt_dtype dt,
-                              cudaStream_t st) {
+                              cudaStream_t st, bool col) {
   AttnWs w = carve_attn(ws, dt, tot, order, H, d);
   const int Hd = H * d;
   const bool pair = order == NT_ORDER_PAIR_IJC;
@@ -289,7 +289,21 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       pa.W1 = W->W_b; pa.Nout = H; pa.out = w.bias; pa.out_mode = O_CHANNEL_MAJOR;
       if ((r = launch_proj<T>(pa, m, st, "generic_attn_in_bias")) != NT_OK) return r;
     }
-    if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d) && (!W->W_b || tc_in))
+    if (col) {
+      // column-wise attention: the tcgen05 core takes the samples whose key range fits its accumulator, the
+      // shape-generic core the others (the bias is stored times sqrt(d) when the tensor-core projections wrote it)
+      int n_tc = 0;
+      if (dt == NT_BF16 && !g_force_generic && (d == 16 || d == 32) && (!W->W_b || tc_in)) {
+        n_tc = fast_attn_tc_max_n(d, W->W_b != nullptr);
+        if (n_tc > 0) {
+          r = fast_attn_core_tc(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, m, n_tc, L->status_d, st, true);
+          if (r == NT_ERR_UNSUPPORTED) n_tc = 0;
+          else if (r != NT_OK) return r;
+        }
+      }
+      r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, W->W_b ? (const T*)w.bias : nullptr,
+                              (T*)w.o, H, d, 2, m, st, n_tc, tc_in ? rsqrtf((float)d) : 1.0f);
+    } else if (dt == NT_BF16 && !g_force_generic && fast_attn_core_supported(H, d) && (!W->W_b || tc_in))
       r = fast_attn_core(w.q, w.k, w.v, W->W_b ? w.bias : nullptr, w.o, H, d, pair ? 1 : 0, tc_in ? 1 : 0, m,
                          L->status_d, st);
     else
@@ -384,8 +398,27 @@ nt_status nt_row_attn_pairbias(const nt_layout* L, nt_order order, nt_dtype dt, 
   if (!zx || !workspace || !aligned16(zx) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
   if (workspace_bytes < carve_attn(nullptr, dt, tot, order, H, d).bytes) return NT_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
-  if (dt == NT_F32) return attn_generic<float>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st);
-  return attn_generic<__nv_bfloat16>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st);
+  if (dt == NT_F32) return attn_generic<float>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st, false);
+  return attn_generic<__nv_bfloat16>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st, false);
+}
+
+nt_status nt_col_attn_pairbias(const nt_layout* L, nt_dtype dt, int32_t c, int32_t H, int32_t d,
+                               const nt_attn_weights* W, float ln_eps, void* z, void* workspace,
+                               size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c <= 0 || H <= 0 || d <= 0 || !W) return NT_ERR_INVALID_ARG;
+  if (!W->W_q || !W->W_k || !W->W_v || !W->W_o) return NT_ERR_INVALID_ARG;
+  if ((W->ln_gamma == nullptr) != (W->ln_beta == nullptr)) return NT_ERR_INVALID_ARG;
+  if (d > 128) return NT_ERR_UNSUPPORTED;
+  if (tot.T2 == 0) return NT_OK;
+  if (!z || !workspace || !aligned16(z) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < carve_attn(nullptr, dt, tot, NT_ORDER_PAIR_IJC, H, d).bytes) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32) return attn_generic<float>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, true);
+  return attn_generic<__nv_bfloat16>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, true);
 }
 
 nt_status nt_segment_reduce(nt_dtype dt, nt_reduce op, int32_t C, int64_t G, int64_t rows, const int64_t* splits_d,

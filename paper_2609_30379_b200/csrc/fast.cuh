@@ -28,7 +28,7 @@ nt_status fast_attn_core(const void* q, const void* k, const void* v, const void
 // fast_attn_tc_max_n gives the largest N whose score row and bias tiles fit (0: not supported)
 int fast_attn_tc_max_n(int d, bool has_bias);
 nt_status fast_attn_core_tc(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
-                            const BatchMeta& m, int n_max, int* status, cudaStream_t st);
+                            const BatchMeta& m, int n_max, int* status, cudaStream_t st, bool col = false);
 
 // triangle contraction on tcgen05: a, b, t are three equally spaced channel-major buffers
 // (b = a + stride, t = a + 2 * stride); incoming = contraction over the first index (sum_k a[k][i] b[k][j])

@@ -39,6 +39,9 @@ constexpr float TCA_LOG2E = 1.4426950408889634f;
 struct AttnTcParams {
   CUtensorMap qmap;       // flat {H d, rows}, box {d, 128}
   CUtensorMap kmap, vmap; // box {d, 32}
+  // column mode (queries and keys run along the first pair index of a column): one map per sample,
+  // {H d, first index (stride N H d), column (stride H d), which of q / k / v}, box {d, 32, 1, 1}
+  CUtensorMap cmap[MAXB];
   BatchMeta m;
   long long item_off[MAXB + 1];   // prefix of N_s * H * ceil(N_s / 128) over the samples this kernel takes
   const __nv_bfloat16* bias;      // head-major channel-major, stored times sqrt(d); nullable
@@ -84,7 +87,7 @@ __device__ inline unsigned long long tca_desc(unsigned saddr, int span) {
   return d;
 }
 
-template <int D>
+template <int D, bool COL>
 __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_constant__ AttnTcParams p) {
   constexpr int SPAN = 2 * D;                 // bytes per tile row = swizzle span
   constexpr int Q_BYTES = 128 * SPAN;
@@ -160,11 +163,30 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
       // (rows of K that belong to other pair rows) get a large negative bias, so their weights come out as exact
       // zeros and neither softmax pass needs a mask.
       const int chunks = Nk / 8;
-      for (int idx = threadIdx.x - 96; idx < njb * 128 * chunks; idx += 512) {
-        const int q = idx / chunks, c = idx - q * chunks;
-        const bool ok = has_bias && q < N && c * 8 < ld;
-        tca_cp_async16(sBias + (q >> 7) * p.bias_tile_bytes + (q & 127) * bstride + c * 16,
-                       ok ? bias_h + (long long)q * ld + c * 8 : p.o, ok);
+      if (COL) {
+        // the bias of (query q, key k) is element [k][q] of the plane: read 8 consecutive queries of a key row,
+        // scatter them into the 8 query rows of the tile
+        const int qchunks = ld / 8;
+        for (int idx = threadIdx.x - 96; idx < N * qchunks; idx += 512) {
+          const int k = idx / qchunks, c = idx - k * qchunks;
+          uint4 val = make_uint4(0, 0, 0, 0);
+          if (has_bias) val = *reinterpret_cast<const uint4*>(bias_h + (long long)k * ld + c * 8);
+          const unsigned w4[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int q = c * 8 + e;
+            if (q < njb * 128)
+              *reinterpret_cast<unsigned short*>(sBias + (q >> 7) * p.bias_tile_bytes + (q & 127) * bstride + k * 2) =
+                  (unsigned short)(e & 1 ? w4[e >> 1] >> 16 : w4[e >> 1] & 0xffffu);
+          }
+        }
+      } else {
+        for (int idx = threadIdx.x - 96; idx < njb * 128 * chunks; idx += 512) {
+          const int q = idx / chunks, c = idx - q * chunks;
+          const bool ok = has_bias && q < N && c * 8 < ld;
+          tca_cp_async16(sBias + (q >> 7) * p.bias_tile_bytes + (q & 127) * bstride + c * 16,
+                         ok ? bias_h + (long long)q * ld + c * 8 : p.o, ok);
+        }
       }
       asm volatile("cp.async.wait_all;\n" ::: "memory");
       named_bar_sync(3, 512);
@@ -202,8 +224,13 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
           mbar_expect_tx(&qkfull[st], Q_BYTES + nb * 32 * SPAN);
         }
         __syncwarp();
-        if (lane == 0) tma_load_2d(stg, &p.qmap, &qkfull[st], h * D, base + jb * 128);
-        else if (lane <= nb) tma_load_2d(stg + Q_BYTES + (lane - 1) * 32 * SPAN, &p.kmap, &qkfull[st], h * D, base + (lane - 1) * 32);
+        if (COL) {     // i is the column; the query block and the keys run along the first pair index
+          if (lane < 4) tma_load_4d(stg + lane * 32 * SPAN, &p.cmap[s], &qkfull[st], h * D, jb * 128 + lane * 32, i, 0);
+          else if (lane < 4 + nb) tma_load_4d(stg + Q_BYTES + (lane - 4) * 32 * SPAN, &p.cmap[s], &qkfull[st], h * D, (lane - 4) * 32, i, 1);
+        } else {
+          if (lane == 0) tma_load_2d(stg, &p.qmap, &qkfull[st], h * D, base + jb * 128);
+          else if (lane <= nb) tma_load_2d(stg + Q_BYTES + (lane - 1) * 32 * SPAN, &p.kmap, &qkfull[st], h * D, base + (lane - 1) * 32);
+        }
         if (++st == (unsigned)p.nqk) { st = 0; ++k; }
       }
     } else if (warp == 2) {
@@ -218,7 +245,10 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
           mbar_expect_tx(&vfull[st], nb * 32 * SPAN);
         }
         __syncwarp();
-        if (lane < nb) tma_load_2d(sV + st * kv_bytes + lane * 32 * SPAN, &p.vmap, &vfull[st], h * D, base + lane * 32);
+        if (lane < nb) {
+          if (COL) tma_load_4d(sV + st * kv_bytes + lane * 32 * SPAN, &p.cmap[s], &vfull[st], h * D, lane * 32, i, 2);
+          else tma_load_2d(sV + st * kv_bytes + lane * 32 * SPAN, &p.vmap, &vfull[st], h * D, base + lane * 32);
+        }
         if (++st == (unsigned)p.nv) { st = 0; ++k; }
       }
     } else if (warp == 1) {
@@ -374,7 +404,8 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
           const float inv = 1.0f / (xm[256 + row] + xm[256 + 128 + row]);
           tmem_ld_wait16(ra);
           if (j < N) {
-            __nv_bfloat16* op = p.o + (p.row0 + row_base + (long long)i * N + j) * Hd + h * D + hf * CPT;
+            const long long orow = COL ? (long long)j * N + i : (long long)i * N + j;
+            __nv_bfloat16* op = p.o + (p.row0 + row_base + orow) * Hd + h * D + hf * CPT;
             unsigned w[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) w[e] = tca_pack(__uint_as_float(ra[2 * e]) * inv, __uint_as_float(ra[2 * e + 1]) * inv);
@@ -403,7 +434,7 @@ static size_t tca_smem_bytes(int D, int n_max, bool has_bias, int nqk, int nv, i
          (size_t)njb * *tile_bytes + 1024;
 }
 
-template <int D>
+template <int D, bool COL>
 static nt_status launch_attn_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                                 const __nv_bfloat16* bias, __nv_bfloat16* o, int H, const BatchMeta& m, int n_max,
                                 int* status, cudaStream_t st) {
@@ -440,7 +471,20 @@ static nt_status launch_attn_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, 
   }
   if (smem > limit) return NT_ERR_UNSUPPORTED;
   const int Hd = H * D;
-  {
+  if (COL) {
+    // q, k, v must be three equally spaced buffers (they are carved that way): the map's outermost dimension picks one
+    const long long gap = (const char*)k - (const char*)q;
+    if (gap <= 0 || (const char*)v - (const char*)k != gap || gap % 16 != 0) return NT_ERR_UNSUPPORTED;
+    for (int s = 0; s < m.B; ++s) {
+      const int N = m.N[s];
+      if (N < 1 || N > n_max) continue;
+      const unsigned long long dims[4] = {(unsigned long long)Hd, (unsigned long long)N, (unsigned long long)N, 3};
+      const unsigned long long strides[3] = {(unsigned long long)N * Hd * 2, (unsigned long long)Hd * 2, (unsigned long long)gap};
+      const unsigned box[4] = {(unsigned)D, 32, 1, 1};
+      if (!make_tmap_16bit(&p.cmap[s], q + m.pair_off[s] * Hd, 4, dims, strides, box, 2 * D, 2 * D >= 128 ? 128 : 2 * D))
+        return cuda_fail("attn tc column map");
+    }
+  } else {
     const unsigned long long dims[2] = {(unsigned long long)Hd, (unsigned long long)rows};
     const unsigned long long strides[1] = {(unsigned long long)Hd * 2};
     const unsigned qbox[2] = {(unsigned)D, 128}, kbox[2] = {(unsigned)D, 32};
@@ -450,14 +494,14 @@ static nt_status launch_attn_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, 
   }
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit - 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_tc_kernel<D, COL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit - 1024) != cudaSuccess)
       return cuda_fail("attention tc smem attribute");
     attr_set = true;
   }
   const unsigned grid = (unsigned)(total < 148 ? total : 148);
   {
-    LaunchScope ls("attn_core", st);
-    attn_tc_kernel<D><<<grid, TCA_THREADS, smem, st>>>(p);
+    LaunchScope ls(COL ? "attn_core_col" : "attn_core", st);
+    attn_tc_kernel<D, COL><<<grid, TCA_THREADS, smem, st>>>(p);
   }
   return cuda_ok("attention tc launch");
 }
@@ -471,14 +515,19 @@ int fast_attn_tc_max_n(int d, bool has_bias) {
 }
 
 nt_status fast_attn_core_tc(const void* q, const void* k, const void* v, const void* bias, void* o, int H, int d,
-                            const BatchMeta& m, int n_max, int* status, cudaStream_t st) {
+                            const BatchMeta& m, int n_max, int* status, cudaStream_t st, bool col) {
   const __nv_bfloat16* qq = (const __nv_bfloat16*)q;
   const __nv_bfloat16* kk = (const __nv_bfloat16*)k;
   const __nv_bfloat16* vv = (const __nv_bfloat16*)v;
   const __nv_bfloat16* bb = (const __nv_bfloat16*)bias;
   __nv_bfloat16* oo = (__nv_bfloat16*)o;
-  if (d == 16) return launch_attn_tc<16>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
-  if (d == 32) return launch_attn_tc<32>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+  if (col) {
+    if (d == 16) return launch_attn_tc<16, true>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+    if (d == 32) return launch_attn_tc<32, true>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+    return NT_ERR_UNSUPPORTED;
+  }
+  if (d == 16) return launch_attn_tc<16, false>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
+  if (d == 32) return launch_attn_tc<32, false>(qq, kk, vv, bb, oo, H, m, n_max, status, st);
   return NT_ERR_UNSUPPORTED;
 }
 

@@ -304,7 +304,9 @@ template nt_status launch_broadcast_ln<__nv_bfloat16>(const float*, const float*
                                                       const BatchMeta&, cudaStream_t);
 
 // ------------------------------------------------------------------------------------------
-// attention core: one warp per (attention row, head, query); lanes over keys; online softmax
+// attention core: one warp per (attention row, head, query); lanes over keys; online softmax.
+// pair_order: 0 = token segments, 1 = pair rows (queries and keys run along j of row i), 2 = pair columns (queries
+// and keys run along the first index of column i; the bias of (query, key) is bias[key][query]).
 // ------------------------------------------------------------------------------------------
 constexpr int AQB = 8;      // queries (warps) per block
 constexpr int AD_MAX = 128; // head dim limit of the generic core
@@ -313,14 +315,14 @@ template <typename T>
 __global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                             const T* __restrict__ v, const T* __restrict__ bias,
                                                             T* __restrict__ o, int H, int d, int pair_order,
-                                                            BatchMeta m) {
+                                                            BatchMeta m, int skip_max_n, float bias_scale) {
   __shared__ float qs[AQB][AD_MAX];
   long long w = blockIdx.x;
   int s = 0, N = 0, nqb = 0;
   for (; s < m.B; ++s) {
     N = m.N[s];
     nqb = (N + AQB - 1) / AQB;
-    long long cnt = (long long)(pair_order ? N : (N > 0 ? 1 : 0)) * H * nqb;
+    long long cnt = N <= skip_max_n ? 0 : (long long)(pair_order ? N : (N > 0 ? 1 : 0)) * H * nqb;
     if (w < cnt) break;
     w -= cnt;
   }
@@ -328,17 +330,19 @@ __global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict
   const int jb = (int)(w % nqb);
   const int h = (int)((w / nqb) % H);
   const long long i = w / ((long long)nqb * H);
-  const long long base = pair_order ? m.pair_off[s] + i * N : m.tok_off[s];
+  const long long base = pair_order == 1 ? m.pair_off[s] + i * N : pair_order == 2 ? m.pair_off[s] + i : m.tok_off[s];
+  const long long step = pair_order == 2 ? N : 1;          // packed rows between consecutive queries / keys
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = jb * AQB + warp;
   const int Hd = H * d;
   const bool active = j < N;
   if (active)
-    for (int e = lane; e < d; e += 32) qs[warp][e] = Cvt<T>::ld(q + (base + j) * Hd + h * d + e);
+    for (int e = lane; e < d; e += 32) qs[warp][e] = Cvt<T>::ld(q + (base + j * step) * Hd + h * d + e);
   __syncwarp();
   if (!active) return;
   const int ld = round_up8(N);
-  const T* brow = bias ? bias + (long long)H * m.cm_off[s] + (long long)h * N * ld + (long long)j * ld : nullptr;
+  const T* brow = bias ? bias + (long long)H * m.cm_off[s] + (long long)h * N * ld + (pair_order == 2 ? (long long)j : (long long)j * ld) : nullptr;
+  const long long bstep = pair_order == 2 ? ld : 1;
   const float scale = rsqrtf((float)d);
   float mrun = -INFINITY, lrun = 0.f;
   float oacc[AD_MAX / 32] = {};
@@ -347,11 +351,11 @@ __global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict
     const int kk = c0 + lane;
     float sc = -INFINITY;
     if (kk < N) {
-      const T* kr = k + (base + kk) * Hd + h * d;
+      const T* kr = k + (base + kk * step) * Hd + h * d;
       float dot = 0.f;
       for (int e = 0; e < d; ++e) dot = fmaf(qs[warp][e], Cvt<T>::ld(kr + e), dot);
       sc = dot * scale;
-      if (brow) sc += Cvt<T>::ld(brow + kk);
+      if (brow) sc += Cvt<T>::ld(brow + kk * bstep) * bias_scale;
     }
     float cmax = sc;
 #pragma unroll
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict
     const int lim = min(32, N - c0);
     for (int k2 = 0; k2 < lim; ++k2) {
       const float pk = __shfl_sync(0xffffffffu, pr, k2);
-      const T* vr = v + (base + c0 + k2) * Hd + h * d;
+      const T* vr = v + (base + (c0 + k2) * step) * Hd + h * d;
       for (int u = 0; u < ne; ++u) {
         const int e = u * 32 + lane;
         if (e < d) oacc[u] = fmaf(pk, Cvt<T>::ld(vr + e), oacc[u]);
@@ -378,32 +382,33 @@ __global__ void __launch_bounds__(AQB * 32) attn_core_kernel(const T* __restrict
   const float inv = 1.0f / lrun;
   for (int u = 0; u < ne; ++u) {
     const int e = u * 32 + lane;
-    if (e < d) Cvt<T>::st(o + (base + j) * Hd + h * d + e, oacc[u] * inv);
+    if (e < d) Cvt<T>::st(o + (base + j * step) * Hd + h * d + e, oacc[u] * inv);
   }
 }
 
 template <typename T>
 nt_status launch_attn_core(const T* q, const T* k, const T* v, const T* bias, T* o, int H, int d, int pair_order,
-                           const BatchMeta& m, cudaStream_t st) {
+                           const BatchMeta& m, cudaStream_t st, int skip_max_n, float bias_scale) {
   if (d > AD_MAX) return NT_ERR_UNSUPPORTED;
   long long blocks = 0;
   for (int s = 0; s < m.B; ++s) {
     long long N = m.N[s], nqb = (N + AQB - 1) / AQB;
+    if (N <= skip_max_n) continue;
     blocks += (pair_order ? N : (N > 0 ? 1 : 0)) * H * nqb;
   }
   if (blocks == 0) return NT_OK;
   if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
   {
-    LaunchScope ls("generic_attn_core", st);
-    attn_core_kernel<T><<<(unsigned)blocks, AQB * 32, 0, st>>>(q, k, v, bias, o, H, d, pair_order, m);
+    LaunchScope ls(pair_order == 2 ? "generic_attn_core_col" : "generic_attn_core", st);
+    attn_core_kernel<T><<<(unsigned)blocks, AQB * 32, 0, st>>>(q, k, v, bias, o, H, d, pair_order, m, skip_max_n, bias_scale);
   }
   return cuda_ok();
 }
 template nt_status launch_attn_core<float>(const float*, const float*, const float*, const float*, float*, int, int,
-                                           int, const BatchMeta&, cudaStream_t);
+                                           int, const BatchMeta&, cudaStream_t, int, float);
 template nt_status launch_attn_core<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
                                                    const __nv_bfloat16*, __nv_bfloat16*, int, int, int,
-                                                   const BatchMeta&, cudaStream_t);
+                                                   const BatchMeta&, cudaStream_t, int, float);
 
 // ------------------------------------------------------------------------------------------
 // segmented reduction (generic widths): one block per group

@@ -45,7 +45,7 @@ nt_status launch_broadcast_ln(const float* u, const float* v, const T* gamma, co
 // head-major channel-major buffer; token order: one row per sample.
 template <typename T>
 nt_status launch_attn_core(const T* q, const T* k, const T* v, const T* bias, T* o, int H, int d, int pair_order,
-                           const BatchMeta& m, cudaStream_t st);
+                           const BatchMeta& m, cudaStream_t st, int skip_max_n = -1, float bias_scale = 1.0f);
 
 template <typename T>
 nt_status launch_segment_reduce(const T* v, T* out, const int64_t* splits, long long G, int C, int mean,
