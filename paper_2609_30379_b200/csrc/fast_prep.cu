@@ -12,6 +12,7 @@ struct PrepJob {
   const __nv_bfloat16* src[6];
   int rows[6];
   float scale[6];   // extra factor on the rows of a source (and on its c0, c1)
+  int bf16out[6];   // rows of this source are written as bf16 (for an MMA whose activation operand stays bf16)
   int nsrc, K, total;
   const __nv_bfloat16* gamma;
   const __nv_bfloat16* beta;
@@ -34,13 +35,17 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
   float c0 = 0.f, c1 = 0.f;
   for (int k = lane; k < J.K; k += 32) {
     const float wv = w ? __bfloat162float(w[k]) * J.scale[src] : 0.f;
-    __half o = __float2half_rn(wv);
-    if (J.gamma) {
-      o = __float2half_rn(wv * __bfloat162float(J.gamma[k]));
-      c0 = fmaf(wv, __bfloat162float(J.beta[k]), c0);
-      c1 += __half2float(o);
+    const float folded = J.gamma ? wv * __bfloat162float(J.gamma[k]) : wv;
+    if (J.gamma) c0 = fmaf(wv, __bfloat162float(J.beta[k]), c0);
+    if (J.bf16out[src]) {
+      const __nv_bfloat16 ob = __float2bfloat16_rn(folded);
+      if (J.gamma) c1 += __bfloat162float(ob);
+      reinterpret_cast<__nv_bfloat16*>(J.out)[(long long)n * J.K + k] = ob;
+    } else {
+      const __half o = __float2half_rn(folded);
+      if (J.gamma) c1 += __half2float(o);
+      J.out[(long long)n * J.K + k] = o;
     }
-    J.out[(long long)n * J.K + k] = o;
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) {
@@ -64,13 +69,15 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
 }
 
 static void add_job(PrepArgs& a, const void* const* srcs, const int* rows, int nsrc, int K, const void* gamma,
-                    const void* beta, void* out, void* c01, const float* scale = nullptr, void* aug = nullptr) {
+                    const void* beta, void* out, void* c01, const float* scale = nullptr, void* aug = nullptr,
+                    const int* bf16out = nullptr) {
   PrepJob& J = a.job[a.njobs++];
   J.total = 0;
   for (int i = 0; i < nsrc; ++i) {
     J.src[i] = (const __nv_bfloat16*)srcs[i];
     J.rows[i] = rows[i];
     J.scale[i] = scale ? scale[i] : 1.0f;
+    J.bf16out[i] = bf16out ? bf16out[i] : 0;
     J.total += rows[i];
   }
   J.nsrc = nsrc;
@@ -119,7 +126,9 @@ nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep
   const int r0[5] = {c_h, c_h, c_h, c_h, c_z};
   // gate and value rows are folded times 1/2 (exact): sigmoid(g) v = (tanh(g / 2) + 1) (v / 2) costs one MUFU and one FMA
   const float sc[5] = {0.5f, 0.5f, 0.5f, 0.5f, 1.0f};
-  add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, sc, out.aug1);
+  // W_g meets the bf16 state itself in the output stage (no conversion pass there): its folded rows are bf16
+  const int asbf16[5] = {0, 0, 0, 0, 1};
+  add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, sc, out.aug1, asbf16);
   const void* s1[1] = {W->W_o};
   const int r1[1] = {c_z};
   add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o, nullptr, out.augo);

@@ -1,20 +1,20 @@
-// Triangle-update output stage on tcgen05 (bf16, float accumulate), in place on the pair state:
+// Triangle-update output stage on tcgen05 (float accumulate), in place on the pair state:
 //   z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T)
 // t is the contraction result in channel-major layout (t[c][i][j], j contiguous), so a run of 64
 // positions of one pair row is, per channel, 128 contiguous bytes: exactly the MN-major operand
 // form of the MMA (positions are M, channels are K).  The output gate is recomputed here from z
 // instead of being stored by the input projection, which saves one write and one read of a
-// [T2, c_z] buffer.  Both LayerNorms are folded into the weights (see fast_tri_in.cu) and their mean
-// terms into the MMA: one more K step multiplies (-mean_hi, -mean_lo, -mean_hi) per position with
-// (c1_hi, c1_hi, c1_lo) per output channel, so the epilogue is left with
-//   o / 2 = (rstd_t / 2) acc_o + c0_o / 2,  g / 2 = (rstd_z / 2) acc_g + c0_g / 2,
-//   z += (tanh(g / 2) + 1) (o / 2).
-// The row statistics come from the shared-memory tiles; z stays an exact fp16 copy of the bf16 state.
+// [T2, c_z] buffer.  Both LayerNorms are folded into the weights (W' = W gamma; W_o' fp16 against the
+// fp16 t, W_g' bf16 against the bf16 state itself), so NOTHING has to touch the tiles between the TMA
+// load and the MMA: the MMAs start as soon as the tiles land, four warps take the row statistics of t
+// and z from the same tiles meanwhile, and the epilogue applies them:
+//   o / 2 = (rstd_t / 2) (acc_o - mean_t c1_o) + c0_o / 2,  g / 2 = (rstd_z / 2) (acc_g - mean_z c1_g) + c0_g / 2,
+//   z += (tanh(g / 2) + 1) (o / 2)        with c1 = sum_k W'[n][k], c0 = sum_k W[n][k] beta[k].
 //
-// A tile is two 64-position chunks (s, i, j0).  Per tile the producer brings the t chunk
-// [c_h][64] and the z chunk [64][c_z]; the MMA warp issues t^T W_o'^T and z W_g'^T into one TMEM
-// buffer; eight epilogue warps combine them with the residual, write the new z into the z tile in
-// shared memory and TMA-store it (clipped at the row end, so nothing outside sum N^2 is touched).
+// A tile is two 64-position chunks (s, i, j0).  The t chunks and the z tile travel through rings of
+// their own: a t stage is free once the MMAs and the statistics have read it, a z stage only after the
+// epilogue has written the new z into it and the TMA stores have read it (clipped at the row end, so
+// nothing outside sum N^2 is touched) -- so the t loads of the tile after next start one epilogue early.
 #include <cstring>
 
 #include "fast.cuh"
@@ -30,8 +30,6 @@ struct TriOutParams {
   CUtensorMap tmap[TO_MAXB];     // {N (j), N (i), c_h, 1}, box {64, 1, c_h, 1}
   CUtensorMap womap;             // {c_h, c_z}, box {64, c_z}
   CUtensorMap wgmap;             // {c_z, c_z}, box {64, c_z}
-  CUtensorMap wgxmap, woxmap;    // augmentation columns of W_g / W_o: {8, rows}, box {8, 64}, no swizzle
-  int wgx_row0, wgx_rows, wox_rows;   // first row of W_g in its table; rows per region of each table
   long long chunk_off[TO_MAXB + 1];
   int N[TO_MAXB];
   int B, c_z, c_h;
@@ -61,8 +59,8 @@ __device__ inline float to_tanh(float x) {
 
 __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_constant__ TriOutParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[11];
-  __shared__ float2 sStats[2][128];        // per stage and position: (rstd_t / 2, rstd_z / 2)
+  __shared__ __align__(8) unsigned long long bars[17];
+  __shared__ float4 sStats[2][128];        // per z stage and position: (rstd_t / 2, rstd_z / 2, -mean_t rstd_t / 2, -mean_z rstd_z / 2)
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_flag;
   unsigned char* smem = smem_raw + ((1024 - (smem_u32(smem_raw) & 1023)) & 1023);
@@ -72,33 +70,35 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   const int wo_bytes = hslab * wo_slab, wg_bytes = zslab * wg_slab;
   const int t_chunk = c_h * 128;                             // [c_h][64 positions]
   const int z_slab = 128 * 128;                              // [128 positions][64 channels]
-  const int stage_bytes = 2 * t_chunk + zslab * z_slab;
+  const int t_stage = 2 * t_chunk, z_stage = zslab * z_slab;
   unsigned char* sWo = smem;
   unsigned char* sWg = sWo + wo_bytes;
-  unsigned char* sSt = sWg + wg_bytes;                       // 2 stages: t chunks then z slabs
-  float* sCo = reinterpret_cast<float*>(sSt + 2 * stage_bytes);   // c0 of W_o / 2 per channel
-  float* sCg = sCo + c_z;                                         // c0 of W_g / 2
-  const int wx_region = c_z * 16;                                 // one 8-column region of a weight augmentation
-  unsigned char* sWox = reinterpret_cast<unsigned char*>(sCg + c_z);   // [2 regions][c_z][8] fp16, K-major no swizzle
-  unsigned char* sWgx = sWox + 2 * wx_region;
-  unsigned char* sZx = sWgx + 2 * wx_region;                      // 2 stages x [2 regions][128 positions][8] fp16 (K-major)
-  unsigned char* sTx = sZx + 2 * 2 * 2048;                        // 2 stages x [2 k groups][16 position groups][8 k][8 positions] (MN-major)
-  unsigned long long* afull = bars;
-  unsigned long long* aempty = bars + 2;
-  unsigned long long* tfull = bars + 4;
-  unsigned long long* tempty = bars + 6;
-  unsigned long long* wfull = bars + 8;
-  unsigned long long* aconv = bars + 9;  // [2]
+  unsigned char* sT = sWg + wg_bytes;                        // 2 stages of the two t chunks
+  unsigned char* sZ = sT + 2 * t_stage;                      // 2 stages of the z tile
+  float* sCo = reinterpret_cast<float*>(sZ + 2 * z_stage);   // c0 of W_o / 2 per channel
+  float* sCg = sCo + c_z;                                    // c0 of W_g / 2
+  float* sKo = sCg + c_z;                                    // c1 of W_o
+  float* sKg = sKo + c_z;                                    // c1 of W_g
+  unsigned long long* tfullb = bars;        // [2] t chunks landed
+  unsigned long long* tfree = bars + 2;     // [2] MMAs and statistics have read them
+  unsigned long long* zfullb = bars + 4;    // [2] z tile landed
+  unsigned long long* zfree = bars + 6;     // [2] MMAs have read it, the new z has been stored from it
+  unsigned long long* tfull = bars + 8;     // [2] accumulators complete
+  unsigned long long* tempty = bars + 10;   // [2]
+  unsigned long long* sconv = bars + 12;    // [2] statistics published
+  unsigned long long* wfull = bars + 14;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&afull[s], 1);
-      mbar_init(&aempty[s], 1 + 4 * (p.c_z / 64));   // MMA commit + the storing epilogue lanes
+      mbar_init(&tfullb[s], 1);
+      mbar_init(&tfree[s], 1 + 4);                   // MMA commit + the four statistics warps
+      mbar_init(&zfullb[s], 1);
+      mbar_init(&zfree[s], 1 + 4 + 4 * (p.c_z / 64)); // MMA commit + the statistics warps + the storing epilogue lanes
       mbar_init(&tfull[s], 1);
       mbar_init(&tempty[s], 8);
-      mbar_init(&aconv[s], 4);
+      mbar_init(&sconv[s], 4);
     }
     mbar_init(wfull, 1);
     mbar_fence_init();
@@ -107,11 +107,9 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   for (int n = threadIdx.x; n < c_z; n += TO_THREADS) {
     sCo[n] = 0.5f * p.c01o[n].x;
     sCg[n] = 0.5f * p.c01g[n].x;
+    sKo[n] = p.c01o[n].y;
+    sKg[n] = p.c01g[n].y;
   }
-  // activation augmentation tiles start as zeros; the converters fill the three mean columns of every position
-  for (int idx = threadIdx.x; idx < 2 * (2 * 2048 + 4096) / 16; idx += TO_THREADS)
-    *reinterpret_cast<uint4*>(sZx + idx * 16) = make_uint4(0, 0, 0, 0);
-  fence_proxy_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -123,12 +121,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
   if (warp == 0) {
     // ------------------------------------------------------------------ producer (lane q decodes and loads chunk q)
     if (lane == 0) {
-      mbar_expect_tx(wfull, wo_bytes + wg_bytes + 4 * wx_region);
-      for (int reg = 0; reg < 2; ++reg)
-        for (int r = 0; r < c_z; r += 64) {
-          tma_load_2d(sWox + reg * wx_region + r * 16, &p.woxmap, wfull, 0, reg * p.wox_rows + r);
-          tma_load_2d(sWgx + reg * wx_region + r * 16, &p.wgxmap, wfull, 0, reg * p.wgx_rows + p.wgx_row0 + r);
-        }
+      mbar_expect_tx(wfull, wo_bytes + wg_bytes);
       for (int sl = 0; sl < hslab; ++sl) tma_load_2d(sWo + sl * wo_slab, &p.womap, wfull, sl * 64, 0);
       for (int sl = 0; sl < zslab; ++sl) tma_load_2d(sWg + sl * wg_slab, &p.wgmap, wfull, sl * 64, 0);
     }
@@ -137,20 +130,23 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       int s = 0, i = 0, j0 = 0;
       const bool valid = lane < 2 && to_decode(p, 2 * t + lane, s, i, j0);
+      const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
       if (lane == 0) {
-        const int nvalid = (2 * t + 1 < nchunks) ? 2 : 1;
-        mbar_wait(&aempty[stage], phase ^ 1, ab);
-        mbar_expect_tx(&afull[stage], nvalid * (t_chunk + zslab * 64 * 128));
+        mbar_wait(&tfree[stage], phase ^ 1, ab);
+        mbar_expect_tx(&tfullb[stage], nvalid * t_chunk);
       }
       __syncwarp();
-      if (valid) {
-        unsigned char* st = sSt + stage * stage_bytes;
-        tma_load_4d(st + lane * t_chunk, &p.tmap[s], &afull[stage], j0, i, 0, 0);
+      if (valid) tma_load_4d(sT + stage * t_stage + lane * t_chunk, &p.tmap[s], &tfullb[stage], j0, i, 0, 0);
+      if (lane == 0) {
+        mbar_wait(&zfree[stage], phase ^ 1, ab);
+        mbar_expect_tx(&zfullb[stage], nvalid * zslab * 64 * 128);
+      }
+      __syncwarp();
+      if (valid)
         for (int sl = 0; sl < zslab; ++sl)
           for (int sub = 0; sub < 2; ++sub)      // 32-position boxes (the size the epilogue warps store)
-            tma_load_4d(st + 2 * t_chunk + sl * z_slab + (lane * 64 + sub * 32) * 128, &p.zmap[s], &afull[stage], sl * 64,
+            tma_load_4d(sZ + stage * z_stage + sl * z_slab + (lane * 64 + sub * 32) * 128, &p.zmap[s], &zfullb[stage], sl * 64,
                         j0 + sub * 32, i, 0);
-      }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp == 1) {
@@ -159,50 +155,46 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     int stage = 0;
     unsigned phase = 0, tph0 = 0, tph1 = 0;
     unsigned n = 0;
-    const unsigned idesc_t = idesc_f16(128, c_z, 1, 0, FMT_F16, FMT_F16);   // A = t (fp16, MN-major), W_o' fp16
-    const unsigned idesc_z = idesc_f16(128, c_z, 0, 0, FMT_F16, FMT_F16);   // A = z tile converted to fp16, W_g' fp16
+    const unsigned idesc_t = idesc_f16(128, c_z, 1, 0, FMT_F16, FMT_F16);     // A = t (fp16, MN-major), W_o' fp16
+    const unsigned idesc_z = idesc_f16(128, c_z, 0, 0, FMT_BF16, FMT_BF16);   // A = the bf16 z tile, W_g' bf16
     const unsigned long long wo_desc = desc_kmajor_sw128(smem_u32(sWo)), wg_desc = desc_kmajor_sw128(smem_u32(sWg));
     const unsigned wo16 = (unsigned)wo_slab >> 4, wg16 = (unsigned)wg_slab >> 4, z16 = (unsigned)z_slab >> 4;
-    const unsigned long long wox_desc = desc_kmajor_nosw(smem_u32(sWox), wx_region, 128);
-    const unsigned long long wgx_desc = desc_kmajor_nosw(smem_u32(sWgx), wx_region, 128);
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const unsigned buf = n & 1;
       if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
       else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
-      mbar_wait(&aconv[stage], phase, ab);
-      tc_fence_after();
-      const unsigned st = smem_u32(sSt + stage * stage_bytes);
       const unsigned d1 = tmem_base + buf * 256, d2 = d1 + c_z;
-      const unsigned long long t_desc = desc_mnmajor_sw128(st, t_chunk, 1024);
-      const unsigned long long z_desc = desc_kmajor_sw128(st + 2 * t_chunk);
+      mbar_wait(&tfullb[stage], phase, ab);
+      tc_fence_after();
+      const unsigned long long t_desc = desc_mnmajor_sw128(smem_u32(sT + stage * t_stage), t_chunk, 1024);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)                       // K = channels of t, 16 per step (2048 bytes of the MN-major tile)
         if (ks < c_h / 16 && elect_one())
           umma_bf16(d1, t_desc + ks * 128, wo_desc + ((ks >> 2) * wo16 + (ks & 3) * 2), idesc_t, ks != 0);
+      if (elect_one()) tc_commit(&tfree[stage]);
+      __syncwarp();
+      mbar_wait(&zfullb[stage], phase, ab);
+      tc_fence_after();
+      const unsigned long long z_desc = desc_kmajor_sw128(smem_u32(sZ + stage * z_stage));
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
         if (ks < c_z / 16 && elect_one())
           umma_bf16(d2, z_desc + ((ks >> 2) * z16 + (ks & 3) * 2), wg_desc + ((ks >> 2) * wg16 + (ks & 3) * 2), idesc_z, ks != 0);
-      // augmentation K steps: the mean terms of both LayerNorms.  t side: MN-major without swizzle (8 positions
-      // further = 128 bytes, 8 k further = 2048); z side: K-major without swizzle (8 k further = 2048, 8 rows = 128).
       if (elect_one()) {
-        umma_bf16(d1, desc_kmajor_nosw(smem_u32(sTx + stage * 4096), 2048, 128), wox_desc, idesc_t, 1);
-        umma_bf16(d2, desc_kmajor_nosw(smem_u32(sZx + stage * 4096), 2048, 128), wgx_desc, idesc_z, 1);
         tc_commit(&tfull[buf]);
-        tc_commit(&aempty[stage]);
+        tc_commit(&zfree[stage]);
       }
       __syncwarp();
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------------ converters (4 warps, one position per thread)
+    // ------------------------------------------------------------------ statistics (4 warps, one position per thread)
     const int row = (warp - 2) * 32 + lane;
     const int q = row >> 6;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
-      mbar_wait(&afull[stage], phase, ab);
-      unsigned char* st = sSt + stage * stage_bytes;
+      mbar_wait(&tfullb[stage], phase, ab);
       // Statistics of t over channels (columns of the MN-major fp16 tile).  Eight lanes share a group of eight
       // positions: lane cg sums channels cg, cg + 8, ... with 16-byte loads (8 positions each), then a
       // reduce-scatter over the eight lanes leaves every lane with the two sums of one position -- its own row.
@@ -210,7 +202,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       {
         const int cg = lane & 7, pgl = ((warp - 2) * 4 + (lane >> 3)) & 7;      // position group inside the 64-position chunk
         float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, q8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        const unsigned char* tb = st + q * t_chunk + cg * 128 + ((pgl ^ cg) << 4);   // channel c = cc * 8 + cg: c & 7 = cg
+        const unsigned char* tb = sT + stage * t_stage + q * t_chunk + cg * 128 + ((pgl ^ cg) << 4);   // channel c = cc * 8 + cg: c & 7 = cg
 #pragma unroll 4
         for (int cc = 0; cc < c_h / 8; ++cc) {
           const uint4 v = *reinterpret_cast<const uint4*>(tb + cc * 1024);
@@ -247,6 +239,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
           tq = kq + __shfl_xor_sync(0xffffffffu, sq_, 1);
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tfree[stage]);
       // t arrives scaled by 1 / N_s (see the contraction); LayerNorm is scale-free once eps is scaled alike
       float eps_t = p.eps;
       {
@@ -255,26 +249,34 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       }
       const float tmean = ts / (float)c_h;
       const float trstd = rsqrtf(fmaxf(tq / (float)c_h - tmean * tmean, 0.f) + eps_t);
-      // z row: convert to fp16 in place and take its statistics
+      // z row: statistics of the bf16 tile (read only)
+      mbar_wait(&zfullb[stage], phase, ab);
       float zs, zq;
-      convert_row_bf16_to_f16(st + 2 * t_chunk, zslab, z_slab, row, zs, zq);
+      {
+        float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
+        const unsigned char* zt = sZ + stage * z_stage;
+        for (int g8 = 0; g8 < c_z / 8; ++g8) {
+          const uint4 v = *reinterpret_cast<const uint4*>(zt + (g8 >> 3) * z_slab + sw128_off(row, g8 & 7));
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+            s4[e] += lo + hi;
+            q4[e] = fmaf(lo, lo, q4[e]);
+            q4[e] = fmaf(hi, hi, q4[e]);
+          }
+        }
+        zs = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        zq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
+      }
       const float zmean = zs / (float)c_z;
       const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
-      sStats[stage][row] = make_float2(0.5f * trstd, 0.5f * zrstd);
-      {
-        const __half th = __float2half_rn(-tmean), tl = __float2half_rn(-tmean - __half2float(th));
-        const __half zh = __float2half_rn(-zmean), zl = __float2half_rn(-zmean - __half2float(zh));
-        // t side: element (position, k) at (position / 8) * 128 + k * 16 + (position % 8) * 2
-        __half* tx = reinterpret_cast<__half*>(sTx + stage * 4096 + (row >> 3) * 128 + (row & 7) * 2);
-        tx[0] = th; tx[8] = tl; tx[16] = th;
-        // z side: row's 16 bytes (k = 0 .. 7)
-        __half2 p0 = __halves2half2(zh, zl), p1 = __halves2half2(zh, __float2half_rn(0.f));
-        *reinterpret_cast<uint2*>(sZx + stage * 4096 + row * 16) =
-            make_uint2(*reinterpret_cast<unsigned*>(&p0), *reinterpret_cast<unsigned*>(&p1));
-      }
-      fence_proxy_async_smem();
+      sStats[stage][row] = make_float4(0.5f * trstd, 0.5f * zrstd, -0.5f * trstd * tmean, -0.5f * zrstd * zmean);
       __syncwarp();
-      if (lane == 0) mbar_arrive(&aconv[stage]);
+      if (lane == 0) {
+        mbar_arrive(&sconv[stage]);
+        mbar_arrive(&zfree[stage]);
+      }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 6) {
@@ -287,13 +289,13 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     long long n = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++n) {
       const int buf = (int)(n & 1);
-      unsigned char* st = sSt + stage * stage_bytes;
-      unsigned char* zrow = st + 2 * t_chunk;
-      mbar_wait(&tfull[buf], tph[buf], ab);         // MMAs done, hence the statistics are published too
+      unsigned char* zrow = sZ + stage * z_stage;
+      mbar_wait(&sconv[stage], phase, ab);
+      const float4 stt = sStats[stage][row];
+      const float trh = stt.x, zrh = stt.y, tmh = stt.z, zmh = stt.w;
+      mbar_wait(&tfull[buf], tph[buf], ab);
       tph[buf] ^= 1;
       tc_fence_after();
-      const float2 stt = sStats[stage][row];
-      const float trh = stt.x, zrh = stt.y;
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       for (int c0 = half * (c_z / 2); c0 < (half + 1) * (c_z / 2); c0 += 32) {
         unsigned r1[32], r2[32];
@@ -307,18 +309,24 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
           uint4* ptr = reinterpret_cast<uint4*>(zp + sw128_off(row, chunk16));
           uint4 v = *ptr;
           unsigned w[4] = {v.x, v.y, v.z, v.w};
-          const float4 co0 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8), co1 = *reinterpret_cast<const float4*>(sCo + c0 + ch * 8 + 4);
-          const float4 cg0 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8), cg1 = *reinterpret_cast<const float4*>(sCg + c0 + ch * 8 + 4);
-          const float ko[8] = {co0.x, co0.y, co0.z, co0.w, co1.x, co1.y, co1.z, co1.w};
-          const float kg[8] = {cg0.x, cg0.y, cg0.z, cg0.w, cg1.x, cg1.y, cg1.z, cg1.w};
+          const int cb = c0 + ch * 8;
+          const float4 co0 = *reinterpret_cast<const float4*>(sCo + cb), co1 = *reinterpret_cast<const float4*>(sCo + cb + 4);
+          const float4 cg0 = *reinterpret_cast<const float4*>(sCg + cb), cg1 = *reinterpret_cast<const float4*>(sCg + cb + 4);
+          const float4 ko0 = *reinterpret_cast<const float4*>(sKo + cb), ko1 = *reinterpret_cast<const float4*>(sKo + cb + 4);
+          const float4 kg0 = *reinterpret_cast<const float4*>(sKg + cb), kg1 = *reinterpret_cast<const float4*>(sKg + cb + 4);
+          // per channel: c0 / 2 - mean rstd c1 / 2, the part of the LayerNorm that does not depend on the accumulator
+          const float bo[8] = {fmaf(tmh, ko0.x, co0.x), fmaf(tmh, ko0.y, co0.y), fmaf(tmh, ko0.z, co0.z), fmaf(tmh, ko0.w, co0.w),
+                               fmaf(tmh, ko1.x, co1.x), fmaf(tmh, ko1.y, co1.y), fmaf(tmh, ko1.z, co1.z), fmaf(tmh, ko1.w, co1.w)};
+          const float bg[8] = {fmaf(zmh, kg0.x, cg0.x), fmaf(zmh, kg0.y, cg0.y), fmaf(zmh, kg0.z, cg0.z), fmaf(zmh, kg0.w, cg0.w),
+                               fmaf(zmh, kg1.x, cg1.x), fmaf(zmh, kg1.y, cg1.y), fmaf(zmh, kg1.z, cg1.z), fmaf(zmh, kg1.w, cg1.w)};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            const float2 zo = unpack_h2(w[e]);         // the z tile holds fp16 after conversion
-            const float oh0 = fmaf(trh, __uint_as_float(r1[n0]), ko[e * 2]), oh1 = fmaf(trh, __uint_as_float(r1[n0 + 1]), ko[e * 2 + 1]);
-            const float t0 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0]), kg[e * 2]));
-            const float t1 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0 + 1]), kg[e * 2 + 1]));
-            __nv_bfloat162 hh = __floats2bfloat162_rn(fmaf(oh0, t0, oh0) + zo.x, fmaf(oh1, t1, oh1) + zo.y);
+            const float z0 = __uint_as_float(w[e] << 16), z1 = __uint_as_float(w[e] & 0xffff0000u);   // the bf16 state
+            const float oh0 = fmaf(trh, __uint_as_float(r1[n0]), bo[e * 2]), oh1 = fmaf(trh, __uint_as_float(r1[n0 + 1]), bo[e * 2 + 1]);
+            const float t0 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0]), bg[e * 2]));
+            const float t1 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0 + 1]), bg[e * 2 + 1]));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(fmaf(oh0, t0, oh0) + z0, fmaf(oh1, t1, oh1) + z1);
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);
@@ -340,7 +348,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
                        j0 + sub * 32, i, 0);
         tma_store_commit();
         tma_store_wait_read0();
-        mbar_arrive(&aempty[stage]);
+        mbar_arrive(&zfree[stage]);
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
@@ -362,8 +370,7 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
   const float2* c01g = (const float2*)tp.c01g;
   const int zslab = c_z / 64, hslab = c_h / 64;
   const size_t smem = (size_t)hslab * c_z * 128 + (size_t)zslab * c_z * 128 +
-                      2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 2 * c_z * 4 + 4 * (size_t)c_z * 16 +
-                      2 * (2 * 2048 + 4096) + 1024;
+                      2 * ((size_t)2 * c_h * 128 + (size_t)zslab * 128 * 128) + 4 * c_z * 4 + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(tri_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -388,14 +395,6 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
       const unsigned long long dims2[2] = {(unsigned long long)c_z, (unsigned long long)c_z};
       const unsigned long long strides2[1] = {(unsigned long long)c_z * 2};
       if (!make_tmap_bf16(&p.wgmap, wg, 2, dims2, strides2, box)) return cuda_fail("tri_out W_g map");
-      const unsigned long long xstr[1] = {16};
-      const unsigned xbox[2] = {8, 64};
-      const unsigned long long gdims[2] = {8, (unsigned long long)2 * tp.aug1_rows}, odims[2] = {8, (unsigned long long)2 * c_z};
-      if (!make_tmap_16bit(&p.wgxmap, tp.aug1, 2, gdims, xstr, xbox, 0)) return cuda_fail("tri_out W_g augmentation map");
-      if (!make_tmap_16bit(&p.woxmap, tp.augo, 2, odims, xstr, xbox, 0)) return cuda_fail("tri_out W_o augmentation map");
-      p.wgx_row0 = 4 * c_h;
-      p.wgx_rows = tp.aug1_rows;
-      p.wox_rows = c_z;
     }
     p.chunk_off[0] = 0;
     for (int l = 0; l < TO_MAXB; ++l) {
