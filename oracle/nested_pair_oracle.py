@@ -26,6 +26,9 @@ What each function follows:
   col_attn_pairbias    the second (column-wise, "ending node") triangle attention of Sec. 4.3: the mirror image of
                        row_attn_pairbias; pinned by the exact transposition relation to it, library attention, and
                        scalar loops.
+  single_attn_pairbias the pair-biased single attention of Sec. 4.3 (tokens attend tokens of the same sample, logits
+                       biased by a projection of the pair state); pinned by library attention with an additive mask,
+                       scalar loops, and its reduction to the token-order attention when the bias weights are zero.
   segment_reduce       Eq. 4 (pair reduction) and the mean of Eq. 1 line 3; App. A batch-axis
                        convention (``[1,2],[3,4]`` sums to ``[3,7]``).
   token_update         Eq. 1 line 3: ``X~ = X + g(mean_b P~[a,b,:])`` with ``g`` a bias-free projection.
@@ -296,6 +299,44 @@ def col_attn_pairbias(z, lengths, W, H, d, eps=LN_EPS, dtype=np.float64, return_
             parts.append(dict(q=q, k=k, v=v, A=A, o=ov))
         o += n * n
     res = np.concatenate(out, axis=0) if out else z.copy()
+    return (res, parts) if return_parts else res
+
+
+def single_attn_pairbias(x, z, lengths, W, H, d, eps=LN_EPS, dtype=np.float64, return_parts=False):
+    """Pair-biased single attention (Sec. 4.3: the tokens of a sample attend the tokens of the same sample, the
+    logits biased by a projection of the pair state), with residual, per sample:
+        xh = LN_x(x); q,k,v = xh W_{q,k,v}^T viewed [N,H,d]; g = sig(xh W_g^T); bias = LN_z(z) W_b^T [N,N,H]
+        S[h,j,k] = <q[j,h,:], k[k,h,:]>/sqrt(d) + bias[j,k,h];  A = softmax_k S
+        o[j,h,:] = sum_k A[h,j,k] v[k,h,:];  x <- x + (g * o) W_o^T
+    x [T1, c_s] packed tokens, z [T2, c_z] packed pair state (read only).
+    """
+    x = np.asarray(x, dtype=dtype)
+    z = np.asarray(z, dtype=dtype)
+    Wd = {k: (None if v is None else np.asarray(v, dtype=dtype)) for k, v in W.items()}
+    scale = 1.0 / np.sqrt(float(d))
+    out, parts, ot, op_ = [], [], 0, 0
+    for n in (int(v) for v in lengths):
+        if n == 0:
+            continue
+        xs = x[ot:ot + n]
+        zs = z[op_:op_ + n * n].reshape(n, n, z.shape[1])
+        xh = layer_norm(xs, Wd["ln_gamma"], Wd["ln_beta"], eps)
+        q = (xh @ Wd["W_q"].T).reshape(n, H, d)
+        k = (xh @ Wd["W_k"].T).reshape(n, H, d)
+        v = (xh @ Wd["W_v"].T).reshape(n, H, d)
+        bias = layer_norm(zs, Wd["ln_z_gamma"], Wd["ln_z_beta"], eps) @ Wd["W_b"].T      # [j, k, H]
+        S = np.matmul(q.transpose(1, 0, 2), k.transpose(1, 2, 0)) * scale + bias.transpose(2, 0, 1)   # [H, j, k]
+        S = S - S.max(axis=-1, keepdims=True)
+        A = np.exp(S)
+        A = A / A.sum(axis=-1, keepdims=True)
+        ov = np.matmul(A, v.transpose(1, 0, 2)).transpose(1, 0, 2).reshape(n, H * d)
+        ov = sigmoid(xh @ Wd["W_g"].T) * ov
+        out.append(xs + ov @ Wd["W_o"].T)
+        if return_parts:
+            parts.append(dict(q=q, k=k, v=v, bias=bias, A=A, o=ov))
+        ot += n
+        op_ += n * n
+    res = np.concatenate(out, axis=0) if out else x.copy()
     return (res, parts) if return_parts else res
 
 

@@ -146,6 +146,16 @@ def make_transition_weights(cfg: Config, block: int = 0, expansion: int = 4) -> 
                 W_2=st.weight(c, hid))
 
 
+def make_single_attn_weights(cfg: Config, block: int = 0) -> dict:
+    """Weights of the pair-biased single attention of one block (tokens of width c_s, bias from the pair state of
+    width c_z, H heads of d).  A stream of its own (seed + 104729 * (block + 1)): the frozen draws are unchanged."""
+    st = _Stream(cfg.seed + 104729 * (block + 1), cfg.dtype == "bf16")
+    c, cz, Hd = cfg.c_s, cfg.c_z, cfg.H * cfg.d
+    return dict(ln_gamma=st.ln_gamma(c), ln_beta=st.ln_beta(c), W_q=st.weight(Hd, c), W_k=st.weight(Hd, c),
+                W_v=st.weight(Hd, c), W_g=st.weight(Hd, c), W_o=st.weight(c, Hd),
+                ln_z_gamma=st.ln_gamma(cz), ln_z_beta=st.ln_beta(cz), W_b=st.weight(cfg.H, cz))
+
+
 def make_token_weights(st: _Stream, cfg: Config) -> dict:
     """Weights of the single-ragged special case: attention over the token axis, no LN/gate/bias."""
     c, Hd = cfg.c_z, cfg.H * cfg.d
