@@ -79,6 +79,10 @@ def kernel_work(cfg: wl.Config):
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
     w["token_update"] = dict(bytes=T1 * (c_z + 2 * c_s) * e + c_s * c_z * e, flops=2 * T1 * c_s * c_z)
+    # pair-biased single attention: the bias planes are the only part that touches the pair state (read z, write H values)
+    w["single_attn_bias"] = dict(bytes=T2 * (c_z + H) * e, flops=2 * T2 * c_z * H)
+    # its attention core runs over the token axis: one exponential per (query, key, head) of every sample
+    w["single_attn_core"] = dict(bytes=T1 * 4 * Hd * e + T2 * H * e, flops=4 * T2 * Hd, exps=T2 * H)
     # SwiGLU pair transition with expansion 4: read and write the state once, three GEMMs of c_z x 4 c_z per row
     w["transition"] = w["generic_transition"] = dict(bytes=2 * T2 * c_z * e, flops=6 * T2 * c_z * 4 * c_z)
     return w
@@ -243,6 +247,8 @@ def main():
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
     ap.add_argument("--only-transition", action="store_true",
                     help="run just the pair-transition measurement (the row after the block; for ncu captures)")
+    ap.add_argument("--only-single-attn", action="store_true",
+                    help="run just the pair-biased single attention measurement (for ncu captures)")
     ap.add_argument("--only-col-attn", action="store_true",
                     help="run just the column-wise attention measurement (for ncu captures)")
     ap.add_argument("--only-tri-mul-in", action="store_true",
@@ -360,6 +366,42 @@ def main():
             out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
         return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
 
+    def single_attn_pass(n_calls):
+        """Pair-biased single attention (a row after the block): tokens [T1, c_s] attend within their sample, bias from
+        the pair state the first block's broadcast produces.  Not part of the step or of `value`."""
+        if cfg.kind != "pair":
+            return None
+        w0 = stack.W[0]
+        b = w0["broadcast"]
+        nt.nt_pair_broadcast(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        Ws = {k: torch.from_numpy(np.ascontiguousarray(v)).to("cuda", stack.dtype) for k, v in wl.make_single_attn_weights(cfg).items()}
+        ws = torch.empty(max(nt.nt_single_attn_workspace_bytes(stack.dtype, cfg.lengths, cfg.c_s, cfg.H, cfg.d), 256), dtype=torch.uint8, device="cuda")
+        xs = x0.clone()
+        for _ in range(3):
+            nt.nt_single_attn_pairbias(stack.L, Ws, cfg.H, cfg.d, 1e-5, xs, stack.z, ws)
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            nt.nt_single_attn_pairbias(stack.L, Ws, cfg.H, cfg.d, 1e-5, xs, stack.z, ws)
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        out = {}
+        for k, v in tp.items():
+            name = "single_attn_core" if k in ("attn_core", "generic_attn_core") else k     # token-axis work, not the pair rows'
+            wk = dict(kernel_work(cfg))
+            wk[k] = wk.get(name, wk.get(k))
+            r = roofline_entry(k, v[0], v[1], n_calls, wk, peaks_t, kind_t) if wk.get(k) else None
+            out[name] = dict(r, kernel=name) if r else dict(kernel=name, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
+
+    if args.only_single_attn:
+        res = dict(single_attn=single_attn_pass(steps))
+        if rank == 0:
+            print(json.dumps(res))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.only_transition or args.only_tri_mul_in or args.only_col_attn:
         res = (dict(pair_transition=transition_pass(steps)) if args.only_transition else
                dict(tri_mul_in=tri_mul_in_pass(steps)) if args.only_tri_mul_in else dict(col_attn=col_attn_pass(steps)))
@@ -430,7 +472,8 @@ def main():
     if roofline and cfg.name == "cfg2" and not args.force_generic:
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
-    next_rows = (dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps), col_attn=col_attn_pass(steps))
+    next_rows = (dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps), col_attn=col_attn_pass(steps),
+                      single_attn=single_attn_pass(steps))
                  if not args.force_generic else None)
 
     # ---- end to end through the public API with host buffers

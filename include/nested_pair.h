@@ -87,6 +87,15 @@ typedef struct {                /* row-wise attention; all device, dtype = dt   
   const void *W_o;                          /* [c, H*d]                                     */
 } nt_attn_weights;
 
+typedef struct {                /* pair-biased single attention; all device, dtype = dt     */
+  const void *ln_gamma, *ln_beta;           /* [c_s]    LayerNorm of the tokens             */
+  const void *W_q, *W_k, *W_v;              /* [H*d, c_s]                                   */
+  const void *W_g;                          /* [H*d, c_s]                                   */
+  const void *W_o;                          /* [c_s, H*d]                                   */
+  const void *ln_z_gamma, *ln_z_beta;       /* [c_z]    LayerNorm of the pair state         */
+  const void *W_b;                          /* [H, c_z]                                     */
+} nt_single_attn_weights;
+
 /*
  * nt_offsets_build -- prefix sums and position decode (Sec. 3.1 offsets o; Fig. 2 two-level row
  * splits; Eq. 3 coordinate map; the rows/columns gather indices of the program figure).
@@ -166,6 +175,20 @@ nt_status nt_row_attn_pairbias(const nt_layout *L, nt_order order, nt_dtype dt,
 nt_status nt_col_attn_pairbias(const nt_layout *L, nt_dtype dt, int32_t c, int32_t H, int32_t d,
                                const nt_attn_weights *W, float ln_eps, void *z,
                                void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
+ * nt_single_attn_pairbias -- pair-biased single attention (Sec. 4.3): the tokens of a sample attend the tokens of
+ * the same sample, the logits biased by a projection of the sample's pair state; one segmented call for the
+ * whole batch (Sec. 3.3 "Attention through packed blocks": segments from the offsets).
+ *   xh = LN(x); q,k,v = xh W_{q,k,v}^T; g = sig(xh W_g^T); bias[j,k,h] = (LN_z(z_jk) W_b^T)[h]
+ *   S[h,j,k] = <q_jh, k_kh>/sqrt(d) + bias[j,k,h]; P = softmax_k S; o_jh = sum_k P[h,j,k] v_kh; x += (g * o) W_o^T
+ *   x [T1, c_s] in/out (in place); z [T2, c_z] in (not modified).  No weight pointer may be NULL.  d <= 128.
+ *   Workspace: nt_single_attn_workspace_bytes (0 when the batch is empty or an argument is invalid).
+ */
+nt_status nt_single_attn_pairbias(const nt_layout *L, nt_dtype dt, int32_t c_s, int32_t c_z, int32_t H, int32_t d,
+                                  const nt_single_attn_weights *W, float ln_eps, void *x, const void *z,
+                                  void *workspace, size_t workspace_bytes, nt_stream stream);
+size_t nt_single_attn_workspace_bytes(nt_dtype dt, const int64_t *lengths_h, int32_t B, int32_t c_s, int32_t H, int32_t d);
 
 /*
  * nt_segment_reduce -- segmented sum or mean of contiguous row groups (Eq. 4 pair reduction; the

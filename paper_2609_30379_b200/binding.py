@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3:
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
 EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-           "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
+           "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
+           "nt_single_attn_workspace_bytes", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
            "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
 
@@ -52,6 +53,11 @@ class nt_attn_weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("ln_gamma", "ln_beta", "W_q", "W_k", "W_v", "W_b", "W_g", "W_o")]
 
 
+class nt_single_attn_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ln_gamma", "ln_beta", "W_q", "W_k", "W_v", "W_g", "W_o", "ln_z_gamma",
+                                          "ln_z_beta", "W_b")]
+
+
 class nt_transition_weights(C.Structure):
     _fields_ = [(k, C.c_void_p) for k in ("ln_gamma", "ln_beta", "W_a", "W_b", "W_2")]
 
@@ -68,6 +74,10 @@ def _load() -> C.CDLL:
     lib.nt_pair_broadcast_static.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.nt_tri_mul_out.argtypes = [C.POINTER(nt_layout), i32, i32, i32, C.POINTER(nt_trimul_weights), f32, vp, vp, sz, vp]
     lib.nt_tri_mul_in.argtypes = lib.nt_tri_mul_out.argtypes
+    lib.nt_single_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_single_attn_weights),
+                                            f32, vp, vp, vp, sz, vp]
+    lib.nt_single_attn_workspace_bytes.argtypes = [i32, vp, i32, i32, i32, i32]
+    lib.nt_single_attn_workspace_bytes.restype = sz
     lib.nt_col_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, C.POINTER(nt_attn_weights), f32, vp, vp, sz, vp]
     lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
                                          f32, vp, vp, sz, vp]
@@ -90,7 +100,8 @@ def _load() -> C.CDLL:
     lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
     lib.nt_profile_end.restype = i32
     for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-                 "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_segment_reduce", "nt_token_update"):
+                 "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias", "nt_segment_reduce",
+                 "nt_token_update"):
         getattr(lib, name).restype = i32
     return lib
 
@@ -214,6 +225,21 @@ def nt_row_attn_pairbias(L: Layout, order: int, W: dict, H: int, d: int, ln_eps,
                                   _ptr(zx), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                   _stream(stream))
     _check(st, "nt_row_attn_pairbias")
+
+
+def nt_single_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, x, z, workspace, stream=None):
+    """Pair-biased single attention: x [T1, c_s] updated in place, z [T2, c_z] read only."""
+    c_s, c_z = int(W["W_q"].shape[1]), int(W["W_b"].shape[1])
+    w = nt_single_attn_weights(*[_ptr(W[n]) for n, _ in nt_single_attn_weights._fields_])
+    st = lib.nt_single_attn_pairbias(C.byref(L.c), dtype_code(x.dtype), c_s, c_z, H, d, C.byref(w), float(ln_eps),
+                                     _ptr(x), _ptr(z), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _stream(stream))
+    _check(st, "nt_single_attn_pairbias")
+
+
+def nt_single_attn_workspace_bytes(dtype, lengths, c_s: int, H: int, d: int) -> int:
+    arr = (C.c_int64 * max(len(lengths), 1))(*[int(v) for v in lengths])
+    return int(lib.nt_single_attn_workspace_bytes(dtype_code(dtype), arr, len(lengths), c_s, H, d))
 
 
 def nt_col_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, z, workspace, stream=None):

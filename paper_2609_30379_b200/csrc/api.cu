@@ -146,6 +146,22 @@ static AttnWs carve_attn(void* ws, nt_dtype dt, const Totals& t, nt_order order,
   return w;
 }
 
+struct SingleWs { void *q, *k, *v, *o, *g, *xh, *bias; size_t bytes; };
+static SingleWs carve_single(void* ws, nt_dtype dt, const Totals& t, int c_s, int H, int d) {
+  Carver c(ws);
+  SingleWs w;
+  const size_t e = esize(dt), Hd = (size_t)H * d;
+  w.q = c.take(t.T1 * Hd * e);
+  w.k = c.take(t.T1 * Hd * e);
+  w.v = c.take(t.T1 * Hd * e);
+  w.o = c.take(t.T1 * Hd * e);
+  w.g = c.take(t.T1 * Hd * e);
+  w.xh = c.take(t.T1 * (size_t)c_s * e);
+  w.bias = c.take((size_t)H * t.cm * e);
+  w.bytes = c.off;
+  return w;
+}
+
 static size_t broadcast_ws_bytes(const Totals& t, int c_z) {
   return 2 * align_up((size_t)t.T1 * c_z * sizeof(float), 256);
 }
@@ -324,6 +340,66 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
   return NT_OK;
 }
 
+// Pair-biased single attention: token projections (T1 rows), the bias planes from the pair state (T2 rows, the
+// only part that touches the pair state), the segmented attention core over the token axis, gate + output projection.
+template <typename T>
+static nt_status single_attn_impl(const nt_layout* L, const Totals& tot, int c_s, int c_z, int H, int d,
+                                  const nt_single_attn_weights* W, float eps, void* x, const void* z, void* ws,
+                                  nt_dtype dt, cudaStream_t st) {
+  SingleWs w = carve_single(ws, dt, tot, c_s, H, d);
+  const int Hd = H * d;
+  const bool fast = dt == NT_BF16 && !g_force_generic && fast_single_attn_supported(c_s, c_z, H, d);
+  GroupIter it(L->lengths_h, L->B);
+  BatchMeta m;
+  while (it.next(m)) {
+    const long long trow0 = m.tok_off[0], trows = m.tok_off[m.B] - trow0;
+    const long long prow0 = m.pair_off[0], prows = m.pair_off[m.B] - prow0;
+    if (trows == 0) continue;
+    nt_status r;
+    if (fast) {
+      // tensor-core path: LayerNorm once (bf16), token GEMMs on mma.sync, bias planes written times sqrt(d) as the
+      // attention core wants them, the segmented core over the token axis, gate, output GEMM accumulated into x
+      const size_t e = 2;
+      char* xr = (char*)x + (size_t)trow0 * c_s * e;
+      char* xh = (char*)w.xh + (size_t)trow0 * c_s * e;
+      const size_t to = (size_t)trow0 * Hd * e;
+      if ((r = fast_ln_rows(xr, W->ln_gamma, W->ln_beta, eps, c_s, trows, xh, st)) != NT_OK) return r;
+      if ((r = fast_token_gemm(xh, trows, c_s, W->W_q, Hd, (char*)w.q + to, W->W_k, Hd, (char*)w.k + to, 0, 0, "single_attn_in_qk", st)) != NT_OK) return r;
+      if ((r = fast_token_gemm(xh, trows, c_s, W->W_v, Hd, (char*)w.v + to, W->W_g, Hd, (char*)w.g + to, 0, 0, "single_attn_in_vg", st)) != NT_OK) return r;
+      if ((r = fast_single_bias(z, W->ln_z_gamma, W->ln_z_beta, W->W_b, eps, c_z, H, sqrtf((float)d), m, w.bias, st)) != NT_OK) return r;
+      if ((r = fast_attn_core(w.q, w.k, w.v, w.bias, w.o, H, d, 0, 1, m, L->status_d, st)) != NT_OK) return r;
+      if ((r = fast_gate_mul((char*)w.g + to, (char*)w.o + to, trows * Hd, st)) != NT_OK) return r;
+      if ((r = fast_token_gemm((char*)w.o + to, trows, Hd, W->W_o, c_s, xr, nullptr, 0, nullptr, 0, 1, "single_attn_out", st)) != NT_OK) return r;
+      continue;
+    }
+    ProjArgs pa{};
+    pa.A = x; pa.a_mode = A_ROWMAJOR; pa.row0 = trow0; pa.rows = trows; pa.K = c_s;
+    pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = eps;
+    pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
+    pa.W1 = W->W_q; pa.out = w.q;
+    if ((r = launch_proj<T>(pa, m, st, "single_attn_in_q")) != NT_OK) return r;
+    pa.W1 = W->W_k; pa.out = w.k;
+    if ((r = launch_proj<T>(pa, m, st, "single_attn_in_k")) != NT_OK) return r;
+    pa.W1 = W->W_v; pa.out = w.v;
+    if ((r = launch_proj<T>(pa, m, st, "single_attn_in_v")) != NT_OK) return r;
+    pa.W1 = W->W_g; pa.out = w.g; pa.act = ACT_SIGMOID;
+    if ((r = launch_proj<T>(pa, m, st, "single_attn_in_g")) != NT_OK) return r;
+    ProjArgs pb{};
+    pb.A = z; pb.a_mode = A_ROWMAJOR; pb.row0 = prow0; pb.rows = prows; pb.K = c_z;
+    pb.ln_g = W->ln_z_gamma; pb.ln_b = W->ln_z_beta; pb.eps = eps;
+    pb.W1 = W->W_b; pb.Nout = H; pb.act = ACT_NONE; pb.out = w.bias; pb.out_mode = O_CHANNEL_MAJOR;
+    if ((r = launch_proj<T>(pb, m, st, "single_attn_bias")) != NT_OK) return r;
+    r = launch_attn_core<T>((const T*)w.q, (const T*)w.k, (const T*)w.v, (const T*)w.bias, (T*)w.o, H, d, 0, m, st);
+    if (r != NT_OK) return r;
+    ProjArgs po{};
+    po.A = w.o; po.a_mode = A_ROWMAJOR; po.row0 = trow0; po.rows = trows; po.K = Hd;
+    po.gateA = w.g;
+    po.W1 = W->W_o; po.Nout = c_s; po.act = ACT_NONE; po.out = x; po.out_mode = O_ACCUM;
+    if ((r = launch_proj<T>(po, m, st, "single_attn_out")) != NT_OK) return r;
+  }
+  return NT_OK;
+}
+
 }  // namespace ntp
 
 using namespace ntp;
@@ -419,6 +495,33 @@ nt_status nt_col_attn_pairbias(const nt_layout* L, nt_dtype dt, int32_t c, int32
   cudaStream_t st = (cudaStream_t)stream;
   if (dt == NT_F32) return attn_generic<float>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, true);
   return attn_generic<__nv_bfloat16>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, true);
+}
+
+nt_status nt_single_attn_pairbias(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_t c_z, int32_t H, int32_t d,
+                                  const nt_single_attn_weights* W, float ln_eps, void* x, const void* z,
+                                  void* workspace, size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c_s <= 0 || c_z <= 0 || H <= 0 || d <= 0 || !W) return NT_ERR_INVALID_ARG;
+  if (!W->ln_gamma || !W->ln_beta || !W->W_q || !W->W_k || !W->W_v || !W->W_g || !W->W_o || !W->ln_z_gamma ||
+      !W->ln_z_beta || !W->W_b)
+    return NT_ERR_INVALID_ARG;
+  if (d > 128) return NT_ERR_UNSUPPORTED;
+  if (tot.T1 == 0) return NT_OK;
+  if (!x || !z || !workspace || !aligned16(x) || !aligned16(z) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < carve_single(nullptr, dt, tot, c_s, H, d).bytes) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32) return single_attn_impl<float>(L, tot, c_s, c_z, H, d, W, ln_eps, x, z, workspace, dt, st);
+  return single_attn_impl<__nv_bfloat16>(L, tot, c_s, c_z, H, d, W, ln_eps, x, z, workspace, dt, st);
+}
+
+size_t nt_single_attn_workspace_bytes(nt_dtype dt, const int64_t* lengths_h, int32_t B, int32_t c_s, int32_t H, int32_t d) {
+  if (B <= 0 || !lengths_h || c_s <= 0 || H <= 0 || d <= 0 || (dt != NT_F32 && dt != NT_BF16)) return 0;
+  Totals tot;
+  if (totals_of(lengths_h, B, tot) != NT_OK) return 0;
+  return carve_single(nullptr, dt, tot, c_s, H, d).bytes;
 }
 
 nt_status nt_segment_reduce(nt_dtype dt, nt_reduce op, int32_t C, int64_t G, int64_t rows, const int64_t* splits_d,

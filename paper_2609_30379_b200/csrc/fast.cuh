@@ -18,6 +18,14 @@ bool fast_token_gemm_supported(int K, int N0, int N1);
 nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, int N0, void* out0, const void* W1,
                           int N1, void* out1, int out_f32, int accumulate, const char* name, cudaStream_t st);
 
+// pair-biased single attention: LayerNorm of the token rows (bf16 out), o <- sigmoid(g) * o, and the bias planes
+// bias[s][h][i][j] = scale * (LN(z_ij) W_b^T)[h] in the head-major padded layout of the attention core
+bool fast_single_attn_supported(int c_s, int c_z, int H, int d);
+nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st);
+nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st);
+nt_status fast_single_bias(const void* z, const void* g, const void* b, const void* Wb, float eps, int C, int H, float scale,
+                           const BatchMeta& m, void* bias, cudaStream_t st);
+
 // attention core on tensor cores (bf16, d in {16, 32, 64}); q, k, v, o row-major [rows, H*d], bias
 // head-major channel-major (nullable)
 bool fast_attn_core_supported(int H, int d);

@@ -397,3 +397,362 @@ nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, 
 }
 
 }  // namespace ntp
+
+// ------------------------------------------------------------------------------------------------------------------
+// Pair-biased single attention: the CUDA-core pieces around the token GEMMs and the attention core.
+// ------------------------------------------------------------------------------------------------------------------
+namespace ntp {
+
+// LayerNorm of token rows, bf16 in / bf16 out: one warp per row, 16-byte loads.
+__global__ void __launch_bounds__(256) ln_rows_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gamma,
+                                                      const __nv_bfloat16* __restrict__ beta, float eps, int C, long long rows,
+                                                      __nv_bfloat16* __restrict__ out) {
+  const long long r = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= rows) return;
+  const int nch = C / 8;
+  uint4 v[8];
+  float s = 0.f, q = 0.f;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int c8 = lane + u * 32;
+    if (c8 < nch) {
+      v[u] = *reinterpret_cast<const uint4*>(x + r * C + c8 * 8);
+      const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+        s += lo + hi;
+        q = fmaf(lo, lo, q);
+        q = fmaf(hi, hi, q);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, o);
+    q += __shfl_xor_sync(0xffffffffu, q, o);
+  }
+  const float mean = s / (float)C;
+  const float rstd = rsqrtf(fmaxf(q / (float)C - mean * mean, 0.f) + eps);
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int c8 = lane + u * 32;
+    if (c8 < nch) {
+      const uint4 g4 = *reinterpret_cast<const uint4*>(gamma + c8 * 8), b4 = *reinterpret_cast<const uint4*>(beta + c8 * 8);
+      const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w}, gw[4] = {g4.x, g4.y, g4.z, g4.w}, bw[4] = {b4.x, b4.y, b4.z, b4.w};
+      unsigned o4[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = (__uint_as_float(w[e] << 16) - mean) * rstd, hi = (__uint_as_float(w[e] & 0xffff0000u) - mean) * rstd;
+        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf(lo, __uint_as_float(gw[e] << 16), __uint_as_float(bw[e] << 16)),
+                                                 fmaf(hi, __uint_as_float(gw[e] & 0xffff0000u), __uint_as_float(bw[e] & 0xffff0000u)));
+        o4[e] = *reinterpret_cast<unsigned*>(&h);
+      }
+      *reinterpret_cast<uint4*>(out + r * C + c8 * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+    }
+  }
+}
+
+// o <- sigmoid(g) * o, elementwise on bf16 (eight elements per thread)
+__global__ void __launch_bounds__(256) gate_mul_kernel(const __nv_bfloat16* __restrict__ g, __nv_bfloat16* __restrict__ o, long long n8) {
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= n8) return;
+  const uint4 gv = *reinterpret_cast<const uint4*>(g + i * 8);
+  uint4 ov = *reinterpret_cast<const uint4*>(o + i * 8);
+  const unsigned gw[4] = {gv.x, gv.y, gv.z, gv.w};
+  unsigned ow[4] = {ov.x, ov.y, ov.z, ov.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float g0 = __uint_as_float(gw[e] << 16), g1 = __uint_as_float(gw[e] & 0xffff0000u);
+    const float o0 = __uint_as_float(ow[e] << 16), o1 = __uint_as_float(ow[e] & 0xffff0000u);
+    __nv_bfloat162 h = __floats2bfloat162_rn(o0 / (1.0f + __expf(-g0)), o1 / (1.0f + __expf(-g1)));
+    ow[e] = *reinterpret_cast<unsigned*>(&h);
+  }
+  *reinterpret_cast<uint4*>(o + i * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+}
+
+// Bias planes of the pair-biased single attention: bias[s][h][i][j] = scale * (LN(z_ij) W_b^T)[h], head-major with the
+// padded row stride of the channel-major buffers.  The pair state is read once; the H results per position are tiny.
+// A warp takes 32 consecutive packed positions: sixteen lanes work on one position (16-byte loads, LayerNorm folded
+// into the H weight rows kept in shared memory), the results are handed to the lane that owns the position, and the
+// warp writes each head's 32 values as one run.
+constexpr int SB_MAXH = 8;
+template <int HT>      // heads the arithmetic runs over (H <= HT; rows H .. HT - 1 of the weight table are zeros)
+__global__ void __launch_bounds__(256) single_bias_kernel(const __nv_bfloat16* __restrict__ z, const __nv_bfloat16* __restrict__ gamma,
+                                                          const __nv_bfloat16* __restrict__ beta, const __nv_bfloat16* __restrict__ Wb,
+                                                          float eps, int C, int H, float scale, BatchMeta m,
+                                                          __nv_bfloat16* __restrict__ bias) {
+  extern __shared__ float sbw[];            // [HT][C] folded weights, then c0[HT], c1[HT]
+  float* c0 = sbw + HT * C;
+  float* c1 = c0 + SB_MAXH;
+  for (int idx = threadIdx.x; idx < HT * C; idx += 256) {
+    const int c = idx % C;
+    sbw[idx] = idx < H * C ? __bfloat162float(Wb[idx]) * __bfloat162float(gamma[c]) : 0.f;
+  }
+  if (threadIdx.x < 2 * SB_MAXH) c0[threadIdx.x] = 0.f;
+  __syncthreads();
+  if ((threadIdx.x >> 5) < H) {            // warp h sums row h (H <= 8 = warps per block)
+    const int h = threadIdx.x >> 5;
+    float a0 = 0.f, a1 = 0.f;
+    for (int c = threadIdx.x & 31; c < C; c += 32) {
+      a0 = fmaf(__bfloat162float(Wb[h * C + c]), __bfloat162float(beta[c]), a0);
+      a1 += sbw[h * C + c];
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+      a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+      c0[h] = a0;
+      c1[h] = a1;
+    }
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, hw = lane >> 4, l16 = lane & 15;
+  const long long p0 = m.pair_off[0], p1 = m.pair_off[m.B];
+  const long long nblk = (p1 - p0 + 31) / 32;
+  const int nch = C / 8;
+  for (long long blk = (long long)blockIdx.x * 8 + warp; blk < nblk; blk += (long long)gridDim.x * 8) {
+    const long long base = p0 + blk * 32;
+    float keep[HT];
+#pragma unroll
+    for (int h = 0; h < HT; ++h) keep[h] = 0.f;
+    // four positions' loads are issued before the first is used (one 16-byte chunk per lane covers C <= 128;
+    // wider rows take further chunks inside the step)
+    for (int t0 = 0; t0 < 16; t0 += 4) {
+      uint4 first[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const long long p = base + 2 * (t0 + u) + hw;
+        first[u] = (p < p1 && l16 < nch) ? *reinterpret_cast<const uint4*>(z + p * C + l16 * 8) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int t = t0 + u;
+        const long long p = base + 2 * t + hw;
+        float s = 0.f, q = 0.f, dot[HT];
+#pragma unroll
+        for (int h = 0; h < HT; ++h) dot[h] = 0.f;
+        for (int c8 = l16; c8 < nch; c8 += 16) {
+          uint4 v = first[u];
+          if (c8 != l16) v = p < p1 ? *reinterpret_cast<const uint4*>(z + p * C + c8 * 8) : make_uint4(0, 0, 0, 0);
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+          float f[8];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            f[2 * e] = __uint_as_float(w[e] << 16);
+            f[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            s += f[e];
+            q = fmaf(f[e], f[e], q);
+          }
+#pragma unroll
+          for (int h = 0; h < HT; ++h) {
+              const float4 w0 = *reinterpret_cast<const float4*>(sbw + h * C + c8 * 8), w1 = *reinterpret_cast<const float4*>(sbw + h * C + c8 * 8 + 4);
+              dot[h] = fmaf(f[0], w0.x, fmaf(f[1], w0.y, fmaf(f[2], w0.z, fmaf(f[3], w0.w, dot[h]))));
+              dot[h] = fmaf(f[4], w1.x, fmaf(f[5], w1.y, fmaf(f[6], w1.z, fmaf(f[7], w1.w, dot[h]))));
+            }
+        }
+#pragma unroll
+        for (int o = 8; o; o >>= 1) {
+          s += __shfl_xor_sync(0xffffffffu, s, o);
+          q += __shfl_xor_sync(0xffffffffu, q, o);
+#pragma unroll
+          for (int h = 0; h < HT; ++h) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], o);
+        }
+        const float mean = s / (float)C;
+        const float rstd = rsqrtf(fmaxf(q / (float)C - mean * mean, 0.f) + eps);
+#pragma unroll
+        for (int h = 0; h < HT; ++h) {
+            const float r = (rstd * (dot[h] - mean * c1[h]) + c0[h]) * scale;
+            const float got = __shfl_sync(0xffffffffu, r, (lane & 1) * 16);     // from the half-warp that holds position 2 t + (lane & 1)
+            if ((lane >> 1) == t) keep[h] = got;
+          }
+      }
+    }
+    const long long p = base + lane;
+    if (p < p1) {
+      const int s_ = find_sample(m.pair_off, m.B, p);
+      const int N = m.N[s_], ld = round_up8(N);
+      const long long r = p - m.pair_off[s_];
+      const int i = (int)(r / N), j = (int)(r - (long long)i * N);
+      __nv_bfloat16* bp = bias + (long long)H * m.cm_off[s_] + (long long)i * ld + j;
+#pragma unroll
+      for (int h = 0; h < HT; ++h)
+        if (h < H) bp[(long long)h * N * ld] = __float2bfloat16_rn(keep[h]);
+    }
+  }
+}
+
+// The same planes on the tensor cores (H <= 4, C = 16 NK): per 16 positions one m16n8k16 MMA per 16 channels against
+// B = [W'_0 .. W'_3 | 1 | 0 ..] gives the H dot products and the row sum; a second MMA of the squared inputs against
+// a ones column adds the sum of squares as column 5 of the same accumulator, so the LayerNorm statistics cost no
+// shuffle reductions at all.  A fragments come straight from global memory (each k step reads one 32-byte sector of a
+// row).  W' = W_b gamma is rounded to bf16; c1 is the sum of the rounded values.
+__device__ inline void mma_bf16_16816(float (&c)[4], const unsigned (&a)[4], unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <int NK>
+__global__ void __launch_bounds__(256) single_bias_mma_kernel(const __nv_bfloat16* __restrict__ z, const __nv_bfloat16* __restrict__ gamma,
+                                                              const __nv_bfloat16* __restrict__ beta, const __nv_bfloat16* __restrict__ Wb,
+                                                              float eps, int H, float scale, BatchMeta m,
+                                                              __nv_bfloat16* __restrict__ bias) {
+  constexpr int C = 16 * NK;
+  __shared__ __nv_bfloat16 sW[4][C];        // W' rounded to bf16 (rows H .. 3 zero)
+  __shared__ float c0[4], c1[4];
+  for (int idx = threadIdx.x; idx < 4 * C; idx += 256) {
+    const int h = idx / C, c = idx - h * C;
+    sW[h][c] = __float2bfloat16_rn(h < H ? __bfloat162float(Wb[h * C + c]) * __bfloat162float(gamma[c]) : 0.f);
+  }
+  __syncthreads();
+  if ((threadIdx.x >> 5) < 4) {
+    const int h = threadIdx.x >> 5;
+    float a0 = 0.f, a1 = 0.f;
+    for (int c = threadIdx.x & 31; c < C; c += 32) {
+      if (h < H) a0 = fmaf(__bfloat162float(Wb[h * C + c]), __bfloat162float(beta[c]), a0);
+      a1 += __bfloat162float(sW[h][c]);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      a0 += __shfl_xor_sync(0xffffffffu, a0, o);
+      a1 += __shfl_xor_sync(0xffffffffu, a1, o);
+    }
+    if ((threadIdx.x & 31) == 0) { c0[h] = a0; c1[h] = a1; }
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  // B fragments: column n = g of the MMA is head g (g < 4), the ones column (g == 4) or zero
+  unsigned bw[NK][2];
+#pragma unroll
+  for (int ks = 0; ks < NK; ++ks) {
+    if (g < 4) {
+      bw[ks][0] = *reinterpret_cast<const unsigned*>(&sW[g][ks * 16 + 2 * t]);
+      bw[ks][1] = *reinterpret_cast<const unsigned*>(&sW[g][ks * 16 + 2 * t + 8]);
+    } else {
+      bw[ks][0] = bw[ks][1] = g == 4 ? 0x3F803F80u : 0u;
+    }
+  }
+  const unsigned bsq = g == 5 ? 0x3F803F80u : 0u;
+  const float k0a = c0[(2 * t) & 3], k0b = c0[(2 * t + 1) & 3], k1a = c1[(2 * t) & 3], k1b = c1[(2 * t + 1) & 3];
+  const long long p0 = m.pair_off[0], p1 = m.pair_off[m.B];
+  const long long ntile = (p1 - p0 + 15) / 16;
+  for (long long tile = (long long)blockIdx.x * 8 + warp; tile < ntile; tile += (long long)gridDim.x * 8) {
+    const long long pa = p0 + tile * 16 + g, pb = pa + 8;
+    const __nv_bfloat16* ra = z + (pa < p1 ? pa : p1 - 1) * C + 2 * t;
+    const __nv_bfloat16* rb = z + (pb < p1 ? pb : p1 - 1) * C + 2 * t;
+    unsigned a[NK][4];
+#pragma unroll
+    for (int ks = 0; ks < NK; ++ks) {
+      a[ks][0] = *reinterpret_cast<const unsigned*>(ra + ks * 16);
+      a[ks][1] = *reinterpret_cast<const unsigned*>(rb + ks * 16);
+      a[ks][2] = *reinterpret_cast<const unsigned*>(ra + ks * 16 + 8);
+      a[ks][3] = *reinterpret_cast<const unsigned*>(rb + ks * 16 + 8);
+    }
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < NK; ++ks) {
+      mma_bf16_16816(acc, a[ks], bw[ks][0], bw[ks][1]);
+      unsigned sq[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&a[ks][e]);
+        const __nv_bfloat162 v2 = __hmul2(v, v);
+        sq[e] = *reinterpret_cast<const unsigned*>(&v2);
+      }
+      mma_bf16_16816(acc, sq, bsq, bsq);
+    }
+    // columns 4 / 5 (lanes with t == 2) hold the row sum and the sum of squares
+    const int src = (lane & ~3) | 2;
+    const float sa = __shfl_sync(0xffffffffu, acc[0], src), qa = __shfl_sync(0xffffffffu, acc[1], src);
+    const float sb = __shfl_sync(0xffffffffu, acc[2], src), qb = __shfl_sync(0xffffffffu, acc[3], src);
+    if (t < 2) {
+      const float ma = sa / (float)C, mb = sb / (float)C;
+      const float rsa = rsqrtf(fmaxf(qa / (float)C - ma * ma, 0.f) + eps), rsb = rsqrtf(fmaxf(qb / (float)C - mb * mb, 0.f) + eps);
+      const float out[2][2] = {{(rsa * (acc[0] - ma * k1a) + k0a) * scale, (rsa * (acc[1] - ma * k1b) + k0b) * scale},
+                               {(rsb * (acc[2] - mb * k1a) + k0a) * scale, (rsb * (acc[3] - mb * k1b) + k0b) * scale}};
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const long long p = rr ? pb : pa;
+        if (p < p1) {
+          const int s_ = find_sample(m.pair_off, m.B, p);
+          const int N = m.N[s_], ld = round_up8(N);
+          const long long r = p - m.pair_off[s_];
+          const int i = (int)(r / N), j = (int)(r - (long long)i * N);
+          __nv_bfloat16* bp = bias + (long long)H * m.cm_off[s_] + (long long)i * ld + j;
+          if (2 * t < H) bp[(long long)(2 * t) * N * ld] = __float2bfloat16_rn(out[rr][0]);
+          if (2 * t + 1 < H) bp[(long long)(2 * t + 1) * N * ld] = __float2bfloat16_rn(out[rr][1]);
+        }
+      }
+    }
+  }
+}
+
+bool fast_single_attn_supported(int c_s, int c_z, int H, int d) {
+  const int Hd = H * d;
+  return c_s % 8 == 0 && c_s <= 2048 && c_z % 8 == 0 && c_z <= 1024 && H >= 1 && H <= SB_MAXH && fast_attn_core_supported(H, d) &&
+         fast_token_gemm_supported(c_s, Hd, Hd) && fast_token_gemm_supported(Hd, c_s, 0);
+}
+
+nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st) {
+  if (rows <= 0) return NT_OK;
+  {
+    LaunchScope ls("single_attn_ln", st);
+    ln_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b, eps, C,
+                                                               rows, (__nv_bfloat16*)out);
+  }
+  return cuda_ok("single attention LayerNorm launch");
+}
+
+nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st) {
+  if (n <= 0) return NT_OK;
+  const long long n8 = n / 8;
+  {
+    LaunchScope ls("single_attn_gate", st);
+    gate_mul_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)g, (__nv_bfloat16*)o, n8);
+  }
+  return cuda_ok("single attention gate launch");
+}
+
+nt_status fast_single_bias(const void* z, const void* g, const void* b, const void* Wb, float eps, int C, int H, float scale,
+                           const BatchMeta& m, void* bias, cudaStream_t st) {
+  const long long rows = m.pair_off[m.B] - m.pair_off[0];
+  if (rows <= 0) return NT_OK;
+  const long long nblk = (rows + 31) / 32;
+  const long long want = (nblk + 7) / 8;
+  const unsigned grid = (unsigned)(want < 148 * 3 ? want : 148 * 3);      // 3 blocks of 256 threads fit an SM at 79 registers
+  if (H <= 4 && (C == 128 || C == 64)) {
+    const long long ntile = (rows + 15) / 16, wantb = (ntile + 7) / 8;
+    const unsigned gridm = (unsigned)(wantb < 148 * 8 ? wantb : 148 * 8);
+    {
+      LaunchScope ls("single_attn_bias", st);
+      if (C == 128)
+        single_bias_mma_kernel<8><<<gridm, 256, 0, st>>>((const __nv_bfloat16*)z, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b,
+                                                         (const __nv_bfloat16*)Wb, eps, H, scale, m, (__nv_bfloat16*)bias);
+      else
+        single_bias_mma_kernel<4><<<gridm, 256, 0, st>>>((const __nv_bfloat16*)z, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b,
+                                                         (const __nv_bfloat16*)Wb, eps, H, scale, m, (__nv_bfloat16*)bias);
+    }
+    return cuda_ok("single attention bias launch");
+  }
+  const int HT = H <= 4 ? 4 : SB_MAXH;
+  const size_t smem = ((size_t)HT * C + 2 * SB_MAXH) * sizeof(float);
+  {
+    LaunchScope ls("single_attn_bias", st);
+    if (HT == 4)
+      single_bias_kernel<4><<<grid, 256, smem, st>>>((const __nv_bfloat16*)z, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b,
+                                                     (const __nv_bfloat16*)Wb, eps, C, H, scale, m, (__nv_bfloat16*)bias);
+    else
+      single_bias_kernel<8><<<grid, 256, smem, st>>>((const __nv_bfloat16*)z, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b,
+                                                     (const __nv_bfloat16*)Wb, eps, C, H, scale, m, (__nv_bfloat16*)bias);
+  }
+  return cuda_ok("single attention bias launch");
+}
+
+}  // namespace ntp

@@ -1,0 +1,101 @@
+"""GPU parity of the pair-biased single attention (tokens attend tokens of their sample, logits biased by a
+projection of the pair state) against the CPU oracle, through the C ABI.  The pair state is the one the block's
+broadcast produces from the seeded tokens."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nested_pair_oracle as orc
+from paper_2609_30379_b200 import workloads as wl
+from tests.parity_utils import check
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nt():
+    from paper_2609_30379_b200 import binding
+    return binding
+
+
+def host(t):
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def _run(nt, cfg, force_generic=False):
+    from paper_2609_30379_b200 import runner
+    inp = wl.make_inputs(cfg)
+    W = wl.make_single_attn_weights(cfg)
+    prev = nt.nt_force_generic(force_generic)
+    try:
+        st = runner.PairStack(cfg, cfg.lengths, inp["blocks"][:1])
+        x_d = runner.to_device(inp["x"], st.dtype)
+        b = st.W[0]["broadcast"]
+        nt.nt_pair_broadcast(st.L, x_d, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, st.z, st.workspace)
+        z0 = st.z.clone()
+        W_d = {k: torch.from_numpy(np.ascontiguousarray(v)).to("cuda", st.dtype) for k, v in W.items()}
+        nbytes = nt.nt_single_attn_workspace_bytes(st.dtype, cfg.lengths, cfg.c_s, cfg.H, cfg.d)
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        x_in = x_d.clone()
+        nt.nt_single_attn_pairbias(st.L, W_d, cfg.H, cfg.d, 1e-5, x_d, st.z, ws)
+        torch.cuda.synchronize()
+        assert st.L.device_status() == 0
+        assert torch.equal(st.z, z0)                       # the pair state is read only
+        return host(x_in), host(z0), host(x_d), W
+    finally:
+        nt.nt_force_generic(prev)
+
+
+def _check(cfg, x0, z0, x1, W, samples):
+    tok = np.concatenate([[0], np.cumsum(np.asarray(cfg.lengths, dtype=np.int64))])
+    po = np.concatenate([[0], np.cumsum(np.asarray(cfg.lengths, dtype=np.int64) ** 2)])
+    for s in samples:
+        n = cfg.lengths[s]
+        if n == 0:
+            continue
+        ref = orc.single_attn_pairbias(x0[tok[s]:tok[s + 1]], z0[po[s]:po[s + 1]], (n,), W, cfg.H, cfg.d)
+        check(cfg.dtype, x1[tok[s]:tok[s + 1]], ref, f"single attention s={s} n={n}")
+
+
+def test_single_attn_cfg1_f32(nt):
+    cfg = wl.CONFIGS["cfg1"]
+    x0, z0, x1, W = _run(nt, cfg)
+    _check(cfg, x0, z0, x1, W, range(cfg.B))
+
+
+@pytest.mark.parametrize("dtype,generic", [("f32", False), ("bf16", False), ("bf16", True)])
+def test_single_attn_edge_lengths(nt, dtype, generic):
+    bf = dtype == "bf16"
+    cfg = wl.Config("edge_single", dtype, (0, 1, 7, 31, 33, 64, 0, 129, 200), c_s=64 if bf else 24, c_z=128 if bf else 16,
+                    c_h=128 if bf else 16, H=4 if bf else 2, d=32 if bf else 8, blocks=1, seed=61)
+    x0, z0, x1, W = _run(nt, cfg, force_generic=generic)
+    _check(cfg, x0, z0, x1, W, range(cfg.B))
+    assert np.all(np.isfinite(x1))
+
+
+def test_single_attn_cfg2(nt):
+    """The bench workload, every sample in full (the token axis is short: the oracle finishes in seconds)."""
+    cfg = wl.CONFIGS["cfg2"]
+    x0, z0, x1, W = _run(nt, cfg)
+    _check(cfg, x0, z0, x1, W, range(cfg.B))
+
+
+def test_single_attn_long_sample(nt):
+    cfg = wl.Config("single600", "bf16", (600, 40), c_s=128, c_z=64, c_h=64, H=4, d=16, blocks=1, seed=62)
+    x0, z0, x1, W = _run(nt, cfg)
+    _check(cfg, x0, z0, x1, W, range(cfg.B))
+
+
+def test_single_attn_workspace_and_errors(nt):
+    cfg = wl.CONFIGS["cfg1"]
+    assert nt.nt_single_attn_workspace_bytes(torch.float32, (), cfg.c_s, cfg.H, cfg.d) == 0
+    need = nt.nt_single_attn_workspace_bytes(torch.float32, cfg.lengths, cfg.c_s, cfg.H, cfg.d)
+    assert need > 0
+    from paper_2609_30379_b200 import runner
+    inp = wl.make_inputs(cfg)
+    st = runner.PairStack(cfg, cfg.lengths, inp["blocks"][:1])
+    x_d = runner.to_device(inp["x"], st.dtype)
+    W_d = {k: torch.from_numpy(np.ascontiguousarray(v)).to("cuda", st.dtype) for k, v in wl.make_single_attn_weights(cfg).items()}
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(nt.NtError):
+        nt.nt_single_attn_pairbias(st.L, W_d, cfg.H, cfg.d, 1e-5, x_d, st.z, small)
