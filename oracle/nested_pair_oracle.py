@@ -473,11 +473,21 @@ def col_attn_pairbias_at(zs, W, H, d, positions, eps=LN_EPS, dtype=np.float64):
     return np.stack(out)
 
 
-def block_forward(x, lengths, w, H, d, eps=LN_EPS, dtype=np.float64):
+def pair_broadcast_add(z_prev, x, lengths, W_a, W_b, ln_gamma, ln_beta, eps=LN_EPS, dtype=np.float64):
+    """Persistent pair stream: z = z_prev + LN(u_i + v_j) gamma + beta, the broadcast of Eq. 1 line 1 accumulated onto
+    the state of the previous block instead of replacing it."""
+    return np.asarray(z_prev, dtype=dtype) + pair_broadcast(x, lengths, W_a, W_b, ln_gamma, ln_beta, eps=eps, dtype=dtype)
+
+
+def block_forward(x, lengths, w, H, d, eps=LN_EPS, dtype=np.float64, z_prev=None):
     """One Pairformer-style block: broadcast+LN, outgoing triangle update, row-wise pair-biased
-    attention, segmented mean over j and token update.  Returns (x', z)."""
+    attention, segmented mean over j and token update.  Returns (x', z).  With z_prev the broadcast is
+    accumulated onto it (persistent pair stream)."""
     _, _, row_splits = offsets_only(lengths)
-    z = pair_broadcast(x, lengths, eps=eps, dtype=dtype, **w["broadcast"])
+    if z_prev is None:
+        z = pair_broadcast(x, lengths, eps=eps, dtype=dtype, **w["broadcast"])
+    else:
+        z = pair_broadcast_add(z_prev, x, lengths, eps=eps, dtype=dtype, **w["broadcast"])
     z = tri_mul_out(z, lengths, w["trimul"], eps=eps, dtype=dtype)
     z = row_attn_pairbias(z, lengths, w["attn"], H, d, eps=eps, order="pair", dtype=dtype)
     m = segment_reduce(z, row_splits, "mean", dtype=dtype)
@@ -485,12 +495,14 @@ def block_forward(x, lengths, w, H, d, eps=LN_EPS, dtype=np.float64):
     return x2, z
 
 
-def stack_forward(x, lengths, blocks, H, d, eps=LN_EPS, dtype=np.float64):
-    """Stacked blocks: block b+1 rebuilds the pair state from the tokens block b returned."""
+def stack_forward(x, lengths, blocks, H, d, eps=LN_EPS, dtype=np.float64, persistent=False):
+    """Stacked blocks.  persistent=False: block b+1 rebuilds the pair state from the tokens block b returned (Eq. 1).
+    persistent=True: the pair state is a stream of its own, z_b = z_{b-1} + LN(broadcast of the tokens) before the
+    pair sub-layers of block b (the Pairformer keeps a persistent pair state, Sec. 2); block 0 starts it."""
     z = None
     x = np.asarray(x, dtype=dtype)
     for w in blocks:
-        x, z = block_forward(x, lengths, w, H, d, eps=eps, dtype=dtype)
+        x, z = block_forward(x, lengths, w, H, d, eps=eps, dtype=dtype, z_prev=z if persistent else None)
     return x, z
 
 

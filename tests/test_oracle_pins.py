@@ -542,6 +542,30 @@ def test_stack_rebuilds_pair_state_from_tokens():
     assert np.array_equal(x2, xb) and np.array_equal(z2, zb)
 
 
+def test_persistent_pair_stream():
+    cfg, inp = tiny_inputs((3, 5))
+    w = inp["blocks"][0]["broadcast"]
+    rng = np.random.default_rng(71)
+    zp = rng.standard_normal((cfg.T2, cfg.c_z))
+    z0 = orc.pair_broadcast(inp["x"], cfg.lengths, **w)
+    # accumulated broadcast: zero previous state gives the plain broadcast; the previous state enters additively
+    assert np.array_equal(orc.pair_broadcast_add(np.zeros_like(zp), inp["x"], cfg.lengths, **w), z0)
+    assert np.allclose(orc.pair_broadcast_add(zp, inp["x"], cfg.lengths, **w) - zp, z0, rtol=1e-12, atol=1e-12)
+    # a stack of one block is the same in both modes; with two blocks the second one sees z_1 + broadcast(x_1)
+    blocks = [inp["blocks"][0], wl.make_inputs(wl.Config("tiny2", "f32", cfg.lengths, c_s=cfg.c_s, c_z=cfg.c_z, c_h=cfg.c_h,
+                                                         H=cfg.H, d=cfg.d, blocks=1, seed=99))["blocks"][0]]
+    x1a, z1a = orc.stack_forward(inp["x"], cfg.lengths, blocks[:1], cfg.H, cfg.d)
+    x1b, z1b = orc.stack_forward(inp["x"], cfg.lengths, blocks[:1], cfg.H, cfg.d, persistent=True)
+    assert np.array_equal(x1a, x1b) and np.array_equal(z1a, z1b)
+    x2, z2 = orc.stack_forward(inp["x"], cfg.lengths, blocks, cfg.H, cfg.d, persistent=True)
+    zin = z1a + orc.pair_broadcast(x1a, cfg.lengths, **blocks[1]["broadcast"])
+    zt = orc.tri_mul_out(zin, cfg.lengths, blocks[1]["trimul"])
+    zt = orc.row_attn_pairbias(zt, cfg.lengths, blocks[1]["attn"], cfg.H, cfg.d)
+    assert np.allclose(z2, zt, rtol=1e-12, atol=1e-12)
+    xr, zr = orc.stack_forward(inp["x"], cfg.lengths, blocks, cfg.H, cfg.d)
+    assert not np.allclose(z2, zr)
+
+
 def test_bf16_rounding_helpers():
     a = np.array([1.0, 1.00390625, 1.001953125, 3.1415927, -2.7182817, 1e-3], dtype=np.float32)
     ref = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
