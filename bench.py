@@ -61,6 +61,8 @@ def kernel_work(cfg: wl.Config):
     w["tok_proj"] = dict(bytes=T1 * c_s * e + 2 * c_z * c_s * e + 2 * T1 * c_z * 4, flops=4 * T1 * c_s * c_z)
     bc = dict(bytes=T2 * c_z * e + 2 * T1 * c_z * 4, flops=8 * T2 * c_z)
     w["broadcast_ln"] = w["generic_broadcast_ln"] = bc
+    # accumulated onto the state (persistent pair stream): the state is read as well as written
+    w["broadcast_ln_add"] = w["generic_broadcast_ln_add"] = dict(bytes=2 * T2 * c_z * e + 2 * T1 * c_z * 4, flops=9 * T2 * c_z)
     w["generic_tri_in_a"] = w["generic_tri_in_b"] = dict(bytes=T2 * (c_z + c_h) * e, flops=2 * T2 * c_z * 2 * c_h)
     w["generic_tri_in_g"] = dict(bytes=2 * T2 * c_z * e, flops=2 * T2 * c_z * c_z)
     w["tri_in"] = dict(bytes=T2 * (c_z + 2 * c_h) * e, flops=2 * T2 * c_z * 4 * c_h)
@@ -395,6 +397,27 @@ def main():
             out[name] = dict(r, kernel=name) if r else dict(kernel=name, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
         return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
 
+    def stream_pass(n_calls):
+        """The accumulated broadcast of a persistent pair stream (z += LN(u_i + v_j)); not part of the step."""
+        if cfg.kind != "pair":
+            return None
+        b = stack.W[0]["broadcast"]
+        nt.nt_pair_broadcast(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        for _ in range(3):
+            nt.nt_pair_broadcast_add(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            nt.nt_pair_broadcast_add(stack.L, x0, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, stack.z, stack.workspace)
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        out = {}
+        for k, v in tp.items():
+            r = roofline_entry(k, v[0], v[1], n_calls, kernel_work(cfg), peaks_t, kind_t)
+            out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
+
     if args.only_single_attn:
         res = dict(single_attn=single_attn_pass(steps))
         if rank == 0:
@@ -473,7 +496,7 @@ def main():
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
     next_rows = (dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps), col_attn=col_attn_pass(steps),
-                      single_attn=single_attn_pass(steps))
+                      single_attn=single_attn_pass(steps), pair_stream=stream_pass(steps))
                  if not args.force_generic else None)
 
     # ---- end to end through the public API with host buffers

@@ -125,6 +125,16 @@ nt_status nt_pair_broadcast(const nt_layout *L, nt_dtype dt, int32_t c_s, int32_
                             void *z, void *workspace, size_t workspace_bytes, nt_stream stream);
 
 /*
+ * nt_pair_broadcast_add -- the same broadcast accumulated onto the state: z[p,:] += LN(u_i + v_j) * gamma + beta.
+ * For a pair state that persists across blocks (the Pairformer's pair stream) instead of being rebuilt from the
+ * tokens by every block (Eq. 1).  z [T2, c_z] in/out; everything else as nt_pair_broadcast.
+ */
+nt_status nt_pair_broadcast_add(const nt_layout *L, nt_dtype dt, int32_t c_s, int32_t c_z,
+                            const void *x, const void *W_a, const void *W_b,
+                            const void *ln_gamma, const void *ln_beta, float ln_eps,
+                            void *z, void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
  * nt_tri_mul_out -- outgoing triangle multiplicative update (the Pairformer block's triangle
  * multiplication, Sec. 4.3), a per-sample grouped contraction over channels:
  *   zh = LN_in(z); a = sig(zh W_ag^T) * (zh W_ap^T); b = sig(zh W_bg^T) * (zh W_bp^T); g = sig(zh W_g^T)

@@ -25,7 +25,7 @@ NT_OP_PAIR_BROADCAST, NT_OP_TRI_MUL_OUT, NT_OP_ROW_ATTN, NT_OP_BLOCK = 0, 1, 2, 
 STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3: "NT_ERR_WORKSPACE",
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
-EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
+EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_add", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
            "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
            "nt_single_attn_workspace_bytes", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
@@ -71,6 +71,7 @@ def _load() -> C.CDLL:
     vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
     lib.nt_offsets_build.argtypes = [vp, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.nt_pair_broadcast.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp, sz, vp]
+    lib.nt_pair_broadcast_add.argtypes = lib.nt_pair_broadcast.argtypes
     lib.nt_pair_broadcast_static.argtypes = [C.POINTER(nt_layout), i32, i32, i32, vp, vp, vp, vp, vp, f32, vp, vp]
     lib.nt_tri_mul_out.argtypes = [C.POINTER(nt_layout), i32, i32, i32, C.POINTER(nt_trimul_weights), f32, vp, vp, sz, vp]
     lib.nt_tri_mul_in.argtypes = lib.nt_tri_mul_out.argtypes
@@ -99,7 +100,7 @@ def _load() -> C.CDLL:
     lib.nt_profile_begin.restype = i32
     lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
     lib.nt_profile_end.restype = i32
-    for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
+    for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_add", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
                  "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias", "nt_segment_reduce",
                  "nt_token_update"):
         getattr(lib, name).restype = i32
@@ -190,6 +191,14 @@ def nt_pair_broadcast(L: Layout, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, work
                                _ptr(ln_gamma), _ptr(ln_beta), float(ln_eps), _ptr(z), _ptr(workspace),
                                workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "nt_pair_broadcast")
+
+
+def nt_pair_broadcast_add(L: Layout, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, stream=None):
+    c_s, c_z = int(W_a.shape[1]), int(W_a.shape[0])
+    st = lib.nt_pair_broadcast_add(C.byref(L.c), dtype_code(x.dtype), c_s, c_z, _ptr(x), _ptr(W_a), _ptr(W_b),
+                               _ptr(ln_gamma), _ptr(ln_beta), float(ln_eps), _ptr(z), _ptr(workspace),
+                               workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_pair_broadcast_add")
 
 
 def nt_pair_broadcast_static(L: Layout, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, stream=None):

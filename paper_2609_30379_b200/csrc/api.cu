@@ -170,7 +170,7 @@ static size_t broadcast_ws_bytes(const Totals& t, int c_z) {
 template <typename T>
 static nt_status pair_broadcast_impl(const nt_layout* L, const Totals& tot, int c_s, int c_z, const void* x,
                                      const void* W_a, const void* W_b, const void* g, const void* b, float eps,
-                                     void* z, void* ws, cudaStream_t st, bool fast) {
+                                     void* z, void* ws, cudaStream_t st, bool fast, bool accumulate = false) {
   Carver c(ws);
   float* u = (float*)c.take((size_t)tot.T1 * c_z * sizeof(float));
   float* v = (float*)c.take((size_t)tot.T1 * c_z * sizeof(float));
@@ -193,8 +193,8 @@ static nt_status pair_broadcast_impl(const nt_layout* L, const Totals& tot, int 
   GroupIter it(L->lengths_h, L->B);
   BatchMeta m;
   while (it.next(m)) {
-    if (fast) r = fast_broadcast_ln(u, v, g, b, eps, c_z, z, m, st);
-    else r = launch_broadcast_ln<T>(u, v, (const T*)g, (const T*)b, eps, c_z, (T*)z, m, st);
+    if (fast) r = fast_broadcast_ln(u, v, g, b, eps, c_z, z, m, st, accumulate);
+    else r = launch_broadcast_ln<T>(u, v, (const T*)g, (const T*)b, eps, c_z, (T*)z, m, st, accumulate);
     if (r != NT_OK) return r;
   }
   return NT_OK;
@@ -425,6 +425,27 @@ nt_status nt_pair_broadcast(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_
   const bool fast = !g_force_generic && fast_broadcast_supported(c_z);
   return pair_broadcast_impl<__nv_bfloat16>(L, tot, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, st,
                                             fast);
+}
+
+nt_status nt_pair_broadcast_add(const nt_layout* L, nt_dtype dt, int32_t c_s, int32_t c_z, const void* x,
+                            const void* W_a, const void* W_b, const void* ln_gamma, const void* ln_beta,
+                            float ln_eps, void* z, void* workspace, size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c_s <= 0 || c_z <= 0) return NT_ERR_INVALID_ARG;
+  if (tot.T2 == 0) return NT_OK;
+  if (!x || !W_a || !W_b || !ln_gamma || !ln_beta || !z || !workspace) return NT_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(z) || !aligned16(workspace) || !aligned16(W_a) || !aligned16(W_b))
+    return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < broadcast_ws_bytes(tot, c_z)) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32)
+    return pair_broadcast_impl<float>(L, tot, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, st, false, true);
+  const bool fast = !g_force_generic && fast_broadcast_supported(c_z);
+  return pair_broadcast_impl<__nv_bfloat16>(L, tot, c_s, c_z, x, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, st,
+                                            fast, true);
 }
 
 static nt_status tri_mul_entry(const nt_layout* L, nt_dtype dt, int32_t c_z, int32_t c_h, const nt_trimul_weights* W,

@@ -7,7 +7,7 @@ namespace ntp {
 
 bool fast_broadcast_supported(int c_z);
 nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
-                            void* z, const BatchMeta& m, cudaStream_t st);
+                            void* z, const BatchMeta& m, cudaStream_t st, bool accumulate = false);
 
 bool fast_segment_reduce_supported(int C);
 nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, long long G, int C, int mean,

@@ -12,7 +12,7 @@ namespace ntp {
 // ------------------------------------------------------------------------------------------
 constexpr int BJ = 64;
 
-template <int LP>
+template <int LP, bool ACC>      // ACC: z += the broadcast (persistent pair stream) instead of z = the broadcast
 __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __restrict__ u,
                                                                 const float* __restrict__ v,
                                                                 const __nv_bfloat16* __restrict__ gamma,
@@ -79,13 +79,19 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
       }
       const float ma = sa * (1.0f / C), mc = sc * (1.0f / C);
       const float ra = rsqrtf(fmaxf(qa * (1.0f / C) - ma * ma, 0.f) + eps), rc = rsqrtf(fmaxf(qc * (1.0f / C) - mc * mc, 0.f) + eps);
-      unsigned pa[4], pc[4];
+      unsigned pa[4] = {0, 0, 0, 0}, pc[4] = {0, 0, 0, 0};
+      if (ACC) {
+        if (oka) { const uint4 o = *reinterpret_cast<const uint4*>(zrow + (long long)ja * C + cl * 8); pa[0] = o.x; pa[1] = o.y; pa[2] = o.z; pa[3] = o.w; }
+        if (okc) { const uint4 o = *reinterpret_cast<const uint4*>(zrow + (long long)jc * C + cl * 8); pc[0] = o.x; pc[1] = o.y; pc[2] = o.z; pc[3] = o.w; }
+      }
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float g0 = g[2 * e], g1 = g[2 * e + 1];
-        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf((xa[2 * e] - ma) * ra, g0, b[2 * e]), fmaf((xa[2 * e + 1] - ma) * ra, g1, b[2 * e + 1]));
+        const float oa0 = ACC ? __uint_as_float(pa[e] << 16) : 0.f, oa1 = ACC ? __uint_as_float(pa[e] & 0xffff0000u) : 0.f;
+        const float oc0 = ACC ? __uint_as_float(pc[e] << 16) : 0.f, oc1 = ACC ? __uint_as_float(pc[e] & 0xffff0000u) : 0.f;
+        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf((xa[2 * e] - ma) * ra, g0, b[2 * e]) + oa0, fmaf((xa[2 * e + 1] - ma) * ra, g1, b[2 * e + 1]) + oa1);
         pa[e] = *reinterpret_cast<unsigned*>(&h);
-        h = __floats2bfloat162_rn(fmaf((xc[2 * e] - mc) * rc, g0, b[2 * e]), fmaf((xc[2 * e + 1] - mc) * rc, g1, b[2 * e + 1]));
+        h = __floats2bfloat162_rn(fmaf((xc[2 * e] - mc) * rc, g0, b[2 * e]) + oc0, fmaf((xc[2 * e + 1] - mc) * rc, g1, b[2 * e + 1]) + oc1);
         pc[e] = *reinterpret_cast<unsigned*>(&h);
       }
       if (oka) *reinterpret_cast<uint4*>(zrow + (long long)ja * C + cl * 8) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
@@ -97,7 +103,7 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
 bool fast_broadcast_supported(int c_z) { return c_z == 64 || c_z == 128 || c_z == 256; }
 
 nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
-                            void* z, const BatchMeta& m, cudaStream_t st) {
+                            void* z, const BatchMeta& m, cudaStream_t st, bool accumulate) {
   long long items = 0;
   for (int s = 0; s < m.B; ++s) items += (long long)m.N[s] * ((m.N[s] + BJ - 1) / BJ);
   if (items == 0) return NT_OK;
@@ -108,10 +114,16 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
   const __nv_bfloat16* b = (const __nv_bfloat16*)beta;
   __nv_bfloat16* zz = (__nv_bfloat16*)z;
   {
-    LaunchScope ls("broadcast_ln", st);
-    if (c_z == 64) broadcast_ln_fast_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-    else if (c_z == 128) broadcast_ln_fast_kernel<16><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-    else broadcast_ln_fast_kernel<32><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+    LaunchScope ls(accumulate ? "broadcast_ln_add" : "broadcast_ln", st);
+    if (accumulate) {
+      if (c_z == 64) broadcast_ln_fast_kernel<8, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else if (c_z == 128) broadcast_ln_fast_kernel<16, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else broadcast_ln_fast_kernel<32, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+    } else {
+      if (c_z == 64) broadcast_ln_fast_kernel<8, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else if (c_z == 128) broadcast_ln_fast_kernel<16, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else broadcast_ln_fast_kernel<32, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+    }
   }
   return cuda_ok();
 }

@@ -256,7 +256,7 @@ template nt_status launch_contract<__nv_bfloat16>(const __nv_bfloat16*, const __
 template <typename T>
 __global__ void __launch_bounds__(256) broadcast_ln_kernel(const float* __restrict__ u, const float* __restrict__ v,
                                                           const T* __restrict__ gamma, const T* __restrict__ beta,
-                                                          float eps, int c_z, T* __restrict__ z, BatchMeta m) {
+                                                          float eps, int c_z, T* __restrict__ z, BatchMeta m, int accumulate) {
   const int lane = threadIdx.x & 31;
   const long long p = m.pair_off[0] + (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (p >= m.pair_off[m.B]) return;
@@ -281,27 +281,27 @@ __global__ void __launch_bounds__(256) broadcast_ln_kernel(const float* __restri
   const float rs = rsqrtf(q / (float)c_z + eps);
   T* zr = z + p * c_z;
   for (int c = lane; c < c_z; c += 32)
-    Cvt<T>::st(zr + c, (ur[c] + vr[c] - mean) * rs * Cvt<T>::ld(gamma + c) + Cvt<T>::ld(beta + c));
+    Cvt<T>::st(zr + c, (ur[c] + vr[c] - mean) * rs * Cvt<T>::ld(gamma + c) + Cvt<T>::ld(beta + c) + (accumulate ? Cvt<T>::ld(zr + c) : 0.f));
 }
 
 template <typename T>
 nt_status launch_broadcast_ln(const float* u, const float* v, const T* gamma, const T* beta, float eps, int c_z,
-                              T* z, const BatchMeta& m, cudaStream_t st) {
+                              T* z, const BatchMeta& m, cudaStream_t st, bool accumulate) {
   long long npos = m.pair_off[m.B] - m.pair_off[0];
   if (npos <= 0) return NT_OK;
   long long blocks = (npos + 7) / 8;
   if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
   {
-    LaunchScope ls("generic_broadcast_ln", st);
-    broadcast_ln_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(u, v, gamma, beta, eps, c_z, z, m);
+    LaunchScope ls(accumulate ? "generic_broadcast_ln_add" : "generic_broadcast_ln", st);
+    broadcast_ln_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(u, v, gamma, beta, eps, c_z, z, m, accumulate ? 1 : 0);
   }
   return cuda_ok();
 }
 template nt_status launch_broadcast_ln<float>(const float*, const float*, const float*, const float*, float, int,
-                                              float*, const BatchMeta&, cudaStream_t);
+                                              float*, const BatchMeta&, cudaStream_t, bool);
 template nt_status launch_broadcast_ln<__nv_bfloat16>(const float*, const float*, const __nv_bfloat16*,
                                                       const __nv_bfloat16*, float, int, __nv_bfloat16*,
-                                                      const BatchMeta&, cudaStream_t);
+                                                      const BatchMeta&, cudaStream_t, bool);
 
 // ------------------------------------------------------------------------------------------
 // attention core: one warp per (attention row, head, query); lanes over keys; online softmax.

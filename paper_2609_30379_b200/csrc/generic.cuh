@@ -39,7 +39,7 @@ nt_status launch_contract(const T* a, const T* b, T* t, int C, const BatchMeta& 
 // z[p,:] = LN(u[row(p)] + v[col(p)]) * gamma + beta;  u, v float [T1, c_z]
 template <typename T>
 nt_status launch_broadcast_ln(const float* u, const float* v, const T* gamma, const T* beta, float eps, int c_z,
-                              T* z, const BatchMeta& m, cudaStream_t st);
+                              T* z, const BatchMeta& m, cudaStream_t st, bool accumulate = false);
 
 // softmax attention over attention rows.  pair order: rows are (s, i) and bias (nullable) is the
 // head-major channel-major buffer; token order: one row per sample.

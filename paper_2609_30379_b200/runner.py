@@ -61,21 +61,23 @@ class PairStack:
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=self.device)
 
     # one block, in place on x; z is rebuilt from x
-    def block(self, x: torch.Tensor, w: dict, stream=None):
+    def block(self, x: torch.Tensor, w: dict, stream=None, accumulate=False):
         cfg, L = self.cfg, self.L
         b = w["broadcast"]
-        nt.nt_pair_broadcast(L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], LN_EPS, self.z, self.workspace, stream)
+        bc = nt.nt_pair_broadcast_add if accumulate else nt.nt_pair_broadcast
+        bc(L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], LN_EPS, self.z, self.workspace, stream)
         nt.nt_tri_mul_out(L, w["trimul"], LN_EPS, self.z, self.workspace, stream)
         nt.nt_row_attn_pairbias(L, nt.NT_ORDER_PAIR_IJC, w["attn"], cfg.H, cfg.d, LN_EPS, self.z, self.workspace, stream)
         nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, self.z, self.m, L.status, stream)
         nt.nt_token_update(self.m, w["reduce"]["W_r"], x, stream)
 
-    def forward(self, x: torch.Tensor, stream=None):
+    def forward(self, x: torch.Tensor, stream=None, persistent=False):
         """Runs every block in place on ``x`` [T1, c_s]; returns (x, z) for pair configs or
-        (x, pooled) for the token-only configuration."""
+        (x, pooled) for the token-only configuration.  persistent=True keeps the pair state as a stream of its
+        own: from the second block on the broadcast is accumulated onto it instead of replacing it."""
         if self.cfg.kind == "pair":
-            for w in self.W:
-                self.block(x, w, stream)
+            for n, w in enumerate(self.W):
+                self.block(x, w, stream, accumulate=persistent and n > 0)
             return x, self.z
         for w in self.W:
             nt.nt_row_attn_pairbias(self.L, nt.NT_ORDER_TOKEN_NC, w, self.cfg.H, self.cfg.d, LN_EPS, x,
