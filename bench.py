@@ -189,13 +189,13 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------------------------
 def oracle_sample_rate(cfg, inp, n_samples, repeats=1):
-    """Times the NumPy oracle (as it stands, float32 on the same bf16-rounded inputs) on one block over
+    """Times the NumPy oracle as it stands (float64, on the same bf16-rounded inputs) on one block over
     the first n_samples samples of the batch.  Returns (positions/s, seconds, sample description)."""
     from oracle import nested_pair_oracle as orc
     lengths = list(cfg.lengths[:n_samples])
     T1s = sum(lengths)
     x = inp["x"][:T1s]
-    dt = np.float64 if cfg.dtype == "f32" else np.float32
+    dt = np.float64
     best = None
     for _ in range(repeats):
         t0 = time.perf_counter()
@@ -230,7 +230,7 @@ def run_reference(args):
     cores = len(os.sched_getaffinity(0))
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=min(warm, 1), ms_per_step=el / max(args.steps, 1) * 1e3, higher_is_better=True,
-                scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
                 config=dict(workload=f"{cfg.name}: per step {desc}", lengths=list(cfg.lengths[:1])),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=desc),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
@@ -529,7 +529,7 @@ def main():
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        n_s = {"cfg1": cfg.B, "cfg2": 4, "cfg3": 8, "cfg4": cfg.B, "cfg5": 1}[cfg.name]
+        n_s = {"cfg1": cfg.B, "cfg2": 8, "cfg3": 8, "cfg4": cfg.B, "cfg5": 1}[cfg.name]
         rate, sec, desc = oracle_sample_rate(cfg, inp, n_s)
         cpu = dict(value=rate, unit=UNIT, cores=len(os.sched_getaffinity(0)), kind="oracle",
                    sample=f"{desc}; {sec:.1f} s")
