@@ -92,8 +92,9 @@ def kernel_work(cfg: wl.Config):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (cfg2 only);
 # other workloads report traffic = None.
-NCU_TRAFFIC_CFG2 = {"attn_core": 375.1e6, "tri_out": 243.3e6, "attn_in": 324.7e6, "tri_in": 233.1e6, "attn_out": 240.1e6,
-                    "tri_contract": 255.0e6}
+NCU_TRAFFIC_CFG2 = {"attn_core": 375.2e6, "tri_out": 242.2e6, "attn_in": 324.4e6, "tri_in": 232.0e6, "attn_out": 240.4e6,
+                    "tri_contract": 255.4e6, "transition": 130.3e6, "tri_contract_in": 255.5e6, "attn_core_col": 375.1e6,
+                    "single_attn_bias": 97.8e6}
 
 
 # Exponentials per second of the special-function units: 16 per clock and SM (measured: 15.99 with ex2.approx.f32,

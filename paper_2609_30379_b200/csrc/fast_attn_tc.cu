@@ -317,12 +317,19 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
         if (warp_live) {
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
           int g = gb;
-          if ((g & 1) && g < ge) {
+          // reading needs no alignment of the granule index: four granules (64 columns) per wait while they last
+#pragma unroll 1
+          for (; g + 4 <= ge; g += 4) {
+            unsigned rc[16], rd[16];
             tmem_ld16(t_row + g * 16, ra);
-            tmem_ld_wait16(ra);
+            tmem_ld16(t_row + g * 16 + 16, rb);
+            tmem_ld16(t_row + g * 16 + 32, rc);
+            tmem_ld16(t_row + g * 16 + 48, rd);
+            tmem_ld_wait2(ra, rb);
+            tmem_ld_wait2(rc, rd);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(ra[e]));
-            ++g;
+            for (int e = 0; e < 16; ++e)
+              m4[e & 3] = fmaxf(m4[e & 3], fmaxf(fmaxf(__uint_as_float(ra[e]), __uint_as_float(rb[e])), fmaxf(__uint_as_float(rc[e]), __uint_as_float(rd[e]))));
           }
 #pragma unroll 1
           for (; g + 2 <= ge; g += 2) {
