@@ -1,9 +1,10 @@
 // Attention output stage on tcgen05 (bf16, float accumulate), in place on the pair state:
 //   z += (sigmoid(LN(z) W_g^T) * o) W_o^T
-// The gate is recomputed from z here (LayerNorm folded into W_g, see fast_tri_in.cu) instead of
+// The gate is recomputed from z here (LayerNorm folded into W_g: W_g' = bf16(W_g gamma) meets the bf16 state
+// directly, the row statistics are taken beside the MMA and applied in the epilogue) instead of
 // being written by the input projection.  Per 128-position tile: TMA brings the z tile and the o
-// tile; the MMA warp computes the gate pre-activation into TMEM; the epilogue warps turn it into
-// sigmoid(.) * o, written back over the o tile in shared memory; the MMA warp multiplies that by
+// tile; the MMA warp computes the gate pre-activation into TMEM as soon as they land; the epilogue warps turn it
+// into sigmoid(.) * o, written back over the o tile in shared memory; the MMA warp multiplies that by
 // W_o; the epilogue adds the residual into the z tile and TMA-stores it.
 #include <cstring>
 
@@ -12,7 +13,7 @@
 
 namespace ntp {
 
-constexpr int AO_THREADS = 64 + 128 + 256;   // producer, MMA, 4 converter warps, 8 epilogue warps
+constexpr int AO_THREADS = 64 + 128 + 256;   // producer, MMA, 4 statistics warps, 8 epilogue warps
 
 struct AttnOutParams {
   CUtensorMap zmap;              // {c, rows}, box {64, 128}: load and store
@@ -103,7 +104,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
     int stage = 0;
     unsigned phase = 0, tph0 = 0, tph1 = 0, gph0 = 0, gph1 = 0;
     unsigned n = 0;
-    const unsigned idesc_g = idesc_f16(128, Hd, 0, 0, FMT_F16, FMT_F16);    // z tile converted to fp16, folded W_g fp16
+    const unsigned idesc_g = idesc_f16(128, Hd, 0, 0, FMT_BF16, FMT_BF16);  // the bf16 z tile, folded W_g bf16
     const unsigned idesc_o = idesc_f16(128, c, 0, 0, FMT_BF16, FMT_BF16);   // gated o bf16, W_o as given (bf16)
     const unsigned long long wg_desc = desc_kmajor_sw128(smem_u32(sWg)), wo_desc = desc_kmajor_sw128(smem_u32(sWo));
     const unsigned slab16 = (unsigned)slab >> 4, wg16 = (unsigned)wg_slab >> 4, wo16 = (unsigned)wo_slab >> 4;
@@ -111,7 +112,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       const unsigned buf = n & 1;
       if (buf == 0) { mbar_wait(&tempty[0], tph0 ^ 1, ab); tph0 ^= 1; }
       else { mbar_wait(&tempty[1], tph1 ^ 1, ab); tph1 ^= 1; }
-      mbar_wait(&aconv[stage], phase, ab);
+      mbar_wait(&afull[stage], phase, ab);
       tc_fence_after();
       const unsigned long long st_desc = desc_kmajor_sw128(smem_u32(sSt + stage * stage_bytes));
       const unsigned dg = tmem_base + buf * 256, dout = dg + Hd;
@@ -138,17 +139,29 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
   } else if (warp >= 2 && warp < 6) {
-    // ------------------------------------------------------------------ converters (4 warps, one row per thread)
+    // ------------------------------------------------------------------ row statistics (4 warps, one row per thread),
+    // beside the gate MMA
     const int row = (warp - 2) * 32 + lane;
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
-      float sum, sq;
-      convert_row_bf16_to_f16(sSt + stage * stage_bytes, zslab, slab, row, sum, sq);
+      float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
+      const unsigned char* zt = sSt + stage * stage_bytes;
+      for (int g8 = 0; g8 < c / 8; ++g8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(zt + (g8 >> 3) * slab + sw128_off(row, g8 & 7));
+        const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+          s4[e] += lo + hi;
+          q4[e] = fmaf(lo, lo, q4[e]);
+          q4[e] = fmaf(hi, hi, q4[e]);
+        }
+      }
+      const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]), sq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
       const float mean = sum / (float)c;
       sStats[stage][row] = make_float2(mean, rsqrtf(fmaxf(sq / (float)c - mean * mean, 0.f) + p.eps));
-      fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&aconv[stage]);
       if (++stage == 2) { stage = 0; phase ^= 1; }
@@ -166,7 +179,8 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       const int buf = (int)(n & 1);
       unsigned char* st = sSt + stage * stage_bytes;
       // ---- phase 1: o <- sigmoid(gate) * o, in place in shared memory
-      mbar_wait(&gfull[buf], gph[buf], ab);         // gate MMA done, hence the statistics are published too
+      mbar_wait(&aconv[stage], (unsigned)((n >> 1) & 1), ab);   // the row statistics are published
+      mbar_wait(&gfull[buf], gph[buf], ab);
       gph[buf] ^= 1;
       tc_fence_after();
       const float mean = sStats[stage][row].x, rstd = sStats[stage][row].y;
@@ -215,8 +229,8 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            const float2 zo = unpack_h2(w[e]);        // the z tile holds fp16 after conversion
-            __nv_bfloat162 hh = __floats2bfloat162_rn(zo.x + __uint_as_float(r[n0]), zo.y + __uint_as_float(r[n0 + 1]));
+            const float z0 = __uint_as_float(w[e] << 16), z1 = __uint_as_float(w[e] & 0xffff0000u);   // the bf16 state
+            __nv_bfloat162 hh = __floats2bfloat162_rn(z0 + __uint_as_float(r[n0]), z1 + __uint_as_float(r[n0 + 1]));
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);

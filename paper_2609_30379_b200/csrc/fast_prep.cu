@@ -152,7 +152,9 @@ nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* pr
   const void* s0[6] = {W->W_q, W->W_k, W->W_v, W->W_b, nullptr, W->W_g};
   const int r0[6] = {Hd, Hd, Hd, W->W_b ? H : 0, W->W_b ? 16 - H : 16, W->W_g ? Hd : 0};
   const float sc[6] = {1.f, 1.f, 1.f, sqrtf((float)d), 1.f, 1.f};   // bias rows times sqrt(d)
-  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01, sc, out.aug);
+  // W_g meets the bf16 state itself in the output stage (no conversion pass there): its folded rows are bf16
+  const int asbf16[6] = {0, 0, 0, 0, 0, 1};
+  add_job(a, s0, r0, 6, c, W->ln_gamma, W->ln_beta, out.w, out.c01, sc, out.aug, asbf16);
   return run_prep(a, st);
 }
 
