@@ -29,6 +29,8 @@ What each function follows:
   single_attn_pairbias the pair-biased single attention of Sec. 4.3 (tokens attend tokens of the same sample, logits
                        biased by a projection of the pair state); pinned by library attention with an additive mask,
                        scalar loops, and its reduction to the token-order attention when the bias weights are zero.
+  rect_*               the rectangular pair layout (N_i, M_i): Eq. 2 packing (sum N_i M_i rows), Eq. 4 (column reduction
+                       over the M_i cells of a row; its mean divides by M_i, App. A.1), distinct row and column inputs.
   segment_reduce       Eq. 4 (pair reduction) and the mean of Eq. 1 line 3; App. A batch-axis
                        convention (``[1,2],[3,4]`` sums to ``[3,7]``).
   token_update         Eq. 1 line 3: ``X~ = X + g(mean_b P~[a,b,:])`` with ``g`` a bias-free projection.
@@ -338,6 +340,60 @@ def single_attn_pairbias(x, z, lengths, W, H, d, eps=LN_EPS, dtype=np.float64, r
         op_ += n * n
     res = np.concatenate(out, axis=0) if out else x.copy()
     return (res, parts) if return_parts else res
+
+
+# --------------------------------------------------------------------------------------------
+# rectangular pairs (N_i, M_i): the paper's second pair layout (Eq. 2: pairs (N_i, M_i, C) pack as (sum N_i M_i, C);
+# Eq. 4: a column reduction groups the M_i cells of one row; App. A.1: the rectangular variant has distinct row and
+# column inputs and divides its column mean by M_i)
+# --------------------------------------------------------------------------------------------
+def rect_offsets(lengths_n, lengths_m):
+    """Offsets of a batch of rectangular pairs: tokn_off / tokm_off (prefix sums of N_i / M_i), pair_off (prefix sums
+    of N_i M_i), the level-2 row splits (one group of M_s cells per row (s, a): sum N + 1 entries), and the decode of
+    every packed cell p = pair_off[s] + a M_s + b into (s, a, b)."""
+    n = np.asarray(lengths_n, dtype=np.int64)
+    m = np.asarray(lengths_m, dtype=np.int64)
+    assert n.shape == m.shape and np.all(n >= 0) and np.all(m >= 0)
+    tokn = np.concatenate([[0], np.cumsum(n)]).astype(np.int64)
+    tokm = np.concatenate([[0], np.cumsum(m)]).astype(np.int64)
+    po = np.concatenate([[0], np.cumsum(n * m)]).astype(np.int64)
+    rs = np.empty(int(tokn[-1]) + 1, dtype=np.int64)
+    ps, pi, pj = [], [], []
+    for s in range(len(n)):
+        for a in range(int(n[s])):
+            rs[tokn[s] + a] = po[s] + a * m[s]
+        if n[s] and m[s]:
+            ps.append(np.full(int(n[s] * m[s]), s, dtype=np.int32))
+            pi.append(np.repeat(np.arange(n[s], dtype=np.int32), int(m[s])))
+            pj.append(np.tile(np.arange(m[s], dtype=np.int32), int(n[s])))
+    rs[-1] = po[-1]
+    cat = lambda l: np.concatenate(l) if l else np.zeros(0, dtype=np.int32)
+    return dict(tokn_off=tokn, tokm_off=tokm, pair_off=po, row_splits=rs, pos_sample=cat(ps), pos_i=cat(pi), pos_j=cat(pj))
+
+
+def rect_pair_broadcast(x, y, lengths_n, lengths_m, W_a, W_b, ln_gamma, ln_beta, eps=LN_EPS, dtype=np.float64):
+    """Rectangular broadcast: z[(s, a, b), :] = LN(W_a x_{s,a} + W_b y_{s,b}) gamma + beta with x the row tokens
+    [sum N, c_s] and y the column tokens [sum M, c_s]; output [sum N M, c_z]."""
+    x, y, W_a, W_b, g, bt = _as(dtype, x, y, W_a, W_b, ln_gamma, ln_beta)
+    out, on, om = [], 0, 0
+    for n, m in zip((int(v) for v in lengths_n), (int(v) for v in lengths_m)):
+        u = x[on:on + n] @ W_a.T
+        v = y[om:om + m] @ W_b.T
+        out.append(layer_norm(u[:, None, :] + v[None, :, :], g, bt, eps).reshape(n * m, -1))
+        on += n
+        om += m
+    return np.concatenate(out, axis=0) if out else np.zeros((0, W_a.shape[0]), dtype=dtype)
+
+
+def rect_block_forward(x, y, lengths_n, lengths_m, w, eps=LN_EPS, dtype=np.float64):
+    """Single-pair-single block on rectangular pairs (Eq. 1 with distinct row and column inputs): broadcast + LN,
+    the position-wise SwiGLU transition, the mean over the column axis (divided by M_s, Eq. 4) and the token update of
+    the row tokens.  Returns (x', z)."""
+    off = rect_offsets(lengths_n, lengths_m)
+    z = rect_pair_broadcast(x, y, lengths_n, lengths_m, eps=eps, dtype=dtype, **w["broadcast"])
+    z = pair_transition(z, w["transition"], eps=eps, dtype=dtype)
+    mrow = segment_reduce(z, off["row_splits"], "mean", dtype=dtype)
+    return token_update(x, mrow, w["reduce"]["W_r"], dtype=dtype), z
 
 
 def segment_reduce(v, splits, op="mean", dtype=np.float64):

@@ -653,3 +653,113 @@ def test_transition_is_position_wise():
     z, W = _transition_case(rows=13, c=8, seed=2)
     perm = np.random.default_rng(0).permutation(z.shape[0])
     np.testing.assert_allclose(orc.pair_transition(z[perm], W), orc.pair_transition(z, W)[perm], rtol=1e-13, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------------------------
+# rectangular pairs (N_i, M_i): Eq. 2 packing, Eq. 4 column reduction, distinct row / column inputs
+# ---------------------------------------------------------------------------------------------
+def _rect_case(ln, lm, seed=5, c_s=6, c_z=8):
+    cfg = wl.Config("rect", "f32", tuple(ln), c_s=c_s, c_z=c_z, c_h=4, H=2, d=4, blocks=1, seed=seed)
+    inp = wl.make_inputs(cfg)
+    rng = np.random.default_rng(seed + 100)
+    y = rng.standard_normal((int(sum(lm)), c_s))
+    w = dict(broadcast=inp["blocks"][0]["broadcast"], transition=wl.make_transition_weights(cfg), reduce=inp["blocks"][0]["reduce"])
+    return inp["x"].astype(np.float64), y, w
+
+
+def test_rect_offsets_structure():
+    ln, lm = (2, 3, 0, 1), (3, 1, 4, 0)
+    off = orc.rect_offsets(ln, lm)
+    assert off["tokn_off"].tolist() == [0, 2, 5, 5, 6] and off["tokm_off"].tolist() == [0, 3, 4, 8, 8]
+    assert off["pair_off"].tolist() == [0, 6, 9, 9, 9]                     # o_0 = 0, o_{s+1} - o_s = N_s M_s, o_B = T
+    assert off["row_splits"].tolist() == [0, 3, 6, 7, 8, 9, 9]            # one group of M_s cells per row; sum N + 1 entries
+    assert off["pos_sample"].tolist() == [0] * 6 + [1] * 3
+    assert off["pos_i"].tolist() == [0, 0, 0, 1, 1, 1, 0, 1, 2] and off["pos_j"].tolist() == [0, 1, 2, 0, 1, 2, 0, 0, 0]
+    # coordinate map o_s + a M_s + b composed with the decode is the identity
+    for p_, (s_, a, b) in enumerate(zip(off["pos_sample"], off["pos_i"], off["pos_j"])):
+        assert off["pair_off"][s_] + a * lm[s_] + b == p_
+    # square lengths reproduce the square layout
+    sq = orc.offsets_build((2, 3))
+    r = orc.rect_offsets((2, 3), (2, 3))
+    assert np.array_equal(r["pair_off"], sq["pair_off"]) and np.array_equal(r["row_splits"], sq["row_splits"])
+
+
+def test_rect_broadcast_and_reduction_definitions():
+    ln, lm = (3, 1, 4), (2, 5, 3)
+    x, y, w = _rect_case(ln, lm)
+    z = orc.rect_pair_broadcast(x, y, ln, lm, **w["broadcast"])
+    assert z.shape == (sum(n * m for n, m in zip(ln, lm)), 8)              # exactly sum N_s M_s rows
+    off = orc.rect_offsets(ln, lm)
+    b = {k: np.asarray(v, dtype=np.float64) for k, v in w["broadcast"].items()}
+    # cell by cell from the decode (the explicit-packed form u[rows] + v[cols])
+    u, v = x @ b["W_a"].T, y @ b["W_b"].T
+    rows = off["tokn_off"][off["pos_sample"]] + off["pos_i"]
+    cols = off["tokm_off"][off["pos_sample"]] + off["pos_j"]
+    assert np.allclose(z, orc.layer_norm(u[rows] + v[cols], b["ln_gamma"], b["ln_beta"]), rtol=1e-12, atol=1e-12)
+    # the column reduction of Eq. 4, written out: V_Y[eta_s + a] = sum_b V_P[o_s + a M_s + b]; the mean divides by M_s
+    want_sum = np.zeros((sum(ln), z.shape[1]))
+    for s_ in range(len(ln)):
+        for a in range(ln[s_]):
+            for bb in range(lm[s_]):
+                want_sum[off["tokn_off"][s_] + a] += z[off["pair_off"][s_] + a * lm[s_] + bb]
+    assert np.allclose(orc.segment_reduce(z, off["row_splits"], "sum"), want_sum, rtol=1e-12, atol=1e-12)
+    cnt = np.repeat(np.asarray(lm, dtype=np.float64), ln)[:, None]
+    assert np.allclose(orc.segment_reduce(z, off["row_splits"], "mean"), want_sum / cnt, rtol=1e-12, atol=1e-12)
+    # square special case: same lengths and the same tokens on both sides give the square broadcast
+    xs = x[:sum((3, 1))]
+    zs = orc.rect_pair_broadcast(xs, xs, (3, 1), (3, 1), **w["broadcast"])
+    assert np.array_equal(zs, orc.pair_broadcast(xs, (3, 1), **w["broadcast"]))
+
+
+def test_rect_block_equals_padded_and_masked_computation():
+    ln, lm = (3, 1, 4), (2, 5, 3)
+    x, y, w = _rect_case(ln, lm)
+    x2, z = orc.rect_block_forward(x, y, ln, lm, w)
+    # an independent dense computation on a [B, Nmax, Mmax] envelope with a validity mask and the true counts
+    B, Nx, Mx = len(ln), max(ln), max(lm)
+    b = {k: np.asarray(v, dtype=np.float64) for k, v in w["broadcast"].items()}
+    tw = {k: np.asarray(v, dtype=np.float64) for k, v in w["transition"].items()}
+    xp, yp = np.zeros((B, Nx, x.shape[1])), np.zeros((B, Mx, x.shape[1]))
+    on = om = 0
+    for s_, (n, m) in enumerate(zip(ln, lm)):
+        xp[s_, :n], yp[s_, :m] = x[on:on + n], y[om:om + m]
+        on, om = on + n, om + m
+    U, V = xp @ b["W_a"].T, yp @ b["W_b"].T
+    Z = U[:, :, None, :] + V[:, None, :, :]
+    Z = (Z - Z.mean(-1, keepdims=True)) / np.sqrt(Z.var(-1, keepdims=True) + 1e-5) * b["ln_gamma"] + b["ln_beta"]
+    Zh = (Z - Z.mean(-1, keepdims=True)) / np.sqrt(Z.var(-1, keepdims=True) + 1e-5) * tw["ln_gamma"] + tw["ln_beta"]
+    ga = Zh @ tw["W_a"].T
+    Z = Z + ((ga / (1 + np.exp(-ga))) * (Zh @ tw["W_b"].T)) @ tw["W_2"].T
+    mask = np.zeros((B, Nx, Mx, 1))
+    for s_, (n, m) in enumerate(zip(ln, lm)):
+        mask[s_, :n, :m] = 1
+    mean = (Z * mask).sum(2) / np.maximum(np.asarray(lm, dtype=np.float64), 1)[:, None, None]
+    Xn = xp + mean @ np.asarray(w["reduce"]["W_r"], dtype=np.float64).T
+    on = op_ = 0
+    for s_, (n, m) in enumerate(zip(ln, lm)):
+        assert np.allclose(z[op_:op_ + n * m], Z[s_, :n, :m].reshape(n * m, -1), rtol=1e-10, atol=1e-10)
+        assert np.allclose(x2[on:on + n], Xn[s_, :n], rtol=1e-10, atol=1e-10)
+        on, op_ = on + n, op_ + n * m
+
+
+RECT_PATTERNS = [   # the kinds of structure change the paper's validation patterns name (App. A.1)
+    ((4, 2, 6), (3, 6, 2)), ((2, 4, 6), (6, 3, 2)), ((6, 6), (3, 3)),          # changed partitions, fixed total of 36 cells
+    ((5, 1), (2, 7)), ((8, 3, 2), (1, 9, 4)),                                    # changed packed extents and maxima
+    ((3, 3, 3), (3, 3, 3)), ((3, 3, 3), (4, 4, 4)), ((1,), (1,)),                # fresh equal structures
+]
+
+
+@pytest.mark.parametrize("ln,lm", RECT_PATTERNS)
+def test_rect_validation_patterns_structure_and_sample_locality(ln, lm):
+    off = orc.rect_offsets(ln, lm)
+    n, m = np.asarray(ln), np.asarray(lm)
+    assert off["pair_off"][0] == 0 and np.array_equal(np.diff(off["pair_off"]), n * m) and off["pair_off"][-1] == int((n * m).sum())
+    assert len(off["row_splits"]) == n.sum() + 1 and np.array_equal(np.diff(off["row_splits"]), np.repeat(m, n))
+    x, y, w = _rect_case(ln, lm, seed=11)
+    x2, z = orc.rect_block_forward(x, y, ln, lm, w)
+    # every sample's result is what it gets alone (sample-local semantics)
+    for s_ in range(len(ln)):
+        xa, ya = x[off["tokn_off"][s_]:off["tokn_off"][s_ + 1]], y[off["tokm_off"][s_]:off["tokm_off"][s_ + 1]]
+        x1, z1 = orc.rect_block_forward(xa, ya, (ln[s_],), (lm[s_],), w)
+        assert np.allclose(z[off["pair_off"][s_]:off["pair_off"][s_ + 1]], z1, rtol=1e-12, atol=1e-12)
+        assert np.allclose(x2[off["tokn_off"][s_]:off["tokn_off"][s_ + 1]], x1, rtol=1e-12, atol=1e-12)
