@@ -201,6 +201,34 @@ nt_status nt_single_attn_pairbias(const nt_layout *L, nt_dtype dt, int32_t c_s, 
 size_t nt_single_attn_workspace_bytes(nt_dtype dt, const int64_t *lengths_h, int32_t B, int32_t c_s, int32_t H, int32_t d);
 
 /*
+ * Rectangular pairs (N_s, M_s): the method's second pair layout (Eq. 2: pairs (N_i, M_i, C) pack as (sum N_i M_i, C);
+ * cell (s, a, b) lives at packed row pair_off[s] + a M_s + b).
+ *
+ * nt_rect_offsets_build -- prefix sums and cell decode of a batch of rectangular pairs.
+ *   tokn_off[s] = sum_{s'<s} N_s', tokm_off[s] = sum_{s'<s} M_s', pair_off[s] = sum_{s'<s} N_s' M_s'   (each [B+1])
+ *   row_splits[tokn_off[s]+a] = pair_off[s] + a M_s, row_splits[T1n] = T2  ([T1n+1], nullable): one group of M_s cells
+ *     per row, the groups the column reduction of Eq. 4 consumes (nt_segment_reduce over them; its mean divides by M_s)
+ *   pos_sample / pos_i / pos_j [T2] (int32, nullable as a group): the decode of every cell
+ *   lengths_n_d, lengths_m_d [B] device int64.  Integer work, bit-exact; inconsistent totals or a negative length
+ *   write NT_ERR_INCONSISTENT to *status_d.
+ *
+ * nt_rect_pair_broadcast -- z[(s,a,b),:] = LN(W_a x_{s,a} + W_b y_{s,b}) * gamma + beta from distinct row tokens
+ *   x [T1n, c_s] and column tokens y [T1m, c_s] (App. A.1); z [T2, c_z] out (exactly T2 * c_z elements).
+ *   lengths_n_h, lengths_m_h [B] HOST int64 (read during the call).  Workspace: nt_rect_broadcast_workspace_bytes.
+ *   Errors as nt_pair_broadcast.
+ */
+nt_status nt_rect_offsets_build(const int64_t *lengths_n_d, const int64_t *lengths_m_d, int32_t B,
+                                int64_t T1n, int64_t T1m, int64_t T2,
+                                int64_t *tokn_off_d, int64_t *tokm_off_d, int64_t *pair_off_d, int64_t *row_splits_d,
+                                int32_t *pos_sample_d, int32_t *pos_i_d, int32_t *pos_j_d,
+                                int32_t *status_d, nt_stream stream);
+nt_status nt_rect_pair_broadcast(nt_dtype dt, int32_t B, const int64_t *lengths_n_h, const int64_t *lengths_m_h,
+                                 int32_t c_s, int32_t c_z, const void *x, const void *y,
+                                 const void *W_a, const void *W_b, const void *ln_gamma, const void *ln_beta,
+                                 float ln_eps, void *z, void *workspace, size_t workspace_bytes, nt_stream stream);
+size_t nt_rect_broadcast_workspace_bytes(const int64_t *lengths_n_h, const int64_t *lengths_m_h, int32_t B, int32_t c_z);
+
+/*
  * nt_segment_reduce -- segmented sum or mean of contiguous row groups (Eq. 4 pair reduction; the
  * mean over j of Eq. 1 line 3 divides by the group's count; App. A batch-axis convention).
  *   out[g,:] = (1/len_g or 1) * sum_{r = splits[g]}^{splits[g+1]-1} v[r,:],  empty group -> 0.

@@ -379,7 +379,7 @@ def rect_pair_broadcast(x, y, lengths_n, lengths_m, W_a, W_b, ln_gamma, ln_beta,
     for n, m in zip((int(v) for v in lengths_n), (int(v) for v in lengths_m)):
         u = x[on:on + n] @ W_a.T
         v = y[om:om + m] @ W_b.T
-        out.append(layer_norm(u[:, None, :] + v[None, :, :], g, bt, eps).reshape(n * m, -1))
+        out.append(layer_norm(u[:, None, :] + v[None, :, :], g, bt, eps).reshape(n * m, W_a.shape[0]))
         on += n
         om += m
     return np.concatenate(out, axis=0) if out else np.zeros((0, W_a.shape[0]), dtype=dtype)

@@ -27,7 +27,8 @@ STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3:
 
 EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_add", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
            "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
-           "nt_single_attn_workspace_bytes", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
+           "nt_single_attn_workspace_bytes", "nt_rect_offsets_build", "nt_rect_pair_broadcast",
+           "nt_rect_broadcast_workspace_bytes", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
            "nt_launch_count", "nt_force_generic", "nt_profile_begin", "nt_profile_end")
 
@@ -79,6 +80,12 @@ def _load() -> C.CDLL:
                                             f32, vp, vp, vp, sz, vp]
     lib.nt_single_attn_workspace_bytes.argtypes = [i32, vp, i32, i32, i32, i32]
     lib.nt_single_attn_workspace_bytes.restype = sz
+    lib.nt_rect_offsets_build.argtypes = [vp, vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.nt_rect_offsets_build.restype = i32
+    lib.nt_rect_pair_broadcast.argtypes = [i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, f32, vp, vp, sz, vp]
+    lib.nt_rect_pair_broadcast.restype = i32
+    lib.nt_rect_broadcast_workspace_bytes.argtypes = [vp, vp, i32, i32]
+    lib.nt_rect_broadcast_workspace_bytes.restype = sz
     lib.nt_col_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, C.POINTER(nt_attn_weights), f32, vp, vp, sz, vp]
     lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
                                          f32, vp, vp, sz, vp]
@@ -249,6 +256,56 @@ def nt_single_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, x, z, wo
 def nt_single_attn_workspace_bytes(dtype, lengths, c_s: int, H: int, d: int) -> int:
     arr = (C.c_int64 * max(len(lengths), 1))(*[int(v) for v in lengths])
     return int(lib.nt_single_attn_workspace_bytes(dtype_code(dtype), arr, len(lengths), c_s, H, d))
+
+
+class RectLayout:
+    """Device offsets of a batch of rectangular pairs (N_s, M_s): tokn_off, tokm_off, pair_off, the level-2 row
+    splits and (optionally) the cell decode, all built on the device by nt_rect_offsets_build."""
+
+    def __init__(self, lengths_n, lengths_m, with_maps=False, device="cuda", stream=None):
+        import torch
+        self.lengths_n = [int(v) for v in lengths_n]
+        self.lengths_m = [int(v) for v in lengths_m]
+        assert len(self.lengths_n) == len(self.lengths_m)
+        self.B = len(self.lengths_n)
+        self.T1n, self.T1m = sum(self.lengths_n), sum(self.lengths_m)
+        self.T2 = sum(n * m for n, m in zip(self.lengths_n, self.lengths_m))
+        self.ln_h = (C.c_int64 * max(self.B, 1))(*self.lengths_n)
+        self.lm_h = (C.c_int64 * max(self.B, 1))(*self.lengths_m)
+        i64t = dict(dtype=torch.int64, device=device)
+        self.ln_d = torch.tensor(self.lengths_n, **i64t)
+        self.lm_d = torch.tensor(self.lengths_m, **i64t)
+        self.tokn_off = torch.empty(self.B + 1, **i64t)
+        self.tokm_off = torch.empty(self.B + 1, **i64t)
+        self.pair_off = torch.empty(self.B + 1, **i64t)
+        self.row_splits = torch.empty(self.T1n + 1, **i64t)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.pos_sample = self.pos_i = self.pos_j = None
+        if with_maps:
+            self.pos_sample = torch.empty(self.T2, dtype=torch.int32, device=device)
+            self.pos_i = torch.empty(self.T2, dtype=torch.int32, device=device)
+            self.pos_j = torch.empty(self.T2, dtype=torch.int32, device=device)
+        st = lib.nt_rect_offsets_build(_ptr(self.ln_d) if self.B else None, _ptr(self.lm_d) if self.B else None, self.B, self.T1n,
+                                       self.T1m, self.T2, _ptr(self.tokn_off), _ptr(self.tokm_off), _ptr(self.pair_off),
+                                       _ptr(self.row_splits), _ptr(self.pos_sample), _ptr(self.pos_i), _ptr(self.pos_j),
+                                       _ptr(self.status), _stream(stream))
+        _check(st, "nt_rect_offsets_build")
+
+    def device_status(self) -> int:
+        return int(self.status.item())
+
+
+def nt_rect_broadcast_workspace_bytes(L: RectLayout, c_z: int) -> int:
+    return int(lib.nt_rect_broadcast_workspace_bytes(L.ln_h, L.lm_h, L.B, c_z))
+
+
+def nt_rect_pair_broadcast(L: RectLayout, x, y, W_a, W_b, ln_gamma, ln_beta, ln_eps, z, workspace, stream=None):
+    """Rectangular broadcast from row tokens x [T1n, c_s] and column tokens y [T1m, c_s] into z [T2, c_z]."""
+    c_s, c_z = int(W_a.shape[1]), int(W_a.shape[0])
+    st = lib.nt_rect_pair_broadcast(dtype_code(x.dtype), L.B, L.ln_h, L.lm_h, c_s, c_z, _ptr(x), _ptr(y), _ptr(W_a), _ptr(W_b),
+                                    _ptr(ln_gamma), _ptr(ln_beta), float(ln_eps), _ptr(z), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_rect_pair_broadcast")
 
 
 def nt_col_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, z, workspace, stream=None):

@@ -1,0 +1,354 @@
+// Rectangular pairs (N_s, M_s): the second pair layout of the method (Eq. 2: pairs (N_i, M_i, C) pack as
+// (sum N_i M_i, C)).  Two entry points:
+//   nt_rect_offsets_build     prefix sums of N_s, M_s and N_s M_s, the level-2 row splits (one group of M_s cells per
+//                             row: the groups the column reduction of Eq. 4 consumes) and the cell decode
+//   nt_rect_pair_broadcast    z[(s, a, b), :] = LN(W_a x_{s,a} + W_b y_{s,b}) gamma + beta from distinct row and
+//                             column tokens (App. A.1: the rectangular variant has distinct row and column inputs)
+// Everything downstream of the broadcast is position-wise or a segmented reduction over the row splits and is served
+// by the existing calls (nt_pair_transition, nt_segment_reduce with these splits: its mean divides by M_s,
+// nt_token_update).  Integer work is bit-exact; the broadcast is a pure streaming write of the packed state.
+#include "fast.cuh"
+#include "generic.cuh"
+
+namespace ntp {
+
+constexpr int RS_THREADS = 1024;
+
+__global__ void __launch_bounds__(RS_THREADS)
+rect_scan_kernel(const int64_t* __restrict__ ln, const int64_t* __restrict__ lm, int B, long long T1n, long long T1m,
+                 long long T2, int64_t* __restrict__ tokn_off, int64_t* __restrict__ tokm_off,
+                 int64_t* __restrict__ pair_off, int32_t* status) {
+  __shared__ long long s1[RS_THREADS], s2[RS_THREADS], s3[RS_THREADS];
+  const int t = threadIdx.x;
+  const int per = (B + RS_THREADS - 1) / RS_THREADS;
+  const int lo = min(B, t * per), hi = min(B, lo + per);
+  long long a = 0, b = 0, c = 0;
+  bool neg = false;
+  for (int s = lo; s < hi; ++s) {
+    const long long n = ln[s], m = lm[s];
+    neg |= n < 0 || m < 0;
+    a += n;
+    b += m;
+    c += n * m;
+  }
+  s1[t] = a;
+  s2[t] = b;
+  s3[t] = c;
+  __syncthreads();
+  for (int off = 1; off < RS_THREADS; off <<= 1) {   // inclusive Hillis-Steele scan
+    long long va = 0, vb = 0, vc = 0;
+    if (t >= off) { va = s1[t - off]; vb = s2[t - off]; vc = s3[t - off]; }
+    __syncthreads();
+    s1[t] += va;
+    s2[t] += vb;
+    s3[t] += vc;
+    __syncthreads();
+  }
+  long long ea = s1[t] - a, eb = s2[t] - b, ec = s3[t] - c;
+  for (int s = lo; s < hi; ++s) {
+    const long long n = ln[s], m = lm[s];
+    tokn_off[s] = ea;
+    tokm_off[s] = eb;
+    pair_off[s] = ec;
+    ea += n;
+    eb += m;
+    ec += n * m;
+  }
+  if (t == RS_THREADS - 1) {
+    tokn_off[B] = s1[t];
+    tokm_off[B] = s2[t];
+    pair_off[B] = s3[t];
+    if ((s1[t] != T1n || s2[t] != T1m || s3[t] != T2) && status) atomicCAS(status, 0, (int)NT_ERR_INCONSISTENT);
+  }
+  if (neg && status) atomicCAS(status, 0, (int)NT_ERR_INCONSISTENT);
+}
+
+__device__ inline int rect_search(const int64_t* off, int B, long long p) {   // largest s with off[s] <= p
+  int lo = 0, hi = B;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (off[mid] <= p) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void rect_row_splits_kernel(const int64_t* __restrict__ lm, const int64_t* __restrict__ tokn_off,
+                                       const int64_t* __restrict__ pair_off, int B, long long T1n, long long T2,
+                                       int64_t* __restrict__ row_splits) {
+  if (tokn_off[B] != T1n || pair_off[B] != T2) return;   // inconsistent totals: flagged by the scan
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t > T1n) return;
+  if (t == T1n) { row_splits[t] = T2; return; }
+  const int s = rect_search(tokn_off, B, t);
+  row_splits[t] = pair_off[s] + (t - tokn_off[s]) * lm[s];
+}
+
+__global__ void __launch_bounds__(256)
+rect_decode_kernel(const int64_t* __restrict__ lm, const int64_t* __restrict__ pair_off, int B, long long T2,
+                   int32_t* __restrict__ ps, int32_t* __restrict__ pi, int32_t* __restrict__ pj) {
+  if (pair_off[B] != T2) return;
+  const long long p = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (p >= T2) return;
+  const int s = rect_search(pair_off, B, p);
+  const unsigned long long r = (unsigned long long)(p - pair_off[s]), m = (unsigned long long)lm[s];
+  const unsigned long long a = r / m;
+  ps[p] = s;
+  pi[p] = (int32_t)a;
+  pj[p] = (int32_t)(r - a * m);
+}
+
+// ---- broadcast + LayerNorm
+struct RectMeta {
+  int B;
+  int N[MAXB], M[MAXB];
+  long long tokn_off[MAXB + 1], tokm_off[MAXB + 1], pair_off[MAXB + 1];
+};
+
+// Shape-generic form: one warp per packed cell (any c_z, float or bf16).
+template <typename T>
+__global__ void __launch_bounds__(256) rect_broadcast_ln_kernel(const float* __restrict__ u, const float* __restrict__ v,
+                                                               const T* __restrict__ gamma, const T* __restrict__ beta,
+                                                               float eps, int c_z, T* __restrict__ z, RectMeta m) {
+  const int lane = threadIdx.x & 31;
+  const long long p = m.pair_off[0] + (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (p >= m.pair_off[m.B]) return;
+  const int s = find_sample(m.pair_off, m.B, p);
+  const int M = m.M[s];
+  const long long r = p - m.pair_off[s];
+  const long long a = r / M, b = r - a * M;
+  const float* ur = u + (m.tokn_off[s] + a) * c_z;
+  const float* vr = v + (m.tokm_off[s] + b) * c_z;
+  float sum = 0.f;
+  for (int c = lane; c < c_z; c += 32) sum += ur[c] + vr[c];
+#pragma unroll
+  for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  const float mean = sum / (float)c_z;
+  float q = 0.f;
+  for (int c = lane; c < c_z; c += 32) {
+    const float dlt = ur[c] + vr[c] - mean;
+    q += dlt * dlt;
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+  const float rs = rsqrtf(q / (float)c_z + eps);
+  T* zr = z + p * c_z;
+  for (int c = lane; c < c_z; c += 32)
+    Cvt<T>::st(zr + c, (ur[c] + vr[c] - mean) * rs * Cvt<T>::ld(gamma + c) + Cvt<T>::ld(beta + c));
+}
+
+// bf16, c_z = 8 LP: a work item is a run of up to RBJ consecutive cells b of one row (s, a); LP lanes share a cell
+// (16-byte stores), the row term u stays in registers for the run, two cells per lane group and iteration share one
+// round of shuffles.
+constexpr int RBJ = 64;
+
+template <int LP>
+__global__ void __launch_bounds__(256) rect_broadcast_ln_fast_kernel(const float* __restrict__ u, const float* __restrict__ v,
+                                                                     const __nv_bfloat16* __restrict__ gamma,
+                                                                     const __nv_bfloat16* __restrict__ beta, float eps,
+                                                                     __nv_bfloat16* __restrict__ z, RectMeta m, long long n_items) {
+  constexpr int C = LP * 8;
+  constexpr int PPW = 32 / LP;
+  __shared__ long long item_off[MAXB + 1];
+  if (threadIdx.x == 0) {
+    long long acc = 0;
+    for (int s = 0; s < m.B; ++s) {
+      item_off[s] = acc;
+      acc += (long long)m.N[s] * ((m.M[s] + RBJ - 1) / RBJ);
+    }
+    item_off[m.B] = acc;
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, sub = lane / LP, cl = lane % LP;
+  float g[8], b[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    g[e] = __bfloat162float(gamma[cl * 8 + e]);
+    b[e] = __bfloat162float(beta[cl * 8 + e]);
+  }
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long it = wid; it < n_items; it += nw) {
+    const int s = find_sample(item_off, m.B, it);
+    const int M = m.M[s];
+    const int cps = (M + RBJ - 1) / RBJ;
+    const long long r = it - item_off[s];
+    const int a = (int)(r / cps), j0 = (int)(r - (long long)a * cps) * RBJ;
+    const int j1 = min(M, j0 + RBJ);
+    const float4* up = reinterpret_cast<const float4*>(u + (m.tokn_off[s] + a) * C + cl * 8);
+    const float4 u0 = up[0], u1 = up[1];
+    const float ur[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+    __nv_bfloat16* zrow = z + (m.pair_off[s] + (long long)a * M) * C;
+    for (int jb = j0; jb < j1; jb += 2 * PPW) {
+      const int ja = jb + sub, jc = jb + PPW + sub;
+      const bool oka = ja < j1, okc = jc < j1;
+      const float4* vpa = reinterpret_cast<const float4*>(v + (m.tokm_off[s] + (oka ? ja : j1 - 1)) * C + cl * 8);
+      const float4* vpc = reinterpret_cast<const float4*>(v + (m.tokm_off[s] + (okc ? jc : j1 - 1)) * C + cl * 8);
+      const float4 a0 = vpa[0], a1 = vpa[1], c0 = vpc[0], c1 = vpc[1];
+      const float xa[8] = {ur[0] + a0.x, ur[1] + a0.y, ur[2] + a0.z, ur[3] + a0.w, ur[4] + a1.x, ur[5] + a1.y, ur[6] + a1.z, ur[7] + a1.w};
+      const float xc[8] = {ur[0] + c0.x, ur[1] + c0.y, ur[2] + c0.z, ur[3] + c0.w, ur[4] + c1.x, ur[5] + c1.y, ur[6] + c1.z, ur[7] + c1.w};
+      float sa = ((xa[0] + xa[1]) + (xa[2] + xa[3])) + ((xa[4] + xa[5]) + (xa[6] + xa[7]));
+      float sc = ((xc[0] + xc[1]) + (xc[2] + xc[3])) + ((xc[4] + xc[5]) + (xc[6] + xc[7]));
+      float qa = 0.f, qc = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        qa = fmaf(xa[e], xa[e], qa);
+        qc = fmaf(xc[e], xc[e], qc);
+      }
+#pragma unroll
+      for (int o = LP / 2; o; o >>= 1) {
+        sa += __shfl_xor_sync(0xffffffffu, sa, o);
+        sc += __shfl_xor_sync(0xffffffffu, sc, o);
+        qa += __shfl_xor_sync(0xffffffffu, qa, o);
+        qc += __shfl_xor_sync(0xffffffffu, qc, o);
+      }
+      const float ma = sa * (1.0f / C), mc = sc * (1.0f / C);
+      const float ra = rsqrtf(fmaxf(qa * (1.0f / C) - ma * ma, 0.f) + eps), rc = rsqrtf(fmaxf(qc * (1.0f / C) - mc * mc, 0.f) + eps);
+      unsigned pa[4], pc[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float g0 = g[2 * e], g1 = g[2 * e + 1];
+        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf((xa[2 * e] - ma) * ra, g0, b[2 * e]), fmaf((xa[2 * e + 1] - ma) * ra, g1, b[2 * e + 1]));
+        pa[e] = *reinterpret_cast<unsigned*>(&h);
+        h = __floats2bfloat162_rn(fmaf((xc[2 * e] - mc) * rc, g0, b[2 * e]), fmaf((xc[2 * e + 1] - mc) * rc, g1, b[2 * e + 1]));
+        pc[e] = *reinterpret_cast<unsigned*>(&h);
+      }
+      if (oka) *reinterpret_cast<uint4*>(zrow + (long long)ja * C + cl * 8) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
+      if (okc) *reinterpret_cast<uint4*>(zrow + (long long)jc * C + cl * 8) = make_uint4(pc[0], pc[1], pc[2], pc[3]);
+    }
+  }
+}
+
+static bool rect_totals(const int64_t* ln, const int64_t* lm, int B, long long& t1n, long long& t1m, long long& t2) {
+  t1n = t1m = t2 = 0;
+  for (int s = 0; s < B; ++s) {
+    if (ln[s] < 0 || lm[s] < 0 || ln[s] > 0x7FFFFFFFll || lm[s] > 0x7FFFFFFFll) return false;
+    t1n += ln[s];
+    t1m += lm[s];
+    t2 += ln[s] * lm[s];
+  }
+  return true;
+}
+
+template <typename T>
+static nt_status rect_broadcast_impl(nt_dtype dt, int B, const int64_t* ln, const int64_t* lm, int c_s, int c_z, const void* x,
+                                     const void* y, const void* W_a, const void* W_b, const void* g, const void* b, float eps,
+                                     void* z, void* ws, long long t1n, long long t1m, cudaStream_t st) {
+  float* u = (float*)ws;
+  float* v = (float*)((char*)ws + align_up((size_t)t1n * c_z * sizeof(float), 256));
+  const bool fast = dt == NT_BF16 && !g_force_generic && fast_broadcast_supported(c_z);
+  nt_status r;
+  BatchMeta dummy;
+  fill_meta(dummy, nullptr, 0, 0, 0, 0, 0);
+  if (fast && fast_token_gemm_supported(c_s, c_z, 0)) {
+    if ((r = fast_token_gemm(x, t1n, c_s, W_a, c_z, u, nullptr, 0, nullptr, 1, 0, "rect_tok_proj_u", st)) != NT_OK) return r;
+    if ((r = fast_token_gemm(y, t1m, c_s, W_b, c_z, v, nullptr, 0, nullptr, 1, 0, "rect_tok_proj_v", st)) != NT_OK) return r;
+  } else {
+    ProjArgs pa{};
+    pa.a_mode = A_ROWMAJOR; pa.row0 = 0; pa.K = c_s; pa.Nout = c_z; pa.act = ACT_NONE; pa.out_mode = O_STORE; pa.out_f32 = 1;
+    pa.A = x; pa.rows = t1n; pa.W1 = W_a; pa.out = u;
+    if (t1n > 0 && (r = launch_proj<T>(pa, dummy, st, "rect_tok_proj_u")) != NT_OK) return r;
+    pa.A = y; pa.rows = t1m; pa.W1 = W_b; pa.out = v;
+    if (t1m > 0 && (r = launch_proj<T>(pa, dummy, st, "rect_tok_proj_v")) != NT_OK) return r;
+  }
+  long long tn = 0, tm = 0, po = 0;
+  for (int s0 = 0; s0 < B; s0 += MAXB) {
+    RectMeta m;
+    m.B = B - s0 < MAXB ? B - s0 : MAXB;
+    long long items = 0;
+    for (int l = 0; l <= MAXB; ++l) {
+      m.tokn_off[l] = tn; m.tokm_off[l] = tm; m.pair_off[l] = po;
+      if (l < m.B) {
+        m.N[l] = (int)ln[s0 + l];
+        m.M[l] = (int)lm[s0 + l];
+        items += (long long)m.N[l] * ((m.M[l] + RBJ - 1) / RBJ);
+        tn += m.N[l]; tm += m.M[l]; po += (long long)m.N[l] * m.M[l];
+      } else if (l < MAXB) {
+        m.N[l] = m.M[l] = 0;
+      }
+    }
+    const long long cells = m.pair_off[m.B] - m.pair_off[0];
+    if (cells == 0) continue;
+    if (fast) {
+      long long blocks = (items + 7) / 8;
+      if (blocks > 148 * 8) blocks = 148 * 8;
+      LaunchScope ls("rect_broadcast_ln", st);
+      const __nv_bfloat16* gg = (const __nv_bfloat16*)g;
+      const __nv_bfloat16* bb = (const __nv_bfloat16*)b;
+      if (c_z == 64) rect_broadcast_ln_fast_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
+      else if (c_z == 128) rect_broadcast_ln_fast_kernel<16><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
+      else rect_broadcast_ln_fast_kernel<32><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
+    } else {
+      const long long blocks = (cells + 7) / 8;
+      if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+      LaunchScope ls("generic_rect_broadcast_ln", st);
+      rect_broadcast_ln_kernel<T><<<(unsigned)blocks, 256, 0, st>>>(u, v, (const T*)g, (const T*)b, eps, c_z, (T*)z, m);
+    }
+    if (cudaPeekAtLastError() != cudaSuccess) return cuda_fail("rectangular broadcast launch");
+  }
+  return NT_OK;
+}
+
+}  // namespace ntp
+
+using namespace ntp;
+
+extern "C" {
+
+nt_status nt_rect_offsets_build(const int64_t* lengths_n_d, const int64_t* lengths_m_d, int32_t B, int64_t T1n, int64_t T1m,
+                                int64_t T2, int64_t* tokn_off_d, int64_t* tokm_off_d, int64_t* pair_off_d,
+                                int64_t* row_splits_d, int32_t* pos_sample_d, int32_t* pos_i_d, int32_t* pos_j_d,
+                                int32_t* status_d, nt_stream stream_) {
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (B < 0 || T1n < 0 || T1m < 0 || T2 < 0) return NT_ERR_INVALID_ARG;
+  if (!tokn_off_d || !tokm_off_d || !pair_off_d) return NT_ERR_INVALID_ARG;
+  if (B > 0 && (!lengths_n_d || !lengths_m_d)) return NT_ERR_INVALID_ARG;
+  const bool want_pos = pos_sample_d || pos_i_d || pos_j_d;
+  if (want_pos && !(pos_sample_d && pos_i_d && pos_j_d)) return NT_ERR_INVALID_ARG;
+  {
+    LaunchScope ls("rect_offsets_scan", stream);
+    rect_scan_kernel<<<1, RS_THREADS, 0, stream>>>(lengths_n_d, lengths_m_d, B, T1n, T1m, T2, tokn_off_d, tokm_off_d, pair_off_d,
+                                                   status_d);
+  }
+  if (row_splits_d) {
+    const long long n = T1n + 1;
+    LaunchScope ls("rect_offsets_row_splits", stream);
+    rect_row_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(lengths_m_d, tokn_off_d, pair_off_d, B, T1n, T2,
+                                                                           row_splits_d);
+  }
+  if (want_pos && T2 > 0) {
+    const long long blocks = (T2 + 255) / 256;
+    if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+    LaunchScope ls("rect_offsets_decode", stream);
+    rect_decode_kernel<<<(unsigned)blocks, 256, 0, stream>>>(lengths_m_d, pair_off_d, B, T2, pos_sample_d, pos_i_d, pos_j_d);
+  }
+  return cuda_ok();
+}
+
+size_t nt_rect_broadcast_workspace_bytes(const int64_t* lengths_n_h, const int64_t* lengths_m_h, int32_t B, int32_t c_z) {
+  long long t1n, t1m, t2;
+  if (B <= 0 || c_z <= 0 || !lengths_n_h || !lengths_m_h || !rect_totals(lengths_n_h, lengths_m_h, B, t1n, t1m, t2)) return 0;
+  return align_up((size_t)t1n * c_z * sizeof(float), 256) + align_up((size_t)t1m * c_z * sizeof(float), 256);
+}
+
+nt_status nt_rect_pair_broadcast(nt_dtype dt, int32_t B, const int64_t* lengths_n_h, const int64_t* lengths_m_h, int32_t c_s,
+                                 int32_t c_z, const void* x, const void* y, const void* W_a, const void* W_b,
+                                 const void* ln_gamma, const void* ln_beta, float ln_eps, void* z, void* workspace,
+                                 size_t workspace_bytes, nt_stream stream) {
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (B < 0 || c_s <= 0 || c_z <= 0) return NT_ERR_INVALID_ARG;
+  if (B == 0) return NT_OK;
+  long long t1n, t1m, t2;
+  if (!lengths_n_h || !lengths_m_h || !rect_totals(lengths_n_h, lengths_m_h, B, t1n, t1m, t2)) return NT_ERR_INVALID_ARG;
+  if (t2 == 0) return NT_OK;
+  if (!x || !y || !W_a || !W_b || !ln_gamma || !ln_beta || !z || !workspace) return NT_ERR_INVALID_ARG;
+  if (((uintptr_t)x | (uintptr_t)y | (uintptr_t)z | (uintptr_t)workspace | (uintptr_t)W_a | (uintptr_t)W_b) & 15) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < nt_rect_broadcast_workspace_bytes(lengths_n_h, lengths_m_h, B, c_z)) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dt == NT_F32)
+    return rect_broadcast_impl<float>(dt, B, lengths_n_h, lengths_m_h, c_s, c_z, x, y, W_a, W_b, ln_gamma, ln_beta, ln_eps, z,
+                                      workspace, t1n, t1m, st);
+  return rect_broadcast_impl<__nv_bfloat16>(dt, B, lengths_n_h, lengths_m_h, c_s, c_z, x, y, W_a, W_b, ln_gamma, ln_beta, ln_eps,
+                                            z, workspace, t1n, t1m, st);
+}
+
+}  // extern "C"

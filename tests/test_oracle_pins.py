@@ -742,6 +742,18 @@ def test_rect_block_equals_padded_and_masked_computation():
         on, op_ = on + n, op_ + n * m
 
 
+def test_rect_empty_rows_and_columns_contribute_nothing():
+    ln, lm = (0, 2, 3, 1), (4, 0, 2, 5)
+    x, y, w = _rect_case(ln, lm)
+    x2, z = orc.rect_block_forward(x, y, ln, lm, w)
+    assert z.shape[0] == 3 * 2 + 1 * 5
+    # a sample without columns has rows but no cells: its rows' mean is the empty-group zero, the tokens pass through
+    assert np.array_equal(x2[0:2], x[0:2])
+    keep_n, keep_m = (3, 1), (2, 5)
+    xk, zk = orc.rect_block_forward(x[2:], y[4:], keep_n, keep_m, w)
+    assert np.allclose(z, zk, rtol=1e-12, atol=1e-12) and np.allclose(x2[2:], xk, rtol=1e-12, atol=1e-12)
+
+
 RECT_PATTERNS = [   # the kinds of structure change the paper's validation patterns name (App. A.1)
     ((4, 2, 6), (3, 6, 2)), ((2, 4, 6), (6, 3, 2)), ((6, 6), (3, 3)),          # changed partitions, fixed total of 36 cells
     ((5, 1), (2, 7)), ((8, 3, 2), (1, 9, 4)),                                    # changed packed extents and maxima

@@ -1,0 +1,119 @@
+"""GPU parity of the rectangular-pair path (N_s, M_s) against the CPU oracle, through the C ABI: offsets (bit-exact),
+broadcast from distinct row and column tokens, and the whole single-pair-single block (broadcast, position-wise
+transition, column mean divided by M_s, token update)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nested_pair_oracle as orc
+from paper_2609_30379_b200 import workloads as wl
+from tests.parity_utils import check
+
+pytestmark = pytest.mark.gpu
+
+PATTERNS = [   # the kinds of structure change the paper's validation patterns name
+    ((4, 2, 6), (3, 6, 2)), ((2, 4, 6), (6, 3, 2)), ((6, 6), (3, 3)),
+    ((5, 1), (2, 7)), ((8, 3, 2), (1, 9, 4)),
+    ((3, 3, 3), (3, 3, 3)), ((3, 3, 3), (4, 4, 4)), ((1,), (1,)),
+]
+
+
+@pytest.fixture(scope="module")
+def nt():
+    from paper_2609_30379_b200 import binding
+    return binding
+
+
+def host(t):
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("ln,lm", PATTERNS + [((0, 3, 0, 5), (4, 0, 2, 7)), ((), ()), (tuple(range(1, 70)), tuple(range(69, 0, -1)))])
+def test_rect_offsets_bit_exact(nt, ln, lm):
+    L = nt.RectLayout(ln, lm, with_maps=True)
+    ref = orc.rect_offsets(ln, lm)
+    torch.cuda.synchronize()
+    assert L.device_status() == 0
+    for got, key in ((L.tokn_off, "tokn_off"), (L.tokm_off, "tokm_off"), (L.pair_off, "pair_off"), (L.row_splits, "row_splits"),
+                     (L.pos_sample, "pos_sample"), (L.pos_i, "pos_i"), (L.pos_j, "pos_j")):
+        g = got.cpu().numpy()
+        assert g.dtype == ref[key].dtype and np.array_equal(g, ref[key]), key
+
+
+def _inputs(dtype, ln, lm, c_s, c_z, seed):
+    cfg = wl.Config("rect", dtype, tuple(ln), c_s=c_s, c_z=c_z, c_h=c_z, H=2, d=c_z // 2 if c_z <= 32 else 32, blocks=1, seed=seed)
+    inp = wl.make_inputs(cfg)
+    rng = np.random.default_rng(seed + 100)
+    y = rng.standard_normal((int(sum(lm)), c_s)).astype(np.float32)
+    if dtype == "bf16":
+        y = wl.round_to_bf16(y)
+    w = dict(broadcast=inp["blocks"][0]["broadcast"], transition=wl.make_transition_weights(cfg), reduce=inp["blocks"][0]["reduce"])
+    return cfg, inp["x"], y, w
+
+
+def _run_block(nt, dtype, ln, lm, c_s, c_z, seed, force_generic=False):
+    cfg, x, y, w = _inputs(dtype, ln, lm, c_s, c_z, seed)
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to("cuda", tdt)
+    prev = nt.nt_force_generic(force_generic)
+    try:
+        L = nt.RectLayout(ln, lm)
+        x_d, y_d = dev(x), dev(y)
+        b = {k: dev(v) for k, v in w["broadcast"].items()}
+        tw = {k: dev(v) for k, v in w["transition"].items()}
+        W_r = dev(w["reduce"]["W_r"])
+        z = torch.empty((L.T2, c_z), dtype=tdt, device="cuda")
+        ws = torch.empty(max(nt.nt_rect_broadcast_workspace_bytes(L, c_z), 256), dtype=torch.uint8, device="cuda")
+        nt.nt_rect_pair_broadcast(L, x_d, y_d, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, z, ws)
+        z0 = z.clone()
+        hidden = w["transition"]["W_a"].shape[0]
+        tws = torch.empty(max(nt.nt_transition_workspace_bytes(tdt, c_z, hidden, max(L.T2, 1)), 256), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        nt.nt_pair_transition(tw, 1e-5, z, tws, status)
+        z1 = z.clone()
+        mrow = torch.empty((L.T1n, c_z), dtype=tdt, device="cuda")
+        nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, z, mrow, L.status)
+        x_before = x_d.clone()
+        nt.nt_token_update(mrow, W_r, x_d)
+        torch.cuda.synchronize()
+        assert L.device_status() == 0 and int(status.item()) == 0
+    finally:
+        nt.nt_force_generic(prev)
+    # teacher-forced, call by call
+    ref0 = orc.rect_pair_broadcast(x, y, ln, lm, **w["broadcast"])
+    check(dtype, host(z0), ref0, "rect broadcast", already_normalised=True)
+    check(dtype, host(z1), orc.pair_transition(host(z0), w["transition"]), "rect transition")
+    off = orc.rect_offsets(ln, lm)
+    mref = orc.segment_reduce(host(z1), off["row_splits"], "mean")
+    if L.T1n:
+        check(dtype, host(mrow), mref, "rect column mean")
+        check(dtype, host(x_d), orc.token_update(host(x_before), host(mrow), w["reduce"]["W_r"]), "rect token update")
+    assert z.shape[0] == sum(n * m for n, m in zip(ln, lm))
+    return host(x_d), host(z1)
+
+
+@pytest.mark.parametrize("ln,lm", PATTERNS)
+def test_rect_validation_patterns_f32(nt, ln, lm):
+    x2, z = _run_block(nt, "f32", ln, lm, c_s=24, c_z=16, seed=3)
+    # and the whole block against the oracle end to end (fp32: no drift to speak of)
+    cfg, x, y, w = _inputs("f32", ln, lm, 24, 16, 3)
+    rx, rz = orc.rect_block_forward(x, y, ln, lm, w)
+    check("f32", z, rz, "rect block z")
+    check("f32", x2, rx, "rect block x")
+
+
+@pytest.mark.parametrize("generic", [False, True])
+def test_rect_edge_lengths_bf16(nt, generic):
+    # empty rows / columns, single cells, ragged tails around the 64-cell run and 128-row tile edges
+    ln = (0, 1, 7, 63, 64, 65, 3, 130)
+    lm = (5, 1, 64, 65, 0, 2, 200, 129)
+    _run_block(nt, "bf16", ln, lm, c_s=64, c_z=128, seed=4, force_generic=generic)
+
+
+def test_rect_c64_and_rectangular_workload_shape(nt):
+    _run_block(nt, "bf16", (40, 9, 77), (13, 90, 31), c_s=64, c_z=64, seed=5)
+    # the rectangular workload of the paper's table: B = 8, rows 130-221, columns 148-224 (seeded stand-in)
+    rng = np.random.default_rng(6)
+    ln = tuple(int(v) for v in rng.integers(130, 222, 8))
+    lm = tuple(int(v) for v in rng.integers(148, 225, 8))
+    _run_block(nt, "bf16", ln, lm, c_s=384, c_z=128, seed=6)
