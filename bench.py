@@ -419,6 +419,54 @@ def main():
             out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
         return dict(calls=n_calls, us_per_call=round(sum(v[0] for v in tp.values()) / n_calls * 1e3, 2), kernels=out)
 
+    def rect_pass(n_calls):
+        """Single-pair-single block on RECTANGULAR pairs of the paper's rectangular workload shape (B = 8, rows 130-221,
+        columns 148-224, seeded): broadcast from distinct row / column tokens, the transition, the column mean over
+        M_s, the token update.  Not part of the step or of `value`."""
+        if cfg.kind != "pair" or cfg.dtype != "bf16":
+            return None
+        rng = np.random.default_rng(6)
+        ln = tuple(int(v) for v in rng.integers(130, 222, 8))
+        lm = tuple(int(v) for v in rng.integers(148, 225, 8))
+        L = nt.RectLayout(ln, lm)
+        dt = stack.dtype
+        xr = torch.randn((L.T1n, cfg.c_s), device="cuda").to(dt)
+        yr = torch.randn((L.T1m, cfg.c_s), device="cuda").to(dt)
+        b = stack.W[0]["broadcast"]
+        Wt = {k: torch.from_numpy(np.ascontiguousarray(v)).to("cuda", dt) for k, v in wl.make_transition_weights(cfg).items()}
+        W_r = stack.W[0]["reduce"]["W_r"]
+        zr = torch.empty((L.T2, cfg.c_z), dtype=dt, device="cuda")
+        mr = torch.empty((L.T1n, cfg.c_z), dtype=dt, device="cuda")
+        ws = torch.empty(max(nt.nt_rect_broadcast_workspace_bytes(L, cfg.c_z), 256), dtype=torch.uint8, device="cuda")
+        tws = torch.empty(max(nt.nt_transition_workspace_bytes(dt, cfg.c_z, 4 * cfg.c_z, L.T2), 256), dtype=torch.uint8, device="cuda")
+
+        def one():
+            nt.nt_rect_pair_broadcast(L, xr, yr, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], 1e-5, zr, ws)
+            nt.nt_pair_transition(Wt, 1e-5, zr, tws)
+            nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, zr, mr, L.status)
+            nt.nt_token_update(mr, W_r, xr)
+
+        for _ in range(3):
+            one()
+        torch.cuda.synchronize()
+        nt.nt_profile_begin()
+        for _ in range(n_calls):
+            one()
+        torch.cuda.synchronize()
+        tp = nt.nt_profile_end()
+        peaks_t, kind_t = load_peaks()
+        e = 2
+        wk = dict(rect_broadcast_ln=dict(bytes=L.T2 * cfg.c_z * e + (L.T1n + L.T1m) * cfg.c_z * 4, flops=8 * L.T2 * cfg.c_z),
+                  transition=dict(bytes=2 * L.T2 * cfg.c_z * e, flops=6 * L.T2 * cfg.c_z * 4 * cfg.c_z),
+                  segment_reduce=dict(bytes=L.T2 * cfg.c_z * e + L.T1n * cfg.c_z * e, flops=L.T2 * cfg.c_z))
+        out = {}
+        for k, v in tp.items():
+            r = roofline_entry(k, v[0], v[1], n_calls, wk, peaks_t, kind_t)
+            out[k] = r if r else dict(kernel=k, us_per_call=round(v[0] / n_calls * 1e3, 2), launches=v[1])
+        tot_us = sum(v[0] for v in tp.values()) / n_calls * 1e3
+        return dict(workload=f"B=8, rows {min(ln)}..{max(ln)}, columns {min(lm)}..{max(lm)}, T2={L.T2}", calls=n_calls,
+                    us_per_call=round(tot_us, 2), cells_per_s=round(L.T2 / (tot_us * 1e-6), 1), kernels=out)
+
     if args.only_single_attn:
         res = dict(single_attn=single_attn_pass(steps))
         if rank == 0:
@@ -497,7 +545,7 @@ def main():
         roofline["traffic"] = NCU_TRAFFIC_CFG2.get(dominant)
 
     next_rows = (dict(pair_transition=transition_pass(steps), tri_mul_in=tri_mul_in_pass(steps), col_attn=col_attn_pass(steps),
-                      single_attn=single_attn_pass(steps), pair_stream=stream_pass(steps))
+                      single_attn=single_attn_pass(steps), pair_stream=stream_pass(steps), rect_block=rect_pass(steps))
                  if not args.force_generic else None)
 
     # ---- end to end through the public API with host buffers
