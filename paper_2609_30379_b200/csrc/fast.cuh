@@ -45,7 +45,7 @@ nt_status fast_contract(const void* a, size_t buf_stride_bytes, int C, const Bat
                         cudaStream_t st, bool incoming = false);
 
 // ---- tensor-core projections (tcgen05, LayerNorm folded into fp16 weights prepared once per call)
-struct TriPrep { void *w1, *c01_1, *wg, *c01g, *wo, *c01o, *aug1, *augo; int aug1_rows; };
+struct TriPrep { void *w1, *c01_1, *wg, *c01g, *wo, *c01o, *aug1; int aug1_rows; };
 struct AttnPrep { void *w, *c01, *wg, *c01g, *aug; int aug_rows; };
 nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep, TriPrep& out, cudaStream_t st);
 // the bias rows are folded times sqrt(d): the attention core keeps scores in units of q.k

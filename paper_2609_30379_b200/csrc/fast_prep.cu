@@ -116,8 +116,6 @@ nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep
   p += align_up((size_t)c_z * sizeof(float2), 256);
   out.aug1 = p;                         // [2][rows1][8] fp16
   out.aug1_rows = rows1;
-  p += align_up((size_t)2 * rows1 * 16, 256);
-  out.augo = p;                         // [2][c_z][8] fp16
   PrepArgs a{};
   // The input projection computes D^T = W' z^T with 128 weight rows per MMA and pairs the gate rows of an
   // accumulator with the value rows of the next one: c_h = 128 -> [ag, ap, bg, bp]; c_h = 64 -> [ag, bg, ap, bp].
@@ -131,7 +129,7 @@ nt_status fast_tri_prep(const nt_trimul_weights* W, int c_z, int c_h, void* prep
   add_job(a, c_h == 64 ? s64 : s128, r0, 5, c_z, W->ln_in_gamma, W->ln_in_beta, out.w1, out.c01_1, sc, out.aug1, asbf16);
   const void* s1[1] = {W->W_o};
   const int r1[1] = {c_z};
-  add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o, nullptr, out.augo);
+  add_job(a, s1, r1, 1, c_h, W->ln_out_gamma, W->ln_out_beta, out.wo, out.c01o);
   return run_prep(a, st);
 }
 
