@@ -56,6 +56,16 @@ def kernel_work(cfg: wl.Config):
     c_s, c_z, c_h, H, d = cfg.c_s, cfg.c_z, cfg.c_h, cfg.H, cfg.d
     Hd = H * d
     w = {}
+    if cfg.kind == "token":
+        # single-ragged special case: the attention works on the T1 token rows (c_z is the token width); one
+        # exponential per (query, key, head) of every sample = sum N^2 per head
+        R = T1
+        for n in ("q", "k", "v", "g"):
+            w[f"generic_attn_in_{n}"] = dict(bytes=R * (c_z + Hd) * e, flops=2 * R * c_z * Hd)
+        w["generic_attn_core"] = w["attn_core"] = dict(bytes=R * 4 * Hd * e, flops=4 * T2 * Hd, exps=T2 * H)
+        w["generic_attn_out"] = w["attn_out"] = dict(bytes=R * (Hd + 2 * c_z) * e + c_z * Hd * e, flops=2 * R * Hd * c_z)
+        w["segment_reduce"] = w["generic_segment_reduce"] = dict(bytes=R * c_z * e, flops=R * c_z)
+        return w
     tok = dict(bytes=T1 * c_s * e + c_z * c_s * e + T1 * c_z * 4, flops=2 * T1 * c_s * c_z)
     w["tok_proj_u"] = w["tok_proj_v"] = tok
     w["tok_proj"] = dict(bytes=T1 * c_s * e + 2 * c_z * c_s * e + 2 * T1 * c_z * 4, flops=4 * T1 * c_s * c_z)
