@@ -107,3 +107,36 @@ def test_workspace_bytes_scale_with_packed_size_not_envelope(lib):
     T2 = 4 * 64 * 64
     assert a >= T2 * 128 * 2 * 5     # q, k, v, o, g
     assert a < T2 * 128 * 2 * 8
+
+
+def test_host_validation_of_the_calls_after_the_block(lib):
+    """Argument checks of the later entry points return before anything touches the device."""
+    L, keep = _layout(lib, [3, 4])
+    w = lib.nt_trimul_weights()
+    assert lib.lib.nt_tri_mul_in(C.byref(L), lib.NT_BF16, 8, 8, C.byref(w), 1e-5, FAKE, FAKE, 1 << 20, None) == 1   # null weights
+    aw = lib.nt_attn_weights(*([FAKE] * 8))
+    assert lib.lib.nt_col_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 8, None) == 3          # workspace
+    assert lib.lib.nt_col_attn_pairbias(C.byref(L), 7, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None) == 2              # dtype
+    assert lib.lib.nt_col_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 2, 200, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None) == 2  # head dim
+    sw = lib.nt_single_attn_weights()
+    assert lib.lib.nt_single_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 8, 2, 4, C.byref(sw), 1e-5, FAKE, FAKE, FAKE, 1 << 20, None) == 1
+    sw = lib.nt_single_attn_weights(*([FAKE] * 10))
+    assert lib.lib.nt_single_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 8, 2, 4, C.byref(sw), 1e-5, FAKE, FAKE, FAKE, 8, None) == 3
+    assert lib.lib.nt_pair_broadcast_add(C.byref(L), lib.NT_BF16, 8, 8, None, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE, 1 << 20, None) == 1
+    # rectangular pairs: host length vectors are validated and sized on the host
+    ln = (C.c_int64 * 2)(3, 4)
+    lm = (C.c_int64 * 2)(5, 2)
+    need = lib.lib.nt_rect_broadcast_workspace_bytes(ln, lm, 2, 8)
+    assert need == 2 * 256                                   # u [7, 8] and v [7, 8] floats, each rounded up to 256 bytes
+    assert lib.lib.nt_rect_broadcast_workspace_bytes(ln, lm, 0, 8) == 0
+    bad = (C.c_int64 * 2)(3, -1)
+    assert lib.lib.nt_rect_broadcast_workspace_bytes(bad, lm, 2, 8) == 0
+    args = (FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, 1e-5, FAKE, FAKE)
+    assert lib.lib.nt_rect_pair_broadcast(lib.NT_BF16, 2, bad, lm, 8, 8, *args, 1 << 20, None) == 1
+    assert lib.lib.nt_rect_pair_broadcast(lib.NT_BF16, 2, ln, lm, 8, 8, *args, 16, None) == 3
+    assert lib.lib.nt_rect_pair_broadcast(9, 2, ln, lm, 8, 8, *args, 1 << 20, None) == 2
+    assert lib.lib.nt_rect_pair_broadcast(lib.NT_BF16, 0, ln, lm, 8, 8, *args, 0, None) == 0    # empty batch: nothing to do
+    assert lib.lib.nt_rect_offsets_build(FAKE, FAKE, -1, 0, 0, 0, FAKE, FAKE, FAKE, None, None, None, None, None, None) == 1
+    assert lib.lib.nt_rect_offsets_build(FAKE, FAKE, 2, 7, 7, 23, FAKE, FAKE, FAKE, None, FAKE, None, None, None, None) == 1   # decode as a group
+    # transition: the workspace size is a host function
+    assert lib.nt_transition_workspace_bytes is not None
