@@ -260,6 +260,8 @@ def main():
     ap.add_argument("--force-generic", action="store_true", help="time the shape-generic CUDA-core kernels")
     ap.add_argument("--only-transition", action="store_true",
                     help="run just the pair-transition measurement (the row after the block; for ncu captures)")
+    ap.add_argument("--only-rect-block", action="store_true",
+                    help="run just the rectangular-pair block measurement (for ncu captures)")
     ap.add_argument("--only-single-attn", action="store_true",
                     help="run just the pair-biased single attention measurement (for ncu captures)")
     ap.add_argument("--only-col-attn", action="store_true",
@@ -477,6 +479,13 @@ def main():
         return dict(workload=f"B=8, rows {min(ln)}..{max(ln)}, columns {min(lm)}..{max(lm)}, T2={L.T2}", calls=n_calls,
                     us_per_call=round(tot_us, 2), cells_per_s=round(L.T2 / (tot_us * 1e-6), 1), kernels=out)
 
+    if args.only_rect_block:
+        res = dict(rect_block=rect_pass(steps))
+        if rank == 0:
+            print(json.dumps(res))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.only_single_attn:
         res = dict(single_attn=single_attn_pass(steps))
         if rank == 0:
