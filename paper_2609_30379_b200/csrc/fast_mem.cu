@@ -5,71 +5,150 @@
 namespace ntp {
 
 // ------------------------------------------------------------------------------------------
-// z[p,:] = LN(u[tok_off[s]+i] + v[tok_off[s]+j]) * gamma + beta, bf16 out, 16-byte stores.
-// A work item is a run of up to BJ consecutive j of one pair row (s, i); LP = c_z / 8 lanes share a
-// position, so a warp normalises 32 / LP positions per step with shuffle reductions inside the
-// lane group.  The row term u is held in registers for the whole run.
+// z[p,:] = LN(u[tok_off[s]+i] + v[tok_off[s]+j]) * gamma + beta, bf16 out.
+// The state is cut into bands of BI pair rows i; the columns of all bands, laid end to end, are split
+// evenly over a persistent grid, and a block walks its share in chunks of up to BJ columns of one
+// band.  The chunk's column-token rows of v are shared by the BI rows: they are staged in shared
+// memory with asynchronous copies, the next chunk's while the current one is computed.  Each warp
+// takes one i, holds its row term u in registers and walks the chunk.  LP = c_z / 16 lanes share a
+// position: a lane owns four chunks of four channels, LP chunks apart, so every warp-wide
+// shared-memory read and every store of the bf16 state is contiguous.  A warp normalises 2 * 32 / LP
+// positions per step; the statistics cross the lane group by shuffles and the arithmetic around them
+// runs on packed float pairs.  The kernel is bound by instruction issue and latency, not by the
+// 2 c_z bytes it writes per position.
 // ------------------------------------------------------------------------------------------
-constexpr int BJ = 64;
+constexpr int BI = 8;            // pair rows per band = warps per block
+#define BL_TJ(C) ((C) <= 64 ? 64 : (C) <= 128 ? 32 : 16)   // columns per chunk: four steps of a warp, ~17 KB of v rows
 
-template <int LP, bool ACC>      // ACC: z += the broadcast (persistent pair stream) instead of z = the broadcast
+__device__ inline float2 bl_f2(float x, float y) { return make_float2(x, y); }
+__device__ inline unsigned bl_pack(float2 v) {
+  unsigned y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(y) : "f"(v.y), "f"(v.x));
+  return y;
+}
+
+struct BlChunk { int s, i0, j, len; };
+__device__ inline BlChunk bl_chunk(const long long* band_off, const BatchMeta& m, long long cur, long long end,
+                                   int bj) {
+  BlChunk c{0, 0, 0, 0};
+  if (cur >= end) return c;
+  c.s = find_sample(band_off, m.B, cur);
+  const int N = m.N[c.s];
+  const int r = (int)(cur - band_off[c.s]);
+  c.i0 = (r / N) * BI;
+  c.j = r % N;
+  c.len = (int)min((long long)min(bj, N - c.j), end - cur);
+  return c;
+}
+
+template <int C, bool ACC>       // ACC: z += the broadcast (persistent pair stream) instead of z = the broadcast
 __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __restrict__ u,
                                                                 const float* __restrict__ v,
                                                                 const __nv_bfloat16* __restrict__ gamma,
                                                                 const __nv_bfloat16* __restrict__ beta, float eps,
                                                                 __nv_bfloat16* __restrict__ z, BatchMeta m,
-                                                                long long n_items) {
-  constexpr int C = LP * 8;
-  constexpr int PPW = 32 / LP;   // positions per warp step
-  __shared__ long long item_off[MAXB + 1];
+                                                                long long n_cols) {
+  constexpr int LP = C / 16;     // lanes per position
+  constexpr int PPW = 32 / LP;   // positions per warp-wide instruction
+  constexpr int VS = C / 4 + 1;  // float4 per staged v row: one of padding keeps lane groups on distinct banks
+  constexpr int BJ = BL_TJ(C);
+  __shared__ long long band_off[MAXB + 1];     // prefix of bands x columns per sample
+  __shared__ float4 sV[2][BJ * VS];
   if (threadIdx.x == 0) {
     long long acc = 0;
     for (int s = 0; s < m.B; ++s) {
-      item_off[s] = acc;
-      acc += (long long)m.N[s] * ((m.N[s] + BJ - 1) / BJ);
+      band_off[s] = acc;
+      acc += (long long)((m.N[s] + BI - 1) / BI) * m.N[s];
     }
-    item_off[m.B] = acc;
+    band_off[m.B] = acc;
   }
   __syncthreads();
-  const int lane = threadIdx.x & 31, sub = lane / LP, cl = lane % LP;
-  float g[8], b[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane / LP, cl = lane % LP;
+  float2 g2[8], b2[8];           // channels (q LP + cl) 4 .. + 4 for q = 0 .. 3, as pairs
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    g[e] = __bfloat162float(gamma[cl * 8 + e]);
-    b[e] = __bfloat162float(beta[cl * 8 + e]);
+  for (int q = 0; q < 4; ++q) {
+    const uint2 gw = *reinterpret_cast<const uint2*>(gamma + (q * LP + cl) * 4);
+    const uint2 bw = *reinterpret_cast<const uint2*>(beta + (q * LP + cl) * 4);
+    g2[2 * q] = bl_f2(__uint_as_float(gw.x << 16), __uint_as_float(gw.x & 0xffff0000u));
+    g2[2 * q + 1] = bl_f2(__uint_as_float(gw.y << 16), __uint_as_float(gw.y & 0xffff0000u));
+    b2[2 * q] = bl_f2(__uint_as_float(bw.x << 16), __uint_as_float(bw.x & 0xffff0000u));
+    b2[2 * q + 1] = bl_f2(__uint_as_float(bw.y << 16), __uint_as_float(bw.y & 0xffff0000u));
   }
-  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
-  for (long long it = wid; it < n_items; it += nw) {
-    const int s = find_sample(item_off, m.B, it);
-    const int N = m.N[s];
-    const int cps = (N + BJ - 1) / BJ;
-    const long long r = it - item_off[s];
-    const int i = (int)(r / cps), j0 = (int)(r - (long long)i * cps) * BJ;
-    const int j1 = min(N, j0 + BJ);
-    const float4* up = reinterpret_cast<const float4*>(u + (m.tok_off[s] + i) * C + cl * 8);
-    const float4 u0 = up[0], u1 = up[1];
-    const float ur[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
-    __nv_bfloat16* zrow = z + (m.pair_off[s] + (long long)i * N) * C;
-    // two positions per lane group and iteration: their four partial sums share one round of shuffles
-    for (int jb = j0; jb < j1; jb += 2 * PPW) {
-      const int ja = jb + sub, jc = jb + PPW + sub;
-      const bool oka = ja < j1, okc = jc < j1;
-      const float4* vpa = reinterpret_cast<const float4*>(v + (m.tok_off[s] + (oka ? ja : j1 - 1)) * C + cl * 8);
-      const float4* vpc = reinterpret_cast<const float4*>(v + (m.tok_off[s] + (okc ? jc : j1 - 1)) * C + cl * 8);
-      const float4 a0 = vpa[0], a1 = vpa[1], c0 = vpc[0], c1 = vpc[1];
-      const float xa[8] = {ur[0] + a0.x, ur[1] + a0.y, ur[2] + a0.z, ur[3] + a0.w, ur[4] + a1.x, ur[5] + a1.y, ur[6] + a1.z, ur[7] + a1.w};
-      const float xc[8] = {ur[0] + c0.x, ur[1] + c0.y, ur[2] + c0.z, ur[3] + c0.w, ur[4] + c1.x, ur[5] + c1.y, ur[6] + c1.z, ur[7] + c1.w};
-      float sa = ((xa[0] + xa[1]) + (xa[2] + xa[3])) + ((xa[4] + xa[5]) + (xa[6] + xa[7]));
-      float sc = ((xc[0] + xc[1]) + (xc[2] + xc[3])) + ((xc[4] + xc[5]) + (xc[6] + xc[7]));
+  long long cur = n_cols * blockIdx.x / gridDim.x;
+  const long long end = n_cols * (blockIdx.x + 1) / gridDim.x;
+  auto stage = [&](const BlChunk& c, float4* dst) {      // asynchronous copies, 16 bytes each
+    const float4* src = reinterpret_cast<const float4*>(v + (m.tok_off[c.s] + c.j) * C);
+    for (int e = threadIdx.x; e < c.len * (C / 4); e += 256) {
+      const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + (e / (C / 4)) * VS + e % (C / 4));
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa), "l"(src + e));
+    }
+    asm volatile("cp.async.commit_group;\n" ::);
+  };
+  BlChunk ck = bl_chunk(band_off, m, cur, end, BJ);
+  stage(ck, sV[0]);
+  for (int k = 0; ck.len > 0; ++k) {
+    cur += ck.len;
+    const BlChunk nx = bl_chunk(band_off, m, cur, end, BJ);
+    stage(nx, sV[(k + 1) & 1]);                // an empty group when nothing is left
+    const int N = m.N[ck.s];
+    const int i = ck.i0 + warp, nj = ck.len;
+    float2 ur[8];
+    if (i < N) {
+      const float4* up = reinterpret_cast<const float4*>(u + (m.tok_off[ck.s] + i) * C) + cl;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 t = up[q * LP];
+        ur[2 * q] = bl_f2(t.x, t.y);
+        ur[2 * q + 1] = bl_f2(t.z, t.w);
+      }
+    }
+    asm volatile("cp.async.wait_group 1;\n" ::);
+    __syncthreads();
+    if (i < N) {
+    uint2* zp = reinterpret_cast<uint2*>(z + (m.pair_off[ck.s] + (long long)i * N + ck.j) * C) + sub * (C / 4) + cl;
+    const float4* vp = sV[k & 1] + sub * VS + cl;
+    // two positions per lane group and iteration: independent work for the scheduler between the shuffles
+    for (int jb = 0; jb < nj; jb += 2 * PPW, zp += 2 * PPW * (C / 4), vp += 2 * PPW * VS) {
+      const bool oka = jb + sub < nj, okc = jb + PPW + sub < nj;
+      float4 la[4], lc[4];             // rows past the run are stale shared memory: computed, never stored
+#pragma unroll
+      for (int q = 0; q < 4; ++q) la[q] = vp[q * LP];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) lc[q] = vp[PPW * VS + q * LP];
+      uint2 olda[4], oldc[4];
+      if (ACC) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          olda[q] = oka ? zp[q * LP] : make_uint2(0, 0);
+          oldc[q] = okc ? zp[PPW * (C / 4) + q * LP] : make_uint2(0, 0);
+        }
+      }
+      float2 xa[8], xc[8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        xa[2 * q] = __fadd2_rn(ur[2 * q], bl_f2(la[q].x, la[q].y));
+        xa[2 * q + 1] = __fadd2_rn(ur[2 * q + 1], bl_f2(la[q].z, la[q].w));
+        xc[2 * q] = __fadd2_rn(ur[2 * q], bl_f2(lc[q].x, lc[q].y));
+        xc[2 * q + 1] = __fadd2_rn(ur[2 * q + 1], bl_f2(lc[q].z, lc[q].w));
+      }
+      const float2 sa2 = __fadd2_rn(__fadd2_rn(__fadd2_rn(xa[0], xa[1]), __fadd2_rn(xa[2], xa[3])),
+                                    __fadd2_rn(__fadd2_rn(xa[4], xa[5]), __fadd2_rn(xa[6], xa[7])));
+      const float2 sc2 = __fadd2_rn(__fadd2_rn(__fadd2_rn(xc[0], xc[1]), __fadd2_rn(xc[2], xc[3])),
+                                    __fadd2_rn(__fadd2_rn(xc[4], xc[5]), __fadd2_rn(xc[6], xc[7])));
       // centred second moments would need a second round of shuffles; x = u + v is O(1..10) and float carries
       // E[x^2] - mean^2 with a relative error near 1e-6, far below the bf16 output
-      float qa = 0.f, qc = 0.f;
+      float2 qa2 = __fmul2_rn(xa[0], xa[0]), qa3 = __fmul2_rn(xa[1], xa[1]);
+      float2 qc2 = __fmul2_rn(xc[0], xc[0]), qc3 = __fmul2_rn(xc[1], xc[1]);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        qa = fmaf(xa[e], xa[e], qa);
-        qc = fmaf(xc[e], xc[e], qc);
+      for (int e = 2; e < 8; e += 2) {
+        qa2 = __ffma2_rn(xa[e], xa[e], qa2);
+        qa3 = __ffma2_rn(xa[e + 1], xa[e + 1], qa3);
+        qc2 = __ffma2_rn(xc[e], xc[e], qc2);
+        qc3 = __ffma2_rn(xc[e + 1], xc[e + 1], qc3);
       }
+      qa2 = __fadd2_rn(qa2, qa3);
+      qc2 = __fadd2_rn(qc2, qc3);
+      float sa = sa2.x + sa2.y, sc = sc2.x + sc2.y, qa = qa2.x + qa2.y, qc = qc2.x + qc2.y;
 #pragma unroll
       for (int o = LP / 2; o; o >>= 1) {
         sa += __shfl_xor_sync(0xffffffffu, sa, o);
@@ -78,25 +157,29 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
         qc += __shfl_xor_sync(0xffffffffu, qc, o);
       }
       const float ma = sa * (1.0f / C), mc = sc * (1.0f / C);
-      const float ra = rsqrtf(fmaxf(qa * (1.0f / C) - ma * ma, 0.f) + eps), rc = rsqrtf(fmaxf(qc * (1.0f / C) - mc * mc, 0.f) + eps);
-      unsigned pa[4] = {0, 0, 0, 0}, pc[4] = {0, 0, 0, 0};
-      if (ACC) {
-        if (oka) { const uint4 o = *reinterpret_cast<const uint4*>(zrow + (long long)ja * C + cl * 8); pa[0] = o.x; pa[1] = o.y; pa[2] = o.z; pa[3] = o.w; }
-        if (okc) { const uint4 o = *reinterpret_cast<const uint4*>(zrow + (long long)jc * C + cl * 8); pc[0] = o.x; pc[1] = o.y; pc[2] = o.z; pc[3] = o.w; }
-      }
+      const float ra = rsqrtf(fmaxf(fmaf(-ma, ma, qa * (1.0f / C)), 0.f) + eps);
+      const float rc = rsqrtf(fmaxf(fmaf(-mc, mc, qc * (1.0f / C)), 0.f) + eps);
+      const float2 ra2 = bl_f2(ra, ra), rc2 = bl_f2(rc, rc);
+      const float2 na2 = bl_f2(-ma * ra, -ma * ra), nc2 = bl_f2(-mc * rc, -mc * rc);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float g0 = g[2 * e], g1 = g[2 * e + 1];
-        const float oa0 = ACC ? __uint_as_float(pa[e] << 16) : 0.f, oa1 = ACC ? __uint_as_float(pa[e] & 0xffff0000u) : 0.f;
-        const float oc0 = ACC ? __uint_as_float(pc[e] << 16) : 0.f, oc1 = ACC ? __uint_as_float(pc[e] & 0xffff0000u) : 0.f;
-        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf((xa[2 * e] - ma) * ra, g0, b[2 * e]) + oa0, fmaf((xa[2 * e + 1] - ma) * ra, g1, b[2 * e + 1]) + oa1);
-        pa[e] = *reinterpret_cast<unsigned*>(&h);
-        h = __floats2bfloat162_rn(fmaf((xc[2 * e] - mc) * rc, g0, b[2 * e]) + oc0, fmaf((xc[2 * e + 1] - mc) * rc, g1, b[2 * e + 1]) + oc1);
-        pc[e] = *reinterpret_cast<unsigned*>(&h);
+      for (int q = 0; q < 4; ++q) {
+        float2 ya0 = __ffma2_rn(__ffma2_rn(xa[2 * q], ra2, na2), g2[2 * q], b2[2 * q]);
+        float2 ya1 = __ffma2_rn(__ffma2_rn(xa[2 * q + 1], ra2, na2), g2[2 * q + 1], b2[2 * q + 1]);
+        float2 yc0 = __ffma2_rn(__ffma2_rn(xc[2 * q], rc2, nc2), g2[2 * q], b2[2 * q]);
+        float2 yc1 = __ffma2_rn(__ffma2_rn(xc[2 * q + 1], rc2, nc2), g2[2 * q + 1], b2[2 * q + 1]);
+        if (ACC) {
+          ya0 = __fadd2_rn(ya0, bl_f2(__uint_as_float(olda[q].x << 16), __uint_as_float(olda[q].x & 0xffff0000u)));
+          ya1 = __fadd2_rn(ya1, bl_f2(__uint_as_float(olda[q].y << 16), __uint_as_float(olda[q].y & 0xffff0000u)));
+          yc0 = __fadd2_rn(yc0, bl_f2(__uint_as_float(oldc[q].x << 16), __uint_as_float(oldc[q].x & 0xffff0000u)));
+          yc1 = __fadd2_rn(yc1, bl_f2(__uint_as_float(oldc[q].y << 16), __uint_as_float(oldc[q].y & 0xffff0000u)));
+        }
+        if (oka) zp[q * LP] = make_uint2(bl_pack(ya0), bl_pack(ya1));
+        if (okc) zp[PPW * (C / 4) + q * LP] = make_uint2(bl_pack(yc0), bl_pack(yc1));
       }
-      if (oka) *reinterpret_cast<uint4*>(zrow + (long long)ja * C + cl * 8) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-      if (okc) *reinterpret_cast<uint4*>(zrow + (long long)jc * C + cl * 8) = make_uint4(pc[0], pc[1], pc[2], pc[3]);
     }
+    }
+    __syncthreads();                           // the chunk's readers are done before its buffer is refilled
+    ck = nx;
   }
 }
 
@@ -104,11 +187,11 @@ bool fast_broadcast_supported(int c_z) { return c_z == 64 || c_z == 128 || c_z =
 
 nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
                             void* z, const BatchMeta& m, cudaStream_t st, bool accumulate) {
-  long long items = 0;
-  for (int s = 0; s < m.B; ++s) items += (long long)m.N[s] * ((m.N[s] + BJ - 1) / BJ);
+  long long items = 0;      // columns of all bands of BI pair rows, laid end to end
+  for (int s = 0; s < m.B; ++s) items += (long long)((m.N[s] + BI - 1) / BI) * m.N[s];
   if (items == 0) return NT_OK;
-  long long blocks = (items + 7) / 8;
-  const long long cap = 148 * 8;
+  long long blocks = (items + 15) / 16;
+  const long long cap = 148 * 2;
   if (blocks > cap) blocks = cap;
   const __nv_bfloat16* g = (const __nv_bfloat16*)gamma;
   const __nv_bfloat16* b = (const __nv_bfloat16*)beta;
@@ -116,13 +199,13 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
   {
     LaunchScope ls(accumulate ? "broadcast_ln_add" : "broadcast_ln", st);
     if (accumulate) {
-      if (c_z == 64) broadcast_ln_fast_kernel<8, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-      else if (c_z == 128) broadcast_ln_fast_kernel<16, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-      else broadcast_ln_fast_kernel<32, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      if (c_z == 64) broadcast_ln_fast_kernel<64, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else if (c_z == 128) broadcast_ln_fast_kernel<128, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else broadcast_ln_fast_kernel<256, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
     } else {
-      if (c_z == 64) broadcast_ln_fast_kernel<8, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-      else if (c_z == 128) broadcast_ln_fast_kernel<16, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
-      else broadcast_ln_fast_kernel<32, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      if (c_z == 64) broadcast_ln_fast_kernel<64, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else if (c_z == 128) broadcast_ln_fast_kernel<128, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
+      else broadcast_ln_fast_kernel<256, false><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
     }
   }
   return cuda_ok();
