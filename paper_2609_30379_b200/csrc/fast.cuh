@@ -5,6 +5,16 @@
 
 namespace ntp {
 
+// Geometry of a broadcast z[s][i][j] = LN(u[s][i] + v[s][j]): rows x cols cells per sample, token-row offsets of
+// the two operands and cell offset of the result.  Square pairs use the same tokens for both operands.
+struct BcastGeom {
+  int B;
+  int rows[MAXB], cols[MAXB];
+  long long u_off[MAXB], v_off[MAXB], z_off[MAXB];
+};
+nt_status fast_broadcast_ln_geom(const float* u, const float* v, const void* gamma, const void* beta, float eps,
+                                 int c_z, void* z, const BcastGeom& m, cudaStream_t st, bool accumulate,
+                                 const char* scope);
 bool fast_broadcast_supported(int c_z);
 nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
                             void* z, const BatchMeta& m, cudaStream_t st, bool accumulate = false);

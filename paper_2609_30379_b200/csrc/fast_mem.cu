@@ -28,12 +28,12 @@ __device__ inline unsigned bl_pack(float2 v) {
 }
 
 struct BlChunk { int s, i0, j, len; };
-__device__ inline BlChunk bl_chunk(const long long* band_off, const BatchMeta& m, long long cur, long long end,
+__device__ inline BlChunk bl_chunk(const long long* band_off, const BcastGeom& m, long long cur, long long end,
                                    int bj) {
   BlChunk c{0, 0, 0, 0};
   if (cur >= end) return c;
   c.s = find_sample(band_off, m.B, cur);
-  const int N = m.N[c.s];
+  const int N = m.cols[c.s];
   const int r = (int)(cur - band_off[c.s]);
   c.i0 = (r / N) * BI;
   c.j = r % N;
@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
                                                                 const float* __restrict__ v,
                                                                 const __nv_bfloat16* __restrict__ gamma,
                                                                 const __nv_bfloat16* __restrict__ beta, float eps,
-                                                                __nv_bfloat16* __restrict__ z, BatchMeta m,
+                                                                __nv_bfloat16* __restrict__ z, BcastGeom m,
                                                                 long long n_cols) {
   constexpr int LP = C / 16;     // lanes per position
   constexpr int PPW = 32 / LP;   // positions per warp-wide instruction
@@ -58,7 +58,7 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
     long long acc = 0;
     for (int s = 0; s < m.B; ++s) {
       band_off[s] = acc;
-      acc += (long long)((m.N[s] + BI - 1) / BI) * m.N[s];
+      acc += (long long)((m.rows[s] + BI - 1) / BI) * m.cols[s];
     }
     band_off[m.B] = acc;
   }
@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
   long long cur = n_cols * blockIdx.x / gridDim.x;
   const long long end = n_cols * (blockIdx.x + 1) / gridDim.x;
   auto stage = [&](const BlChunk& c, float4* dst) {      // asynchronous copies, 16 bytes each
-    const float4* src = reinterpret_cast<const float4*>(v + (m.tok_off[c.s] + c.j) * C);
+    const float4* src = reinterpret_cast<const float4*>(v + (m.v_off[c.s] + c.j) * C);
     for (int e = threadIdx.x; e < c.len * (C / 4); e += 256) {
       const unsigned sa = (unsigned)__cvta_generic_to_shared(dst + (e / (C / 4)) * VS + e % (C / 4));
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(sa), "l"(src + e));
@@ -90,11 +90,12 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
     cur += ck.len;
     const BlChunk nx = bl_chunk(band_off, m, cur, end, BJ);
     stage(nx, sV[(k + 1) & 1]);                // an empty group when nothing is left
-    const int N = m.N[ck.s];
+    const int N = m.cols[ck.s];
     const int i = ck.i0 + warp, nj = ck.len;
+    const bool live = i < m.rows[ck.s];
     float2 ur[8];
-    if (i < N) {
-      const float4* up = reinterpret_cast<const float4*>(u + (m.tok_off[ck.s] + i) * C) + cl;
+    if (live) {
+      const float4* up = reinterpret_cast<const float4*>(u + (m.u_off[ck.s] + i) * C) + cl;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const float4 t = up[q * LP];
@@ -104,8 +105,8 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
     }
     asm volatile("cp.async.wait_group 1;\n" ::);
     __syncthreads();
-    if (i < N) {
-    uint2* zp = reinterpret_cast<uint2*>(z + (m.pair_off[ck.s] + (long long)i * N + ck.j) * C) + sub * (C / 4) + cl;
+    if (live) {
+    uint2* zp = reinterpret_cast<uint2*>(z + (m.z_off[ck.s] + (long long)i * N + ck.j) * C) + sub * (C / 4) + cl;
     const float4* vp = sV[k & 1] + sub * VS + cl;
     // two positions per lane group and iteration: independent work for the scheduler between the shuffles
     for (int jb = 0; jb < nj; jb += 2 * PPW, zp += 2 * PPW * (C / 4), vp += 2 * PPW * VS) {
@@ -185,10 +186,11 @@ __global__ void __launch_bounds__(256) broadcast_ln_fast_kernel(const float* __r
 
 bool fast_broadcast_supported(int c_z) { return c_z == 64 || c_z == 128 || c_z == 256; }
 
-nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
-                            void* z, const BatchMeta& m, cudaStream_t st, bool accumulate) {
+nt_status fast_broadcast_ln_geom(const float* u, const float* v, const void* gamma, const void* beta, float eps,
+                                 int c_z, void* z, const BcastGeom& m, cudaStream_t st, bool accumulate,
+                                 const char* scope) {
   long long items = 0;      // columns of all bands of BI pair rows, laid end to end
-  for (int s = 0; s < m.B; ++s) items += (long long)((m.N[s] + BI - 1) / BI) * m.N[s];
+  for (int s = 0; s < m.B; ++s) items += (long long)((m.rows[s] + BI - 1) / BI) * m.cols[s];
   if (items == 0) return NT_OK;
   long long blocks = (items + 15) / 16;
   const long long cap = 148 * 2;
@@ -197,7 +199,7 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
   const __nv_bfloat16* b = (const __nv_bfloat16*)beta;
   __nv_bfloat16* zz = (__nv_bfloat16*)z;
   {
-    LaunchScope ls(accumulate ? "broadcast_ln_add" : "broadcast_ln", st);
+    LaunchScope ls(scope, st);
     if (accumulate) {
       if (c_z == 64) broadcast_ln_fast_kernel<64, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
       else if (c_z == 128) broadcast_ln_fast_kernel<128, true><<<(unsigned)blocks, 256, 0, st>>>(u, v, g, b, eps, zz, m, items);
@@ -209,6 +211,19 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
     }
   }
   return cuda_ok();
+}
+
+nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, const void* beta, float eps, int c_z,
+                            void* z, const BatchMeta& m, cudaStream_t st, bool accumulate) {
+  BcastGeom g;
+  g.B = m.B;
+  for (int s = 0; s < MAXB; ++s) {
+    g.rows[s] = g.cols[s] = s < m.B ? m.N[s] : 0;
+    g.u_off[s] = g.v_off[s] = m.tok_off[s];
+    g.z_off[s] = m.pair_off[s];
+  }
+  return fast_broadcast_ln_geom(u, v, gamma, beta, eps, c_z, z, g, st, accumulate,
+                                accumulate ? "broadcast_ln_add" : "broadcast_ln");
 }
 
 // ------------------------------------------------------------------------------------------

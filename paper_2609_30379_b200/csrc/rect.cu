@@ -136,87 +136,8 @@ __global__ void __launch_bounds__(256) rect_broadcast_ln_kernel(const float* __r
     Cvt<T>::st(zr + c, (ur[c] + vr[c] - mean) * rs * Cvt<T>::ld(gamma + c) + Cvt<T>::ld(beta + c));
 }
 
-// bf16, c_z = 8 LP: a work item is a run of up to RBJ consecutive cells b of one row (s, a); LP lanes share a cell
-// (16-byte stores), the row term u stays in registers for the run, two cells per lane group and iteration share one
-// round of shuffles.
-constexpr int RBJ = 64;
-
-template <int LP>
-__global__ void __launch_bounds__(256) rect_broadcast_ln_fast_kernel(const float* __restrict__ u, const float* __restrict__ v,
-                                                                     const __nv_bfloat16* __restrict__ gamma,
-                                                                     const __nv_bfloat16* __restrict__ beta, float eps,
-                                                                     __nv_bfloat16* __restrict__ z, RectMeta m, long long n_items) {
-  constexpr int C = LP * 8;
-  constexpr int PPW = 32 / LP;
-  __shared__ long long item_off[MAXB + 1];
-  if (threadIdx.x == 0) {
-    long long acc = 0;
-    for (int s = 0; s < m.B; ++s) {
-      item_off[s] = acc;
-      acc += (long long)m.N[s] * ((m.M[s] + RBJ - 1) / RBJ);
-    }
-    item_off[m.B] = acc;
-  }
-  __syncthreads();
-  const int lane = threadIdx.x & 31, sub = lane / LP, cl = lane % LP;
-  float g[8], b[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    g[e] = __bfloat162float(gamma[cl * 8 + e]);
-    b[e] = __bfloat162float(beta[cl * 8 + e]);
-  }
-  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long nw = (long long)gridDim.x * (blockDim.x >> 5);
-  for (long long it = wid; it < n_items; it += nw) {
-    const int s = find_sample(item_off, m.B, it);
-    const int M = m.M[s];
-    const int cps = (M + RBJ - 1) / RBJ;
-    const long long r = it - item_off[s];
-    const int a = (int)(r / cps), j0 = (int)(r - (long long)a * cps) * RBJ;
-    const int j1 = min(M, j0 + RBJ);
-    const float4* up = reinterpret_cast<const float4*>(u + (m.tokn_off[s] + a) * C + cl * 8);
-    const float4 u0 = up[0], u1 = up[1];
-    const float ur[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
-    __nv_bfloat16* zrow = z + (m.pair_off[s] + (long long)a * M) * C;
-    for (int jb = j0; jb < j1; jb += 2 * PPW) {
-      const int ja = jb + sub, jc = jb + PPW + sub;
-      const bool oka = ja < j1, okc = jc < j1;
-      const float4* vpa = reinterpret_cast<const float4*>(v + (m.tokm_off[s] + (oka ? ja : j1 - 1)) * C + cl * 8);
-      const float4* vpc = reinterpret_cast<const float4*>(v + (m.tokm_off[s] + (okc ? jc : j1 - 1)) * C + cl * 8);
-      const float4 a0 = vpa[0], a1 = vpa[1], c0 = vpc[0], c1 = vpc[1];
-      const float xa[8] = {ur[0] + a0.x, ur[1] + a0.y, ur[2] + a0.z, ur[3] + a0.w, ur[4] + a1.x, ur[5] + a1.y, ur[6] + a1.z, ur[7] + a1.w};
-      const float xc[8] = {ur[0] + c0.x, ur[1] + c0.y, ur[2] + c0.z, ur[3] + c0.w, ur[4] + c1.x, ur[5] + c1.y, ur[6] + c1.z, ur[7] + c1.w};
-      float sa = ((xa[0] + xa[1]) + (xa[2] + xa[3])) + ((xa[4] + xa[5]) + (xa[6] + xa[7]));
-      float sc = ((xc[0] + xc[1]) + (xc[2] + xc[3])) + ((xc[4] + xc[5]) + (xc[6] + xc[7]));
-      float qa = 0.f, qc = 0.f;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        qa = fmaf(xa[e], xa[e], qa);
-        qc = fmaf(xc[e], xc[e], qc);
-      }
-#pragma unroll
-      for (int o = LP / 2; o; o >>= 1) {
-        sa += __shfl_xor_sync(0xffffffffu, sa, o);
-        sc += __shfl_xor_sync(0xffffffffu, sc, o);
-        qa += __shfl_xor_sync(0xffffffffu, qa, o);
-        qc += __shfl_xor_sync(0xffffffffu, qc, o);
-      }
-      const float ma = sa * (1.0f / C), mc = sc * (1.0f / C);
-      const float ra = rsqrtf(fmaxf(qa * (1.0f / C) - ma * ma, 0.f) + eps), rc = rsqrtf(fmaxf(qc * (1.0f / C) - mc * mc, 0.f) + eps);
-      unsigned pa[4], pc[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float g0 = g[2 * e], g1 = g[2 * e + 1];
-        __nv_bfloat162 h = __floats2bfloat162_rn(fmaf((xa[2 * e] - ma) * ra, g0, b[2 * e]), fmaf((xa[2 * e + 1] - ma) * ra, g1, b[2 * e + 1]));
-        pa[e] = *reinterpret_cast<unsigned*>(&h);
-        h = __floats2bfloat162_rn(fmaf((xc[2 * e] - mc) * rc, g0, b[2 * e]), fmaf((xc[2 * e + 1] - mc) * rc, g1, b[2 * e + 1]));
-        pc[e] = *reinterpret_cast<unsigned*>(&h);
-      }
-      if (oka) *reinterpret_cast<uint4*>(zrow + (long long)ja * C + cl * 8) = make_uint4(pa[0], pa[1], pa[2], pa[3]);
-      if (okc) *reinterpret_cast<uint4*>(zrow + (long long)jc * C + cl * 8) = make_uint4(pc[0], pc[1], pc[2], pc[3]);
-    }
-  }
-}
+// bf16 with c_z = 64, 128 or 256 goes through the band kernel of the square broadcast with rows x cols = N x M and
+// distinct row / column token offsets.
 
 static bool rect_totals(const int64_t* ln, const int64_t* lm, int B, long long& t1n, long long& t1m, long long& t2) {
   t1n = t1m = t2 = 0;
@@ -254,13 +175,11 @@ static nt_status rect_broadcast_impl(nt_dtype dt, int B, const int64_t* ln, cons
   for (int s0 = 0; s0 < B; s0 += MAXB) {
     RectMeta m;
     m.B = B - s0 < MAXB ? B - s0 : MAXB;
-    long long items = 0;
     for (int l = 0; l <= MAXB; ++l) {
       m.tokn_off[l] = tn; m.tokm_off[l] = tm; m.pair_off[l] = po;
       if (l < m.B) {
         m.N[l] = (int)ln[s0 + l];
         m.M[l] = (int)lm[s0 + l];
-        items += (long long)m.N[l] * ((m.M[l] + RBJ - 1) / RBJ);
         tn += m.N[l]; tm += m.M[l]; po += (long long)m.N[l] * m.M[l];
       } else if (l < MAXB) {
         m.N[l] = m.M[l] = 0;
@@ -269,14 +188,14 @@ static nt_status rect_broadcast_impl(nt_dtype dt, int B, const int64_t* ln, cons
     const long long cells = m.pair_off[m.B] - m.pair_off[0];
     if (cells == 0) continue;
     if (fast) {
-      long long blocks = (items + 7) / 8;
-      if (blocks > 148 * 8) blocks = 148 * 8;
-      LaunchScope ls("rect_broadcast_ln", st);
-      const __nv_bfloat16* gg = (const __nv_bfloat16*)g;
-      const __nv_bfloat16* bb = (const __nv_bfloat16*)b;
-      if (c_z == 64) rect_broadcast_ln_fast_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
-      else if (c_z == 128) rect_broadcast_ln_fast_kernel<16><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
-      else rect_broadcast_ln_fast_kernel<32><<<(unsigned)blocks, 256, 0, st>>>(u, v, gg, bb, eps, (__nv_bfloat16*)z, m, items);
+      BcastGeom geo;
+      geo.B = m.B;
+      for (int l = 0; l < MAXB; ++l) {
+        geo.rows[l] = m.N[l]; geo.cols[l] = m.M[l];
+        geo.u_off[l] = m.tokn_off[l]; geo.v_off[l] = m.tokm_off[l]; geo.z_off[l] = m.pair_off[l];
+      }
+      const nt_status r = fast_broadcast_ln_geom(u, v, g, b, eps, c_z, z, geo, st, false, "rect_broadcast_ln");
+      if (r != NT_OK) return r;
     } else {
       const long long blocks = (cells + 7) / 8;
       if (blocks > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
