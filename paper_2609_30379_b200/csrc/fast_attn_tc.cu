@@ -69,6 +69,11 @@ __device__ inline float tca_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ inline float tca_max3(float a, float b, float c) {      // one instruction on sm_100
+  float y;
+  asm("max.f32 %0, %1, %2, %3;\n" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
 __device__ inline unsigned tca_pack(float lo, float hi) {
   unsigned y;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;\n" : "=r"(y) : "f"(hi), "f"(lo));
@@ -329,7 +334,7 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
             tmem_ld_wait2(rc, rd);
 #pragma unroll
             for (int e = 0; e < 16; ++e)
-              m4[e & 3] = fmaxf(m4[e & 3], fmaxf(fmaxf(__uint_as_float(ra[e]), __uint_as_float(rb[e])), fmaxf(__uint_as_float(rc[e]), __uint_as_float(rd[e]))));
+              m4[e & 3] = tca_max3(tca_max3(m4[e & 3], __uint_as_float(ra[e]), __uint_as_float(rb[e])), __uint_as_float(rc[e]), __uint_as_float(rd[e]));
           }
 #pragma unroll 1
           for (; g + 2 <= ge; g += 2) {
@@ -337,7 +342,7 @@ __global__ void __launch_bounds__(TCA_THREADS, 1) attn_tc_kernel(const __grid_co
             tmem_ld16(t_row + g * 16 + 16, rb);
             tmem_ld_wait2(ra, rb);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) m4[e & 3] = fmaxf(m4[e & 3], fmaxf(__uint_as_float(ra[e]), __uint_as_float(rb[e])));
+            for (int e = 0; e < 16; ++e) m4[e & 3] = tca_max3(m4[e & 3], __uint_as_float(ra[e]), __uint_as_float(rb[e]));
           }
           if (g < ge) {
             tmem_ld16(t_row + g * 16, ra);

@@ -33,7 +33,41 @@ __global__ void __launch_bounds__(256) ln_fold_prep_kernel(PrepArgs a) {
   while (r >= J.rows[src]) { r -= J.rows[src]; ++src; }
   const __nv_bfloat16* w = J.src[src] ? J.src[src] + (long long)r * J.K : nullptr;
   float c0 = 0.f, c1 = 0.f;
-  for (int k = lane; k < J.K; k += 32) {
+  // eight elements per lane with 16-byte accesses: the weight, gamma and beta loads of a row are all in flight at
+  // once (the kernel is pure latency: a few hundred rows of K <= 1024 elements)
+  const bool vec = J.K % 8 == 0 && (reinterpret_cast<size_t>(w) & 15) == 0 && (reinterpret_cast<size_t>(J.gamma) & 15) == 0 &&
+                   (reinterpret_cast<size_t>(J.beta) & 15) == 0 && (reinterpret_cast<size_t>(J.out) & 15) == 0;
+  for (int k8 = lane; vec && k8 < J.K / 8; k8 += 32) {
+    const uint4 z4 = make_uint4(0, 0, 0, 0);
+    const uint4 wv = w ? *reinterpret_cast<const uint4*>(w + k8 * 8) : z4;
+    const uint4 gv = J.gamma ? *reinterpret_cast<const uint4*>(J.gamma + k8 * 8) : z4;
+    const uint4 bv = J.gamma ? *reinterpret_cast<const uint4*>(J.beta + k8 * 8) : z4;
+    const unsigned ww[4] = {wv.x, wv.y, wv.z, wv.w}, gw[4] = {gv.x, gv.y, gv.z, gv.w}, bw[4] = {bv.x, bv.y, bv.z, bv.w};
+    unsigned ow[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float f[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const float wvf = __uint_as_float(h ? ww[e] & 0xffff0000u : ww[e] << 16) * J.scale[src];
+        const float gf = __uint_as_float(h ? gw[e] & 0xffff0000u : gw[e] << 16);
+        const float bf = __uint_as_float(h ? bw[e] & 0xffff0000u : bw[e] << 16);
+        f[h] = J.gamma ? wvf * gf : wvf;
+        if (J.gamma) c0 = fmaf(wvf, bf, c0);
+      }
+      if (J.bf16out[src]) {
+        const __nv_bfloat162 ob = __floats2bfloat162_rn(f[0], f[1]);
+        if (J.gamma) c1 += __bfloat162float(ob.x) + __bfloat162float(ob.y);
+        ow[e] = *reinterpret_cast<const unsigned*>(&ob);
+      } else {
+        const __half2 o = __floats2half2_rn(f[0], f[1]);
+        if (J.gamma) c1 += __half2float(o.x) + __half2float(o.y);
+        ow[e] = *reinterpret_cast<const unsigned*>(&o);
+      }
+    }
+    *reinterpret_cast<uint4*>(J.out + (long long)n * J.K + k8 * 8) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+  }
+  for (int k = lane; !vec && k < J.K; k += 32) {
     const float wv = w ? __bfloat162float(w[k]) * J.scale[src] : 0.f;
     const float folded = J.gamma ? wv * __bfloat162float(J.gamma[k]) : wv;
     if (J.gamma) c0 = fmaf(wv, __bfloat162float(J.beta[k]), c0);
