@@ -90,6 +90,8 @@ def kernel_work(cfg: wl.Config):
     w["generic_attn_out"] = w["attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
+    # fused mean behind the attention output stage: two float partial sums per 32 positions and channel, read once
+    w["segment_partials"] = dict(bytes=(T2 // 32 + 1) * 2 * c_z * 4 + T1 * c_z * e, flops=(T2 // 32 + 1) * 2 * c_z)
     w["token_update"] = dict(bytes=T1 * (c_z + 2 * c_s) * e + c_s * c_z * e, flops=2 * T1 * c_s * c_z)
     # pair-biased single attention: the bias planes are the only part that touches the pair state (read z, write H values)
     w["single_attn_bias"] = dict(bytes=T2 * (c_z + H) * e, flops=2 * T2 * c_z * H)
@@ -102,7 +104,7 @@ def kernel_work(cfg: wl.Config):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (cfg2 only);
 # other workloads report traffic = None.
-NCU_TRAFFIC_CFG2 = {"attn_core": 375.2e6, "tri_out": 242.2e6, "attn_in": 324.4e6, "tri_in": 232.0e6, "attn_out": 240.4e6,
+NCU_TRAFFIC_CFG2 = {"attn_core": 375.2e6, "tri_out": 242.2e6, "attn_in": 324.4e6, "tri_in": 232.0e6, "attn_out": 250.0e6,
                     "tri_contract": 255.4e6, "transition": 130.3e6, "tri_contract_in": 255.5e6, "attn_core_col": 375.1e6,
                     "single_attn_bias": 97.8e6}
 
@@ -268,6 +270,8 @@ def main():
                     help="run just the column-wise attention measurement (for ncu captures)")
     ap.add_argument("--only-tri-mul-in", action="store_true",
                     help="run just the incoming-triangle-update measurement (for ncu captures)")
+    ap.add_argument("--separate-reduce", action="store_true",
+                    help="nt_row_attn_pairbias + nt_segment_reduce instead of the fused nt_row_attn_pairbias_mean")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the per-kernel timing pass, the end-to-end pass and the CPU baseline (for ncu captures)")
     args = ap.parse_args()
@@ -299,7 +303,7 @@ def main():
         nt.nt_force_generic(True)
     cfg = wl.CONFIGS[args.config]
     inp = wl.make_inputs(cfg)
-    stack = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+    stack = runner.PairStack(cfg, cfg.lengths, inp["blocks"], fused_mean=not args.separate_reduce)
     x0 = runner.to_device(inp["x"], stack.dtype)
     x = torch.empty_like(x0)
     warmup = max(args.warmup, 3)

@@ -173,6 +173,21 @@ nt_status nt_row_attn_pairbias(const nt_layout *L, nt_order order, nt_dtype dt,
                                void *workspace, size_t workspace_bytes, nt_stream stream);
 
 /*
+ * nt_row_attn_pairbias_mean -- nt_row_attn_pairbias in pair order followed by the mean over j of the updated state
+ * (Eq. 1 line 3, Eq. 4), in one call: where the tensor-core output stage runs, the column sums are taken from its
+ * tiles while they are still on chip and the state is not read back for the reduction.
+ *   z [T2, c] in/out as nt_row_attn_pairbias; m_out [T1, c] out (dtype dt): m_out[tok_off[s]+i,:] = mean_j z[(s,i,j),:]
+ *   of the UPDATED state, accumulated in float, i.e. what nt_segment_reduce(NT_REDUCE_MEAN, row_splits) returns on it
+ *   (the order of the float additions differs, so the two may differ by rounding).
+ *   L->row_splits_d must be present (used when a part of the batch takes a path without the fused reduction:
+ *   float data, a sample shorter than 32, shapes outside the tensor-core stage).
+ *   Workspace and errors as nt_row_attn_pairbias.
+ */
+nt_status nt_row_attn_pairbias_mean(const nt_layout *L, nt_dtype dt, int32_t c, int32_t H, int32_t d,
+                                    const nt_attn_weights *W, float ln_eps, void *z, void *m_out,
+                                    void *workspace, size_t workspace_bytes, nt_stream stream);
+
+/*
  * nt_col_attn_pairbias -- column-wise pair-biased softmax attention over ragged N_s: the second triangle
  * attention of the block (Sec. 4.3, "ending node"), the mirror image of nt_row_attn_pairbias in pair order.
  *   Attention rows are the pair COLUMNS (s, j); for each column and head h:

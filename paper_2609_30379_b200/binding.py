@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "NT_OK", 1: "NT_ERR_INVALID_ARG", 2: "NT_ERR_UNSUPPORTED", 3:
                 4: "NT_ERR_CUDA", 5: "NT_ERR_TIMEOUT", 6: "NT_ERR_INCONSISTENT"}
 
 EXPORTS = ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_add", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-           "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
+           "nt_row_attn_pairbias", "nt_row_attn_pairbias_mean", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
            "nt_single_attn_workspace_bytes", "nt_rect_offsets_build", "nt_rect_pair_broadcast",
            "nt_rect_broadcast_workspace_bytes", "nt_segment_reduce", "nt_pair_transition", "nt_transition_workspace_bytes", "nt_token_update",
            "nt_workspace_bytes", "nt_status_string",
@@ -87,6 +87,7 @@ def _load() -> C.CDLL:
     lib.nt_rect_broadcast_workspace_bytes.argtypes = [vp, vp, i32, i32]
     lib.nt_rect_broadcast_workspace_bytes.restype = sz
     lib.nt_col_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, C.POINTER(nt_attn_weights), f32, vp, vp, sz, vp]
+    lib.nt_row_attn_pairbias_mean.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, C.POINTER(nt_attn_weights), f32, vp, vp, vp, sz, vp]
     lib.nt_row_attn_pairbias.argtypes = [C.POINTER(nt_layout), i32, i32, i32, i32, i32, C.POINTER(nt_attn_weights),
                                          f32, vp, vp, sz, vp]
     lib.nt_segment_reduce.argtypes = [i32, i32, i32, i64, i64, vp, vp, vp, vp, vp]
@@ -108,8 +109,8 @@ def _load() -> C.CDLL:
     lib.nt_profile_end.argtypes = [vp, sz, vp, vp, i32]
     lib.nt_profile_end.restype = i32
     for name in ("nt_offsets_build", "nt_pair_broadcast", "nt_pair_broadcast_add", "nt_pair_broadcast_static", "nt_tri_mul_out", "nt_tri_mul_in",
-                 "nt_row_attn_pairbias", "nt_col_attn_pairbias", "nt_single_attn_pairbias", "nt_segment_reduce",
-                 "nt_token_update"):
+                 "nt_row_attn_pairbias", "nt_row_attn_pairbias_mean", "nt_col_attn_pairbias", "nt_single_attn_pairbias",
+                 "nt_segment_reduce", "nt_token_update"):
         getattr(lib, name).restype = i32
     return lib
 
@@ -306,6 +307,17 @@ def nt_rect_pair_broadcast(L: RectLayout, x, y, W_a, W_b, ln_gamma, ln_beta, ln_
                                     _ptr(ln_gamma), _ptr(ln_beta), float(ln_eps), _ptr(z), _ptr(workspace),
                                     workspace.numel() * workspace.element_size(), _stream(stream))
     _check(st, "nt_rect_pair_broadcast")
+
+
+def nt_row_attn_pairbias_mean(L: Layout, W: dict, H: int, d: int, ln_eps, z, m_out, workspace, stream=None):
+    """Row-wise pair-biased attention in pair order followed by the mean over j of the updated state into
+    m_out [T1, c], in one call (the column sums come from the output stage's tiles where that stage runs)."""
+    c = int(W["W_q"].shape[1])
+    w = nt_attn_weights(*[_ptr(W.get(n)) for n, _ in nt_attn_weights._fields_])
+    st = lib.nt_row_attn_pairbias_mean(C.byref(L.c), dtype_code(z.dtype), c, H, d, C.byref(w), float(ln_eps),
+                                       _ptr(z), _ptr(m_out), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream))
+    _check(st, "nt_row_attn_pairbias_mean")
 
 
 def nt_col_attn_pairbias(L: Layout, W: dict, H: int, d: int, ln_eps, z, workspace, stream=None):

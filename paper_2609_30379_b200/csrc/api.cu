@@ -262,8 +262,9 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
 template <typename T>
 static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order order, int c, int H, int d,
                               const nt_attn_weights* W, float eps, void* zx, void* ws, nt_dtype dt,
-                              cudaStream_t st, bool col) {
+                              cudaStream_t st, bool col, void* mean_out = nullptr, bool* mean_done = nullptr) {
   AttnWs w = carve_attn(ws, dt, tot, order, H, d);
+  if (mean_done) *mean_done = mean_out != nullptr;
   const int Hd = H * d;
   const bool pair = order == NT_ORDER_PAIR_IJC;
   const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma && tot.nmax < 60000;
@@ -327,10 +328,22 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
                               (T*)w.o, H, d, pair ? 1 : 0, m, st);
     if (r != NT_OK) return r;
     if (tc_out) {
-      r = fast_attn_out(zx, w.o, W->W_o, aprep, eps, c, H, d, m, L->status_d, st);
+      // the mean over j of the updated state, taken while its tiles are still on chip; q is dead by now and lends
+      // its memory to the partial sums
+      float* partial = nullptr;
+      if (mean_out && fast_attn_out_reduce_supported(m) &&
+          fast_attn_out_partial_bytes(rows, c) <= (size_t)tot.T2 * Hd * sizeof(T))
+        partial = (float*)w.q;
+      r = fast_attn_out(zx, w.o, W->W_o, aprep, eps, c, H, d, m, L->status_d, st, partial);
       if (r != NT_OK) return r;
+      if (partial) {
+        if ((r = fast_segment_partials(partial, m, c, 1, mean_out, st)) != NT_OK) return r;
+      } else if (mean_done) {
+        *mean_done = false;
+      }
       continue;
     }
+    if (mean_done) *mean_done = false;
     ProjArgs po{};
     po.A = w.o; po.a_mode = A_ROWMAJOR; po.row0 = row0; po.rows = rows; po.K = Hd;
     po.gateA = W->W_g ? w.g : nullptr;
@@ -497,6 +510,32 @@ nt_status nt_row_attn_pairbias(const nt_layout* L, nt_order order, nt_dtype dt, 
   cudaStream_t st = (cudaStream_t)stream;
   if (dt == NT_F32) return attn_generic<float>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st, false);
   return attn_generic<__nv_bfloat16>(L, tot, order, c, H, d, W, ln_eps, zx, workspace, dt, st, false);
+}
+
+nt_status nt_row_attn_pairbias_mean(const nt_layout* L, nt_dtype dt, int32_t c, int32_t H, int32_t d,
+                                    const nt_attn_weights* W, float ln_eps, void* z, void* m_out, void* workspace,
+                                    size_t workspace_bytes, nt_stream stream) {
+  Totals tot;
+  nt_status r = check_layout(L, tot);
+  if (r != NT_OK) return r;
+  if (dt != NT_F32 && dt != NT_BF16) return NT_ERR_UNSUPPORTED;
+  if (c <= 0 || H <= 0 || d <= 0 || !W) return NT_ERR_INVALID_ARG;
+  if (!W->W_q || !W->W_k || !W->W_v || !W->W_o) return NT_ERR_INVALID_ARG;
+  if ((W->ln_gamma == nullptr) != (W->ln_beta == nullptr)) return NT_ERR_INVALID_ARG;
+  if (d > 128) return NT_ERR_UNSUPPORTED;
+  if (tot.T1 == 0) return NT_OK;
+  if (!m_out || !aligned16(m_out) || !L->row_splits_d) return NT_ERR_INVALID_ARG;
+  if (!z || !workspace || !aligned16(z) || !aligned16(workspace)) return NT_ERR_INVALID_ARG;
+  if (workspace_bytes < carve_attn(nullptr, dt, tot, NT_ORDER_PAIR_IJC, H, d).bytes) return NT_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  bool done = false;
+  if (dt == NT_F32)
+    r = attn_generic<float>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, false, m_out, &done);
+  else
+    r = attn_generic<__nv_bfloat16>(L, tot, NT_ORDER_PAIR_IJC, c, H, d, W, ln_eps, z, workspace, dt, st, false, m_out, &done);
+  if (r != NT_OK || done) return r;
+  // some part of the batch went through a path without the fused reduction: reduce the finished state as a whole
+  return nt_segment_reduce(dt, NT_REDUCE_MEAN, c, tot.T1, tot.T2, L->row_splits_d, z, m_out, L->status_d, stream);
 }
 
 nt_status nt_col_attn_pairbias(const nt_layout* L, nt_dtype dt, int32_t c, int32_t H, int32_t d,

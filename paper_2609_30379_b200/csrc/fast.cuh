@@ -78,8 +78,13 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
 
 // in place on z: z += (sigmoid(LN(z) W_g^T) * o) W_o^T
 bool fast_attn_out_supported(int c, int H, int d);
+// Fused mean over j behind the attention output stage: column sums of 32-position groups land in `partial`
+// (fast_attn_out_partial_bytes), fast_segment_partials adds them per pair row into out [T1, C] (bf16).
+bool fast_attn_out_reduce_supported(const BatchMeta& m);
+size_t fast_attn_out_partial_bytes(long long rows, int c);
+nt_status fast_segment_partials(const float* partial, const BatchMeta& m, int C, int mean, void* out, cudaStream_t st);
 nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
-                        const BatchMeta& m, int* status, cudaStream_t st);
+                        const BatchMeta& m, int* status, cudaStream_t st, float* partial = nullptr);
 
 // SwiGLU transition, fused on tcgen05: z += (silu(LN(z) W_a^T) * (LN(z) W_b^T)) W_2^T with the hidden activation
 // kept on chip.  prep: at least 1 MiB of device scratch for the folded weights.

@@ -6,6 +6,12 @@
 // tile; the MMA warp computes the gate pre-activation into TMEM as soon as they land; the epilogue warps turn it
 // into sigmoid(.) * o, written back over the o tile in shared memory; the MMA warp multiplies that by
 // W_o; the epilogue adds the residual into the z tile and TMA-stores it.
+//
+// Optional fused reduction (the mean over j that follows the attention in the block): while the finished tile is
+// still in shared memory the epilogue threads add up its columns per group of 32 positions, split at the one pair
+// row boundary such a group can contain (every sample of the batch has N >= 32 or is empty), and write the two
+// partial sums to a scratch array; a second small kernel adds the partials of every pair row in a fixed order.  The
+// state is then never read back for the reduction.
 #include <cstring>
 
 #include "fast.cuh"
@@ -25,6 +31,9 @@ struct AttnOutParams {
   float eps;
   const float2* c01g;            // [Hd]
   int* status;
+  float* partial;                // nullable: [ceil(rows / 32)][2][c] column sums of 32-position groups
+  long long P0;                  // packed position of row 0 of the maps
+  BatchMeta m;                   // read only when partial != nullptr
 };
 
 __device__ inline float sigmoid_fast3(float x) {
@@ -63,7 +72,7 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
     abort_flag = 0;
     for (int s = 0; s < 2; ++s) {
       mbar_init(&afull[s], 1);
-      mbar_init(&aempty[s], 2);
+      mbar_init(&aempty[s], p.partial ? 2 + 8 : 2);   // + the epilogue warps that read the tile for the column sums
       mbar_init(&gfull[s], 1);
       mbar_init(&ogated[s], 8);
       mbar_init(&ofull[s], 1);
@@ -244,6 +253,54 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       if (ep_tid == 0) {
         for (int sl = 0; sl < zslab; ++sl) tma_store_2d(&p.zmap, st + sl * slab, sl * 64, (int)(t * 128));
         tma_store_commit();
+      }
+      if (p.partial) {
+        // thread = (channel pair, quarter of the tile): column sums of 32 positions, split at the pair row boundary
+        const int cp = ep_tid & 63, q = ep_tid >> 6;
+        const long long p0 = t * 128 + q * 32;
+        if (cp < c / 2 && p0 < p.rows) {
+          const int nvalid = (int)min(32ll, p.rows - p0);
+          const int s = find_sample(p.m.pair_off, p.m.B, p.P0 + p0);
+          const unsigned N = (unsigned)p.m.N[s];
+          const unsigned rem = (unsigned)(p.P0 + p0 - p.m.pair_off[s]) % N;        // N^2 < 2^32 on this path
+          const int br = rem == 0 ? nvalid : (int)min((unsigned)nvalid, N - rem);   // positions of the row that holds p0
+          const unsigned char* zt = st + (cp >> 5) * slab + (cp & 3) * 4;
+          const int chunk = (cp & 31) >> 2;
+          float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
+          if (br == 32) {                    // no boundary inside: four independent chains
+            float2 b0 = a0, b1 = a0, b2 = a0;
+#pragma unroll
+            for (int r = 0; r < 32; r += 4) {
+              const unsigned w0 = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r, chunk));
+              const unsigned w1 = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r + 1, chunk));
+              const unsigned w2 = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r + 2, chunk));
+              const unsigned w3 = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r + 3, chunk));
+              a0 = __fadd2_rn(a0, make_float2(__uint_as_float(w0 << 16), __uint_as_float(w0 & 0xffff0000u)));
+              b0 = __fadd2_rn(b0, make_float2(__uint_as_float(w1 << 16), __uint_as_float(w1 & 0xffff0000u)));
+              b1 = __fadd2_rn(b1, make_float2(__uint_as_float(w2 << 16), __uint_as_float(w2 & 0xffff0000u)));
+              b2 = __fadd2_rn(b2, make_float2(__uint_as_float(w3 << 16), __uint_as_float(w3 & 0xffff0000u)));
+            }
+            a0 = __fadd2_rn(__fadd2_rn(a0, b0), __fadd2_rn(b1, b2));
+          } else {
+            for (int r = 0; r < br; ++r) {
+              const unsigned w = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r, chunk));
+              a0.x += __uint_as_float(w << 16);
+              a0.y += __uint_as_float(w & 0xffff0000u);
+            }
+            for (int r = br; r < nvalid; ++r) {
+              const unsigned w = *reinterpret_cast<const unsigned*>(zt + sw128_off(q * 32 + r, chunk));
+              a1.x += __uint_as_float(w << 16);
+              a1.y += __uint_as_float(w & 0xffff0000u);
+            }
+          }
+          float2* dst = reinterpret_cast<float2*>(p.partial + ((t * 4 + q) * 2) * (long long)c) + cp;
+          dst[0] = a0;
+          dst[c / 2] = a1;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&aempty[stage]);      // this warp has read what it needs of the tile
+      }
+      if (ep_tid == 0) {
         tma_store_wait_read0();
         mbar_arrive(&aempty[stage]);
       }
@@ -257,13 +314,61 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
+// Adds the partial column sums of every pair row (= token row g of the group) in ascending position order.  Group
+// mt of 32 positions keeps the sum of the row that holds its first position in slot 0 and of the row that starts
+// inside it in slot 1.
+__global__ void __launch_bounds__(128) segment_partials_kernel(const float* __restrict__ partial, BatchMeta m,
+                                                               long long P0, int C, int mean,
+                                                               __nv_bfloat16* __restrict__ out) {
+  const long long g = m.tok_off[0] + blockIdx.x;
+  const int s = find_sample(m.tok_off, m.B, g);
+  const long long N = m.N[s];
+  const long long lo = m.pair_off[s] + (g - m.tok_off[s]) * N - P0, hi = lo + N;
+  const float sc = mean ? 1.0f / (float)N : 1.0f;
+  const long long mt0 = lo >> 5, mt1 = (hi - 1) >> 5;
+  for (int c = threadIdx.x; c < C; c += 128) {
+    float tot = 0.f;
+    for (long long mb = mt0; mb <= mt1; mb += 8) {     // eight loads in flight, added in ascending order
+      float v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const long long mt = mb + k;
+        v[k] = mt <= mt1 ? partial[(mt * 2 + (lo > (mt << 5) ? 1 : 0)) * C + c] : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) tot += v[k];
+    }
+    out[g * C + c] = __float2bfloat16_rn(tot * sc);
+  }
+}
+
+// The fused reduction needs every 32 consecutive positions to meet at most one pair row boundary.
+bool fast_attn_out_reduce_supported(const BatchMeta& m) {
+  for (int s = 0; s < m.B; ++s)
+    if (m.N[s] > 0 && m.N[s] < 32) return false;
+  return true;
+}
+
+size_t fast_attn_out_partial_bytes(long long rows, int c) { return (size_t)((rows + 31) / 32) * 2 * c * sizeof(float); }
+
+nt_status fast_segment_partials(const float* partial, const BatchMeta& m, int C, int mean, void* out, cudaStream_t st) {
+  const long long G = m.tok_off[m.B] - m.tok_off[0];
+  if (G <= 0) return NT_OK;
+  if (G > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
+  {
+    LaunchScope ls("segment_partials", st);
+    segment_partials_kernel<<<(unsigned)G, 128, 0, st>>>(partial, m, m.pair_off[0], C, mean, (__nv_bfloat16*)out);
+  }
+  return cuda_ok();
+}
+
 bool fast_attn_out_supported(int c, int H, int d) {
   const int Hd = H * d;
   return (c == 64 || c == 128) && (Hd == 64 || Hd == 128);
 }
 
 nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
-                        const BatchMeta& m, int* status, cudaStream_t st) {
+                        const BatchMeta& m, int* status, cudaStream_t st, float* partial) {
   const int Hd = H * d;
   const void* wg = ap.wg;
   const float2* c01g = (const float2*)ap.c01g;
@@ -287,6 +392,9 @@ nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep&
   p.eps = eps;
   p.c01g = c01g;
   p.status = status;
+  p.partial = partial;
+  p.P0 = P0;
+  if (partial) p.m = m;
   {
     const unsigned box[2] = {64, 128};
     const unsigned long long zdims[2] = {(unsigned long long)c, (unsigned long long)p.rows};

@@ -42,8 +42,9 @@ def upload_weights(blocks: List[dict], dtype: torch.dtype, device="cuda") -> Lis
 class PairStack:
     """Device state for running a configuration's stacked blocks on one batch layout."""
 
-    def __init__(self, cfg: Config, lengths, weights_host: List[dict], device="cuda"):
+    def __init__(self, cfg: Config, lengths, weights_host: List[dict], device="cuda", fused_mean=True):
         self.cfg = cfg
+        self.fused_mean = fused_mean   # nt_row_attn_pairbias_mean instead of attention + nt_segment_reduce
         self.dtype = torch_dtype(cfg.dtype)
         self.device = torch.device(device)
         self.L = nt.Layout(lengths, device=device)
@@ -67,8 +68,11 @@ class PairStack:
         bc = nt.nt_pair_broadcast_add if accumulate else nt.nt_pair_broadcast
         bc(L, x, b["W_a"], b["W_b"], b["ln_gamma"], b["ln_beta"], LN_EPS, self.z, self.workspace, stream)
         nt.nt_tri_mul_out(L, w["trimul"], LN_EPS, self.z, self.workspace, stream)
-        nt.nt_row_attn_pairbias(L, nt.NT_ORDER_PAIR_IJC, w["attn"], cfg.H, cfg.d, LN_EPS, self.z, self.workspace, stream)
-        nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, self.z, self.m, L.status, stream)
+        if self.fused_mean:     # attention and the mean over j in one call
+            nt.nt_row_attn_pairbias_mean(L, w["attn"], cfg.H, cfg.d, LN_EPS, self.z, self.m, self.workspace, stream)
+        else:
+            nt.nt_row_attn_pairbias(L, nt.NT_ORDER_PAIR_IJC, w["attn"], cfg.H, cfg.d, LN_EPS, self.z, self.workspace, stream)
+            nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, self.z, self.m, L.status, stream)
         nt.nt_token_update(self.m, w["reduce"]["W_r"], x, stream)
 
     def forward(self, x: torch.Tensor, stream=None, persistent=False):

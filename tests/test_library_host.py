@@ -118,6 +118,11 @@ def test_host_validation_of_the_calls_after_the_block(lib):
     assert lib.lib.nt_col_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 8, None) == 3          # workspace
     assert lib.lib.nt_col_attn_pairbias(C.byref(L), 7, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None) == 2              # dtype
     assert lib.lib.nt_col_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 2, 200, C.byref(aw), 1e-5, FAKE, FAKE, 1 << 20, None) == 2  # head dim
+    # fused attention + mean: same checks as the attention, plus the output and the level-2 splits it may fall back on
+    assert lib.lib.nt_row_attn_pairbias_mean(C.byref(L), lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, None, FAKE, 1 << 20, None) == 1   # no output
+    assert lib.lib.nt_row_attn_pairbias_mean(C.byref(L), lib.NT_BF16, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, FAKE, 8, None) in (1, 3)    # splits / workspace
+    assert lib.lib.nt_row_attn_pairbias_mean(C.byref(L), 7, 8, 2, 4, C.byref(aw), 1e-5, FAKE, FAKE, FAKE, 1 << 20, None) == 2             # dtype
+    assert lib.lib.nt_row_attn_pairbias_mean(C.byref(L), lib.NT_BF16, 8, 2, 200, C.byref(aw), 1e-5, FAKE, FAKE, FAKE, 1 << 20, None) == 2 # head dim
     sw = lib.nt_single_attn_weights()
     assert lib.lib.nt_single_attn_pairbias(C.byref(L), lib.NT_BF16, 8, 8, 2, 4, C.byref(sw), 1e-5, FAKE, FAKE, FAKE, 1 << 20, None) == 1
     sw = lib.nt_single_attn_weights(*([FAKE] * 10))
