@@ -223,7 +223,8 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
     pa.ln_g = W->ln_in_gamma; pa.ln_b = W->ln_in_beta; pa.eps = eps;
     nt_status r;
     if (tc) {
-      r = fast_tri_in(z, tprep, eps, c_z, c_h, w.a, w.b, m, L->status_d, st);
+      // the gate buffer is free on this path (the output stage recomputes the gate): it carries the z row statistics
+      r = fast_tri_in(z, tprep, eps, c_z, c_h, w.a, w.b, m, L->status_d, st, (float2*)w.g);
       if (r != NT_OK) return r;
     } else {
       pa.W1 = W->W_ag; pa.W2 = W->W_ap; pa.Nout = c_h; pa.out = w.a; pa.out_mode = O_CHANNEL_MAJOR;
@@ -245,7 +246,7 @@ static nt_status tri_mul_generic(const nt_layout* L, const Totals& tot, int c_z,
       r = launch_contract<T>((const T*)w.a, (const T*)w.b, (T*)w.t, c_h, m, st, incoming);
     if (r != NT_OK) return r;
     if (tc_out) {
-      r = fast_tri_out(z, w.t, tprep, eps, c_z, c_h, m, L->status_d, st);
+      r = fast_tri_out(z, w.t, tprep, eps, c_z, c_h, m, L->status_d, st, (const float2*)w.g);
       if (r != NT_OK) return r;
       continue;
     }
@@ -287,7 +288,9 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
     pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
     nt_status r;
     if (tc_in) {
-      r = fast_attn_in(zx, aprep, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, m, L->status_d, st);
+      // the gate buffer is free when the output stage recomputes the gate: it carries the z row statistics to it
+      r = fast_attn_in(zx, aprep, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, m, L->status_d, st,
+                       tc_out ? (float2*)w.g : nullptr);
       if (r != NT_OK) return r;
     } else {
       pa.W1 = W->W_q; pa.out = w.q;
@@ -334,7 +337,8 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
       if (mean_out && fast_attn_out_reduce_supported(m) &&
           fast_attn_out_partial_bytes(rows, c) <= (size_t)tot.T2 * Hd * sizeof(T))
         partial = (float*)w.q;
-      r = fast_attn_out(zx, w.o, W->W_o, aprep, eps, c, H, d, m, L->status_d, st, partial);
+      r = fast_attn_out(zx, w.o, W->W_o, aprep, eps, c, H, d, m, L->status_d, st, partial,
+                        tc_in ? (const float2*)w.g : nullptr);
       if (r != NT_OK) return r;
       if (partial) {
         if ((r = fast_segment_partials(partial, m, c, 1, mean_out, st)) != NT_OK) return r;

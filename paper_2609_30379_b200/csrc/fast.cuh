@@ -64,17 +64,17 @@ nt_status fast_attn_prep(const nt_attn_weights* W, int c, int H, int d, void* pr
 // a = sig(LN(z) W_ag^T) * (LN(z) W_ap^T), b likewise: fp16, channel-major
 bool fast_tri_in_supported(int c_z, int c_h);
 nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int c_h, void* a, void* b,
-                      const BatchMeta& m, int* status, cudaStream_t st);
+                      const BatchMeta& m, int* status, cudaStream_t st, float2* zstats = nullptr);
 
 // in place on z: z += sigmoid(LN_in(z) W_g^T) * (LN_out(t) W_o^T); t fp16 channel-major scaled by 1 / N
 bool fast_tri_out_supported(int c_z, int c_h);
 nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int c_z, int c_h, const BatchMeta& m,
-                       int* status, cudaStream_t st);
+                       int* status, cudaStream_t st, const float2* zstats = nullptr);
 
 // q, k, v row-major bf16, bias head-major bf16 (nullable)
 bool fast_attn_in_supported(int c, int H, int d);
 nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int H, int d, void* q, void* k, void* v,
-                       void* bias, const BatchMeta& m, int* status, cudaStream_t st);
+                       void* bias, const BatchMeta& m, int* status, cudaStream_t st, float2* zstats = nullptr);
 
 // in place on z: z += (sigmoid(LN(z) W_g^T) * o) W_o^T
 bool fast_attn_out_supported(int c, int H, int d);
@@ -84,7 +84,7 @@ bool fast_attn_out_reduce_supported(const BatchMeta& m);
 size_t fast_attn_out_partial_bytes(long long rows, int c);
 nt_status fast_segment_partials(const float* partial, const BatchMeta& m, int C, int mean, void* out, cudaStream_t st);
 nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
-                        const BatchMeta& m, int* status, cudaStream_t st, float* partial = nullptr);
+                        const BatchMeta& m, int* status, cudaStream_t st, float* partial = nullptr, const float2* zstats = nullptr);
 
 // SwiGLU transition, fused on tcgen05: z += (silu(LN(z) W_a^T) * (LN(z) W_b^T)) W_2^T with the hidden activation
 // kept on chip.  prep: at least 1 MiB of device scratch for the folded weights.

@@ -35,6 +35,7 @@ struct AttnInParams {
   int aug_rows;
   __nv_bfloat16* bias;           // nullable
   int* status;
+  float2* zstats;                // nullable: (mean, rstd) of every row of the group, for the output stage
 };
 
 __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_constant__ AttnInParams p) {
@@ -166,7 +167,8 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
       mbar_wait(&afull[stage], phase, ab);
-      convert_row_ln_fp16(sA + stage * a_stage, nslab, a_slab, sAx + stage * 2 * zx_region + row * 16, row, hf, c, p.eps);
+      convert_row_ln_fp16(sA + stage * a_stage, nslab, a_slab, sAx + stage * 2 * zx_region + row * 16, row, hf, c, p.eps,
+                          p.zstats && t * 128 + row < p.rows ? p.zstats + t * 128 + row : nullptr);
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&aconv[stage]);
@@ -261,7 +263,7 @@ bool fast_attn_in_supported(int c, int H, int d) {
 }
 
 nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int H, int d, void* q, void* k, void* v,
-                       void* bias, const BatchMeta& m, int* status, cudaStream_t st) {
+                       void* bias, const BatchMeta& m, int* status, cudaStream_t st, float2* zstats) {
   const int Hd = H * d;
   const int wrows = 3 * Hd + 16;
   const void* wprime = ap.w;
@@ -287,6 +289,7 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
     p.bias = (__nv_bfloat16*)bias;
     p.status = status;
     const long long P0 = m.pair_off[g0];
+    p.zstats = zstats ? zstats + P0 : nullptr;
     p.pair_off[0] = 0;
     for (int l = 0; l < AI_MAXB; ++l) {
       const int N = l < p.B ? m.N[g0 + l] : 0;

@@ -31,6 +31,7 @@ struct AttnOutParams {
   float eps;
   const float2* c01g;            // [Hd]
   int* status;
+  const float2* zstats;          // nullable: (mean, rstd) of every z row, left by the input projection
   float* partial;                // nullable: [ceil(rows / 32)][2][c] column sums of 32-position groups
   long long P0;                  // packed position of row 0 of the maps
   BatchMeta m;                   // read only when partial != nullptr
@@ -154,6 +155,15 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      if (p.zstats) {                       // the input projection normalised the same rows: take its statistics
+        const float2 zst = t * 128 + row < p.rows ? __ldg(p.zstats + t * 128 + row) : make_float2(0.f, 1.f);
+        mbar_wait(&afull[stage], phase, ab);
+        sStats[stage][row] = zst;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&aconv[stage]);
+        if (++stage == 2) { stage = 0; phase ^= 1; }
+        continue;
+      }
       mbar_wait(&afull[stage], phase, ab);
       float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
       const unsigned char* zt = sSt + stage * stage_bytes;
@@ -368,7 +378,7 @@ bool fast_attn_out_supported(int c, int H, int d) {
 }
 
 nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep& ap, float eps, int c, int H, int d,
-                        const BatchMeta& m, int* status, cudaStream_t st, float* partial) {
+                        const BatchMeta& m, int* status, cudaStream_t st, float* partial, const float2* zstats) {
   const int Hd = H * d;
   const void* wg = ap.wg;
   const float2* c01g = (const float2*)ap.c01g;
@@ -393,6 +403,7 @@ nt_status fast_attn_out(void* z, const void* o, const void* W_o, const AttnPrep&
   p.c01g = c01g;
   p.status = status;
   p.partial = partial;
+  p.zstats = zstats ? zstats + P0 : nullptr;
   p.P0 = P0;
   if (partial) p.m = m;
   {

@@ -42,6 +42,8 @@ struct TriInParams {
   int B, c_z, c_h, aug_rows;
   float eps;
   int* status;
+  float2* zstats;                          // nullable: (mean, rstd) of every row of z, by packed position, for the output stage
+  long long pos_off[TI_MAXB];              // packed position of the first cell of the sample
 };
 
 __device__ inline bool ti_decode(const TriInParams& p, long long q, int& s, int& i, int& jc) {
@@ -202,9 +204,9 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
     // ------------------------------------------------------------------ converters: two threads per position, each
     // owning four of the eight 16-byte chunks of every 64-channel slab
     const int row = (warp - 2) * 16 + (lane >> 1), hf = lane & 1;
-    int stage = 0;
+    int stage = 0, tn = 0;
     unsigned phase = 0;
-    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+    for (long long t = blockIdx.x; t < ntiles; t += gridDim.x, ++tn) {
       mbar_wait(&afull[stage], phase, ab);
       unsigned char* tile = sZ + stage * z_stage_bytes;
       uint4 raw[2][4];
@@ -249,6 +251,12 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
                 make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
+      if (p.zstats && hf == 0) {             // the output stage normalises the same rows: hand the statistics over
+        const int4 info = tinfo[tn & 7][row / TI_CH];
+        const int j = info.z + (row % TI_CH);
+        if (info.w && j < p.N[info.x])
+          p.zstats[p.pos_off[info.x] + (long long)info.y * p.N[info.x] + j] = make_float2(mean, rstd);
+      }
       if (hf == 0) {
         const float mm = -mean * rstd;
         const __half mh = __float2half_rn(mm), ml = __float2half_rn(mm - __half2float(mh));
@@ -346,7 +354,7 @@ __global__ void __launch_bounds__(TI_THREADS, 1) tri_in_kernel(const __grid_cons
 bool fast_tri_in_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) && (c_h == 64 || c_h == 128); }
 
 nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int c_h, void* a, void* b,
-                      const BatchMeta& m, int* status, cudaStream_t st) {
+                      const BatchMeta& m, int* status, cudaStream_t st, float2* zstats) {
   const int nslab = c_z / 64;
   const int wrows = 4 * c_h;
   const size_t smem = (size_t)nslab * wrows * 128 + (size_t)wrows * 16 + 2 * (size_t)nslab * 128 * 128 +
@@ -377,11 +385,13 @@ nt_status fast_tri_in(const void* z, const TriPrep& tp, float eps, int c_z, int 
       const unsigned xbox[2] = {8, 256};
       if (!make_tmap_16bit(&p.xmap, tp.aug1, 2, xdims, xstr, xbox, 0)) return cuda_fail("tri_in augmentation map");
     }
+    p.zstats = zstats;
     p.chunk_off[0] = 0;
     for (int l = 0; l < TI_MAXB; ++l) {
       const int N = l < p.B ? m.N[g0 + l] : 0;
       p.N[l] = N;
       p.cm_off[l] = l < p.B ? m.cm_off[g0 + l] : 0;
+      p.pos_off[l] = l < p.B ? m.pair_off[g0 + l] : 0;
       p.chunk_off[l + 1] = p.chunk_off[l] + (long long)N * ((N + TI_CH - 1) / TI_CH);
       if (N > 0) {
         const unsigned long long dims[4] = {(unsigned long long)c_z, (unsigned long long)N, (unsigned long long)N, 1};

@@ -37,6 +37,8 @@ struct TriOutParams {
   const float2* c01o;            // [c_z]
   const float2* c01g;            // [c_z]
   int* status;
+  const float2* zstats;          // nullable: (mean, rstd) of every z row by packed position, left by the input projection
+  long long pos_off[TO_MAXB];
 };
 
 __device__ inline bool to_decode(const TriOutParams& p, long long q, int& s, int& i, int& j0) {
@@ -194,6 +196,17 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
     int stage = 0;
     unsigned phase = 0;
     for (long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+      // this row's chunk: scale of eps for t, and the z statistics the input projection left (requested early)
+      float eps_t = p.eps;
+      float2 zst = make_float2(0.f, 1.f);
+      {
+        int s_, i_, j_;
+        if (to_decode(p, 2 * t + q, s_, i_, j_)) {
+          eps_t = p.eps / ((float)p.N[s_] * (float)p.N[s_]);
+          const int j = j_ + (row & 63);
+          if (p.zstats && j < p.N[s_]) zst = __ldg(p.zstats + p.pos_off[s_] + (long long)i_ * p.N[s_] + j);
+        }
+      }
       mbar_wait(&tfullb[stage], phase, ab);
       // Statistics of t over channels (columns of the MN-major fp16 tile).  Eight lanes share a group of eight
       // positions: lane cg sums channels cg, cg + 8, ... with 16-byte loads (8 positions each), then a
@@ -242,17 +255,12 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive(&tfree[stage]);
       // t arrives scaled by 1 / N_s (see the contraction); LayerNorm is scale-free once eps is scaled alike
-      float eps_t = p.eps;
-      {
-        int s_, i_, j_;
-        if (to_decode(p, 2 * t + q, s_, i_, j_)) eps_t = p.eps / ((float)p.N[s_] * (float)p.N[s_]);
-      }
       const float tmean = ts / (float)c_h;
       const float trstd = rsqrtf(fmaxf(tq / (float)c_h - tmean * tmean, 0.f) + eps_t);
       // z row: statistics of the bf16 tile (read only)
       mbar_wait(&zfullb[stage], phase, ab);
-      float zs, zq;
-      {
+      float zs = 0.f, zq = 0.f;
+      if (!p.zstats) {
         float s4[4] = {0.f, 0.f, 0.f, 0.f}, q4[4] = {0.f, 0.f, 0.f, 0.f};
         const unsigned char* zt = sZ + stage * z_stage;
         for (int g8 = 0; g8 < c_z / 8; ++g8) {
@@ -269,8 +277,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
         zs = (s4[0] + s4[1]) + (s4[2] + s4[3]);
         zq = (q4[0] + q4[1]) + (q4[2] + q4[3]);
       }
-      const float zmean = zs / (float)c_z;
-      const float zrstd = rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
+      const float zmean = p.zstats ? zst.x : zs / (float)c_z;
+      const float zrstd = p.zstats ? zst.y : rsqrtf(fmaxf(zq / (float)c_z - zmean * zmean, 0.f) + p.eps);
       sStats[stage][row] = make_float4(0.5f * trstd, 0.5f * zrstd, -0.5f * trstd * tmean, -0.5f * zrstd * zmean);
       __syncwarp();
       if (lane == 0) {
@@ -363,7 +371,7 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
 bool fast_tri_out_supported(int c_z, int c_h) { return (c_z == 64 || c_z == 128) && (c_h == 64 || c_h == 128); }
 
 nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int c_z, int c_h, const BatchMeta& m,
-                       int* status, cudaStream_t st) {
+                       int* status, cudaStream_t st, const float2* zstats) {
   const void* wo = tp.wo;
   const void* wg = tp.wg;
   const float2* c01o = (const float2*)tp.c01o;
@@ -387,6 +395,7 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
     p.c01o = c01o;
     p.c01g = c01g;
     p.status = status;
+    p.zstats = zstats;
     {
       const unsigned long long dims[2] = {(unsigned long long)c_h, (unsigned long long)c_z};
       const unsigned long long strides[1] = {(unsigned long long)c_h * 2};
@@ -400,6 +409,7 @@ nt_status fast_tri_out(void* z, const void* t, const TriPrep& tp, float eps, int
     for (int l = 0; l < TO_MAXB; ++l) {
       const int N = l < p.B ? m.N[g0 + l] : 0;
       p.N[l] = N;
+      p.pos_off[l] = l < p.B ? m.pair_off[g0 + l] : 0;
       p.chunk_off[l + 1] = p.chunk_off[l] + (long long)N * ((N + 63) / 64);
       if (N > 0) {
         const int ld = round_up8(N);

@@ -313,7 +313,7 @@ __device__ inline void convert_row_bf16_to_f16(unsigned char* tile, int nslab, i
 // (c1_hi, c1_hi, c1_lo, c0_hi, c0_lo) one more K step then adds m * c1 + c0, so the accumulator holds LN(z) W^T.
 // The two threads of a row must be neighbouring lanes of a converged warp.
 __device__ inline void convert_row_ln_fp16(unsigned char* tile, int nslab, int slab_bytes, unsigned char* aug_row, int row,
-                                           int hf, int c, float eps) {
+                                           int hf, int c, float eps, float2* stats_out = nullptr) {
   uint4 raw[2][4];
 #pragma unroll
   for (int sl = 0; sl < 2; ++sl)
@@ -354,6 +354,7 @@ __device__ inline void convert_row_ln_fp16(unsigned char* tile, int nslab, int s
         *reinterpret_cast<uint4*>(tile + sl * slab_bytes + sw128_off(row, hf * 4 + j)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
+  if (hf == 0 && stats_out) *stats_out = make_float2(mean, rstd);   // for a later stage that normalises the same row
   if (hf == 0) {
     const float mm = -mean * rstd;
     const __half mh = __float2half_rn(mm), ml = __float2half_rn(mm - __half2float(mh));
