@@ -37,10 +37,10 @@ struct AttnOutParams {
   BatchMeta m;                   // read only when partial != nullptr
 };
 
-__device__ inline float sigmoid_fast3(float x) {
+__device__ inline float ao_tanh(float x) {
   float t;
-  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(0.5f * x));
-  return fmaf(0.5f, t, 0.5f);
+  asm("tanh.approx.f32 %0, %1;\n" : "=f"(t) : "f"(x));
+  return t;
 }
 
 __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_constant__ AttnOutParams p) {
@@ -58,7 +58,8 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
   unsigned char* sWg = smem;                          // zslab slabs of [Hd rows][64]
   unsigned char* sWo = sWg + zslab * wg_slab;         // oslab slabs of [c rows][64]
   unsigned char* sSt = sWo + oslab * wo_slab;         // 2 stages: z slabs then o slabs
-  float2* sC = reinterpret_cast<float2*>(sSt + 2 * stage_bytes);
+  float* sC0 = reinterpret_cast<float*>(sSt + 2 * stage_bytes);   // c0 / 2 per gate channel
+  float* sC1 = sC0 + Hd;                                          // c1 per gate channel
   unsigned long long* afull = bars;        // [2]
   unsigned long long* aempty = bars + 2;   // [2]
   unsigned long long* gfull = bars + 4;    // [2]
@@ -84,7 +85,10 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&tmem_base_s, 512);
-  for (int n = threadIdx.x; n < Hd; n += AO_THREADS) sC[n] = p.c01g[n];
+  for (int n = threadIdx.x; n < Hd; n += AO_THREADS) {
+    sC0[n] = 0.5f * p.c01g[n].x;
+    sC1[n] = p.c01g[n].y;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -202,7 +206,9 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
       mbar_wait(&gfull[buf], gph[buf], ab);
       gph[buf] ^= 1;
       tc_fence_after();
-      const float mean = sStats[stage][row].x, rstd = sStats[stage][row].y;
+      // sigmoid(x) = tanh(x / 2) / 2 + 1 / 2 with x / 2 = (rstd / 2) acc + (c0 / 2 - mean (rstd / 2) c1), on packed float pairs
+      const float rh = 0.5f * sStats[stage][row].y, mh = -sStats[stage][row].x * rh;
+      const float2 rh2 = make_float2(rh, rh), mh2 = make_float2(mh, mh), half2 = make_float2(0.5f, 0.5f);
       const unsigned taddr = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256;
       for (int c0 = half * (Hd / 2); c0 < (half + 1) * (Hd / 2); c0 += 32) {
         unsigned r[32];
@@ -217,11 +223,11 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            const float2 k0 = sC[c0 + n0], k1 = sC[c0 + n0 + 1];
-            const float g0 = sigmoid_fast3(fmaf(rstd, __uint_as_float(r[n0]) - mean * k0.y, k0.x));
-            const float g1 = sigmoid_fast3(fmaf(rstd, __uint_as_float(r[n0 + 1]) - mean * k1.y, k1.x));
-            __nv_bfloat162 hh = __floats2bfloat162_rn(g0 * __uint_as_float(w[e] << 16),
-                                                      g1 * __uint_as_float(w[e] & 0xffff0000u));
+            const float2 k0 = *reinterpret_cast<const float2*>(sC0 + c0 + n0), k1 = *reinterpret_cast<const float2*>(sC1 + c0 + n0);
+            const float2 xh = __ffma2_rn(rh2, make_float2(__uint_as_float(r[n0]), __uint_as_float(r[n0 + 1])), __ffma2_rn(mh2, k1, k0));
+            const float2 g = __ffma2_rn(half2, make_float2(ao_tanh(xh.x), ao_tanh(xh.y)), half2);
+            const float2 go = __fmul2_rn(g, make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u)));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(go.x, go.y);
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);
@@ -248,8 +254,9 @@ __global__ void __launch_bounds__(AO_THREADS, 1) attn_out_kernel(const __grid_co
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            const float z0 = __uint_as_float(w[e] << 16), z1 = __uint_as_float(w[e] & 0xffff0000u);   // the bf16 state
-            __nv_bfloat162 hh = __floats2bfloat162_rn(z0 + __uint_as_float(r[n0]), z1 + __uint_as_float(r[n0 + 1]));
+            const float2 zn = __fadd2_rn(make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u)),   // the bf16 state
+                                         make_float2(__uint_as_float(r[n0]), __uint_as_float(r[n0 + 1])));
+            __nv_bfloat162 hh = __floats2bfloat162_rn(zn.x, zn.y);
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);

@@ -214,7 +214,8 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
       float ts, tq;
       {
         const int cg = lane & 7, pgl = ((warp - 2) * 4 + (lane >> 3)) & 7;      // position group inside the 64-position chunk
-        float a8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, q8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        float2 a2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        float2 q2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         const unsigned char* tb = sT + stage * t_stage + q * t_chunk + cg * 128 + ((pgl ^ cg) << 4);   // channel c = cc * 8 + cg: c & 7 = cg
 #pragma unroll 4
         for (int cc = 0; cc < c_h / 8; ++cc) {
@@ -223,10 +224,12 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float2 f = unpack_h2(w[e]);
-            a8[2 * e] += f.x; a8[2 * e + 1] += f.y;
-            q8[2 * e] = fmaf(f.x, f.x, q8[2 * e]); q8[2 * e + 1] = fmaf(f.y, f.y, q8[2 * e + 1]);
+            a2[e] = __fadd2_rn(a2[e], f);
+            q2[e] = __ffma2_rn(f, f, q2[e]);
           }
         }
+        float a8[8] = {a2[0].x, a2[0].y, a2[1].x, a2[1].y, a2[2].x, a2[2].y, a2[3].x, a2[3].y};
+        float q8[8] = {q2[0].x, q2[0].y, q2[1].x, q2[1].y, q2[2].x, q2[2].y, q2[3].x, q2[3].y};
         // reduce-scatter: after the step with lane bit b, a lane keeps the half of the positions whose bit b equals its own
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -323,18 +326,25 @@ __global__ void __launch_bounds__(TO_THREADS, 1) tri_out_kernel(const __grid_con
           const float4 ko0 = *reinterpret_cast<const float4*>(sKo + cb), ko1 = *reinterpret_cast<const float4*>(sKo + cb + 4);
           const float4 kg0 = *reinterpret_cast<const float4*>(sKg + cb), kg1 = *reinterpret_cast<const float4*>(sKg + cb + 4);
           // per channel: c0 / 2 - mean rstd c1 / 2, the part of the LayerNorm that does not depend on the accumulator
-          const float bo[8] = {fmaf(tmh, ko0.x, co0.x), fmaf(tmh, ko0.y, co0.y), fmaf(tmh, ko0.z, co0.z), fmaf(tmh, ko0.w, co0.w),
-                               fmaf(tmh, ko1.x, co1.x), fmaf(tmh, ko1.y, co1.y), fmaf(tmh, ko1.z, co1.z), fmaf(tmh, ko1.w, co1.w)};
-          const float bg[8] = {fmaf(zmh, kg0.x, cg0.x), fmaf(zmh, kg0.y, cg0.y), fmaf(zmh, kg0.z, cg0.z), fmaf(zmh, kg0.w, cg0.w),
-                               fmaf(zmh, kg1.x, cg1.x), fmaf(zmh, kg1.y, cg1.y), fmaf(zmh, kg1.z, cg1.z), fmaf(zmh, kg1.w, cg1.w)};
+          // (everything on packed float pairs: half the issue slots)
+          const float2 tm2 = make_float2(tmh, tmh), zm2 = make_float2(zmh, zmh), tr2 = make_float2(trh, trh), zr2 = make_float2(zrh, zrh);
+          const float2 bo[4] = {__ffma2_rn(tm2, make_float2(ko0.x, ko0.y), make_float2(co0.x, co0.y)),
+                                __ffma2_rn(tm2, make_float2(ko0.z, ko0.w), make_float2(co0.z, co0.w)),
+                                __ffma2_rn(tm2, make_float2(ko1.x, ko1.y), make_float2(co1.x, co1.y)),
+                                __ffma2_rn(tm2, make_float2(ko1.z, ko1.w), make_float2(co1.z, co1.w))};
+          const float2 bg[4] = {__ffma2_rn(zm2, make_float2(kg0.x, kg0.y), make_float2(cg0.x, cg0.y)),
+                                __ffma2_rn(zm2, make_float2(kg0.z, kg0.w), make_float2(cg0.z, cg0.w)),
+                                __ffma2_rn(zm2, make_float2(kg1.x, kg1.y), make_float2(cg1.x, cg1.y)),
+                                __ffma2_rn(zm2, make_float2(kg1.z, kg1.w), make_float2(cg1.z, cg1.w))};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int n0 = ch * 8 + e * 2;
-            const float z0 = __uint_as_float(w[e] << 16), z1 = __uint_as_float(w[e] & 0xffff0000u);   // the bf16 state
-            const float oh0 = fmaf(trh, __uint_as_float(r1[n0]), bo[e * 2]), oh1 = fmaf(trh, __uint_as_float(r1[n0 + 1]), bo[e * 2 + 1]);
-            const float t0 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0]), bg[e * 2]));
-            const float t1 = to_tanh(fmaf(zrh, __uint_as_float(r2[n0 + 1]), bg[e * 2 + 1]));
-            __nv_bfloat162 hh = __floats2bfloat162_rn(fmaf(oh0, t0, oh0) + z0, fmaf(oh1, t1, oh1) + z1);
+            const float2 z2 = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));   // the bf16 state
+            const float2 oh = __ffma2_rn(tr2, make_float2(__uint_as_float(r1[n0]), __uint_as_float(r1[n0 + 1])), bo[e]);
+            const float2 ta = __ffma2_rn(zr2, make_float2(__uint_as_float(r2[n0]), __uint_as_float(r2[n0 + 1])), bg[e]);
+            const float2 th = make_float2(to_tanh(ta.x), to_tanh(ta.y));
+            const float2 res = __fadd2_rn(__ffma2_rn(oh, th, oh), z2);
+            __nv_bfloat162 hh = __floats2bfloat162_rn(res.x, res.y);
             w[e] = *reinterpret_cast<unsigned*>(&hh);
           }
           *ptr = make_uint4(w[0], w[1], w[2], w[3]);
