@@ -83,11 +83,13 @@ def kernel_work(cfg: wl.Config):
     for n in ("q", "k", "v", "g"):
         w[f"generic_attn_in_{n}"] = dict(bytes=T2 * (c_z + Hd) * e, flops=2 * T2 * c_z * Hd)
     w["generic_attn_in_bias"] = dict(bytes=T2 * (c_z + H) * e, flops=2 * T2 * c_z * H)
-    w["attn_in"] = dict(bytes=T2 * (c_z + 4 * Hd + H) * e, flops=2 * T2 * c_z * (4 * Hd + H))
+    w["attn_in"] = dict(bytes=T2 * (c_z + 3 * Hd + H) * e, flops=2 * T2 * c_z * (3 * Hd + H))   # q, k, v and the bias planes (the gate is recomputed by the output stage)
     # the softmax needs one exponential per (query, key, head): the special-function units retire 16 per clock and SM
     w["generic_attn_core"] = w["attn_core"] = dict(bytes=T2 * (4 * Hd + H) * e, flops=4 * N3 * Hd, exps=N3 * H)
     w["generic_attn_core_col"] = w["attn_core_col"] = w["attn_core"]            # column-wise attention: same work
-    w["generic_attn_out"] = w["attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)
+    w["generic_attn_out"] = dict(bytes=T2 * (2 * Hd + 2 * c_z) * e, flops=2 * T2 * Hd * c_z)     # reads the stored gate
+    # the tensor-core output stage recomputes the gate from z: it reads z and o and writes z
+    w["attn_out"] = dict(bytes=T2 * (Hd + 2 * c_z) * e, flops=2 * T2 * (Hd + c_z) * c_z)
     sr = dict(bytes=T2 * c_z * e + T1 * c_z * e, flops=T2 * c_z)
     w["segment_reduce"] = w["generic_segment_reduce"] = sr
     # fused mean behind the attention output stage: two float partial sums per 32 positions and channel, read once

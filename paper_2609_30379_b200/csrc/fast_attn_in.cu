@@ -24,7 +24,7 @@ struct AttnInParams {
   CUtensorMap zmap;              // {c, rows}, box {64, 128}
   CUtensorMap wmap;              // {c, 3 Hd + 16}, box {64, 128} (q, k, v rows)
   CUtensorMap wbmap;             // same tensor, box {64, 16} (bias rows)
-  CUtensorMap omap[3];           // q, k, v: {Hd, rows}, box {64, 128}
+  CUtensorMap omap[3];           // q, k, v: {Hd, rows}, box {64, 32}: one epilogue warp's rows
   long long pair_off[AI_MAXB + 1];   // relative to the first position of the group
   long long cm_off[AI_MAXB];
   int N[AI_MAXB];
@@ -197,9 +197,14 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
           const int nout = u == 0 ? 2 : 1;
           for (int oi = 0; oi < nout; ++oi) {
             const int o = u == 0 ? oi : 2;          // 0 = q, 1 = k, 2 = v
-            if (store_pending) {                    // previous output still being read from the panels?
-              if (ep_tid == 0) tma_store_wait_read0();
-              named_bar_sync(1, 256);
+            // Every warp stores its own 32 positions x 64 channels as soon as it has written them (Hd = 64: the two
+            // warps of a lane quarter share the slab and meet at a barrier of their own), so no store waits for the
+            // other warps and only the warp's own previous store has to have read its corner of the panels.
+            const bool storer = lane == 0 && (npanel == 2 || half == 0);
+            if (store_pending) {
+              if (storer) tma_store_wait_read0();
+              if (npanel == 1) named_bar_sync(2 + quarter, 64);
+              else __syncwarp();
             }
             for (int c0 = half * cpw; c0 < (half + 1) * cpw; c0 += 32) {
               unsigned r[32];
@@ -219,10 +224,12 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
               }
             }
             fence_proxy_async_smem();
-            named_bar_sync(1, 256);
-            if (ep_tid == 0) {
-              for (int pn = 0; pn < npanel; ++pn)
-                tma_store_2d(&p.omap[o], sOut + pn * a_slab, pn * 64, (int)(t * 128));
+            if (npanel == 1) named_bar_sync(2 + quarter, 64);
+            else __syncwarp();
+            if (storer) {
+              const int pn = npanel == 2 ? half : 0;
+              if (t * 128 + quarter * 32 < p.rows)
+                tma_store_2d(&p.omap[o], sOut + pn * a_slab + quarter * 32 * 128, pn * 64, (int)(t * 128 + quarter * 32));
               tma_store_commit();
             }
             store_pending = true;
@@ -249,7 +256,7 @@ __global__ void __launch_bounds__(AI_THREADS, 1) attn_in_kernel(const __grid_con
       }
       if (++stage == 2) { stage = 0; phase ^= 1; }
     }
-    if (ep_tid == 0) tma_store_wait_all0();
+    if (lane == 0) tma_store_wait_all0();
   }
   tc_fence_before();
   __syncthreads();
@@ -317,8 +324,9 @@ nt_status fast_attn_in(const void* z, const AttnPrep& ap, float eps, int c, int 
       const unsigned long long odims[2] = {(unsigned long long)Hd, (unsigned long long)p.rows};
       const unsigned long long ostr[1] = {(unsigned long long)Hd * 2};
       void* outs[3] = {q, k, v};
+      const unsigned obox[2] = {64, 32};
       for (int o = 0; o < 3; ++o)
-        if (!make_tmap_bf16(&p.omap[o], (char*)outs[o] + (size_t)P0 * Hd * 2, 2, odims, ostr, box))
+        if (!make_tmap_bf16(&p.omap[o], (char*)outs[o] + (size_t)P0 * Hd * 2, 2, odims, ostr, obox))
           return cuda_fail("attn_in out map");
     }
     const long long ntiles = (p.rows + 127) / 128;
