@@ -106,7 +106,7 @@ def kernel_work(cfg: wl.Config):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/ (cfg2 only);
 # other workloads report traffic = None.
-NCU_TRAFFIC_CFG2 = {"attn_core": 375.2e6, "tri_out": 242.2e6, "attn_in": 324.4e6, "tri_in": 232.0e6, "attn_out": 250.0e6,
+NCU_TRAFFIC_CFG2 = {"attn_core": 375.2e6, "tri_out": 247.3e6, "attn_in": 328.4e6, "tri_in": 233.8e6, "attn_out": 253.0e6,
                     "tri_contract": 255.4e6, "transition": 130.3e6, "tri_contract_in": 255.5e6, "attn_core_col": 375.1e6,
                     "single_attn_bias": 97.8e6}
 
