@@ -75,6 +75,16 @@ class PairStack:
             nt.nt_segment_reduce(nt.NT_REDUCE_MEAN, L.row_splits, self.z, self.m, L.status, stream)
         nt.nt_token_update(self.m, w["reduce"]["W_r"], x, stream)
 
+    def capture(self, x: torch.Tensor, persistent=False):
+        """Captures forward(x) in a CUDA graph and returns it; graph.replay() reruns every block on the same buffers
+        (x is updated in place each time).  Possible because no library call allocates or synchronises; valid for the
+        lengths this stack was built with, whose offsets travel by value in the kernel arguments.  Run forward(x) at
+        least once before capturing (first calls set kernel attributes)."""
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.forward(x, persistent=persistent)
+        return graph
+
     def forward(self, x: torch.Tensor, stream=None, persistent=False):
         """Runs every block in place on ``x`` [T1, c_s]; returns (x, z) for pair configs or
         (x, pooled) for the token-only configuration.  persistent=True keeps the pair state as a stream of its
