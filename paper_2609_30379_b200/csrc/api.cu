@@ -271,6 +271,9 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
   const bool tc = dt == NT_BF16 && !g_force_generic && pair && W->ln_gamma && tot.nmax < 60000;
   const bool tc_in = tc && fast_attn_in_supported(c, H, d) && fast_attn_core_supported(H, d);   // bias goes out times sqrt(d)
   const bool tc_out = tc && W->W_g && fast_attn_out_supported(c, H, d);   // recomputes the gate from z
+  const bool tok_fast = dt == NT_BF16 && !g_force_generic && !pair && !W->W_b && c % 8 == 0 && c <= Hd && c <= 2048 &&
+                        fast_attn_core_supported(H, d) && fast_token_gemm_supported(c, Hd, Hd) &&
+                        fast_token_gemm_supported(Hd, c, 0);
   AttnPrep aprep{};
   if (tc_in || tc_out) {
     nt_status r0 = fast_attn_prep(W, c, H, d, w.prep, aprep, st);
@@ -282,11 +285,30 @@ static nt_status attn_generic(const nt_layout* L, const Totals& tot, nt_order or
     const long long row0 = pair ? m.pair_off[0] : m.tok_off[0];
     const long long rows = (pair ? m.pair_off[m.B] : m.tok_off[m.B]) - row0;
     if (rows == 0) continue;
+    nt_status r;
+    if (tok_fast) {
+      // token order: the rows are T1 tokens, so the projections are small GEMMs on mma.sync tiles around the
+      // segmented core: LayerNorm once into the (not yet written) o buffer, q | k and v | g in two launches that share
+      // the normalised rows, the core, the gate, the output GEMM accumulated into x
+      const size_t e = 2, to = (size_t)row0 * Hd * e;
+      char* xr = (char*)zx + (size_t)row0 * c * e;
+      char* xh = xr;
+      if (W->ln_gamma) {
+        xh = (char*)w.o + to;
+        if ((r = fast_ln_rows(xr, W->ln_gamma, W->ln_beta, eps, c, rows, xh, st, "tok_attn_ln")) != NT_OK) return r;
+      }
+      if ((r = fast_token_gemm(xh, rows, c, W->W_q, Hd, (char*)w.q + to, W->W_k, Hd, (char*)w.k + to, 0, 0, "tok_attn_in_qk", st)) != NT_OK) return r;
+      if ((r = fast_token_gemm(xh, rows, c, W->W_v, Hd, (char*)w.v + to, W->W_g, W->W_g ? Hd : 0, W->W_g ? (char*)w.g + to : nullptr, 0, 0,
+                               "tok_attn_in_vg", st)) != NT_OK) return r;
+      if ((r = fast_attn_core(w.q, w.k, w.v, nullptr, w.o, H, d, 0, 0, m, L->status_d, st)) != NT_OK) return r;
+      if (W->W_g && (r = fast_gate_mul((char*)w.g + to, (char*)w.o + to, rows * Hd, st, "tok_attn_gate")) != NT_OK) return r;
+      if ((r = fast_token_gemm((char*)w.o + to, rows, Hd, W->W_o, c, xr, nullptr, 0, nullptr, 0, 1, "tok_attn_out", st)) != NT_OK) return r;
+      continue;
+    }
     ProjArgs pa{};
     pa.A = zx; pa.a_mode = A_ROWMAJOR; pa.row0 = row0; pa.rows = rows; pa.K = c;
     pa.ln_g = W->ln_gamma; pa.ln_b = W->ln_beta; pa.eps = eps;
     pa.Nout = Hd; pa.act = ACT_NONE; pa.out_mode = O_STORE;
-    nt_status r;
     if (tc_in) {
       // the gate buffer is free when the output stage recomputes the gate: it carries the z row statistics to it
       r = fast_attn_in(zx, aprep, eps, c, H, d, w.q, w.k, w.v, W->W_b ? w.bias : nullptr, m, L->status_d, st,

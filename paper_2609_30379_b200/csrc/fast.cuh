@@ -31,8 +31,9 @@ nt_status fast_token_gemm(const void* A, long long rows, int K, const void* W0, 
 // pair-biased single attention: LayerNorm of the token rows (bf16 out), o <- sigmoid(g) * o, and the bias planes
 // bias[s][h][i][j] = scale * (LN(z_ij) W_b^T)[h] in the head-major padded layout of the attention core
 bool fast_single_attn_supported(int c_s, int c_z, int H, int d);
-nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st);
-nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st);
+nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st,
+                       const char* name = "single_attn_ln");
+nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st, const char* name = "single_attn_gate");
 nt_status fast_single_bias(const void* z, const void* g, const void* b, const void* Wb, float eps, int C, int H, float scale,
                            const BatchMeta& m, void* bias, cudaStream_t st);
 

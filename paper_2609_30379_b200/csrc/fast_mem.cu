@@ -810,21 +810,22 @@ bool fast_single_attn_supported(int c_s, int c_z, int H, int d) {
          fast_token_gemm_supported(c_s, Hd, Hd) && fast_token_gemm_supported(Hd, c_s, 0);
 }
 
-nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st) {
+nt_status fast_ln_rows(const void* x, const void* g, const void* b, float eps, int C, long long rows, void* out, cudaStream_t st,
+                       const char* name) {
   if (rows <= 0) return NT_OK;
   {
-    LaunchScope ls("single_attn_ln", st);
+    LaunchScope ls(name, st);
     ln_rows_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)x, (const __nv_bfloat16*)g, (const __nv_bfloat16*)b, eps, C,
                                                                rows, (__nv_bfloat16*)out);
   }
   return cuda_ok("single attention LayerNorm launch");
 }
 
-nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st) {
+nt_status fast_gate_mul(const void* g, void* o, long long n, cudaStream_t st, const char* name) {
   if (n <= 0) return NT_OK;
   const long long n8 = n / 8;
   {
-    LaunchScope ls("single_attn_gate", st);
+    LaunchScope ls(name, st);
     gate_mul_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, st>>>((const __nv_bfloat16*)g, (__nv_bfloat16*)o, n8);
   }
   return cuda_ok("single attention gate launch");
