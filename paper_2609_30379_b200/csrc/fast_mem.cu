@@ -233,13 +233,18 @@ nt_status fast_broadcast_ln(const float* u, const float* v, const void* gamma, c
 // ------------------------------------------------------------------------------------------
 constexpr int SR_THREADS = 128;
 constexpr int SR_UNROLL = 4;
+constexpr int SR_CHUNK = 128;     // channels per block
 
 __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const __nv_bfloat16* __restrict__ v,
                                                                         __nv_bfloat16* __restrict__ out,
                                                                         const int64_t* __restrict__ splits, int C,
                                                                         int mean) {
-  extern __shared__ float part[];   // [RS][C]
-  const int VL = C >> 3;
+  extern __shared__ float part[];   // [RS][Cc]
+  // a block reduces one group over a chunk of up to 128 channels (blockIdx.y): wide rows keep several row slots
+  const int CV = C >> 3;                                  // 16-byte vectors per row
+  const int cb = blockIdx.y * SR_CHUNK;                   // first channel of the chunk
+  const int Cc = min(SR_CHUNK, C - cb);
+  const int VL = Cc >> 3;
   const int RS = SR_THREADS / VL;
   const int t = threadIdx.x;
   const int slot = t / VL, vl = t - slot * VL;
@@ -247,12 +252,12 @@ __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const _
   const long long lo = splits[g], hi = splits[g + 1];
   float acc[8] = {};
   if (slot < RS) {
-    const uint4* base = reinterpret_cast<const uint4*>(v) + vl;
+    const uint4* base = reinterpret_cast<const uint4*>(v) + (cb >> 3) + vl;
     long long r = lo + slot;
     for (; r + (long long)(SR_UNROLL - 1) * RS < hi; r += (long long)SR_UNROLL * RS) {
       uint4 d[SR_UNROLL];
 #pragma unroll
-      for (int uu = 0; uu < SR_UNROLL; ++uu) d[uu] = __ldg(base + (r + (long long)uu * RS) * VL);
+      for (int uu = 0; uu < SR_UNROLL; ++uu) d[uu] = __ldg(base + (r + (long long)uu * RS) * CV);
 #pragma unroll
       for (int uu = 0; uu < SR_UNROLL; ++uu) {
         const unsigned w[4] = {d[uu].x, d[uu].y, d[uu].z, d[uu].w};
@@ -264,7 +269,7 @@ __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const _
       }
     }
     for (; r < hi; r += RS) {
-      const uint4 d = __ldg(base + r * VL);
+      const uint4 d = __ldg(base + r * CV);
       const unsigned w[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -273,15 +278,15 @@ __global__ void __launch_bounds__(SR_THREADS) segment_reduce_fast_kernel(const _
       }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) part[slot * C + vl * 8 + e] = acc[e];
+    for (int e = 0; e < 8; ++e) part[slot * Cc + vl * 8 + e] = acc[e];
   }
   __syncthreads();
   const long long n = hi - lo;
   const float sc = (mean && n > 0) ? 1.0f / (float)n : 1.0f;
-  for (int c = t; c < C; c += SR_THREADS) {
+  for (int c = t; c < Cc; c += SR_THREADS) {
     float tot = 0.f;
-    for (int sl = 0; sl < RS; ++sl) tot += part[sl * C + c];
-    out[g * C + c] = __float2bfloat16_rn(tot * sc);
+    for (int sl = 0; sl < RS; ++sl) tot += part[sl * Cc + c];
+    out[g * C + cb + c] = __float2bfloat16_rn(tot * sc);
   }
 }
 
@@ -291,11 +296,11 @@ nt_status fast_segment_reduce(const void* v, void* out, const int64_t* splits, l
                               cudaStream_t st) {
   if (G <= 0) return NT_OK;
   if (G > 0x7FFFFFFFll) return NT_ERR_UNSUPPORTED;
-  const int VL = C / 8, RS = SR_THREADS / VL;
-  const size_t smem = (size_t)RS * C * sizeof(float);
+  const size_t smem = (size_t)SR_THREADS * 8 * sizeof(float);   // row slots x chunk channels never exceed threads x 8
+  const dim3 grid((unsigned)G, (unsigned)((C + SR_CHUNK - 1) / SR_CHUNK));
   {
     LaunchScope ls("segment_reduce", st);
-    segment_reduce_fast_kernel<<<(unsigned)G, SR_THREADS, smem, st>>>((const __nv_bfloat16*)v, (__nv_bfloat16*)out,
+    segment_reduce_fast_kernel<<<grid, SR_THREADS, smem, st>>>((const __nv_bfloat16*)v, (__nv_bfloat16*)out,
                                                                      splits, C, mean);
   }
   return cuda_ok();
