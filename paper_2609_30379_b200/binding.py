@@ -175,6 +175,19 @@ class Layout:
                            _ptr(self.lengths_d) if self.B else None, _ptr(self.tok_off), _ptr(self.pair_off),
                            _ptr(self.row_splits), _ptr(self.status))
 
+    def rebuild(self, lengths: Sequence[int], stream=None):
+        """Takes the lengths of another batch with the same B, T1 and T2 (the buffer sizes) and builds its offsets
+        into the same device buffers, so that pointers held elsewhere (a captured graph, a cached nt_layout) stay valid."""
+        new = np.ascontiguousarray(np.asarray(lengths, dtype=np.int64))
+        if new.shape != self.lengths_h.shape or int(new.sum()) != self.T1 or int((new * new).sum()) != self.T2:
+            raise ValueError("Layout.rebuild needs the same B, T1 and T2; build a new Layout instead")
+        np.copyto(self.lengths_h, new)
+        if self.B:
+            self.lengths_d.copy_(torch.from_numpy(self.lengths_h), non_blocking=True)
+        nt_offsets_build(self.lengths_d, self.B, self.T1, self.T2, self.tok_off, self.pair_off, self.row_splits,
+                         self.pos_sample, self.pos_i, self.pos_j, self.gather_rows, self.gather_cols,
+                         self.status, stream)
+
     def device_status(self) -> int:
         return int(self.status.item())
 

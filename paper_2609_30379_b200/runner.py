@@ -85,6 +85,24 @@ class PairStack:
             self.forward(x, persistent=persistent)
         return graph
 
+    def forward_cached(self, x: torch.Tensor):
+        """forward(x) through a graph captured the first time this stack sees the current lengths and this x buffer,
+        and replayed afterwards: the kernel arguments carry the batch's offsets by value, so a captured step is valid
+        for one length signature; another signature (Layout.rebuild with other lengths) captures again."""
+        key = (tuple(int(v) for v in self.L.lengths_h), x.data_ptr())
+        cache = self.__dict__.setdefault("_graphs", {})
+        if key not in cache:
+            keep = x.clone()
+            self.forward(x)                    # first calls set kernel attributes; not captured
+            x.copy_(keep)
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                cache[key] = self.capture(x)   # capture does not execute
+            torch.cuda.current_stream().wait_stream(side)
+        cache[key].replay()
+        return (x, self.z) if self.cfg.kind == "pair" else (x, self.pooled)
+
     def forward(self, x: torch.Tensor, stream=None, persistent=False):
         """Runs every block in place on ``x`` [T1, c_s]; returns (x, z) for pair configs or
         (x, pooled) for the token-only configuration.  persistent=True keeps the pair state as a stream of its

@@ -31,3 +31,35 @@ def test_captured_stack_replays_to_the_same_result():
         torch.cuda.synchronize()
         assert torch.equal(x, want_x) and torch.equal(st.z, want_z)
     assert st.L.device_status() == 0
+
+
+def test_graph_cache_follows_the_length_signature():
+    """Layout.rebuild keeps the buffers (same B, T1, T2) and forward_cached captures once per length signature:
+    a batch with the same totals but another partition gets a graph of its own and the result of a fresh stack."""
+    from paper_2609_30379_b200 import runner
+    la, lb = (40, 33, 0, 56), (33, 56, 0, 40)          # same B, sum N and sum N^2
+    cfg_a = wl.Config("sig_a", "bf16", la, c_s=64, c_z=128, c_h=128, H=4, d=32, blocks=1, seed=52)
+    cfg_b = wl.Config("sig_b", "bf16", lb, c_s=64, c_z=128, c_h=128, H=4, d=32, blocks=1, seed=52)
+    inp = wl.make_inputs(cfg_a)
+    x0 = runner.to_device(inp["x"], torch.bfloat16)
+
+    def eager(cfg):
+        st = runner.PairStack(cfg, cfg.lengths, inp["blocks"])
+        x = x0.clone()
+        st.forward(x)
+        torch.cuda.synchronize()
+        return x, st.z.clone()
+
+    want_a, want_b = eager(cfg_a), eager(cfg_b)
+    st = runner.PairStack(cfg_a, la, inp["blocks"])
+    x = x0.clone()
+    for lengths, want in ((la, want_a), (lb, want_b), (la, want_a), (lb, want_b)):
+        st.L.rebuild(lengths)
+        x.copy_(x0)
+        st.forward_cached(x)
+        torch.cuda.synchronize()
+        assert torch.equal(x, want[0]) and torch.equal(st.z, want[1])
+        assert st.L.device_status() == 0
+    assert len(st._graphs) == 2
+    with pytest.raises(ValueError):
+        st.L.rebuild((40, 33, 1, 56))
